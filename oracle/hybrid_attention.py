@@ -1,0 +1,309 @@
+"""CPU oracle for the hybrid attention of Hybrid Forcing.  TEST INFRASTRUCTURE ONLY.
+
+Plain, slow numpy (fp64) restatement of what the hot path computes, written from
+the paper's definitions.  It shares nothing with the CUDA path and must never be
+imported by the product: only tests, the smoke check and the bench's CPU-baseline
+leg may call it.
+
+Inputs are real-valued numpy arrays (the bf16 inputs widened exactly to fp64).
+Nothing is rounded anywhere, except in the *canonical fp32 scorer* below, which
+restates in IEEE float32 the exact operation order in which block means and
+block scores are formed, because a floating-point score decides an integer
+(which blocks are kept) and both sides must take that decision in one precision.
+
+What follows which passage:
+  phi                     activation of the linear branch (Eq. 3; unnamed there, elu+1 here)
+  block_ranges            Alg. 3 "divide Q / K,V into blocks", one chunk at a time
+  block_means, block_scores        Eq. 5 (mean of a query block times mean of a key block)
+  block_means_f32, block_scores_f32   Eq. 5 in the canonical float32 order
+  keep_count, select_blocks         top-K rule after Eq. 5 / Alg. 3 "M_c[i,j] = 1 if in TopK(P_c[i,:], K)"
+  sparse_attention        Eq. 6 as its plain definition: softmax over the kept keys
+  sparse_attention_tiled  Alg. 3 inner loops (running max / sum / rescale), step by step
+  absorb                  Eq. 3 (state update) without the rotation
+  linear_readout          Eq. 4 without the rotation: Linear(phi(Q) L / (phi(Q) H))
+  HybridStream            Alg. 2 cache protocol (evict -> update state -> append) around Alg. 3, Eq. 7 sum
+
+Readings taken where the paper is silent or inconsistent (all listed again in the
+design notes): H is accumulated as the plain sum of phi(K) rows (so that Eq. 4 is a
+normalised kernel average); no rotation inside the linear branch; phi = elu + 1;
+"Linear" is a per-head d x d matrix plus optional bias, y = W x + b; the top-K is
+per query-block row; ties go to the lower (older) block index; each chunk is cut
+into blocks from its own first token, a short last block is averaged over its own
+length; the denominator is phi(q).H + eps.
+
+Parity unpinned (nothing in the paper fixes them, the authors' code is not
+available): the choice of phi, the shape of "Linear", the sum-vs-mean reading of
+H, the rounding of K = ratio * T_n, the blocking of ragged chunks, the tie rule,
+the eps.  Everything else is pinned by tests against brute force, closed forms
+and library routines.
+"""
+from __future__ import annotations
+
+import math
+import numpy as np
+
+F32 = np.float32
+
+
+# --------------------------------------------------------------------------- phi
+def phi(x: np.ndarray) -> np.ndarray:
+    """elu(x) + 1: x + 1 for x > 0, exp(x) otherwise (positive feature map of the linear branch)."""
+    x = np.asarray(x, dtype=np.float64)
+    return np.where(x > 0.0, x + 1.0, np.exp(np.minimum(x, 0.0)))
+
+
+# --------------------------------------------------------------------------- blocks
+def block_ranges(n_tokens: int, b: int):
+    """[(start, stop)] of consecutive blocks of b tokens; the last may be short."""
+    return [(s, min(s + b, n_tokens)) for s in range(0, n_tokens, b)]
+
+
+def key_block_table(chunk_lengths, b: int):
+    """Logical key blocks of a window made of chunks (oldest first, current chunk last).
+
+    Each chunk is cut from its own token 0.  Returns [(chunk_index, start, stop)]."""
+    table = []
+    for c, n in enumerate(chunk_lengths):
+        table += [(c, s, e) for (s, e) in block_ranges(n, b)]
+    return table
+
+
+# --------------------------------------------------------------------------- Eq. 5, fp64
+def block_means(x: np.ndarray, b: int) -> np.ndarray:
+    """x [T, d] -> [ceil(T/b), d]: mean over the tokens of each block (Eq. 5 "Mean")."""
+    x = np.asarray(x, dtype=np.float64)
+    return np.stack([x[s:e].mean(axis=0) for (s, e) in block_ranges(x.shape[0], b)])
+
+
+def block_scores(q_means: np.ndarray, k_means: np.ndarray) -> np.ndarray:
+    """A[i, j] = Mean(q_i) . Mean(k_j)  (Eq. 5)."""
+    return np.asarray(q_means, np.float64) @ np.asarray(k_means, np.float64).T
+
+
+def pooled_softmax(scores: np.ndarray, d: int) -> np.ndarray:
+    """P_c = Softmax(pool(Q) pool(K)^T / sqrt(d)), row-wise (Alg. 3 form of the block score)."""
+    s = np.asarray(scores, np.float64) / math.sqrt(d)
+    s = s - s.max(axis=1, keepdims=True)
+    e = np.exp(s)
+    return e / e.sum(axis=1, keepdims=True)
+
+
+# --------------------------------------------------------------------------- Eq. 5, canonical float32
+def block_means_f32(x: np.ndarray, b: int) -> np.ndarray:
+    """Block means in the canonical float32 order.
+
+    x is float32 [T, d] (bf16 values widened exactly).  Per block and per column:
+    16 running sums, chain r adding tokens r, r+16, r+32, ... of the block in
+    ascending order starting from +0; the 16 chains are then added one after another
+    in ascending r; the total is divided by float32(n), n the block's own length.
+    Every operation is one IEEE float32 operation, round to nearest even."""
+    x = np.asarray(x)
+    assert x.dtype == np.float32 and x.ndim == 2
+    d = x.shape[1]
+    out = []
+    for (s, e) in block_ranges(x.shape[0], b):
+        chains = np.zeros((16, d), dtype=F32)
+        for t0 in range(s, e, 16):
+            rows = x[t0:min(t0 + 16, e)]
+            chains[: rows.shape[0]] = chains[: rows.shape[0]] + rows
+        total = chains[0].copy()
+        for r in range(1, 16):
+            total = total + chains[r]
+        out.append(total / F32(e - s))
+    out = np.stack(out)
+    assert out.dtype == np.float32
+    return out
+
+
+def block_scores_f32(q_means: np.ndarray, k_means: np.ndarray) -> np.ndarray:
+    """A[i, j] in the canonical float32 order.
+
+    32 partial sums: partial l takes columns l, l+32, l+64, ... in ascending order,
+    each term a rounded float32 product added by a rounded float32 add (no fused
+    multiply-add), the first product taken as is.  The 32 partials are then folded
+    as a butterfly: p[l] + p[l+16] for l < 16, then +8, +4, +2, +1."""
+    qm = np.asarray(q_means)
+    km = np.asarray(k_means)
+    assert qm.dtype == np.float32 and km.dtype == np.float32
+    d = qm.shape[1]
+    assert d % 32 == 0
+    prod = qm[:, None, :] * km[None, :, :]                  # float32 products
+    prod = prod.reshape(qm.shape[0], km.shape[0], d // 32, 32)
+    acc = prod[:, :, 0, :].copy()
+    for m in range(1, d // 32):
+        acc = acc + prod[:, :, m, :]
+    width = 16
+    while width >= 1:
+        acc = acc[..., :width] + acc[..., width:2 * width]
+        width //= 2
+    assert acc.dtype == np.float32
+    return acc[..., 0]
+
+
+# --------------------------------------------------------------------------- top-K
+def keep_count(topk: int, keep_permille: int, n_key_blocks: int) -> int:
+    """Blocks kept per query-block row: topk if given, else ceil(permille/1000 * T_n); at least 1, at most T_n."""
+    k = topk if topk > 0 else -(-keep_permille * n_key_blocks // 1000)
+    return max(1, min(k, n_key_blocks))
+
+
+def select_blocks(scores: np.ndarray, k: int) -> np.ndarray:
+    """Binary mask M [T_m, T_n]: per row the k largest scores, equal scores going to the lower index."""
+    scores = np.asarray(scores)
+    mask = np.zeros(scores.shape, dtype=bool)
+    for i in range(scores.shape[0]):
+        order = sorted(range(scores.shape[1]), key=lambda j: (-float(scores[i, j]), j))
+        mask[i, order[:k]] = True
+    return mask
+
+
+# --------------------------------------------------------------------------- Eq. 6
+def sparse_attention(q, k_chunks, v_chunks, b: int, mask: np.ndarray, q_blocks=None) -> np.ndarray:
+    """O_local by definition: every query row attends, with a softmax over q.k/sqrt(d), to exactly
+    the key tokens of the key blocks its query block keeps (Eq. 6).
+
+    q [T_c, d]; k_chunks / v_chunks: lists of [n_c, d] (oldest chunk first, current chunk last);
+    mask [T_m, T_n] over the logical key blocks.  q_blocks: optional subset of query blocks to
+    compute (other rows are returned as NaN)."""
+    q = np.asarray(q, np.float64)
+    d = q.shape[1]
+    table = key_block_table([kc.shape[0] for kc in k_chunks], b)
+    out = np.full(q.shape[:1] + (v_chunks[0].shape[1],), np.nan)
+    for i, (qs, qe) in enumerate(block_ranges(q.shape[0], b)):
+        if q_blocks is not None and i not in q_blocks:
+            continue
+        kept = [table[j] for j in range(len(table)) if mask[i, j]]
+        ks = np.concatenate([np.asarray(k_chunks[c][s:e], np.float64) for (c, s, e) in kept])
+        vs = np.concatenate([np.asarray(v_chunks[c][s:e], np.float64) for (c, s, e) in kept])
+        s_ = q[qs:qe] @ ks.T / math.sqrt(d)
+        s_ = s_ - s_.max(axis=1, keepdims=True)
+        p = np.exp(s_)
+        out[qs:qe] = (p @ vs) / p.sum(axis=1, keepdims=True)
+    return out
+
+
+def sparse_attention_tiled(q, k_chunks, v_chunks, b: int, mask: np.ndarray) -> np.ndarray:
+    """O_local by the tile recurrence of Alg. 3: m = -inf, l = 0, O = 0, then for each kept block
+    S = q_i k_j^T / sqrt(d); m' = max(m, rowmax S); P = exp(S - m'); l = e^{m-m'} l + rowsum P;
+    O = diag(e^{m-m'}) O + P v_j; finally O / l."""
+    q = np.asarray(q, np.float64)
+    d = q.shape[1]
+    table = key_block_table([kc.shape[0] for kc in k_chunks], b)
+    out = np.zeros((q.shape[0], v_chunks[0].shape[1]))
+    for i, (qs, qe) in enumerate(block_ranges(q.shape[0], b)):
+        qi = q[qs:qe]
+        m = np.full(qi.shape[0], -np.inf)
+        l = np.zeros(qi.shape[0])
+        o = np.zeros((qi.shape[0], out.shape[1]))
+        for j, (c, s, e) in enumerate(table):
+            if not mask[i, j]:
+                continue
+            S = qi @ np.asarray(k_chunks[c][s:e], np.float64).T / math.sqrt(d)
+            m_new = np.maximum(m, S.max(axis=1))
+            P = np.exp(S - m_new[:, None])
+            alpha = np.exp(m - m_new)
+            l = alpha * l + P.sum(axis=1)
+            o = alpha[:, None] * o + P @ np.asarray(v_chunks[c][s:e], np.float64)
+            m = m_new
+        out[qs:qe] = o / l[:, None]
+    return out
+
+
+# --------------------------------------------------------------------------- Eq. 3 / Eq. 4
+def absorb(S: np.ndarray, z: np.ndarray, k_ev, v_ev):
+    """Fold evicted tokens into the state (Eq. 3): S += phi(K_ev)^T V_ev (rows: key feature, columns: value
+    dim), z += sum over tokens of phi(K_ev)."""
+    f = phi(k_ev)
+    return S + f.T @ np.asarray(v_ev, np.float64), z + f.sum(axis=0)
+
+
+def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6) -> np.ndarray:
+    """O_history (Eq. 4): h = phi(q) S / (phi(q) . z + eps) per query row, then Linear: y = W h + bias."""
+    f = phi(q)
+    h = (f @ S) / (f @ z + eps)[:, None]
+    if W is not None:
+        h = h @ np.asarray(W, np.float64).T
+    if bias is not None:
+        h = h + np.asarray(bias, np.float64)[None, :]
+    return h
+
+
+# --------------------------------------------------------------------------- Alg. 2 + Alg. 3
+class HybridStream:
+    """Streaming state of one layer (all batches and heads) and the per-chunk forward.
+
+    Alg. 2: the rolling cache holds the clean K/V of the last P = w/c - 1 chunks; a committed clean chunk
+    is appended and whatever then exceeds P chunks is popped from the front and folded into (S, z) --
+    the state is updated before the evicted K/V are dropped.  With P >= 1 this is the paper's
+    "if full: pop(0), update state; append"; with P = 0 a committed chunk goes straight into the state.
+    """
+
+    def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
+                 W=None, bias=None, eps=1e-6):
+        self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
+        self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
+        self.W = None if W is None else np.asarray(W, np.float64)        # [H, d, d]
+        self.bias = None if bias is None else np.asarray(bias, np.float64)  # [H, d]
+        self.past = []                                                   # list of (k [B,H,n,d], v) fp64
+        self.S = np.zeros((batch, heads, d, d))
+        self.z = np.zeros((batch, heads, d))
+        self.absorbed_tokens = 0
+
+    # -- Alg. 2, cache commit
+    def append(self, k_clean, v_clean):
+        self.past.append((np.asarray(k_clean, np.float64), np.asarray(v_clean, np.float64)))
+        while len(self.past) > self.P:
+            k_ev, v_ev = self.past.pop(0)
+            for bi in range(self.B):
+                for h in range(self.H):
+                    self.S[bi, h], self.z[bi, h] = absorb(self.S[bi, h], self.z[bi, h], k_ev[bi, h], v_ev[bi, h])
+            self.absorbed_tokens += k_ev.shape[2]
+
+    # -- Eq. 5 + top-K
+    def n_key_blocks(self, n_cur: int) -> int:
+        return sum(-(-kp.shape[2] // self.b) for kp, _ in self.past) + -(-n_cur // self.b)
+
+    def select(self, q, k_cur, exact: bool = False):
+        """Masks [B, H, T_m, T_n].  exact=False: canonical float32 scores (the bit-exact contract);
+        exact=True: fp64 scores (the ideal the canonical order approximates)."""
+        B, H = self.B, self.H
+        n_kb = self.n_key_blocks(k_cur.shape[2])
+        k = keep_count(self.topk, self.keep_permille, n_kb)
+        masks, scores = [], []
+        for bi in range(B):
+            for h in range(H):
+                if exact:
+                    qm = block_means(q[bi, h], self.b)
+                    km = np.concatenate([block_means(kp[bi, h], self.b) for kp, _ in self.past]
+                                        + [block_means(k_cur[bi, h], self.b)])
+                    a = block_scores(qm, km)
+                else:
+                    as32 = lambda x: np.asarray(x, np.float64).astype(F32)   # exact: values are bf16
+                    qm = block_means_f32(as32(q[bi, h]), self.b)
+                    km = np.concatenate([block_means_f32(as32(kp[bi, h]), self.b) for kp, _ in self.past]
+                                        + [block_means_f32(as32(k_cur[bi, h]), self.b)])
+                    a = block_scores_f32(qm, km)
+                scores.append(a)
+                masks.append(select_blocks(a, k))
+        shape = (B, H) + masks[0].shape
+        return np.stack(masks).reshape(shape), np.stack(scores).reshape(shape)
+
+    # -- Alg. 3 + Eq. 7
+    def forward(self, q, k_cur, v_cur, mask=None, q_blocks=None, parts: bool = False):
+        """O = O_local + O_history for the current chunk's queries against past chunks + the current chunk.
+        mask: [B,H,T_m,T_n] (default: the canonical selection)."""
+        q = np.asarray(q, np.float64); k_cur = np.asarray(k_cur, np.float64); v_cur = np.asarray(v_cur, np.float64)
+        if mask is None:
+            mask, _ = self.select(q, k_cur)
+        o_loc = np.empty_like(q); o_hist = np.empty_like(q)
+        for bi in range(self.B):
+            for h in range(self.H):
+                kc = [kp[bi, h] for kp, _ in self.past] + [k_cur[bi, h]]
+                vc = [vp[bi, h] for _, vp in self.past] + [v_cur[bi, h]]
+                o_loc[bi, h] = sparse_attention(q[bi, h], kc, vc, self.b, mask[bi, h], q_blocks)
+                o_hist[bi, h] = linear_readout(q[bi, h], self.S[bi, h], self.z[bi, h],
+                                               None if self.W is None else self.W[h],
+                                               None if self.bias is None else self.bias[h], self.eps)
+        if parts:
+            return o_loc + o_hist, o_loc, o_hist
+        return o_loc + o_hist

@@ -1,0 +1,373 @@
+"""Pins for the CPU oracle: each oracle function is checked against something other than itself --
+brute force written token by token, a library routine, a closed form, or an invariant of the method.
+The paper prints no numeric worked example of its attention, so none can be quoted; the hand-derived
+cases in tests/golden/hand_cases.json are closed forms of Eq. 3-7.
+"""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import hybrid_attention as oa
+from paper_2604_10103_b200 import inputs as gen
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rnd(shape, seed):
+    """bf16-representable N(0,1) values as fp64."""
+    return gen.bf16_bits_to_f64(gen.normal_bf16(shape, 77, seed))
+
+
+# ----------------------------------------------------------------------------- phi
+def test_phi_matches_library_elu_plus_one():
+    import torch
+    x = np.linspace(-12, 12, 4001)
+    ref = torch.nn.functional.elu(torch.from_numpy(x)).numpy() + 1.0
+    assert np.allclose(oa.phi(x), ref, rtol=0, atol=1e-15)
+    assert oa.phi(0.0) == 1.0 and (oa.phi(x) > 0).all()
+
+
+# ----------------------------------------------------------------------------- blocks
+def test_block_ranges_cover_and_ragged_tail():
+    assert oa.block_ranges(4680, 128)[-1] == (4608, 4680) and len(oa.block_ranges(4680, 128)) == 37
+    assert oa.block_ranges(64, 16) == [(0, 16), (16, 32), (32, 48), (48, 64)]
+    tab = oa.key_block_table([4680, 4680, 4680], 128)
+    assert len(tab) == 111 and tab[37] == (1, 0, 128) and tab[36] == (0, 4608, 4680)
+
+
+def test_keep_count_rule():
+    assert oa.keep_count(2, 0, 12) == 2                 # tiny case: top-2
+    assert oa.keep_count(0, 250, 111) == 28             # ceil(27.75)
+    assert oa.keep_count(0, 100, 110) == 11             # exact multiples do not round up
+    assert oa.keep_count(0, 1000, 111) == 111
+    assert oa.keep_count(5, 0, 3) == 3                  # warm-up: fewer blocks than k
+    assert oa.keep_count(0, 1, 10) == 1                 # never empty
+
+
+# ----------------------------------------------------------------------------- Eq. 5
+def test_block_means_and_scores_brute_force():
+    q = rnd((70, 32), 1); k = rnd((50, 32), 2)
+    qm = oa.block_means(q, 16); km = oa.block_means(k, 16)
+    assert qm.shape == (5, 32) and km.shape == (4, 32)
+    for i, (s, e) in enumerate([(0, 16), (16, 32), (32, 48), (48, 64), (64, 70)]):
+        for c in range(32):
+            assert abs(qm[i, c] - sum(q[t, c] for t in range(s, e)) / (e - s)) < 1e-13
+    a = oa.block_scores(qm, km)
+    for i, j in itertools.product(range(5), range(4)):
+        assert abs(a[i, j] - sum(qm[i, c] * km[j, c] for c in range(32))) < 1e-12
+
+
+def test_canonical_f32_scorer_within_rounding_of_fp64():
+    q = rnd((300, 128), 3); k = rnd((300, 128), 4)
+    qm32 = oa.block_means_f32(q.astype(np.float32), 128)
+    km32 = oa.block_means_f32(k.astype(np.float32), 128)
+    assert np.abs(qm32 - oa.block_means(q, 128)).max() < 2e-6
+    a32 = oa.block_scores_f32(qm32, km32)
+    a64 = oa.block_scores(oa.block_means(q, 128), oa.block_means(k, 128))
+    assert np.abs(a32 - a64).max() < 1e-6
+    # exact in float32 when nothing rounds: small integers
+    xi = np.arange(64 * 32, dtype=np.float32).reshape(64, 32) % 7
+    assert np.array_equal(oa.block_means_f32(xi, 16), oa.block_means(xi, 16).astype(np.float32))
+    assert np.array_equal(oa.block_scores_f32(xi[:4] * 2, xi[4:8]), (xi[:4] * 2).astype(np.float64) @ xi[4:8].T)
+
+
+def test_canonical_f32_order_is_the_documented_one():
+    """Token-by-token scalar restatement of the documented order on a ragged block."""
+    x = rnd((41, 32), 5).astype(np.float32)
+    got = oa.block_means_f32(x, 32)
+    for (s, e), row in zip([(0, 32), (32, 41)], got):
+        for c in range(0, 32, 5):
+            chains = [np.float32(0)] * 16
+            for t in range(s, e):
+                chains[(t - s) % 16] = np.float32(chains[(t - s) % 16] + x[t, c])
+            tot = chains[0]
+            for r in range(1, 16):
+                tot = np.float32(tot + chains[r])
+            assert row[c] == np.float32(tot / np.float32(e - s))
+    qm = rnd((2, 64), 6).astype(np.float32); km = rnd((3, 64), 7).astype(np.float32)
+    a = oa.block_scores_f32(qm, km)
+    for i, j in itertools.product(range(2), range(3)):
+        p = [np.float32(np.float32(qm[i, l] * km[j, l]) + np.float32(qm[i, l + 32] * km[j, l + 32])) for l in range(32)]
+        w = 16
+        while w >= 1:
+            p = [np.float32(p[l] + p[l + w]) for l in range(w)]
+            w //= 2
+        assert a[i, j] == p[0]
+
+
+def test_softmax_form_selects_the_same_blocks_as_raw_scores():
+    q = rnd((128, 64), 8); k = rnd((256, 64), 9)
+    a = oa.block_scores(oa.block_means(q, 16), oa.block_means(k, 16))
+    p = oa.pooled_softmax(a, 64)
+    assert np.allclose(p.sum(axis=1), 1.0)
+    for kk in (1, 3, 8, 16):
+        assert np.array_equal(oa.select_blocks(a, kk), oa.select_blocks(p, kk))
+
+
+def test_select_blocks_rule():
+    a = np.array([[0.1, 0.9, -0.3, 0.9, 0.5]])
+    assert oa.select_blocks(a, 2).tolist() == [[False, True, False, True, False]]
+    assert oa.select_blocks(a, 1).tolist() == [[False, True, False, False, False]]   # tie -> lower index
+    assert oa.select_blocks(np.zeros((3, 6)), 2).tolist() == [[True, True, False, False, False, False]] * 3
+    assert oa.select_blocks(np.array([[0.0, -0.0, 0.0]]), 2).tolist() == [[True, True, False]]
+    m = oa.select_blocks(rnd((7, 13), 10), 4)
+    assert (m.sum(axis=1) == 4).all()
+
+
+# ----------------------------------------------------------------------------- Eq. 6
+def brute_masked_attention(q, keys, vals, token_mask):
+    """Dense softmax with an explicit [T_q, N_k] 0/1 token mask, scalar loops."""
+    d = q.shape[1]
+    out = np.zeros((q.shape[0], vals.shape[1]))
+    for r in range(q.shape[0]):
+        cols = [c for c in range(keys.shape[0]) if token_mask[r, c]]
+        logits = [sum(q[r, x] * keys[c, x] for x in range(d)) / math.sqrt(d) for c in cols]
+        mx = max(logits)
+        w = [math.exp(l - mx) for l in logits]
+        tot = sum(w)
+        for wi, c in zip(w, cols):
+            out[r] += wi / tot * vals[c]
+    return out
+
+
+def expand_mask(mask, q_len, chunk_lens, b):
+    tm = np.zeros((q_len, sum(chunk_lens)), dtype=bool)
+    offs = np.concatenate([[0], np.cumsum(chunk_lens)])
+    table = oa.key_block_table(chunk_lens, b)
+    for i, (qs, qe) in enumerate(oa.block_ranges(q_len, b)):
+        for j, (c, s, e) in enumerate(table):
+            if mask[i, j]:
+                tm[qs:qe, offs[c] + s: offs[c] + e] = True
+    return tm
+
+
+@pytest.mark.parametrize("b,lens", [(8, [24, 24, 24]), (8, [20, 20]), (16, [40])])
+def test_sparse_attention_equals_brute_force_masked_softmax(b, lens):
+    d = 16
+    q = rnd((lens[-1], d), 11)
+    kc = [rnd((n, d), 20 + i) for i, n in enumerate(lens)]
+    vc = [rnd((n, d), 30 + i) for i, n in enumerate(lens)]
+    tm_blocks = -(-lens[-1] // b)
+    tn_blocks = sum(-(-n // b) for n in lens)
+    rng = np.random.default_rng(5)
+    mask = np.zeros((tm_blocks, tn_blocks), dtype=bool)
+    for i in range(tm_blocks):
+        mask[i, rng.choice(tn_blocks, size=2, replace=False)] = True
+    ref = brute_masked_attention(q, np.concatenate(kc), np.concatenate(vc), expand_mask(mask, lens[-1], lens, b))
+    got = oa.sparse_attention(q, kc, vc, b, mask)
+    assert np.abs(got - ref).max() < 1e-13
+    assert np.abs(oa.sparse_attention_tiled(q, kc, vc, b, mask) - got).max() < 1e-12
+
+
+def test_all_blocks_kept_is_dense_window_attention_library_sdpa():
+    import torch
+    d, b, lens = 32, 16, [40, 40, 40]
+    q = rnd((40, d), 12)
+    kc = [rnd((n, d), 40 + i) for i, n in enumerate(lens)]
+    vc = [rnd((n, d), 50 + i) for i, n in enumerate(lens)]
+    mask = np.ones((3, 9), dtype=bool)
+    got = oa.sparse_attention(q, kc, vc, b, mask)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q)[None], torch.from_numpy(np.concatenate(kc))[None], torch.from_numpy(np.concatenate(vc))[None])[0]
+    assert np.abs(got - ref.numpy()).max() < 1e-13
+
+
+def test_sparse_attention_closed_forms():
+    d, b = 16, 8
+    q = rnd((16, d), 13); kc = [rnd((16, d), 14), rnd((16, d), 15)]; vc = [rnd((16, d), 16), rnd((16, d), 17)]
+    mask = np.array([[True, False, True, False], [False, True, True, False]])
+    # V == 1  ->  O == 1
+    ones = [np.ones((16, d))] * 2
+    assert np.abs(oa.sparse_attention(q, kc, ones, b, mask) - 1).max() < 1e-14
+    # q == 0  ->  uniform average of the kept V rows
+    o = oa.sparse_attention(np.zeros((16, d)), kc, vc, b, mask)
+    assert np.abs(o[0] - (vc[0][0:8].sum(0) + vc[1][0:8].sum(0)) / 16).max() < 1e-14
+    assert np.abs(o[8] - (vc[0][8:16].sum(0) + vc[1][0:8].sum(0)) / 16).max() < 1e-14
+    # shifting every logit of a row by a constant leaves O unchanged: k -> k + t * q/|q|^2 is row dependent,
+    # so use one query row
+    q1 = q[:1]
+    kshift = [kk + 3.0 * q1 / (q1 @ q1.T) for kk in kc]
+    m1 = np.array([[True, True, False, True]])
+    a = oa.sparse_attention(np.repeat(q1, 8, 0), kc, vc, b, m1)
+    s = oa.sparse_attention(np.repeat(q1, 8, 0), kshift, vc, b, m1)
+    assert np.abs(a - s).max() < 1e-12
+
+
+def test_hand_worked_cases():
+    cases = json.load(open(os.path.join(GOLDEN, "hand_cases.json")))
+    c = cases["softmax_two_keys"]
+    o = oa.sparse_attention(np.array(c["q"]), [np.array(c["k"])], [np.array(c["v"])], 1, np.array([[True, True]]))
+    assert np.allclose(o, c["o_local"], rtol=0, atol=1e-15)
+    c = cases["state_and_readout"]
+    S, z = oa.absorb(np.zeros((2, 2)), np.zeros(2), np.array(c["k_ev"]), np.array(c["v_ev"]))
+    assert np.allclose(S, c["S"], rtol=0, atol=1e-15) and np.allclose(z, c["z"], rtol=0, atol=1e-15)
+    h = oa.linear_readout(np.array(c["q"]), S, z, np.array(c["W"]), np.array(c["bias"]), eps=0.0)
+    assert np.allclose(h, c["o_history"], rtol=0, atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- Eq. 3 / Eq. 4
+def test_absorb_orientation_and_brute_force():
+    k = rnd((9, 4), 18); v = rnd((9, 6), 19)
+    S, z = oa.absorb(np.zeros((4, 6)), np.zeros(4), k, v)
+    Sb = np.zeros((4, 6)); zb = np.zeros(4)
+    for t in range(9):
+        f = [k[t, a] + 1 if k[t, a] > 0 else math.exp(k[t, a]) for a in range(4)]
+        for a in range(4):
+            zb[a] += f[a]
+            for c in range(6):
+                Sb[a, c] += f[a] * v[t, c]
+    assert np.abs(S - Sb).max() < 1e-13 and np.abs(z - zb).max() < 1e-13
+
+
+def test_readout_equals_direct_kernel_average():
+    d = 8
+    k = rnd((30, d), 21); v = rnd((30, d), 22); q = rnd((5, d), 23)
+    S, z = oa.absorb(np.zeros((d, d)), np.zeros(d), k, v)
+    got = oa.linear_readout(q, S, z, eps=0.0)
+    for r in range(5):
+        w = [float(oa.phi(q[r]) @ oa.phi(k[t])) for t in range(30)]
+        ref = sum(wi * v[t] for t, wi in enumerate(w)) / sum(w)
+        assert np.abs(got[r] - ref).max() < 1e-13
+    # V == 1 -> h == 1 -> O_history = W 1 + bias
+    S1, z1 = oa.absorb(np.zeros((d, d)), np.zeros(d), k, np.ones((30, d)))
+    W = rnd((d, d), 24); bias = rnd((d,), 25)
+    assert np.abs(oa.linear_readout(q, S1, z1, W, bias, eps=0.0) - (W.sum(axis=1) + bias)).max() < 1e-13
+    # Linear is y = W h (+ b), not h W
+    h = oa.linear_readout(q, S, z, eps=0.0)
+    assert np.abs(oa.linear_readout(q, S, z, W, bias, eps=0.0) - np.stack([W @ h[r] + bias for r in range(5)])).max() < 1e-13
+    # empty state: h = 0, O_history = bias
+    assert np.array_equal(oa.linear_readout(q, np.zeros((d, d)), np.zeros(d), W, bias), np.tile(bias, (5, 1)))
+
+
+# ----------------------------------------------------------------------------- Alg. 2 protocol
+def make_stream(P, B=1, H=2, d=16, b=8, topk=2, **kw):
+    return oa.HybridStream(B, H, d, b, P, topk=topk, **kw)
+
+
+@pytest.mark.parametrize("P", [0, 1, 2])
+def test_recurrent_state_equals_from_scratch_sum_and_partition(P):
+    B, H, d, n = 1, 2, 16, 24
+    st = make_stream(P)
+    ks = [rnd((B, H, n, d), 100 + i) for i in range(6)]
+    vs = [rnd((B, H, n, d), 200 + i) for i in range(6)]
+    for i in range(6):
+        st.append(ks[i], vs[i])
+        n_abs = max(0, i + 1 - P)
+        assert st.absorbed_tokens == n_abs * n and len(st.past) == min(P, i + 1)
+        # the window holds exactly the newest min(P, i+1) chunks, the state everything older, once
+        for slot, (kp, _) in enumerate(st.past):
+            assert kp is not None and np.array_equal(kp, ks[i + 1 - len(st.past) + slot])
+        for h in range(H):
+            S = np.zeros((d, d)); z = np.zeros(d)
+            if n_abs:
+                kk = np.concatenate([ks[c][0, h] for c in range(n_abs)]); vv = np.concatenate([vs[c][0, h] for c in range(n_abs)])
+                S = oa.phi(kk).T @ vv; z = oa.phi(kk).sum(0)
+            assert np.abs(st.S[0, h] - S).max() < 1e-11 and np.abs(st.z[0, h] - z).max() < 1e-11
+
+
+def test_state_invariant_under_token_permutation_inside_a_chunk():
+    st1, st2 = make_stream(0), make_stream(0)
+    k = rnd((1, 2, 24, 16), 31); v = rnd((1, 2, 24, 16), 32)
+    perm = np.random.default_rng(3).permutation(24)
+    st1.append(k, v); st2.append(k[:, :, perm], v[:, :, perm])
+    assert np.abs(st1.S - st2.S).max() < 1e-12 and np.abs(st1.z - st2.z).max() < 1e-12
+
+
+def test_stream_forward_equals_brute_force_over_window_plus_state():
+    """Whole Alg. 2 + Alg. 3 + Eq. 7 on a tiny stream against token-level brute force."""
+    B, H, d, n, b, P = 1, 2, 16, 24, 8, 2
+    W = rnd((H, d, d), 41) / 4; bias = rnd((H, d), 42) / 10
+    st = make_stream(P, W=W, bias=bias, eps=1e-6)
+    ks = [rnd((B, H, n, d), 300 + i) for i in range(5)]; vs = [rnd((B, H, n, d), 400 + i) for i in range(5)]
+    for i in range(5):
+        q = rnd((B, H, n, d), 500 + i); kq = rnd((B, H, n, d), 600 + i); vq = rnd((B, H, n, d), 700 + i)
+        mask, _ = st.select(q, kq, exact=True)
+        out, o_loc, o_hist = st.forward(q, kq, vq, mask=mask, parts=True)
+        first = max(0, i - P)
+        assert mask.shape == (B, H, 3, 3 * (i - first + 1)) and (mask.sum(-1) == min(2, mask.shape[-1])).all()
+        for h in range(H):
+            lens = [n] * (i - first + 1)
+            keys = np.concatenate([ks[c][0, h] for c in range(first, i)] + [kq[0, h]])
+            vals = np.concatenate([vs[c][0, h] for c in range(first, i)] + [vq[0, h]])
+            ref_loc = brute_masked_attention(q[0, h], keys, vals, expand_mask(mask[0, h], n, lens, b))
+            assert np.abs(o_loc[0, h] - ref_loc).max() < 1e-12
+            if first > 0:
+                kk = np.concatenate([ks[c][0, h] for c in range(first)]); vv = np.concatenate([vs[c][0, h] for c in range(first)])
+                fq = oa.phi(q[0, h]); wts = fq @ oa.phi(kk).T
+                ref_h = (wts @ vv) / (wts.sum(1, keepdims=True) + 1e-6) @ W[h].T + bias[h]
+            else:
+                ref_h = np.tile(bias[h], (n, 1))
+            assert np.abs(o_hist[0, h] - ref_h).max() < 1e-12
+            assert np.abs(out[0, h] - (ref_loc + ref_h)).max() < 1e-12
+        st.append(ks[i], vs[i])
+
+
+def test_canonical_and_exact_selection_agree_except_near_ties():
+    w = gen.tiny()
+    st = oa.HybridStream(w.batch, w.heads, w.head_dim, w.block, w.past_chunks, topk=w.topk)
+    rows = diff = 0
+    for c in range(4):
+        q, k, v = (gen.bf16_bits_to_f64(t) for t in gen.qkv(w, 0, c, 0))
+        m32, a32 = st.select(q, k); m64, a64 = st.select(q, k, exact=True)
+        assert np.abs(a32 - a64).max() < 1e-6
+        for idx in np.ndindex(m32.shape[:3]):
+            rows += 1
+            if not np.array_equal(m32[idx], m64[idx]):
+                diff += 1
+                srt = np.sort(a64[idx])[::-1]; kk = int(m64[idx].sum())
+                assert srt[kk - 1] - srt[kk] < 1e-6 * np.abs(a64[idx]).max()
+        st.append(*(gen.bf16_bits_to_f64(t) for t in gen.clean_kv(w, 0, c)))
+    assert rows == 32 and diff <= 1
+
+
+# ----------------------------------------------------------------------------- planted mistakes are caught
+def test_pins_catch_planted_mistakes(monkeypatch):
+    """Each mutant of the oracle must fail at least one pin above."""
+    def fails(test, *args):
+        try:
+            test(*args)
+        except AssertionError:
+            return True
+        return False
+
+    real_phi, real_absorb, real_readout = oa.phi, oa.absorb, oa.linear_readout
+    # dropped "+1" on the positive side of phi
+    monkeypatch.setattr(oa, "phi", lambda x: np.where(np.asarray(x) > 0, np.asarray(x, float), np.exp(np.minimum(x, 0))))
+    assert fails(test_phi_matches_library_elu_plus_one)
+    monkeypatch.setattr(oa, "phi", real_phi)
+    # transposed state
+    monkeypatch.setattr(oa, "absorb", lambda S, z, k, v: (S + (real_phi(k).T @ v).T, z + real_phi(k).sum(0)))
+    assert fails(test_readout_equals_direct_kernel_average)
+    monkeypatch.setattr(oa, "absorb", real_absorb)
+    # h W instead of W h
+    def bad_readout(q, S, z, W=None, bias=None, eps=1e-6):
+        return real_readout(q, S, z, None if W is None else np.asarray(W).T, bias, eps)
+    monkeypatch.setattr(oa, "linear_readout", bad_readout)
+    assert fails(test_readout_equals_direct_kernel_average)
+    monkeypatch.setattr(oa, "linear_readout", real_readout)
+    # missing 1/sqrt(d)
+    real_sqrt = math.sqrt
+    monkeypatch.setattr(oa.math, "sqrt", lambda x: 1.0)
+    try:
+        d, b = 32, 16
+        q = rnd((40, d), 12); kc = [rnd((40, d), 40)]; vc = [rnd((40, d), 50)]
+        import torch
+        got = oa.sparse_attention(q, kc, vc, b, np.ones((3, 3), dtype=bool))
+    finally:
+        monkeypatch.setattr(oa.math, "sqrt", real_sqrt)
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(q)[None], torch.from_numpy(kc[0])[None], torch.from_numpy(vc[0])[None])[0].numpy()
+    assert np.abs(got - ref).max() > 1e-3
+    # eviction one chunk too early
+    real_append = oa.HybridStream.append
+    def early(self, k, v):
+        self.P -= 1
+        try:
+            real_append(self, k, v)
+        finally:
+            self.P += 1
+    monkeypatch.setattr(oa.HybridStream, "append", early)
+    assert fails(test_recurrent_state_equals_from_scratch_sum_and_partition, 2)
