@@ -1,0 +1,144 @@
+/*
+ * hf.h -- C ABI of libhf: hybrid attention for an autoregressive streaming video denoiser
+ * (block-sparse sliding-window attention over a rolling KV cache + linear-attention history state).
+ *
+ * One hf_ctx lives on ONE CUDA device and owns, per layer: the rolling cache of the last
+ * P = window_frames/chunk_frames - 1 clean chunks (K, V, pooled K), the linear state
+ * S [B,H,d,d] / z [B,H,d] in fp32, the merge projection, the last block selection and scratch.
+ * The caller owns q/k/v/o.  Unless a parameter says "host", every data pointer is a DEVICE pointer
+ * on the context's device, 16-byte aligned, to a contiguous tensor laid out [B, H, T, d] (d fastest)
+ * of bf16.  `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue
+ * work on `stream` and return; only create / destroy / the *_host calls / hf_get_device_status
+ * synchronise.  Every call returns an hf_status; an invalid argument never launches a kernel.
+ * Nothing here throws, aborts or traps the device.
+ *
+ * Logical key-block order seen by selection and attention: oldest cached chunk first, newest cached
+ * chunk, then the current chunk.  Every chunk is cut into blocks of `block` tokens from its own first
+ * token; a short last block is legal (its mean uses its own length).
+ */
+#ifndef HF_H_
+#define HF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hf_ctx hf_ctx;
+
+typedef enum {
+    HF_OK = 0,
+    HF_ERR_INVALID_ARG = 1,   /* null / misaligned pointer, bad layer index                   */
+    HF_ERR_SHAPE = 2,         /* configuration or size outside what the kernels support       */
+    HF_ERR_STATE = 3,         /* call order: e.g. attention with no selection available       */
+    HF_ERR_UNSUPPORTED = 4,
+    HF_ERR_NOMEM = 5,
+    HF_ERR_CUDA = 6,          /* a CUDA runtime call failed (no device, launch error, ...)    */
+    HF_ERR_DEVICE_TIMEOUT = 7 /* a bounded device-side wait ran out; see hf_get_device_status */
+} hf_status;
+
+enum { HF_PHI_ELU1 = 0 };                                /* phi(x) = elu(x) + 1                 */
+enum { HF_MERGE_IDENTITY = 0, HF_MERGE_PER_HEAD = 1 };   /* "Linear" of Eq. 4: none | W[H,d,d]  */
+enum { HF_SWA_AUTO = 0, HF_SWA_MMA = 1, HF_SWA_TCGEN05 = 2 }; /* sparse-attention kernel choice */
+
+typedef struct {
+    int batch, heads, head_dim;      /* head_dim d in {64, 128}                                         */
+    int tokens_per_frame;            /* tokens of one latent frame                                      */
+    int chunk_frames;                /* latent frames per chunk; T_c = tokens_per_frame * chunk_frames  */
+    int window_frames;               /* sliding window w in frames, counts the current chunk;
+                                        a multiple of chunk_frames, at most 8 chunks                    */
+    int block;                       /* b_q = b_kv in {16, 64, 128}                                     */
+    int topk;                        /* > 0: key blocks kept per query block                            */
+    int keep_permille;               /* used when topk == 0: k = ceil(keep_permille * T_n / 1000)       */
+    int layers;                      /* independent layer states held by the context                    */
+    int phi;                         /* HF_PHI_ELU1                                                     */
+    float eps;                       /* added to the denominator phi(q).z of Eq. 4                      */
+    int merge;                       /* HF_MERGE_IDENTITY | HF_MERGE_PER_HEAD                           */
+    int swa_kernel;                  /* HF_SWA_AUTO | HF_SWA_MMA | HF_SWA_TCGEN05                       */
+} hf_config;
+
+/* Fields of hf_query(). */
+enum {
+    HF_Q_CACHED_CHUNKS = 0,   /* clean chunks now in the rolling cache of the layer                   */
+    HF_Q_KEY_BLOCKS = 1,      /* T_n a forward would see now: (cached + 1) * blocks per chunk          */
+    HF_Q_KEPT_BLOCKS = 2,     /* k_eff = min(k, T_n) for that T_n                                      */
+    HF_Q_ABSORBED_TOKENS = 3, /* tokens folded into (S, z) so far (per batch*head)                     */
+    HF_Q_QUERY_BLOCKS = 4,    /* T_m = ceil(T_c / block)                                               */
+    HF_Q_MASK_WORDS = 5,      /* uint32 words per mask row = ceil(max T_n / 32)                        */
+    HF_Q_SWA_KERNEL = 6       /* kernel hf_sparse_swa resolves to (HF_SWA_MMA | HF_SWA_TCGEN05)        */
+};
+
+/* Create a context on CUDA device `device` (allocates all persistent buffers, zero state).
+ * Errors: HF_ERR_INVALID_ARG (null), HF_ERR_SHAPE (unsupported sizes), HF_ERR_CUDA, HF_ERR_NOMEM. */
+hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out);
+hf_status hf_destroy(hf_ctx* ctx);
+
+/* Empty the rolling cache and zero (S, z) of one layer (layer = -1: all layers). */
+hf_status hf_reset(hf_ctx* ctx, int layer, void* stream);
+
+/* Merge projection of the history branch ("Linear" in Eq. 4; the paper does not give its shape: here one
+ * d x d matrix per head, y = W h + bias).  W: bf16 [H, d, d] row-major (row = output dim), bias: bf16 [H, d]
+ * or NULL.  Copied into the context.  HF_ERR_STATE if the context was created with HF_MERGE_IDENTITY. */
+hf_status hf_set_merge_weights(hf_ctx* ctx, int layer, const void* W, const void* bias, void* stream);
+
+/* Alg. 2, cache commit of a clean chunk: k, v bf16 [B,H,T_c,d].  If the cache already holds P chunks the oldest
+ * is first folded into the state (Eq. 3: S += phi(K_ev)^T V_ev, z += sum phi(K_ev)) and its slot reused; the
+ * chunk's K, V are copied in and its per-block K means stored.  With P = 0 the chunk goes straight into the
+ * state and nothing is cached. */
+hf_status hf_kv_append(hf_ctx* ctx, int layer, const void* k, const void* v, void* stream);
+
+/* Eq. 3 on caller-supplied tokens: k_ev, v_ev bf16 [B,H,n_tokens,d], any n_tokens >= 1. */
+hf_status hf_state_absorb(hf_ctx* ctx, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream);
+
+/* Eq. 5 + top-K rule (Alg. 3: M_c[i,j] = 1 iff block j is among the K best of row i): block means of q and of
+ * the window's keys (cached chunks + k_cur), scores in a fixed float32 operation order, per (batch, head, query
+ * block) the k_eff highest scores kept, equal scores going to the lower block index.  The selection is kept in
+ * the context for hf_sparse_swa and optionally written out:
+ *   mask_out   uint32 [B,H,T_m,HF_Q_MASK_WORDS], bit (j & 31) of word (j >> 5) = block j kept;  or NULL
+ *   idx_out    int32  [B,H,T_m,k_eff] kept block indices ascending;                            or NULL
+ *   scores_out float  [B,H,T_m,T_n] raw scores A_ij;                                           or NULL */
+hf_status hf_block_select(hf_ctx* ctx, int layer, const void* q, const void* k_cur,
+                          uint32_t* mask_out, int32_t* idx_out, float* scores_out, void* stream);
+
+/* Eq. 6 / Alg. 3 inner loops: o_local[r] = softmax_c(q_r . k_c / sqrt(d)) V over the tokens c of the kept key
+ * blocks of r's query block.  idx: int32 [B,H,T_m,k_eff] ascending block indices, or NULL = the context's last
+ * selection for this layer (HF_ERR_STATE if none or if the cache changed since).  o_local: bf16 [B,H,T_c,d].
+ * lse: float [B,H,T_c] natural-log sum of exp of the scaled logits, or NULL. */
+hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur,
+                        const int32_t* idx, void* o_local, float* lse, void* stream);
+
+/* Eq. 4 without rotation: o_hist[r] = W (phi(q_r) S / (phi(q_r) . z + eps)) + bias, bf16 [B,H,T_c,d]. */
+hf_status hf_linear_attn(hf_ctx* ctx, int layer, const void* q, void* o_hist, void* stream);
+
+/* Alg. 3 + Eq. 7 for one denoising step: selection, sparse attention and history read-out of q against the
+ * cache + (k, v), o = o_local + o_history rounded once to bf16 [B,H,T_c,d]. */
+hf_status hf_hybrid_forward(hf_ctx* ctx, int layer, const void* q, const void* k, const void* v, void* o, void* stream);
+
+/* Same two calls for HOST buffers (pinned memory recommended): inputs are copied to staging buffers owned by the
+ * context, the device path runs, o is copied back, and the call returns after the stream has drained. */
+hf_status hf_hybrid_forward_host(hf_ctx* ctx, int layer, const void* q_host, const void* k_host, const void* v_host,
+                                 void* o_host, void* stream);
+hf_status hf_kv_append_host(hf_ctx* ctx, int layer, const void* k_host, const void* v_host, void* stream);
+
+/* Copy the state out: S float [B,H,d,d] (row = key feature, column = value dim), z float [B,H,d]; either may be NULL. */
+hf_status hf_get_state(hf_ctx* ctx, int layer, float* S, float* z, void* stream);
+
+/* Host-side bookkeeping values (HF_Q_*). */
+hf_status hf_query(hf_ctx* ctx, int layer, int what, int64_t* value);
+
+/* Synchronises the device and reports the device status word: flags != 0 means a bounded wait inside a kernel
+ * ran out (detail = where); the result of that launch is invalid, the context stays usable. */
+hf_status hf_get_device_status(hf_ctx* ctx, int* flags, int* detail);
+
+/* Number of kernels the library has launched since the context was created. */
+hf_status hf_launch_count(hf_ctx* ctx, int64_t* launches);
+
+const char* hf_status_string(hf_status s);
+const char* hf_last_error(void);   /* text of the last failure on this thread ("" if none) */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HF_H_ */

@@ -1,0 +1,558 @@
+// libhf host side: context, validation, ring bookkeeping (Alg. 2) and kernel dispatch.
+#include "../../include/hf.h"
+#include "hf_common.cuh"
+#include "k_pool_select.cuh"
+#include "k_swa_mma.cuh"
+#include "k_state_mma.cuh"
+
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+hf_status fail(hf_status s, const char* fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return s;
+}
+
+#define HF_CUDA(call)                                                                                   \
+    do {                                                                                                \
+        cudaError_t e_ = (call);                                                                        \
+        if (e_ != cudaSuccess) return fail(HF_ERR_CUDA, "%s: %s (%s:%d)", #call, cudaGetErrorString(e_), __FILE__, __LINE__); \
+    } while (0)
+
+struct LayerState {
+    bf16* ring_k = nullptr;      // [P][B*H*T_c*d]
+    bf16* ring_v = nullptr;
+    float* pooled_k = nullptr;   // [P][B*H*n_b*d]
+    float* S = nullptr;          // [B*H, d, d]
+    float* z = nullptr;          // [B*H, d]
+    bf16* sf_hi = nullptr;       // folded state S W^T, bf16 hi / lo halves
+    bf16* sf_lo = nullptr;
+    bf16* W = nullptr;           // [H, d, d]
+    bf16* bias = nullptr;        // [H, d]
+    bool has_w = false, has_bias = false;
+    uint32_t* mask = nullptr;    // last selection [B*H, T_m, mask_words]
+    int32_t* idx = nullptr;      // [B*H, T_m, keep]
+    int n_cached = 0, head = 0;  // head = slot of the oldest cached chunk
+    long long absorbed = 0;
+    unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
+    int sel_keep = 0;
+};
+
+}  // namespace
+
+struct hf_ctx {
+    hf_config cfg;
+    int device = 0, sm_count = 0;
+    int BH = 0, Tc = 0, n_b = 0, P = 0, Tm = 0, max_Tn = 0, mask_words = 0, d = 0;
+    size_t chunk_elems = 0, pooled_elems = 0;
+    std::vector<LayerState> layers;
+    float* pooled_q = nullptr;
+    float* pooled_kcur = nullptr;
+    float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
+    float* partials = nullptr;       // absorb split partials
+    unsigned int* counters = nullptr;
+    int nsplit_max = 1;
+    bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
+    int* dev_status = nullptr;
+    long long launches = 0;
+    int swa_kernel = HF_SWA_MMA;
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+hf_status check_ptr(const void* p, const char* name) {
+    if (p == nullptr) return fail(HF_ERR_INVALID_ARG, "%s is null", name);
+    if (!aligned16(p)) return fail(HF_ERR_INVALID_ARG, "%s is not 16-byte aligned", name);
+    return HF_OK;
+}
+hf_status check_layer(hf_ctx* c, int layer) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    if (layer < 0 || layer >= c->cfg.layers) return fail(HF_ERR_INVALID_ARG, "layer %d outside [0, %d)", layer, c->cfg.layers);
+    return HF_OK;
+}
+#define HF_TRY(expr) do { hf_status s_ = (expr); if (s_ != HF_OK) return s_; } while (0)
+
+int keep_for(const hf_ctx* c, int Tn) {
+    long long k = c->cfg.topk > 0 ? c->cfg.topk : ((long long)c->cfg.keep_permille * Tn + 999) / 1000;
+    if (k < 1) k = 1;
+    if (k > Tn) k = Tn;
+    return (int)k;
+}
+
+hf_status validate(const hf_config& g) {
+    if (g.batch < 1 || g.heads < 1 || g.layers < 1) return fail(HF_ERR_SHAPE, "batch, heads, layers must be >= 1");
+    if (g.head_dim != 64 && g.head_dim != 128) return fail(HF_ERR_SHAPE, "head_dim %d not in {64, 128}", g.head_dim);
+    if (g.block != 16 && g.block != 64 && g.block != 128) return fail(HF_ERR_SHAPE, "block %d not in {16, 64, 128}", g.block);
+    if (g.tokens_per_frame < 1 || g.chunk_frames < 1) return fail(HF_ERR_SHAPE, "tokens_per_frame, chunk_frames must be >= 1");
+    if (g.window_frames < g.chunk_frames || g.window_frames % g.chunk_frames != 0)
+        return fail(HF_ERR_SHAPE, "window_frames must be a positive multiple of chunk_frames");
+    if (g.window_frames / g.chunk_frames > HF_MAX_CHUNKS) return fail(HF_ERR_SHAPE, "window spans more than %d chunks", HF_MAX_CHUNKS);
+    if (g.topk < 0 || (g.topk == 0 && (g.keep_permille < 1 || g.keep_permille > 1000)))
+        return fail(HF_ERR_SHAPE, "need topk > 0 or keep_permille in [1, 1000]");
+    if (g.phi != HF_PHI_ELU1) return fail(HF_ERR_UNSUPPORTED, "phi %d unsupported", g.phi);
+    if (g.merge != HF_MERGE_IDENTITY && g.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_UNSUPPORTED, "merge %d unsupported", g.merge);
+    if (!(g.eps >= 0.f)) return fail(HF_ERR_SHAPE, "eps must be >= 0");
+    if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
+    const long long Tc = (long long)g.tokens_per_frame * g.chunk_frames;
+    const long long n_b = (Tc + g.block - 1) / g.block;
+    if (Tc > (1 << 20)) return fail(HF_ERR_SHAPE, "chunk of %lld tokens too large", Tc);
+    if (n_b * (g.window_frames / g.chunk_frames) > HF_MAX_TN)
+        return fail(HF_ERR_SHAPE, "window spans %lld key blocks, more than %d", n_b * (g.window_frames / g.chunk_frames), HF_MAX_TN);
+    if ((long long)g.batch * g.heads > 65535) return fail(HF_ERR_SHAPE, "batch*heads exceeds 65535");
+    return HF_OK;
+}
+
+template <typename T>
+hf_status dmalloc(T** p, size_t count) {
+    *p = nullptr;
+    if (count == 0) return HF_OK;
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(p), count * sizeof(T));
+    if (e == cudaErrorMemoryAllocation) { cudaGetLastError(); return fail(HF_ERR_NOMEM, "cudaMalloc of %zu bytes failed", count * sizeof(T)); }
+    if (e != cudaSuccess) return fail(HF_ERR_CUDA, "cudaMalloc: %s", cudaGetErrorString(e));
+    return HF_OK;
+}
+
+void free_all(hf_ctx* c) {
+    for (auto& L : c->layers) {
+        cudaFree(L.ring_k); cudaFree(L.ring_v); cudaFree(L.pooled_k); cudaFree(L.S); cudaFree(L.z);
+        cudaFree(L.sf_hi); cudaFree(L.sf_lo); cudaFree(L.W); cudaFree(L.bias); cudaFree(L.mask); cudaFree(L.idx);
+    }
+    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials);
+    cudaFree(c->counters); cudaFree(c->dev_status);
+    for (auto& s : c->stage) cudaFree(s);
+}
+
+template <int BLK, int D>
+hf_status set_swa_attr() {
+    HF_CUDA(cudaFuncSetAttribute(k_swa_mma<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaMma<BLK, D>::SMEM_BYTES));
+    return HF_OK;
+}
+template <int D>
+hf_status set_state_attr() {
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbMma<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_readout_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutMma<D>::SMEM_BYTES));
+    return HF_OK;
+}
+
+#define HF_DISPATCH_D(c, FN, ...) ((c)->d == 128 ? FN<128>(__VA_ARGS__) : FN<64>(__VA_ARGS__))
+
+hf_status post_launch(hf_ctx* c, const char* what, int n = 1) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(HF_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+    c->launches += n;
+    return HF_OK;
+}
+
+// ------------------------------------------------------------------------------------------- launches
+template <int D>
+hf_status launch_pool(hf_ctx* c, const PoolJobs& jobs, int njobs, cudaStream_t st) {
+    dim3 grid(c->n_b, c->BH, njobs);
+    k_pool_copy<D><<<grid, 256, 0, st>>>(jobs, c->Tc, c->cfg.block, c->n_b);
+    return post_launch(c, "k_pool_copy");
+}
+
+template <int D>
+hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st) {
+    typedef AbsorbMma<D> A;
+    const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
+    const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
+    dim3 grid(nsplit, c->BH);
+    k_absorb_mma<D><<<grid, A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, c->partials, c->counters, L.S, L.z);
+    HF_TRY(post_launch(c, "k_absorb_mma"));
+    k_fold<D><<<dim3(D / 16, c->BH), D, 0, st>>>(L.S, L.has_w ? L.W : nullptr, c->cfg.heads, L.sf_hi, L.sf_lo);
+    return post_launch(c, "k_fold");
+}
+
+template <int D>
+hf_status launch_fold(hf_ctx* c, LayerState& L, cudaStream_t st) {
+    k_fold<D><<<dim3(D / 16, c->BH), D, 0, st>>>(L.S, L.has_w ? L.W : nullptr, c->cfg.heads, L.sf_hi, L.sf_lo);
+    return post_launch(c, "k_fold");
+}
+
+template <int D>
+hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16, float* out_f32, cudaStream_t st) {
+    typedef ReadoutMma<D> R;
+    dim3 grid((c->Tc + R::ROWS - 1) / R::ROWS, c->BH);
+    k_readout_mma<D><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(q, L.sf_hi, L.sf_lo, L.z, L.has_bias ? L.bias : nullptr,
+                                                             c->cfg.heads, c->Tc, c->cfg.eps, out_bf16, out_f32);
+    return post_launch(c, "k_readout_mma");
+}
+
+ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v_cur) {
+    ChunkTable t;
+    memset(&t, 0, sizeof(t));
+    for (int i = 0; i < L.n_cached; ++i) {
+        const int slot = (L.head + i) % c->P;
+        t.k[i] = L.ring_k + (size_t)slot * c->chunk_elems;
+        t.v[i] = L.ring_v + (size_t)slot * c->chunk_elems;
+        t.pooled[i] = L.pooled_k + (size_t)slot * c->pooled_elems;
+    }
+    t.k[L.n_cached] = k_cur;
+    t.v[L.n_cached] = v_cur;
+    t.pooled[L.n_cached] = c->pooled_kcur;
+    t.n_chunks = L.n_cached + 1;
+    return t;
+}
+
+template <int D>
+hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur,
+                        uint32_t* mask_out, int32_t* idx_out, float* scores_out, cudaStream_t st) {
+    PoolJobs jobs;
+    memset(&jobs, 0, sizeof(jobs));
+    jobs.job[0].src = q;     jobs.job[0].pooled = c->pooled_q;
+    jobs.job[1].src = k_cur; jobs.job[1].pooled = c->pooled_kcur;
+    HF_TRY(launch_pool<D>(c, jobs, 2, st));
+    const int Tn = (L.n_cached + 1) * c->n_b;
+    const int keep = keep_for(c, Tn);
+    ChunkTable tab = make_table(c, L, k_cur, nullptr);
+    k_select<D><<<dim3(c->Tm, c->BH), 128, 0, st>>>(tab, c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+                                                   L.mask, L.idx, mask_out, idx_out, scores_out);
+    HF_TRY(post_launch(c, "k_select"));
+    L.sel_epoch = L.cache_epoch;
+    L.sel_keep = keep;
+    return HF_OK;
+}
+
+template <int BLK, int D>
+hf_status launch_swa_mma_t(hf_ctx* c, const bf16* q, const ChunkTable& tab, const int32_t* idx, int keep,
+                           const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    typedef SwaMma<BLK, D> C;
+    const float scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+    k_swa_mma<BLK, D><<<dim3(c->Tm, c->BH), C::THREADS, C::SMEM_BYTES, st>>>(q, tab, idx, keep, c->Tc, c->n_b, scale_log2, hist, o, lse);
+    return post_launch(c, "k_swa_mma");
+}
+
+hf_status launch_swa(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
+                     int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    ChunkTable tab = make_table(c, L, k_cur, v_cur);
+    const int b = c->cfg.block, d = c->d;
+#define HF_SWA_CASE(B_, D_) if (b == B_ && d == D_) return launch_swa_mma_t<B_, D_>(c, q, tab, idx, keep, hist, o, lse, st)
+    HF_SWA_CASE(16, 64); HF_SWA_CASE(16, 128); HF_SWA_CASE(64, 64); HF_SWA_CASE(64, 128); HF_SWA_CASE(128, 64); HF_SWA_CASE(128, 128);
+#undef HF_SWA_CASE
+    return fail(HF_ERR_UNSUPPORTED, "no attention kernel for block %d, head_dim %d", b, d);
+}
+
+hf_status ensure_staging(hf_ctx* c) {
+    for (int i = 0; i < 4; ++i)
+        if (c->stage[i] == nullptr) HF_TRY(dmalloc(&c->stage[i], c->chunk_elems));
+    return HF_OK;
+}
+
+}  // namespace
+
+// =============================================================================================== C ABI
+extern "C" {
+
+const char* hf_status_string(hf_status s) {
+    switch (s) {
+        case HF_OK: return "HF_OK";
+        case HF_ERR_INVALID_ARG: return "HF_ERR_INVALID_ARG";
+        case HF_ERR_SHAPE: return "HF_ERR_SHAPE";
+        case HF_ERR_STATE: return "HF_ERR_STATE";
+        case HF_ERR_UNSUPPORTED: return "HF_ERR_UNSUPPORTED";
+        case HF_ERR_NOMEM: return "HF_ERR_NOMEM";
+        case HF_ERR_CUDA: return "HF_ERR_CUDA";
+        case HF_ERR_DEVICE_TIMEOUT: return "HF_ERR_DEVICE_TIMEOUT";
+    }
+    return "HF_ERR_UNKNOWN";
+}
+
+const char* hf_last_error(void) { return g_err; }
+
+hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
+    if (cfg == nullptr || out == nullptr) return fail(HF_ERR_INVALID_ARG, "cfg or out is null");
+    *out = nullptr;
+    HF_TRY(validate(*cfg));
+    int count = 0;
+    cudaError_t e = cudaGetDeviceCount(&count);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(HF_ERR_CUDA, "cudaGetDeviceCount: %s", cudaGetErrorString(e)); }
+    if (device < 0 || device >= count) return fail(HF_ERR_INVALID_ARG, "device %d outside [0, %d)", device, count);
+    HF_CUDA(cudaSetDevice(device));
+    hf_ctx* c = new (std::nothrow) hf_ctx();
+    if (c == nullptr) return fail(HF_ERR_NOMEM, "host allocation failed");
+    c->cfg = *cfg;
+    c->device = device;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) { delete c; return fail(HF_ERR_CUDA, "cudaGetDeviceProperties: %s", cudaGetErrorString(e)); }
+    if (prop.major != 10) { delete c; return fail(HF_ERR_UNSUPPORTED, "device is sm_%d%d; this library is built for sm_100a only", prop.major, prop.minor); }
+    c->sm_count = prop.multiProcessorCount;
+    c->d = cfg->head_dim;
+    c->BH = cfg->batch * cfg->heads;
+    c->Tc = cfg->tokens_per_frame * cfg->chunk_frames;
+    c->n_b = (c->Tc + cfg->block - 1) / cfg->block;
+    c->Tm = c->n_b;
+    c->P = cfg->window_frames / cfg->chunk_frames - 1;
+    c->max_Tn = (c->P + 1) * c->n_b;
+    c->mask_words = (c->max_Tn + 31) / 32;
+    c->chunk_elems = (size_t)c->BH * c->Tc * c->d;
+    c->pooled_elems = (size_t)c->BH * c->n_b * c->d;
+    c->nsplit_max = (2 * c->sm_count + c->BH - 1) / c->BH;
+    if (c->nsplit_max > 32) c->nsplit_max = 32;
+    if (c->nsplit_max < 1) c->nsplit_max = 1;
+    c->swa_kernel = HF_SWA_MMA;
+    if (cfg->swa_kernel == HF_SWA_TCGEN05) { delete c; return fail(HF_ERR_UNSUPPORTED, "tcgen05 attention kernel not available for this shape"); }
+
+    hf_status s = HF_OK;
+    c->layers.resize(cfg->layers);
+    const size_t dd = (size_t)c->BH * c->d * c->d, dz = (size_t)c->BH * c->d;
+    for (auto& L : c->layers) {
+        if (s == HF_OK) s = dmalloc(&L.ring_k, (size_t)c->P * c->chunk_elems);
+        if (s == HF_OK) s = dmalloc(&L.ring_v, (size_t)c->P * c->chunk_elems);
+        if (s == HF_OK) s = dmalloc(&L.pooled_k, (size_t)c->P * c->pooled_elems);
+        if (s == HF_OK) s = dmalloc(&L.S, dd);
+        if (s == HF_OK) s = dmalloc(&L.z, dz);
+        if (s == HF_OK) s = dmalloc(&L.sf_hi, dd);
+        if (s == HF_OK) s = dmalloc(&L.sf_lo, dd);
+        if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.W, (size_t)cfg->heads * c->d * c->d);
+        if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
+        if (s == HF_OK) s = dmalloc(&L.mask, (size_t)c->BH * c->Tm * c->mask_words);
+        if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
+        if (s != HF_OK) break;
+        cudaMemset(L.S, 0, dd * 4); cudaMemset(L.z, 0, dz * 4);
+        cudaMemset(L.sf_hi, 0, dd * 2); cudaMemset(L.sf_lo, 0, dd * 2);
+    }
+    if (s == HF_OK) s = dmalloc(&c->pooled_q, c->pooled_elems);
+    if (s == HF_OK) s = dmalloc(&c->pooled_kcur, c->pooled_elems);
+    if (s == HF_OK) s = dmalloc(&c->hist, c->chunk_elems);
+    if (s == HF_OK) s = dmalloc(&c->partials, (size_t)c->BH * c->nsplit_max * ((size_t)c->d * c->d + c->d));
+    if (s == HF_OK) s = dmalloc(&c->counters, (size_t)c->BH);
+    if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)4);
+    if (s == HF_OK) {
+        cudaMemset(c->counters, 0, (size_t)c->BH * 4);
+        cudaMemset(c->dev_status, 0, 16);
+        s = set_swa_attr<16, 64>();
+        if (s == HF_OK) s = set_swa_attr<16, 128>();
+        if (s == HF_OK) s = set_swa_attr<64, 64>();
+        if (s == HF_OK) s = set_swa_attr<64, 128>();
+        if (s == HF_OK) s = set_swa_attr<128, 64>();
+        if (s == HF_OK) s = set_swa_attr<128, 128>();
+        if (s == HF_OK) s = set_state_attr<64>();
+        if (s == HF_OK) s = set_state_attr<128>();
+    }
+    if (s == HF_OK && cudaDeviceSynchronize() != cudaSuccess) s = fail(HF_ERR_CUDA, "device synchronize failed in hf_create");
+    if (s != HF_OK) { free_all(c); delete c; return s; }
+    *out = c;
+    return HF_OK;
+}
+
+hf_status hf_destroy(hf_ctx* c) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    cudaSetDevice(c->device);
+    cudaDeviceSynchronize();
+    free_all(c);
+    delete c;
+    return HF_OK;
+}
+
+hf_status hf_reset(hf_ctx* c, int layer, void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    if (layer != -1) HF_TRY(check_layer(c, layer));
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t dd = (size_t)c->BH * c->d * c->d, dz = (size_t)c->BH * c->d;
+    for (int l = 0; l < c->cfg.layers; ++l) {
+        if (layer != -1 && l != layer) continue;
+        LayerState& L = c->layers[l];
+        HF_CUDA(cudaMemsetAsync(L.S, 0, dd * 4, st));
+        HF_CUDA(cudaMemsetAsync(L.z, 0, dz * 4, st));
+        HF_CUDA(cudaMemsetAsync(L.sf_hi, 0, dd * 2, st));
+        HF_CUDA(cudaMemsetAsync(L.sf_lo, 0, dd * 2, st));
+        L.n_cached = 0; L.head = 0; L.absorbed = 0; L.cache_epoch++; L.sel_epoch = ~0ull;
+    }
+    return HF_OK;
+}
+
+hf_status hf_set_merge_weights(hf_ctx* c, int layer, const void* W, const void* bias, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    if (c->cfg.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_STATE, "context was created with HF_MERGE_IDENTITY");
+    HF_TRY(check_ptr(W, "W"));
+    if (bias != nullptr) HF_TRY(check_ptr(bias, "bias"));
+    cudaStream_t st = (cudaStream_t)stream;
+    LayerState& L = c->layers[layer];
+    HF_CUDA(cudaMemcpyAsync(L.W, W, (size_t)c->cfg.heads * c->d * c->d * 2, cudaMemcpyDeviceToDevice, st));
+    if (bias) HF_CUDA(cudaMemcpyAsync(L.bias, bias, (size_t)c->cfg.heads * c->d * 2, cudaMemcpyDeviceToDevice, st));
+    L.has_w = true;
+    L.has_bias = bias != nullptr;
+    return HF_DISPATCH_D(c, launch_fold, c, L, st);
+}
+
+hf_status hf_state_absorb(hf_ctx* c, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(k_ev, "k_ev"));
+    HF_TRY(check_ptr(v_ev, "v_ev"));
+    if (n_tokens < 1) return fail(HF_ERR_SHAPE, "n_tokens must be >= 1");
+    LayerState& L = c->layers[layer];
+    HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, (const bf16*)k_ev, (const bf16*)v_ev, n_tokens, (cudaStream_t)stream));
+    L.absorbed += n_tokens;
+    return HF_OK;
+}
+
+hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(k, "k"));
+    HF_TRY(check_ptr(v, "v"));
+    LayerState& L = c->layers[layer];
+    cudaStream_t st = (cudaStream_t)stream;
+    if (c->P == 0) {   // window == chunk: a committed chunk leaves the window at once
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, (const bf16*)k, (const bf16*)v, c->Tc, st));
+        L.absorbed += c->Tc;
+        L.cache_epoch++;
+        return HF_OK;
+    }
+    int slot;
+    if (L.n_cached == c->P) {   // cache full: the state is updated before the evicted chunk's slot is reused
+        slot = L.head;
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)slot * c->chunk_elems,
+                             L.ring_v + (size_t)slot * c->chunk_elems, c->Tc, st));
+        L.absorbed += c->Tc;
+        L.head = (L.head + 1) % c->P;
+    } else {
+        slot = (L.head + L.n_cached) % c->P;
+        L.n_cached++;
+    }
+    PoolJobs jobs;
+    memset(&jobs, 0, sizeof(jobs));
+    jobs.job[0].src = (const bf16*)k; jobs.job[0].copy_dst = L.ring_k + (size_t)slot * c->chunk_elems;
+    jobs.job[0].pooled = L.pooled_k + (size_t)slot * c->pooled_elems;
+    jobs.job[1].src = (const bf16*)v; jobs.job[1].copy_dst = L.ring_v + (size_t)slot * c->chunk_elems;
+    HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
+    L.cache_epoch++;
+    return HF_OK;
+}
+
+hf_status hf_block_select(hf_ctx* c, int layer, const void* q, const void* k_cur, uint32_t* mask_out, int32_t* idx_out,
+                          float* scores_out, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q"));
+    HF_TRY(check_ptr(k_cur, "k_cur"));
+    return HF_DISPATCH_D(c, launch_select, c, c->layers[layer], (const bf16*)q, (const bf16*)k_cur, mask_out, idx_out,
+                         scores_out, (cudaStream_t)stream);
+}
+
+hf_status hf_sparse_swa(hf_ctx* c, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
+                        void* o_local, float* lse, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q"));
+    HF_TRY(check_ptr(k_cur, "k_cur"));
+    HF_TRY(check_ptr(v_cur, "v_cur"));
+    HF_TRY(check_ptr(o_local, "o_local"));
+    LayerState& L = c->layers[layer];
+    const int keep = keep_for(c, (L.n_cached + 1) * c->n_b);
+    if (idx == nullptr) {
+        if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
+        idx = L.idx;
+    }
+    return launch_swa(c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, nullptr, (bf16*)o_local, lse,
+                      (cudaStream_t)stream);
+}
+
+hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q"));
+    HF_TRY(check_ptr(o_hist, "o_hist"));
+    return HF_DISPATCH_D(c, launch_readout, c, c->layers[layer], (const bf16*)q, (bf16*)o_hist, (float*)nullptr, (cudaStream_t)stream);
+}
+
+hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, const void* v, void* o, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q"));
+    HF_TRY(check_ptr(k, "k"));
+    HF_TRY(check_ptr(v, "v"));
+    HF_TRY(check_ptr(o, "o"));
+    LayerState& L = c->layers[layer];
+    cudaStream_t st = (cudaStream_t)stream;
+    HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
+    HF_TRY(HF_DISPATCH_D(c, launch_readout, c, L, (const bf16*)q, (bf16*)nullptr, c->hist, st));
+    return launch_swa(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, c->hist, (bf16*)o, nullptr, st);
+}
+
+hf_status hf_hybrid_forward_host(hf_ctx* c, int layer, const void* q_host, const void* k_host, const void* v_host,
+                                 void* o_host, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    if (!q_host || !k_host || !v_host || !o_host) return fail(HF_ERR_INVALID_ARG, "host pointer is null");
+    HF_TRY(ensure_staging(c));
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = c->chunk_elems * 2;
+    HF_CUDA(cudaMemcpyAsync(c->stage[0], q_host, bytes, cudaMemcpyHostToDevice, st));
+    HF_CUDA(cudaMemcpyAsync(c->stage[1], k_host, bytes, cudaMemcpyHostToDevice, st));
+    HF_CUDA(cudaMemcpyAsync(c->stage[2], v_host, bytes, cudaMemcpyHostToDevice, st));
+    HF_TRY(hf_hybrid_forward(c, layer, c->stage[0], c->stage[1], c->stage[2], c->stage[3], stream));
+    HF_CUDA(cudaMemcpyAsync(o_host, c->stage[3], bytes, cudaMemcpyDeviceToHost, st));
+    HF_CUDA(cudaStreamSynchronize(st));
+    return HF_OK;
+}
+
+hf_status hf_kv_append_host(hf_ctx* c, int layer, const void* k_host, const void* v_host, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    if (!k_host || !v_host) return fail(HF_ERR_INVALID_ARG, "host pointer is null");
+    HF_TRY(ensure_staging(c));
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = c->chunk_elems * 2;
+    HF_CUDA(cudaMemcpyAsync(c->stage[1], k_host, bytes, cudaMemcpyHostToDevice, st));
+    HF_CUDA(cudaMemcpyAsync(c->stage[2], v_host, bytes, cudaMemcpyHostToDevice, st));
+    HF_TRY(hf_kv_append(c, layer, c->stage[1], c->stage[2], stream));
+    HF_CUDA(cudaStreamSynchronize(st));
+    return HF_OK;
+}
+
+hf_status hf_get_state(hf_ctx* c, int layer, float* S, float* z, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    LayerState& L = c->layers[layer];
+    cudaStream_t st = (cudaStream_t)stream;
+    if (S) HF_CUDA(cudaMemcpyAsync(S, L.S, (size_t)c->BH * c->d * c->d * 4, cudaMemcpyDeviceToDevice, st));
+    if (z) HF_CUDA(cudaMemcpyAsync(z, L.z, (size_t)c->BH * c->d * 4, cudaMemcpyDeviceToDevice, st));
+    return HF_OK;
+}
+
+hf_status hf_query(hf_ctx* c, int layer, int what, int64_t* value) {
+    HF_TRY(check_layer(c, layer));
+    if (value == nullptr) return fail(HF_ERR_INVALID_ARG, "value is null");
+    LayerState& L = c->layers[layer];
+    const int Tn = (L.n_cached + 1) * c->n_b;
+    switch (what) {
+        case HF_Q_CACHED_CHUNKS: *value = L.n_cached; break;
+        case HF_Q_KEY_BLOCKS: *value = Tn; break;
+        case HF_Q_KEPT_BLOCKS: *value = keep_for(c, Tn); break;
+        case HF_Q_ABSORBED_TOKENS: *value = L.absorbed; break;
+        case HF_Q_QUERY_BLOCKS: *value = c->Tm; break;
+        case HF_Q_MASK_WORDS: *value = c->mask_words; break;
+        case HF_Q_SWA_KERNEL: *value = c->swa_kernel; break;
+        default: return fail(HF_ERR_INVALID_ARG, "unknown query %d", what);
+    }
+    return HF_OK;
+}
+
+hf_status hf_get_device_status(hf_ctx* c, int* flags, int* detail) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    int h[4] = {0, 0, 0, 0};
+    HF_CUDA(cudaDeviceSynchronize());
+    HF_CUDA(cudaMemcpy(h, c->dev_status, 16, cudaMemcpyDeviceToHost));
+    if (flags) *flags = h[0];
+    if (detail) *detail = h[1];
+    if (h[0] != 0) {
+        HF_CUDA(cudaMemset(c->dev_status, 0, 16));
+        return fail(HF_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (flags %d, detail %d)", h[0], h[1]);
+    }
+    return HF_OK;
+}
+
+hf_status hf_launch_count(hf_ctx* c, int64_t* launches) {
+    if (c == nullptr || launches == nullptr) return fail(HF_ERR_INVALID_ARG, "null argument");
+    *launches = c->launches;
+    return HF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,278 @@
+// Linear-attention state kernels on the warp-level tensor path (ldmatrix + mma.sync):
+//   k_absorb_mma   Eq. 3: S += phi(K_ev)^T V_ev, z += sum_t phi(K_ev[t])   (token-split partials + fixed-order reduce)
+//   k_fold         S' = S W^T split into bf16 hi/lo halves (the per-row divisor of Eq. 4 commutes with W)
+//   k_readout_mma  Eq. 4: (phi(Q) S') / (phi(Q).z + eps) + bias
+// phi(K) and phi(Q) are carried as bf16 hi + lo pairs so that the products keep ~16 mantissa bits;
+// accumulation is fp32 throughout.
+#pragma once
+#include "hf_common.cuh"
+
+template <int D>
+struct AbsorbMma {
+    static constexpr int THREADS = D * 2;          // D/16 warps, each owning 16 state rows (key features)
+    static constexpr int TT = 64;                  // tokens per shared-memory tile
+    static constexpr int ROW_BYTES = D * 2;
+    static constexpr int TILE_BYTES = TT * ROW_BYTES;
+    static constexpr int SMEM_BYTES = 4 * TILE_BYTES;   // 2 stages x (K, V)
+    static constexpr int CHUNKS_PER_ROW = D / 8;
+    static constexpr int CHUNKS_PER_THREAD = (TT * CHUNKS_PER_ROW) / THREADS;   // = 4
+    static constexpr int PART_FLOATS = D * D + D;  // one partial: S then z
+};
+
+template <int D>
+__device__ __forceinline__ void absorb_load_tile(uint32_t smem_tile, const bf16* __restrict__ src, int n_valid) {
+    typedef AbsorbMma<D> C;
+#pragma unroll
+    for (int i = 0; i < C::CHUNKS_PER_THREAD; ++i) {
+        const int id = threadIdx.x + i * C::THREADS;
+        const int row = id / C::CHUNKS_PER_ROW, ch = id % C::CHUNKS_PER_ROW;
+        const bool ok = row < n_valid;
+        cp_async16(smem_tile + swz<C::ROW_BYTES>(row, ch), src + (ok ? (size_t)row * D + ch * 8 : 0), ok);
+    }
+}
+
+// grid (nsplit, B*H).  k_ev, v_ev: [B*H, n_tokens, D].  partials: [B*H, nsplit, D*D + D] scratch.
+// counters: [B*H] zero-initialised tickets; the last CTA of a (batch, head) adds the partials to S, z in
+// ascending split order (deterministic) and re-arms the ticket.
+template <int D>
+__global__ void __launch_bounds__(AbsorbMma<D>::THREADS)
+k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n_tokens,
+             float* __restrict__ partials, unsigned int* __restrict__ counters,
+             float* __restrict__ S, float* __restrict__ z) {
+    typedef AbsorbMma<D> C;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t s0 = smem_u32(smem);
+    const int split = blockIdx.x, nsplit = gridDim.x, bh = blockIdx.y;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    // token range of this split, in whole tiles
+    const int n_tiles = (n_tokens + C::TT - 1) / C::TT;
+    const int tile_lo = (int)(((long long)n_tiles * split) / nsplit);
+    const int tile_hi = (int)(((long long)n_tiles * (split + 1)) / nsplit);
+    const bf16* kb = k_ev + (size_t)bh * n_tokens * D;
+    const bf16* vb = v_ev + (size_t)bh * n_tokens * D;
+
+    auto issue = [&](int tile, int stage) {
+        const int t0 = tile * C::TT;
+        const int nv = min(C::TT, n_tokens - t0);
+        absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES, kb + (size_t)t0 * D, nv);
+        absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES + C::TILE_BYTES, vb + (size_t)t0 * D, nv);
+    };
+
+    float acc[D / 8][4];
+#pragma unroll
+    for (int n = 0; n < D / 8; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+    float zs[2] = {0.f, 0.f};
+
+    if (tile_lo < tile_hi) issue(tile_lo, 0);
+    cp_async_commit();
+    for (int tile = tile_lo; tile < tile_hi; ++tile) {
+        const int stage = (tile - tile_lo) & 1;
+        if (tile + 1 < tile_hi) issue(tile + 1, stage ^ 1);
+        cp_async_commit();
+        cp_async_wait<1>();
+        __syncthreads();
+        const uint32_t sK = s0 + stage * 2 * C::TILE_BYTES, sV = sK + C::TILE_BYTES;
+        const int nv = min(C::TT, n_tokens - tile * C::TT);
+#pragma unroll
+        for (int ks = 0; ks < C::TT / 16; ++ks) {
+            // A = phi(K)^T: rows = key features warp*16.., columns = tokens ks*16..
+            uint32_t r[4];
+            ldsm_x4_t(sK + swz<C::ROW_BYTES>(ks * 16 + (lane & 7) + ((lane >> 4) << 3), warp * 2 + ((lane >> 3) & 1)),
+                      r[0], r[1], r[2], r[3]);
+            uint32_t ahi[4], alo[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                float2 kv = unpack_bf16(r[x]);
+                float f0 = phi_elu1(kv.x), f1 = phi_elu1(kv.y);
+                if (nv < C::TT) {   // padded token rows contribute nothing (phi(0) = 1 otherwise)
+                    const int t = ks * 16 + 2 * (lane & 3) + ((x >> 1) << 3);
+                    if (t >= nv) f0 = 0.f;
+                    if (t + 1 >= nv) f1 = 0.f;
+                }
+                zs[x & 1] += f0 + f1;
+                const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+                ahi[x] = pack_bf16(f0, f1);
+                alo[x] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+            }
+#pragma unroll
+            for (int np = 0; np < D / 16; ++np) {
+                uint32_t b0, b1, b2, b3;
+                ldsm_x4_t(sV + swz<C::ROW_BYTES>(ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), np * 2 + (lane >> 4)),
+                          b0, b1, b2, b3);
+                mma_bf16(acc[2 * np], ahi[0], ahi[1], ahi[2], ahi[3], b0, b1);
+                mma_bf16(acc[2 * np], alo[0], alo[1], alo[2], alo[3], b0, b1);
+                mma_bf16(acc[2 * np + 1], ahi[0], ahi[1], ahi[2], ahi[3], b2, b3);
+                mma_bf16(acc[2 * np + 1], alo[0], alo[1], alo[2], alo[3], b2, b3);
+            }
+        }
+        __syncthreads();
+    }
+    cp_async_wait<0>();
+
+    // ---- write this split's partial
+    float* part = partials + ((size_t)bh * nsplit + split) * C::PART_FLOATS;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        zs[r] += __shfl_xor_sync(0xffffffffu, zs[r], 1);
+        zs[r] += __shfl_xor_sync(0xffffffffu, zs[r], 2);
+        const int a = warp * 16 + (lane >> 2) + r * 8;
+        if ((lane & 3) == 0) part[D * D + a] = zs[r];
+#pragma unroll
+        for (int n = 0; n < D / 8; ++n) {
+            const int c = n * 8 + 2 * (lane & 3);
+            *reinterpret_cast<float2*>(part + (size_t)a * D + c) = make_float2(acc[n][2 * r], acc[n][2 * r + 1]);
+        }
+    }
+    // ---- last CTA of this (batch, head) reduces in fixed order
+    __shared__ unsigned int ticket;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) ticket = atomicAdd(&counters[bh], 1u);
+    __syncthreads();
+    if (ticket != (unsigned)(nsplit - 1)) return;
+    __threadfence();
+    const float* base = partials + (size_t)bh * nsplit * C::PART_FLOATS;
+    for (int e = threadIdx.x; e < C::PART_FLOATS; e += C::THREADS) {
+        float sum = __ldcg(base + e);
+        for (int s = 1; s < nsplit; ++s) sum += __ldcg(base + (size_t)s * C::PART_FLOATS + e);
+        if (e < D * D) S[(size_t)bh * D * D + e] += sum;
+        else z[(size_t)bh * D + (e - D * D)] += sum;
+    }
+    if (threadIdx.x == 0) counters[bh] = 0u;
+}
+
+// grid (D/16, B*H), D threads.  Sf = S W_h^T (or S when W == nullptr), written as bf16 hi and lo halves.
+template <int D>
+__global__ void __launch_bounds__(D)
+k_fold(const float* __restrict__ S, const bf16* __restrict__ W, int heads,
+       bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
+    __shared__ float rows[16][D];
+    const int a0 = blockIdx.x * 16, bh = blockIdx.y, h = bh % heads;
+    const int cp = threadIdx.x;
+    for (int e = threadIdx.x; e < 16 * D; e += D) rows[e / D][e % D] = S[((size_t)bh * D + a0) * D + e];
+    __syncthreads();
+    float out[16];
+    if (W == nullptr) {
+#pragma unroll
+        for (int r = 0; r < 16; ++r) out[r] = rows[r][cp];
+    } else {
+#pragma unroll
+        for (int r = 0; r < 16; ++r) out[r] = 0.f;
+        const bf16* wrow = W + ((size_t)h * D + cp) * D;     // W_h[c'][.]
+        for (int c = 0; c < D; c += 8) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(wrow + c));
+            float w[8];
+            float2 t;
+            t = unpack_bf16(u.x); w[0] = t.x; w[1] = t.y;
+            t = unpack_bf16(u.y); w[2] = t.x; w[3] = t.y;
+            t = unpack_bf16(u.z); w[4] = t.x; w[5] = t.y;
+            t = unpack_bf16(u.w); w[6] = t.x; w[7] = t.y;
+#pragma unroll
+            for (int r = 0; r < 16; ++r)
+#pragma unroll
+                for (int e = 0; e < 8; ++e) out[r] = fmaf(rows[r][c + e], w[e], out[r]);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(out[r]);
+        const size_t o = ((size_t)bh * D + a0 + r) * D + cp;
+        sf_hi[o] = hi;
+        sf_lo[o] = __float2bfloat16_rn(out[r] - __bfloat162float(hi));
+    }
+}
+
+template <int D>
+struct ReadoutMma {
+    static constexpr int ROWS = 128, THREADS = 256;
+    static constexpr int ROW_BYTES = D * 2;
+    static constexpr int Q_BYTES = ROWS * ROW_BYTES, S_BYTES = D * ROW_BYTES;
+    static constexpr int SMEM_BYTES = Q_BYTES + 2 * S_BYTES + 2 * D * 4;   // Q, Sf hi, Sf lo, z, bias
+    static constexpr int CHUNKS_PER_ROW = D / 8;
+};
+
+// grid (ceil(T_c/128), B*H).  out_bf16 or out_f32 (exactly one non-null): [B*H, T_c, D].
+template <int D>
+__global__ void __launch_bounds__(256)
+k_readout_mma(const bf16* __restrict__ q, const bf16* __restrict__ sf_hi, const bf16* __restrict__ sf_lo,
+              const float* __restrict__ z, const bf16* __restrict__ bias, int heads, int Tc, float eps,
+              bf16* __restrict__ out_bf16, float* __restrict__ out_f32) {
+    typedef ReadoutMma<D> C;
+    extern __shared__ __align__(128) uint8_t smem[];
+    const uint32_t sQ = smem_u32(smem), sHi = sQ + C::Q_BYTES, sLo = sHi + C::S_BYTES;
+    float* sz = reinterpret_cast<float*>(smem + C::Q_BYTES + 2 * C::S_BYTES);
+    float* sb = sz + D;
+    const int bh = blockIdx.y, h = bh % heads;
+    const int r0 = blockIdx.x * C::ROWS;
+    const int nq = min(C::ROWS, Tc - r0);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    for (int id = threadIdx.x; id < C::ROWS * C::CHUNKS_PER_ROW; id += C::THREADS) {
+        const int row = id / C::CHUNKS_PER_ROW, ch = id % C::CHUNKS_PER_ROW;
+        const bool ok = row < nq;
+        cp_async16(sQ + swz<C::ROW_BYTES>(row, ch), q + ((size_t)bh * Tc + r0 + (ok ? row : 0)) * D + ch * 8, ok);
+    }
+    for (int id = threadIdx.x; id < D * C::CHUNKS_PER_ROW; id += C::THREADS) {
+        const int row = id / C::CHUNKS_PER_ROW, ch = id % C::CHUNKS_PER_ROW;
+        cp_async16(sHi + swz<C::ROW_BYTES>(row, ch), sf_hi + ((size_t)bh * D + row) * D + ch * 8, true);
+        cp_async16(sLo + swz<C::ROW_BYTES>(row, ch), sf_lo + ((size_t)bh * D + row) * D + ch * 8, true);
+    }
+    cp_async_commit();
+    if (threadIdx.x < D) {
+        sz[threadIdx.x] = z[(size_t)bh * D + threadIdx.x];
+        sb[threadIdx.x] = bias ? __bfloat162float(bias[(size_t)h * D + threadIdx.x]) : 0.f;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+
+    float acc[D / 8][4];
+#pragma unroll
+    for (int n = 0; n < D / 8; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+    float den[2] = {0.f, 0.f};
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) {
+        uint32_t r[4];
+        ldsm_x4(sQ + swz<C::ROW_BYTES>(warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), r[0], r[1], r[2], r[3]);
+        uint32_t ahi[4], alo[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+            const float2 qv = unpack_bf16(r[x]);
+            const float f0 = phi_elu1(qv.x), f1 = phi_elu1(qv.y);
+            const int a = ks * 16 + 2 * (lane & 3) + ((x >> 1) << 3);      // key-feature column of f0
+            den[x & 1] = fmaf(f0, sz[a], fmaf(f1, sz[a + 1], den[x & 1]));
+            const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+            ahi[x] = pack_bf16(f0, f1);
+            alo[x] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+        }
+#pragma unroll
+        for (int np = 0; np < D / 16; ++np) {
+            const int row = ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), ch = np * 2 + (lane >> 4);
+            uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
+            ldsm_x4_t(sHi + swz<C::ROW_BYTES>(row, ch), b0, b1, b2, b3);
+            ldsm_x4_t(sLo + swz<C::ROW_BYTES>(row, ch), c0, c1, c2, c3);
+            mma_bf16(acc[2 * np], ahi[0], ahi[1], ahi[2], ahi[3], b0, b1);
+            mma_bf16(acc[2 * np], alo[0], alo[1], alo[2], alo[3], b0, b1);
+            mma_bf16(acc[2 * np], ahi[0], ahi[1], ahi[2], ahi[3], c0, c1);
+            mma_bf16(acc[2 * np + 1], ahi[0], ahi[1], ahi[2], ahi[3], b2, b3);
+            mma_bf16(acc[2 * np + 1], alo[0], alo[1], alo[2], alo[3], b2, b3);
+            mma_bf16(acc[2 * np + 1], ahi[0], ahi[1], ahi[2], ahi[3], c2, c3);
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
+        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
+        const int row = warp * 16 + (lane >> 2) + r * 8;
+        if (row >= nq) continue;
+        const float inv = 1.f / (den[r] + eps);
+        const size_t g = ((size_t)bh * Tc + r0 + row) * D;
+#pragma unroll
+        for (int n = 0; n < D / 8; ++n) {
+            const int col = n * 8 + 2 * (lane & 3);
+            const float x0 = fmaf(acc[n][2 * r], inv, sb[col]), x1 = fmaf(acc[n][2 * r + 1], inv, sb[col + 1]);
+            if (out_f32) *reinterpret_cast<float2*>(out_f32 + g + col) = make_float2(x0, x1);
+            else *reinterpret_cast<uint32_t*>(out_bf16 + g + col) = pack_bf16(x0, x1);
+        }
+    }
+}

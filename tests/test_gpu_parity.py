@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on the same seeded bf16 inputs.  Masks bit-exact; outputs max-abs <= 2e-2 and rel-L2 <= 5e-3;
+state rel-L2 <= 1e-4."""
+import numpy as np
+import pytest
+
+from paper_2604_10103_b200 import inputs as gen
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+
+f64 = gen.bf16_bits_to_f64
+
+
+def stream_compare(w: gen.Workload, chunks: int, merge=True, bias=True, check_parts=True, q_blocks_for=None, swa_kernel=0):
+    """Stream `chunks` chunks (one forward + one append each) on both sides; compare every call."""
+    gpu = hz.GpuStream(w, merge=merge, bias=bias, swa_kernel=swa_kernel)
+    ora = hz.make_oracle(w, merge=merge, bias=bias)
+    worst = {"o": 0.0, "ol": 0.0, "oh": 0.0}
+    try:
+        for c in range(chunks):
+            qb, kb, vb = gen.qkv(w, 0, c, 0)
+            q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+            qf, kf, vf = f64(qb), f64(kb), f64(vb)
+            # Eq. 5 + top-K: bit-exact mask, ascending index list, scores equal to the canonical float32 scores
+            m_gpu, idx_gpu, sc_gpu = gpu.select(q, k)
+            m_ref, sc_ref = ora.select(qf, kf)
+            assert sc_gpu.shape == sc_ref.shape
+            assert np.array_equal(sc_gpu, sc_ref), f"chunk {c}: scores differ in {np.sum(sc_gpu != sc_ref)} places"
+            assert np.array_equal(m_gpu, m_ref), f"chunk {c}: masks differ"
+            keep = int(m_ref[0, 0, 0].sum())
+            assert idx_gpu.shape[-1] == keep
+            ref_idx = np.stack([np.flatnonzero(r) for r in m_ref.reshape(-1, m_ref.shape[-1])]).reshape(idx_gpu.shape)
+            assert np.array_equal(idx_gpu, ref_idx)
+            # Alg. 3 + Eq. 7
+            qbl = None if q_blocks_for is None else q_blocks_for(c)
+            if qbl is not None and len(qbl) == 0:
+                gpu.forward(q, k, v)
+            else:
+                o_ref, ol_ref, oh_ref = ora.forward(qf, kf, vf, mask=m_ref, q_blocks=qbl, parts=True)
+                worst["o"] = max(worst["o"], hz.assert_close_out(gpu.forward(q, k, v), o_ref, f"chunk {c} hybrid O")[1])
+                if check_parts:
+                    worst["ol"] = max(worst["ol"], hz.assert_close_out(gpu.swa(q, k, v), ol_ref, f"chunk {c} O_local")[1])
+                    worst["oh"] = max(worst["oh"], hz.assert_close_out(gpu.linear(q), oh_ref, f"chunk {c} O_history")[1])
+            # Alg. 2 cache commit
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc))
+            ora.append(f64(kc), f64(vc))
+            assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_CACHED_CHUNKS) == len(ora.past)
+            assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_ABSORBED_TOKENS) == ora.absorbed_tokens
+        S, z = gpu.state()
+        if ora.absorbed_tokens:
+            assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2, f"S rel-L2 {hz.rel_l2(S, ora.S):.3e}"
+            assert hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2, f"z rel-L2 {hz.rel_l2(z, ora.z):.3e}"
+        else:
+            assert not S.any() and not z.any()
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
+    return worst
+
+
+def test_tiny_config_stream():
+    """Tiny case: 2 heads of 64, 64-token frames, window 3, 16-token blocks, top-2, 6 chunks (3 evictions seen)."""
+    stream_compare(gen.tiny(), 6)
+
+
+def test_tiny_identity_merge_and_no_bias():
+    stream_compare(gen.tiny(), 5, merge=False)
+    stream_compare(gen.tiny(), 5, merge=True, bias=False)
+
+
+@pytest.mark.parametrize("d,b,tpf,cf,wf,B", [
+    (64, 64, 100, 2, 6, 2),     # ragged 200-token chunks, 64-blocks, batch 2
+    (128, 64, 150, 1, 3, 1),    # ragged, d=128
+    (128, 128, 300, 1, 2, 1),   # several 128-tiles + 44-token tail, P = 1
+    (64, 128, 129, 1, 3, 2),    # 1-token tail block
+    (128, 16, 40, 1, 3, 1),     # 16-blocks with d=128, ragged
+    (128, 128, 200, 1, 1, 1),   # window == chunk: P = 0, chunks go straight to the state
+])
+def test_ragged_shapes(d, b, tpf, cf, wf, B):
+    w = gen.Workload("ragged", batch=B, heads=3, head_dim=d, tokens_per_frame=tpf, chunk_frames=cf, window_frames=wf,
+                     block=b, topk=0, keep_permille=400, seed=11)
+    stream_compare(w, wf // cf + 2)
+
+
+def test_keep_everything_and_keep_one():
+    w = gen.Workload("k_all", batch=1, heads=2, head_dim=64, tokens_per_frame=96, chunk_frames=1, window_frames=3,
+                     block=16, topk=0, keep_permille=1000, seed=12)
+    stream_compare(w, 4)
+    stream_compare(w.with_(topk=1, keep_permille=0), 4)
+
+
+def test_ties_go_to_the_lower_block_index():
+    """q = 0 makes every score 0: the first k blocks must be kept, and O_local is the plain mean of their V rows."""
+    import torch
+    w = gen.tiny()
+    gpu = hz.GpuStream(w)
+    try:
+        for c in range(3):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc))
+        _, kb, vb = gen.qkv(w, 0, 3, 0)
+        q = torch.zeros(gpu.shape, dtype=torch.bfloat16, device="cuda")
+        m, idx, sc = gpu.select(q, gpu.up(kb))
+        assert not sc.any() and m[..., :2].all() and not m[..., 2:].any()
+        assert (idx == np.array([0, 1])).all()
+        o = gpu.swa(q, gpu.up(kb), gpu.up(vb))
+        kc0, vc0 = gen.clean_kv(w, 0, 1)   # oldest cached chunk is chunk 1 (chunk 0 was evicted)
+        ref = f64(vc0)[:, :, :32].mean(axis=2, keepdims=True)
+        assert np.abs(o - ref).max() < 2e-3
+    finally:
+        gpu.close()
+
+
+def test_selection_and_outputs_are_deterministic():
+    w = gen.tiny().with_(seed=21)
+    outs = []
+    for _ in range(2):
+        gpu = hz.GpuStream(w)
+        try:
+            for c in range(4):
+                kc, vc = gen.clean_kv(w, 0, c)
+                gpu.append(gpu.up(kc), gpu.up(vc))
+            qb, kb, vb = gen.qkv(w, 0, 4, 0)
+            o = gpu.forward(gpu.up(qb), gpu.up(kb), gpu.up(vb))
+            S, z = gpu.state()
+            outs.append((o, S, z))
+        finally:
+            gpu.close()
+    for a, b in zip(outs[0], outs[1]):
+        assert np.array_equal(a, b)
+
+
+def test_state_absorb_arbitrary_token_counts():
+    """hf_state_absorb on caller-supplied tokens (Eq. 3), including counts that are not a tile multiple."""
+    from oracle import hybrid_attention as oa
+    w = gen.Workload("abs", batch=2, heads=2, head_dim=128, tokens_per_frame=64, chunk_frames=1, window_frames=2,
+                     block=64, topk=1, keep_permille=0, seed=13)
+    gpu = hz.GpuStream(w, merge=False)
+    try:
+        S = np.zeros((2, 2, 128, 128)); z = np.zeros((2, 2, 128))
+        for i, n in enumerate([1, 63, 64, 65, 1000]):
+            kb = gen.normal_bf16((2, 2, n, 128), 13, i, 1); vb = gen.normal_bf16((2, 2, n, 128), 13, i, 2)
+            gpu.ctx.hf_state_absorb(0, gpu.up(kb), gpu.up(vb), n)
+            for b in range(2):
+                for h in range(2):
+                    S[b, h], z[b, h] = oa.absorb(S[b, h], z[b, h], f64(kb)[b, h], f64(vb)[b, h])
+            Sg, zg = gpu.state()
+            assert hz.rel_l2(Sg, S) <= hz.STATE_REL_L2 and hz.rel_l2(zg, z) <= hz.STATE_REL_L2
+    finally:
+        gpu.close()
+
+
+def test_lse_output():
+    w = gen.tiny().with_(seed=22)
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        qb, kb, vb = gen.qkv(w, 0, 0, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        m, idx, _ = gpu.select(q, k)
+        o, lse = gpu.swa(q, k, v, want_lse=True)
+        qf, kf = f64(qb), f64(kb)
+        for h in range(2):
+            for i in range(4):
+                cols = np.concatenate([np.arange(j * 16, j * 16 + 16) for j in idx[0, h, i]])
+                s = qf[0, h, i * 16:(i + 1) * 16] @ kf[0, h, cols].T / 8.0
+                ref = np.log(np.exp(s).sum(axis=1))
+                assert np.abs(lse[0, h, i * 16:(i + 1) * 16] - ref).max() < 1e-3
+    finally:
+        gpu.close()
+
+
+def test_call_order_errors_do_not_launch():
+    import torch
+    w = gen.tiny()
+    gpu = hz.GpuStream(w)
+    try:
+        qb, kb, vb = gen.qkv(w, 0, 0, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        o = torch.empty_like(q)
+        n0 = gpu.ctx.hf_launch_count()
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_STATE"):
+            gpu.ctx.hf_sparse_swa(0, q, k, v, o)            # no selection yet
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_INVALID_ARG"):
+            gpu.ctx.hf_hybrid_forward(0, q, k, None, o)
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_INVALID_ARG"):
+            gpu.ctx.hf_hybrid_forward(5, q, k, v, o)
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_INVALID_ARG"):
+            gpu.ctx.hf_kv_append(0, k.view(-1)[1:], v)       # misaligned
+        assert gpu.ctx.hf_launch_count() == n0
+        gpu.select(q, k)
+        gpu.ctx.hf_sparse_swa(0, q, k, v, o)
+        gpu.append(k, v)
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_STATE"):
+            gpu.ctx.hf_sparse_swa(0, q, k, v, o)            # cache changed since the selection
+    finally:
+        gpu.close()
+
+
+def test_layer_832x480_single_forward():
+    """One layer at the 832x480 latent shape: prime with 4 clean chunks (2 evicted into the state), then check the
+    forward of chunk 5 on every head for a sample of query blocks (first, a middle one, the ragged last)."""
+    w = gen.layer_832x480()
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        for c in range(4):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        S, z = gpu.state()
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2 and hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        qb, kb, vb = gen.qkv(w, 0, 4, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        m_gpu, idx_gpu, sc_gpu = gpu.select(q, k)
+        m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+        assert m_ref.shape == (1, 12, 37, 111) and int(m_ref[0, 0, 0].sum()) == 28
+        assert np.array_equal(sc_gpu, sc_ref) and np.array_equal(m_gpu, m_ref)
+        qbl = [0, 17, 36]
+        o_ref, ol_ref, oh_ref = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, q_blocks=qbl, parts=True)
+        hz.assert_close_out(gpu.forward(q, k, v), o_ref, "hybrid O")
+        hz.assert_close_out(gpu.swa(q, k, v), ol_ref, "O_local")
+        ok = ~np.isnan(o_ref)
+        oh = gpu.linear(q)
+        assert hz.rel_l2(oh[ok], oh_ref[ok]) <= hz.REL_L2
+    finally:
+        gpu.close()
