@@ -190,3 +190,11 @@ def cuda_to_bits(t):
     import numpy as np
     import torch
     return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+def unpack_mask(words, n_blocks: int):
+    """uint32 mask words [..., W] -> bool [..., n_blocks] (bit j & 31 of word j >> 5 = block j kept)."""
+    import numpy as np
+    words = np.asarray(words).view(np.uint32)
+    bits = ((words[..., :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(bool)
+    return bits.reshape(words.shape[:-1] + (-1,))[..., :n_blocks]

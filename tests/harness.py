@@ -31,10 +31,7 @@ def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool 
                            keep_permille=w.keep_permille, W=W, bias=b, eps=w.eps)
 
 
-def unpack_mask(words: np.ndarray, n_blocks: int) -> np.ndarray:
-    """uint32 [..., words] -> bool [..., n_blocks] (bit j&31 of word j>>5)."""
-    bits = ((words[..., :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(bool)
-    return bits.reshape(words.shape[:-1] + (-1,))[..., :n_blocks]
+from paper_2604_10103_b200.binding import unpack_mask  # noqa: E402,F401
 
 
 class GpuStream:
