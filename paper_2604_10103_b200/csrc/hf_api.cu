@@ -3,6 +3,7 @@
 #include "hf_common.cuh"
 #include "k_pool_select.cuh"
 #include "k_swa_mma.cuh"
+#include "k_swa_tc5.cuh"
 #include "k_state_mma.cuh"
 
 #include <cmath>
@@ -47,6 +48,7 @@ struct LayerState {
     long long absorbed = 0;
     unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
     int sel_keep = 0;
+    CUtensorMap tm_kring, tm_vring;   // 4-D maps over the whole ring [slot, B*H, T_c, d]
 };
 
 }  // namespace
@@ -67,6 +69,7 @@ struct hf_ctx {
     int* dev_status = nullptr;
     long long launches = 0;
     int swa_kernel = HF_SWA_MMA;
+    void* encode_tiled = nullptr;    // cuTensorMapEncodeTiled, resolved through the runtime (no link against libcuda)
 };
 
 namespace {
@@ -235,8 +238,49 @@ hf_status launch_swa_mma_t(hf_ctx* c, const bf16* q, const ChunkTable& tab, cons
     return post_launch(c, "k_swa_mma");
 }
 
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 4-D bf16 map [slots, B*H, T_c, d], box = 64 columns x 128 rows, 128-byte swizzle, out-of-range rows read as zero.
+hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
+    const cuuint64_t dims[4] = {(cuuint64_t)c->d, (cuuint64_t)c->Tc, (cuuint64_t)c->BH, (cuuint64_t)slots};
+    const cuuint64_t strides[3] = {(cuuint64_t)c->d * 2, (cuuint64_t)c->Tc * c->d * 2, (cuuint64_t)c->BH * c->Tc * c->d * 2};
+    const cuuint32_t box[4] = {64, 128, 1, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                                                                  strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(HF_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    return HF_OK;
+}
+
+template <int D>
+hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
+                           int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    typedef SwaTc5<D> C;
+    CUtensorMap tq, tk, tv;
+    HF_TRY(make_map(c, &tq, q, 1));
+    HF_TRY(make_map(c, &tk, k_cur, 1));
+    HF_TRY(make_map(c, &tv, v_cur, 1));
+    Tc5Params p;
+    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head;
+    p.P = c->P > 0 ? c->P : 1;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+    p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
+    const CUtensorMap& rk = c->P > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
+    k_swa_tc5<D><<<dim3(c->Tm, c->BH), C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    return post_launch(c, "k_swa_tc5");
+}
+
 hf_status launch_swa(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
                      int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    if (c->swa_kernel == HF_SWA_TCGEN05) {
+        if (c->d == 128) return launch_swa_tc5_t<128>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+        return launch_swa_tc5_t<64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+    }
     ChunkTable tab = make_table(c, L, k_cur, v_cur);
     const int b = c->cfg.block, d = c->d;
 #define HF_SWA_CASE(B_, D_) if (b == B_ && d == D_) return launch_swa_mma_t<B_, D_>(c, q, tab, idx, keep, hist, o, lse, st)
@@ -303,8 +347,16 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->nsplit_max = (2 * c->sm_count + c->BH - 1) / c->BH;
     if (c->nsplit_max > 32) c->nsplit_max = 32;
     if (c->nsplit_max < 1) c->nsplit_max = 1;
-    c->swa_kernel = HF_SWA_MMA;
-    if (cfg->swa_kernel == HF_SWA_TCGEN05) { delete c; return fail(HF_ERR_UNSUPPORTED, "tcgen05 attention kernel not available for this shape"); }
+    if (cfg->swa_kernel == HF_SWA_TCGEN05 && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the tcgen05 attention kernel needs block == 128"); }
+    c->swa_kernel = (cfg->swa_kernel == HF_SWA_MMA || cfg->block != 128) ? HF_SWA_MMA : HF_SWA_TCGEN05;
+    {
+        cudaDriverEntryPointQueryResult qres;
+        e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || c->encode_tiled == nullptr) {
+            delete c;
+            return fail(HF_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+        }
+    }
 
     hf_status s = HF_OK;
     c->layers.resize(cfg->layers);
@@ -321,6 +373,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
         if (s == HF_OK) s = dmalloc(&L.mask, (size_t)c->BH * c->Tm * c->mask_words);
         if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
+        if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_kring, L.ring_k, c->P);
+        if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_vring, L.ring_v, c->P);
         if (s != HF_OK) break;
         cudaMemset(L.S, 0, dd * 4); cudaMemset(L.z, 0, dz * 4);
         cudaMemset(L.sf_hi, 0, dd * 2); cudaMemset(L.sf_lo, 0, dd * 2);
@@ -340,6 +394,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = set_swa_attr<64, 128>();
         if (s == HF_OK) s = set_swa_attr<128, 64>();
         if (s == HF_OK) s = set_swa_attr<128, 128>();
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }

@@ -1,0 +1,377 @@
+// Block-sparse sliding-window attention (Eq. 6; Alg. 3 inner loops) on the Blackwell tensor path:
+// TMA loads addressed by the kept-block index list, tcgen05.mma with S / P / O in tensor memory,
+// fp32 online softmax with lazy rescaling.  Block size 128, head dim 64 or 128.
+//
+// One CTA per (query block, batch*head), two CTAs per SM so that one CTA's softmax overlaps the other's
+// MMAs.  Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.
+// Warp 5: TMEM allocation and MMA issue.
+//   S = Q K_j^T        A = Q (smem, K-major, 128B swizzle), B = K_j (smem, K-major)     -> TMEM cols [0,128)
+//   P = exp2(S*c - m)  bf16, written over the S columns                                  -> TMEM cols [0,64)
+//   O += P V_j         A = P (TMEM), B = V_j (smem, MN-major, 128B swizzle)              -> TMEM cols [128,128+D)
+// Every wait is bounded (~1 s); on expiry the CTA raises the device status word and leaves through the
+// common exit (drains its copies, frees its TMEM).
+#pragma once
+#include <cuda.h>
+#include "hf_common.cuh"
+
+namespace tc5 {
+
+constexpr long long WAIT_LIMIT_CYCLES = 2000000000LL;   // ~1 s
+
+// ----------------------------------------------------------------------------------------- mbarrier
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 32; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+            *abort_flag = 1;
+            atomicOr(dev_status, HF_DEV_TIMEOUT_FLAG);
+            atomicExch(dev_status + 1, where);
+            return false;
+        }
+    }
+}
+
+// ----------------------------------------------------------------------------------------- TMA
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];\n"
+                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(bar) : "memory");
+}
+
+// ----------------------------------------------------------------------------------------- tcgen05
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void mma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t)
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+                 "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};\n"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+                 "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};\n"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+                 : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1.
+// lbo / sbo in bytes.  K-major operand: sbo = stride between 8-row groups (1024), lbo unused.
+// MN-major operand: lbo = stride between 64-element groups along MN, sbo = stride between 8-row groups along K.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo >> 4) & 0x3FFFu) << 16) |
+           ((uint64_t)((sbo >> 4) & 0x3FFFu) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor, kind::f16: D = f32, A = B = bf16, M = 128.
+__host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+}  // namespace tc5
+
+template <int D>
+struct SwaTc5 {
+    static constexpr int BLK = 128;
+    static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
+    static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
+    static constexpr int TILE_BYTES = SUB * SUB_BYTES;
+    static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = 2 * TILE_BYTES, OFF_BAR = 3 * TILE_BYTES;
+    static constexpr int USED_BYTES = OFF_BAR + 256;
+    // 1 KB slack for manual 1024-byte alignment; at least 80 KB so that at most two CTAs share an SM (TMEM: 2 x 256 columns)
+    static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 80 * 1024 ? (USED_BYTES + 1024) : 80 * 1024;
+    static constexpr int THREADS = 192;
+    static constexpr int TMEM_COLS = 256;
+    static constexpr int COL_S = 0, COL_P = 0, COL_O = 128;
+};
+
+struct Tc5Params {
+    const int32_t* idx;      // [B*H, T_m, keep]
+    int keep, Tc, n_b, n_cached, ring_head, P;
+    float scale_log2;
+    const float* hist;       // optional fp32 [B*H, T_c, D]
+    bf16* o;
+    float* lse;
+    int* dev_status;
+};
+
+template <int D>
+__global__ void __launch_bounds__(SwaTc5<D>::THREADS)
+k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
+          const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
+          const __grid_constant__ CUtensorMap tm_vcur, const Tc5Params p) {
+    using namespace tc5;
+    typedef SwaTc5<D> C;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
+    const uint32_t sQ = s_base + C::OFF_Q, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V;
+    const uint32_t bar0 = s_base + C::OFF_BAR;
+    const uint32_t bar_q = bar0, bar_kf = bar0 + 8, bar_ke = bar0 + 16, bar_vf = bar0 + 24, bar_ve = bar0 + 32,
+                   bar_s = bar0 + 40, bar_p = bar0 + 48, bar_o = bar0 + 56, bar_drain = bar0 + 64;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 132);
+
+    const int i = blockIdx.x, bh = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q0 = i * C::BLK;
+    const int nq = min(C::BLK, p.Tc - q0);
+    const int32_t* my_idx = p.idx + ((size_t)bh * gridDim.x + i) * p.keep;
+    const int keep = p.keep;
+
+    if (threadIdx.x == 0) {
+        mbar_init(bar_q, 1); mbar_init(bar_kf, 1); mbar_init(bar_ke, 1); mbar_init(bar_vf, 1); mbar_init(bar_ve, 1);
+        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        // ================================================================= TMA producer
+        if (lane == 0) {
+            mbar_expect_tx(bar_q, C::TILE_BYTES);
+#pragma unroll
+            for (int s = 0; s < C::SUB; ++s) tma_load_4d(sQ + s * C::SUB_BYTES, &tm_q, s * 64, q0, bh, 0, bar_q);
+            int issued = 0;
+            for (int j = 0; j < keep; ++j) {
+                const int blk = my_idx[j];
+                const int c = blk / p.n_b, jb = blk - c * p.n_b;
+                const bool cur = (c == p.n_cached);
+                const int slot = cur ? 0 : (p.ring_head + c) % p.P;
+                const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
+                const CUtensorMap* mv = cur ? &tm_vcur : &tm_vring;
+                if (j > 0 && !mbar_wait(bar_ke, (j - 1) & 1, abort_flag, p.dev_status, 1)) break;
+                mbar_expect_tx(bar_kf, C::TILE_BYTES);
+#pragma unroll
+                for (int s = 0; s < C::SUB; ++s) tma_load_4d(sK + s * C::SUB_BYTES, mk, s * 64, jb * C::BLK, bh, slot, bar_kf);
+                if (j > 0 && !mbar_wait(bar_ve, (j - 1) & 1, abort_flag, p.dev_status, 2)) { issued = -(j + 1); break; }
+                mbar_expect_tx(bar_vf, C::TILE_BYTES);
+#pragma unroll
+                for (int s = 0; s < C::SUB; ++s) tma_load_4d(sV + s * C::SUB_BYTES, mv, s * 64, jb * C::BLK, bh, slot, bar_vf);
+                issued = j + 1;
+            }
+            // drain: every copy this thread issued has landed before the CTA may leave
+            mbar_wait(bar_q, 0, abort_flag, p.dev_status, 3);
+            if (issued != 0) {
+                const int nk = issued > 0 ? issued : -issued, nvv = issued > 0 ? issued : -issued - 1;
+                long long t0 = clock64();
+                while (!mbar_try_wait(bar_kf, (nk - 1) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+                if (nvv > 0) while (!mbar_try_wait(bar_vf, (nvv - 1) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ================================================================= MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = idesc_bf16(128, false);
+            constexpr uint32_t IDESC_PV = idesc_bf16(D, true);
+            const uint32_t tS = tmem + C::COL_S, tP = tmem + C::COL_P, tO = tmem + C::COL_O;
+            bool ok = mbar_wait(bar_q, 0, abort_flag, p.dev_status, 4);
+            for (int j = 0; ok && j < keep; ++j) {
+                if (!(ok = mbar_wait(bar_kf, j & 1, abort_flag, p.dev_status, 5))) break;
+                fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * C::SUB_BYTES + (ks & 3) * 32;
+                    mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), IDESC_S, ks > 0);
+                }
+                mma_commit(bar_s);
+                mma_commit(bar_ke);
+                if (!(ok = mbar_wait(bar_p, j & 1, abort_flag, p.dev_status, 6))) break;
+                if (!(ok = mbar_wait(bar_vf, j & 1, abort_flag, p.dev_status, 7))) break;
+                fence_after_sync();
+#pragma unroll
+                for (int ks = 0; ks < C::BLK / 16; ++ks)
+                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(sV + ks * 2048, C::SUB_BYTES, 1024), IDESC_PV, (j > 0) || (ks > 0));
+                mma_commit(bar_o);
+                mma_commit(bar_ve);
+            }
+            // drain: all MMAs issued by this thread have completed before TMEM is freed
+            mma_commit(bar_drain);
+            long long t0 = clock64();
+            while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+        }
+    } else {
+        // ================================================================= softmax / correction / epilogue
+        const int row = warp * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t tS = lane_base + C::COL_S, tP = lane_base + C::COL_P, tO = lane_base + C::COL_O;
+        float m_used = -INFINITY, l_run = 0.f;
+        bool ok = true;
+        for (int j = 0; j < keep; ++j) {
+            const int blk = my_idx[j];
+            const int jb = blk % p.n_b;
+            const int nv = min(C::BLK, p.Tc - jb * C::BLK);
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, abort_flag, p.dev_status, 8));
+            if (!ok) break;
+            fence_after_sync();
+            // ---- pass 1: row max
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tS + c * 32, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float x = __uint_as_float(r[e]);
+                    if (nv == C::BLK || c * 32 + e < nv) mx = fmaxf(mx, x);
+                }
+            }
+            const float m_new = fmaxf(m_used, mx * p.scale_log2);
+            // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
+            if (j == 0) {
+                m_used = m_new;
+            } else {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_o, (j - 1) & 1, abort_flag, p.dev_status, 9));
+                if (!ok) break;
+                fence_after_sync();
+                const bool need = (m_new - m_used) > 8.f;
+                if (__any_sync(0xffffffffu, need)) {
+                    const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
+                    if (need) { m_used = m_new; l_run *= alpha; }
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld32(tO + c * 32, r);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                        tmem_st32(tO + c * 32, r);
+                    }
+                }
+            }
+            // ---- pass 2: P = exp2(S*c - m), row sum, bf16 pairs over the S columns
+            float rs = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tS + c * 32, r);
+                tmem_wait_ld();
+                uint32_t pk[16];
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                    float x0 = __uint_as_float(r[e]), x1 = __uint_as_float(r[e + 1]);
+                    float p0 = fast_exp2(fmaf(x0, p.scale_log2, -m_used));
+                    float p1 = fast_exp2(fmaf(x1, p.scale_log2, -m_used));
+                    if (nv < C::BLK) {
+                        if (c * 32 + e >= nv) p0 = 0.f;
+                        if (c * 32 + e + 1 >= nv) p1 = 0.f;
+                    }
+                    rs += p0 + p1;
+                    pk[e >> 1] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tP + c * 16, pk);
+            }
+            l_run += rs;
+            tmem_wait_st();
+            fence_before_sync();
+            mbar_arrive(bar_p);
+        }
+        // ---- epilogue: O / l (+ history term), one rounding to bf16
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_o, (keep - 1) & 1, abort_flag, p.dev_status, 10));
+        if (ok) {
+            fence_after_sync();
+            const float inv = 1.f / l_run;
+            const size_t g = (size_t)bh * p.Tc + q0 + row;
+            if (row < nq && p.lse) p.lse[g] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(tO + c * 32, r);
+                tmem_wait_ld();
+                if (row < nq) {
+                    bf16* dst = p.o + g * D + c * 32;
+                    const float* hsrc = p.hist ? p.hist + g * D + c * 32 : nullptr;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        float x[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(r[v * 8 + e]) * inv;
+                        if (hsrc) {
+                            const float4 h0 = *reinterpret_cast<const float4*>(hsrc + v * 8);
+                            const float4 h1 = *reinterpret_cast<const float4*>(hsrc + v * 8 + 4);
+                            x[0] += h0.x; x[1] += h0.y; x[2] += h0.z; x[3] += h0.w;
+                            x[4] += h1.x; x[5] += h1.y; x[6] += h1.z; x[7] += h1.w;
+                        }
+                        uint4 u;
+                        u.x = pack_bf16(x[0], x[1]); u.y = pack_bf16(x[2], x[3]);
+                        u.z = pack_bf16(x[4], x[5]); u.w = pack_bf16(x[6], x[7]);
+                        *reinterpret_cast<uint4*>(dst + v * 8) = u;
+                    }
+                }
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        fence_after_sync();
+        tmem_dealloc(tmem, C::TMEM_COLS);
+    }
+}
