@@ -122,6 +122,30 @@ hf_status hf_hybrid_forward_host(hf_ctx* ctx, int layer, const void* q_host, con
                                  void* o_host, void* stream);
 hf_status hf_kv_append_host(hf_ctx* ctx, int layer, const void* k_host, const void* v_host, void* stream);
 
+/* State update without any allocation.  (No counterpart in the paper: it is the arithmetic of hf_state_absorb,
+ * offered for callers that cannot allocate.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region whose memory plan is already
+ * frozen (a serving loop that pre-sized its pools and must not perturb them), a callback or plugin that is not
+ * allowed to touch the allocator or to create an hf_ctx (which allocates at creation), or a host thread that must
+ * not take the allocator's implicit device-wide synchronisation.  hf_state_absorb splits the token range over
+ * several thread blocks and needs global scratch for their partial sums; here that scratch is a fixed 16 MiB array
+ * compiled into the library image, which every device that loads the library holds until the process exits.
+ *
+ * Computes, on the current device:  S[bh] += phi(k_ev[bh])^T v_ev[bh],  z[bh] += sum_t phi(k_ev[bh][t])
+ *   k_ev, v_ev  device bf16 [batch_heads, n_tokens, head_dim], read only
+ *   S           device float [batch_heads, head_dim, head_dim], updated in place (caller initialises it)
+ *   z           device float [batch_heads, head_dim], updated in place
+ * Limits: head_dim in {64, 128}; 1 <= batch_heads <= 1024 and batch_heads * (head_dim^2 + head_dim) * 4 bytes must
+ * fit in 16 MiB - 4 KiB (253 batch*heads at head_dim 128, 1007 at head_dim 64); anything larger returns HF_ERR_SHAPE
+ * and launches nothing.  All pointers 16-byte aligned (else HF_ERR_INVALID_ARG).
+ * The first call on a device looks up the device address of the scratch array and sets a kernel attribute; make
+ * that first call outside any stream capture.  No call here uses cudaMalloc, cudaFree or an allocating library routine.
+ * All calls on a device share the one array (its bookkeeping words are cleared at the start of every call): two calls
+ * whose kernels may overlap on the GPU -- different streams, or different threads -- race; keep them stream-ordered. */
+hf_status hf_state_absorb_noalloc(const void* k_ev, const void* v_ev, int batch_heads, int n_tokens, int head_dim,
+                                  float* S, float* z, void* stream);
+
 /* Copy the state out: S float [B,H,d,d] (row = key feature, column = value dim), z float [B,H,d]; either may be NULL. */
 hf_status hf_get_state(hf_ctx* ctx, int layer, float* S, float* z, void* stream);
 

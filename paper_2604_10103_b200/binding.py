@@ -26,7 +26,7 @@ EXPORTS = [
     "hf_create", "hf_destroy", "hf_reset", "hf_set_merge_weights", "hf_kv_append", "hf_state_absorb",
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
-    "hf_status_string", "hf_last_error",
+    "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc",
 ]
 
 
@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
     L.hf_query.argtypes = [vp, ip, ip, C.POINTER(C.c_int64)]
     L.hf_get_device_status.argtypes = [vp, C.POINTER(ip), C.POINTER(ip)]
     L.hf_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+    L.hf_state_absorb_noalloc.argtypes = [vp, vp, ip, ip, ip, vp, vp, vp]
     L.hf_status_string.argtypes = [ip]
     L.hf_status_string.restype = C.c_char_p
     L.hf_last_error.argtypes = []
@@ -176,6 +177,15 @@ class Context:
         v = C.c_int64()
         _check(lib().hf_launch_count(self._h, C.byref(v)))
         return v.value
+
+
+def hf_state_absorb_noalloc(k_ev, v_ev, S, z):
+    """S += phi(k_ev)^T v_ev, z += sum phi(k_ev) without any allocation (see include/hf.h).
+    k_ev, v_ev: bf16 CUDA tensors [..., n_tokens, d] (leading dims = batch*heads); S, z: float32, updated in place."""
+    d = k_ev.shape[-1]
+    n = k_ev.shape[-2]
+    bh = k_ev.numel() // (n * d)
+    _check(lib().hf_state_absorb_noalloc(_ptr(k_ev), _ptr(v_ev), bh, n, d, _ptr(S), _ptr(z), _stream()))
 
 
 def bits_to_cuda(bits, device="cuda"):

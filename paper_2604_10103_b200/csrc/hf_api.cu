@@ -316,6 +316,11 @@ const char* hf_status_string(hf_status s) {
 
 const char* hf_last_error(void) { return g_err; }
 
+// Library-internal (not part of the ABI): lets the other translation units of libhf record their error text.
+void hf_internal_set_error(const char* text) {
+    snprintf(g_err, sizeof(g_err), "%s", text ? text : "");
+}
+
 hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     if (cfg == nullptr || out == nullptr) return fail(HF_ERR_INVALID_ARG, "cfg or out is null");
     *out = nullptr;
