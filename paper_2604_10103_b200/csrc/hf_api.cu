@@ -271,7 +271,9 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
     const CUtensorMap& rk = c->P > 0 ? L.tm_kring : tk;
     const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
-    k_swa_tc5<D><<<dim3(c->Tm, c->BH), C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    k_swa_tc5<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
     return post_launch(c, "k_swa_tc5");
 }
 

@@ -2,12 +2,13 @@
 // TMA loads addressed by the kept-block index list, tcgen05.mma with S / P / O in tensor memory,
 // fp32 online softmax with lazy rescaling.  Block size 128, head dim 64 or 128.
 //
-// One CTA per (query block, batch*head), two CTAs per SM so that one CTA's softmax overlaps the other's
-// MMAs.  Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.
-// Warp 5: TMEM allocation and MMA issue.
-//   S = Q K_j^T        A = Q (smem, K-major, 128B swizzle), B = K_j (smem, K-major)     -> TMEM cols [0,128)
-//   P = exp2(S*c - m)  bf16, written over the S columns                                  -> TMEM cols [0,64)
-//   O += P V_j         A = P (TMEM), B = V_j (smem, MN-major, 128B swizzle)              -> TMEM cols [128,128+D)
+// Persistent kernel, one CTA per SM; a CTA walks its (batch*head, query block) units and their kept key
+// blocks as one stream of tiles.  Warps 0-3: softmax, one query row per thread (TMEM lane = row), the whole
+// S row held in registers.  Warp 4: TMA producer (Q, K, V double-buffered).  Warp 5: TMEM allocation and
+// MMA issue; S is double-buffered in TMEM so that S_{t+1} = Q K^T runs while the softmax of tile t does.
+//   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols [0,128) | [128,256)
+//   P = exp2(S*c - m)  bf16, written over the first 64 columns of its S buffer
+//   O += P V_t         A = P (TMEM), B = V_t (smem, MN-major, 128B swizzle)              -> TMEM cols [256,256+D)
 // Every wait is bounded (~1 s); on expiry the CTA raises the device status word and leaves through the
 // common exit (drains its copies, frees its TMEM).
 #pragma once
@@ -134,18 +135,20 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
-    static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = 2 * TILE_BYTES, OFF_BAR = 3 * TILE_BYTES;
+    static constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = 4 * TILE_BYTES, OFF_BAR = 6 * TILE_BYTES;
     static constexpr int USED_BYTES = OFF_BAR + 256;
-    // 1 KB slack for manual 1024-byte alignment; at least 80 KB so that at most two CTAs share an SM (TMEM: 2 x 256 columns)
-    static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 80 * 1024 ? (USED_BYTES + 1024) : 80 * 1024;
+    // 1 KB slack for manual 1024-byte alignment; more than half an SM's shared memory so that one CTA owns the SM
+    // (it allocates all 512 TMEM columns)
+    static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
     static constexpr int THREADS = 192;
-    static constexpr int TMEM_COLS = 256;
-    static constexpr int COL_S = 0, COL_P = 0, COL_O = 128;
+    static constexpr int TMEM_COLS = 512;
+    static constexpr int COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 };
 
 struct Tc5Params {
     const int32_t* idx;      // [B*H, T_m, keep]
     int keep, Tc, n_b, n_cached, ring_head, P;
+    int Tm, n_units;         // units = (batch*head, query block) pairs, unit u = bh * Tm + i
     float scale_log2;
     const float* hist;       // optional fp32 [B*H, T_c, D]
     bf16* o;
@@ -153,8 +156,10 @@ struct Tc5Params {
     int* dev_status;
 };
 
+// Persistent: CTA c processes units c, c + gridDim.x, ...  All tiles of all its units form one stream t = 0, 1, ...
+// Shared memory: Q x2 (per unit parity), K x2, V x2 (per tile parity).  TMEM: S0 | S1 | O.
 template <int D>
-__global__ void __launch_bounds__(SwaTc5<D>::THREADS)
+__global__ void __launch_bounds__(SwaTc5<D>::THREADS, 1)
 k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
           const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
           const __grid_constant__ CUtensorMap tm_vcur, const Tc5Params p) {
@@ -165,21 +170,24 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t sQ = s_base + C::OFF_Q, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V;
     const uint32_t bar0 = s_base + C::OFF_BAR;
-    const uint32_t bar_q = bar0, bar_kf = bar0 + 8, bar_ke = bar0 + 16, bar_vf = bar0 + 24, bar_ve = bar0 + 32,
-                   bar_s = bar0 + 40, bar_p = bar0 + 48, bar_o = bar0 + 56, bar_drain = bar0 + 64;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 128);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 132);
+    // barrier pairs are indexed [parity]: address = base + 8 * parity
+    const uint32_t bar_qf = bar0, bar_qe = bar0 + 16, bar_kf = bar0 + 32, bar_ke = bar0 + 48, bar_vf = bar0 + 64,
+                   bar_ve = bar0 + 80, bar_sf = bar0 + 96, bar_pf = bar0 + 112, bar_pv = bar0 + 128, bar_drain = bar0 + 136;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 164);
 
-    const int i = blockIdx.x, bh = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int q0 = i * C::BLK;
-    const int nq = min(C::BLK, p.Tc - q0);
-    const int32_t* my_idx = p.idx + ((size_t)bh * gridDim.x + i) * p.keep;
     const int keep = p.keep;
+    const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int n_tiles = my_units * keep;
 
     if (threadIdx.x == 0) {
-        mbar_init(bar_q, 1); mbar_init(bar_kf, 1); mbar_init(bar_ke, 1); mbar_init(bar_vf, 1); mbar_init(bar_ve, 1);
-        mbar_init(bar_s, 1); mbar_init(bar_p, 128); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_qf + 8 * s, 1); mbar_init(bar_qe + 8 * s, 1); mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1);
+            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1); mbar_init(bar_pf + 8 * s, 128);
+        }
+        mbar_init(bar_pv, 1); mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -195,34 +203,42 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     if (warp == 4) {
         // ================================================================= TMA producer
         if (lane == 0) {
-            mbar_expect_tx(bar_q, C::TILE_BYTES);
+            int t = 0;
+            bool ok = true;
+            for (int n = 0; ok && n < my_units; ++n) {
+                const int u = blockIdx.x + n * gridDim.x;
+                const int bh = u / p.Tm, i = u - bh * p.Tm;
+                const int32_t* my_idx = p.idx + (size_t)u * keep;
+                const int qs = n & 1;
+                if (n >= 2 && !(ok = mbar_wait(bar_qe + 8 * qs, ((n >> 1) & 1) ^ 1, abort_flag, p.dev_status, 1))) break;
+                mbar_expect_tx(bar_qf + 8 * qs, C::TILE_BYTES);
 #pragma unroll
-            for (int s = 0; s < C::SUB; ++s) tma_load_4d(sQ + s * C::SUB_BYTES, &tm_q, s * 64, q0, bh, 0, bar_q);
-            int issued = 0;
-            for (int j = 0; j < keep; ++j) {
-                const int blk = my_idx[j];
-                const int c = blk / p.n_b, jb = blk - c * p.n_b;
-                const bool cur = (c == p.n_cached);
-                const int slot = cur ? 0 : (p.ring_head + c) % p.P;
-                const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
-                const CUtensorMap* mv = cur ? &tm_vcur : &tm_vring;
-                if (j > 0 && !mbar_wait(bar_ke, (j - 1) & 1, abort_flag, p.dev_status, 1)) break;
-                mbar_expect_tx(bar_kf, C::TILE_BYTES);
+                for (int s = 0; s < C::SUB; ++s)
+                    tma_load_4d(sQ + qs * C::TILE_BYTES + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_qf + 8 * qs);
+                for (int j = 0; j < keep; ++j, ++t) {
+                    const int blk = my_idx[j];
+                    const int c = blk / p.n_b, jb = blk - c * p.n_b;
+                    const bool cur = (c == p.n_cached);
+                    const int slot = cur ? 0 : (p.ring_head + c) % p.P;
+                    const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
+                    const CUtensorMap* mv = cur ? &tm_vcur : &tm_vring;
+                    const int st = t & 1;
+                    const uint32_t par_e = ((t >> 1) & 1) ^ 1;
+                    if (t >= 2 && !(ok = mbar_wait(bar_ke + 8 * st, par_e, abort_flag, p.dev_status, 2))) break;
+                    mbar_expect_tx(bar_kf + 8 * st, C::TILE_BYTES);
 #pragma unroll
-                for (int s = 0; s < C::SUB; ++s) tma_load_4d(sK + s * C::SUB_BYTES, mk, s * 64, jb * C::BLK, bh, slot, bar_kf);
-                if (j > 0 && !mbar_wait(bar_ve, (j - 1) & 1, abort_flag, p.dev_status, 2)) { issued = -(j + 1); break; }
-                mbar_expect_tx(bar_vf, C::TILE_BYTES);
+                    for (int s = 0; s < C::SUB; ++s)
+                        tma_load_4d(sK + st * C::TILE_BYTES + s * C::SUB_BYTES, mk, s * 64, jb * C::BLK, bh, slot, bar_kf + 8 * st);
+                    if (t >= 2 && !(ok = mbar_wait(bar_ve + 8 * st, par_e, abort_flag, p.dev_status, 3))) break;
+                    mbar_expect_tx(bar_vf + 8 * st, C::TILE_BYTES);
 #pragma unroll
-                for (int s = 0; s < C::SUB; ++s) tma_load_4d(sV + s * C::SUB_BYTES, mv, s * 64, jb * C::BLK, bh, slot, bar_vf);
-                issued = j + 1;
+                    for (int s = 0; s < C::SUB; ++s)
+                        tma_load_4d(sV + st * C::TILE_BYTES + s * C::SUB_BYTES, mv, s * 64, jb * C::BLK, bh, slot, bar_vf + 8 * st);
+                }
             }
-            // drain: every copy this thread issued has landed before the CTA may leave
-            mbar_wait(bar_q, 0, abort_flag, p.dev_status, 3);
-            if (issued != 0) {
-                const int nk = issued > 0 ? issued : -issued, nvv = issued > 0 ? issued : -issued - 1;
-                long long t0 = clock64();
-                while (!mbar_try_wait(bar_kf, (nk - 1) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
-                if (nvv > 0) while (!mbar_try_wait(bar_vf, (nvv - 1) & 1) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
+            if (!ok) {   // gave up: let the copies already in flight land before the CTA leaves
+                const long long t0 = clock64();
+                while (clock64() - t0 < 400000) {}
             }
         }
     } else if (warp == 5) {
@@ -230,120 +246,145 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         if (lane == 0) {
             constexpr uint32_t IDESC_S = idesc_bf16(128, false);
             constexpr uint32_t IDESC_PV = idesc_bf16(D, true);
-            const uint32_t tS = tmem + C::COL_S, tP = tmem + C::COL_P, tO = tmem + C::COL_O;
-            bool ok = mbar_wait(bar_q, 0, abort_flag, p.dev_status, 4);
-            for (int j = 0; ok && j < keep; ++j) {
-                if (!(ok = mbar_wait(bar_kf, j & 1, abort_flag, p.dev_status, 5))) break;
+            const uint32_t tO = tmem + C::COL_O;
+            bool ok = true;
+            auto issue_s = [&](int t) -> bool {       // S_t = Q_unit(t) K_t^T into S buffer t & 1
+                const int n = t / keep, j = t - n * keep;
+                const int qs = n & 1, st = t & 1;
+                if (j == 0 && !mbar_wait(bar_qf + 8 * qs, (n >> 1) & 1, abort_flag, p.dev_status, 4)) return false;
+                if (!mbar_wait(bar_kf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 5)) return false;
                 fence_after_sync();
+                const uint32_t tS = tmem + (st ? C::COL_S1 : C::COL_S0);
+                const uint32_t q_base = sQ + qs * C::TILE_BYTES, k_base = sK + st * C::TILE_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * C::SUB_BYTES + (ks & 3) * 32;
-                    mma_ss(tS, smem_desc_sw128(sQ + off, 16, 1024), smem_desc_sw128(sK + off, 16, 1024), IDESC_S, ks > 0);
+                    mma_ss(tS, smem_desc_sw128(q_base + off, 16, 1024), smem_desc_sw128(k_base + off, 16, 1024), IDESC_S, ks > 0);
                 }
-                mma_commit(bar_s);
-                mma_commit(bar_ke);
-                if (!(ok = mbar_wait(bar_p, j & 1, abort_flag, p.dev_status, 6))) break;
-                if (!(ok = mbar_wait(bar_vf, j & 1, abort_flag, p.dev_status, 7))) break;
+                mma_commit(bar_sf + 8 * st);
+                mma_commit(bar_ke + 8 * st);
+                if (j == keep - 1) mma_commit(bar_qe + 8 * qs);
+                return true;
+            };
+            if (n_tiles > 0) ok = issue_s(0);
+            for (int t = 0; ok && t < n_tiles; ++t) {
+                if (t + 1 < n_tiles && !(ok = issue_s(t + 1))) break;
+                const int st = t & 1;
+                const uint32_t par = (t >> 1) & 1;
+                if (!(ok = mbar_wait(bar_pf + 8 * st, par, abort_flag, p.dev_status, 6))) break;
+                if (!(ok = mbar_wait(bar_vf + 8 * st, par, abort_flag, p.dev_status, 7))) break;
                 fence_after_sync();
+                const uint32_t tP = tmem + (st ? C::COL_S1 : C::COL_S0);
+                const uint32_t v_base = sV + st * C::TILE_BYTES;
+                const bool first = (t % keep) == 0;
 #pragma unroll
                 for (int ks = 0; ks < C::BLK / 16; ++ks)
-                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(sV + ks * 2048, C::SUB_BYTES, 1024), IDESC_PV, (j > 0) || (ks > 0));
-                mma_commit(bar_o);
-                mma_commit(bar_ve);
+                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(v_base + ks * 2048, C::SUB_BYTES, 1024), IDESC_PV, !first || (ks > 0));
+                mma_commit(bar_pv);
+                mma_commit(bar_ve + 8 * st);
             }
             // drain: all MMAs issued by this thread have completed before TMEM is freed
             mma_commit(bar_drain);
-            long long t0 = clock64();
+            const long long t0 = clock64();
             while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
     } else {
         // ================================================================= softmax / correction / epilogue
         const int row = warp * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        const uint32_t tS = lane_base + C::COL_S, tP = lane_base + C::COL_P, tO = lane_base + C::COL_O;
-        float m_used = -INFINITY, l_run = 0.f;
+        const uint32_t tO = lane_base + C::COL_O;
         bool ok = true;
-        for (int j = 0; j < keep; ++j) {
-            const int blk = my_idx[j];
-            const int jb = blk % p.n_b;
-            const int nv = min(C::BLK, p.Tc - jb * C::BLK);
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_s, j & 1, abort_flag, p.dev_status, 8));
-            if (!ok) break;
-            fence_after_sync();
-            // ---- pass 1: row max
-            float mx = -INFINITY;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tS + c * 32, r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float x = __uint_as_float(r[e]);
-                    if (nv == C::BLK || c * 32 + e < nv) mx = fmaxf(mx, x);
-                }
-            }
-            const float m_new = fmaxf(m_used, mx * p.scale_log2);
-            // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
-            if (j == 0) {
-                m_used = m_new;
-            } else {
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_o, (j - 1) & 1, abort_flag, p.dev_status, 9));
+        int t = 0;
+        for (int n = 0; ok && n < my_units; ++n) {
+            const int u = blockIdx.x + n * gridDim.x;
+            const int bh = u / p.Tm, i = u - bh * p.Tm;
+            const int32_t* my_idx = p.idx + (size_t)u * keep;
+            const int q0 = i * C::BLK;
+            const int nq = min(C::BLK, p.Tc - q0);
+            float m_used = -INFINITY, l_run = 0.f;
+            for (int j = 0; j < keep; ++j, ++t) {
+                const int jb = my_idx[j] % p.n_b;
+                const int nv = min(C::BLK, p.Tc - jb * C::BLK);
+                const int st = t & 1;
+                const uint32_t tS = lane_base + (st ? C::COL_S1 : C::COL_S0);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 8));
                 if (!ok) break;
                 fence_after_sync();
-                const bool need = (m_new - m_used) > 8.f;
-                if (__any_sync(0xffffffffu, need)) {
-                    const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
-                    if (need) { m_used = m_new; l_run *= alpha; }
+                // ---- the whole S row in registers
+                uint32_t r[4][32];
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld32(tO + c * 32, r);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                        tmem_st32(tO + c * 32, r);
-                    }
-                }
-            }
-            // ---- pass 2: P = exp2(S*c - m), row sum, bf16 pairs over the S columns
-            float rs = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tS + c * 32, r);
+                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r[c]);
                 tmem_wait_ld();
-                uint32_t pk[16];
+                if (nv < C::BLK) {
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                    float x0 = __uint_as_float(r[e]), x1 = __uint_as_float(r[e + 1]);
-                    float p0 = fast_exp2(fmaf(x0, p.scale_log2, -m_used));
-                    float p1 = fast_exp2(fmaf(x1, p.scale_log2, -m_used));
-                    if (nv < C::BLK) {
-                        if (c * 32 + e >= nv) p0 = 0.f;
-                        if (c * 32 + e + 1 >= nv) p1 = 0.f;
-                    }
-                    rs += p0 + p1;
-                    pk[e >> 1] = pack_bf16(p0, p1);
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; ++e)
+                            if (c * 32 + e >= nv) r[c][e] = 0xff800000u;   // -inf
                 }
-                tmem_st16(tP + c * 16, pk);
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    mx0 = fmaxf(mx0, __uint_as_float(r[0][e])); mx1 = fmaxf(mx1, __uint_as_float(r[1][e]));
+                    mx2 = fmaxf(mx2, __uint_as_float(r[2][e])); mx3 = fmaxf(mx3, __uint_as_float(r[3][e]));
+                }
+                const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
+                if (j == 0) {
+                    m_used = m_new;
+                } else {
+                    // every P.V completion is waited for exactly once and in order (parity waits must not skip a phase);
+                    // P.V of the previous tile has normally finished long before this point
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 9));
+                    if (!ok) break;
+                    const bool need = (m_new - m_used) > 8.f;
+                    if (__any_sync(0xffffffffu, need)) {
+                        fence_after_sync();
+                        const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
+                        if (need) { m_used = m_new; l_run *= alpha; }
+#pragma unroll
+                        for (int c = 0; c < D / 32; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tO + c * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                            tmem_st32(tO + c * 32, o);
+                        }
+                    }
+                }
+                // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the S columns
+                float rs0 = 0.f, rs1 = 0.f;
+                const float neg_m = -m_used;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[c][e]), p.scale_log2, neg_m));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[c][e + 1]), p.scale_log2, neg_m));
+                        rs0 += p0; rs1 += p1;
+                        pk[e >> 1] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                l_run += rs0 + rs1;
+                tmem_wait_st();
+                fence_before_sync();
+                mbar_arrive(bar_pf + 8 * st);
             }
-            l_run += rs;
-            tmem_wait_st();
-            fence_before_sync();
-            mbar_arrive(bar_p);
-        }
-        // ---- epilogue: O / l (+ history term), one rounding to bf16
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_o, (keep - 1) & 1, abort_flag, p.dev_status, 10));
-        if (ok) {
+            if (!ok) break;
+            // ---- epilogue of the unit: O / l (+ history term), one rounding to bf16
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 10));
+            if (!ok) break;
             fence_after_sync();
             const float inv = 1.f / l_run;
             const size_t g = (size_t)bh * p.Tc + q0 + row;
             if (row < nq && p.lse) p.lse[g] = (m_used + log2f(l_run)) * 0.6931471805599453f;
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(tO + c * 32, r);
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
                 if (row < nq) {
                     bf16* dst = p.o + g * D + c * 32;
@@ -352,20 +393,23 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     for (int v = 0; v < 4; ++v) {
                         float x[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(r[v * 8 + e]) * inv;
+                        for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(o[v * 8 + e]) * inv;
                         if (hsrc) {
                             const float4 h0 = *reinterpret_cast<const float4*>(hsrc + v * 8);
                             const float4 h1 = *reinterpret_cast<const float4*>(hsrc + v * 8 + 4);
                             x[0] += h0.x; x[1] += h0.y; x[2] += h0.z; x[3] += h0.w;
                             x[4] += h1.x; x[5] += h1.y; x[6] += h1.z; x[7] += h1.w;
                         }
-                        uint4 u;
-                        u.x = pack_bf16(x[0], x[1]); u.y = pack_bf16(x[2], x[3]);
-                        u.z = pack_bf16(x[4], x[5]); u.w = pack_bf16(x[6], x[7]);
-                        *reinterpret_cast<uint4*>(dst + v * 8) = u;
+                        uint4 w;
+                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
+                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
+                        *reinterpret_cast<uint4*>(dst + v * 8) = w;
                     }
                 }
             }
+            // the next unit's first P.V overwrites O: it is gated by p_full of that tile, which these threads
+            // arrive on only after this epilogue
+            fence_before_sync();
         }
     }
     fence_before_sync();
