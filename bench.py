@@ -223,6 +223,15 @@ def run_ours(args, w):
 
     stage = {}
     roof = None
+    if args.no_extras:      # profiling runs: only the step loop above
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                              "warmup": args.warmup, "ms_per_step": ms_per_step, "gpu_launches": int(launches),
+                              "config": {"workload": w.name, "layers": w.layers}, "extras": "skipped"}))
+        ctx.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
     if rank == 0:
         reps = 2 * L
         stage["select_us"] = timed(lambda r: ctx.hf_block_select(r % L, q[r % L], k[r % L]), reps)
@@ -303,6 +312,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=30)
     ap.add_argument("--denoise-steps", type=int, default=4)
+    ap.add_argument("--no-extras", action="store_true",
+                    help="run only the warm-up and the timed step loop (no stage split, end-to-end leg or CPU baseline): "
+                         "the command profilers are pointed at")
     args = ap.parse_args()
     w = gen.full_depth_832x480(layers=args.layers, steps=args.denoise_steps)
     if args.impl == "reference":

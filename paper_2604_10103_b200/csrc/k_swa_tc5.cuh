@@ -3,8 +3,11 @@
 // fp32 online softmax with lazy rescaling.  Block size 128, head dim 64 or 128.
 //
 // Persistent kernel, one CTA per SM; a CTA walks its (batch*head, query block) units and their kept key
-// blocks as one stream of tiles.  Warps 0-3: softmax, one query row per thread (TMEM lane = row), the whole
-// S row held in registers.  Warp 4: TMA producer (Q, K, V double-buffered).  Warp 5: TMEM allocation and
+// blocks as one stream of tiles.  Softmax warps: NG column groups of four warps; thread (group g, row r) owns
+// columns [g*128/NG, (g+1)*128/NG) of S row r (TMEM lane = row) and the same share of the O columns.  The groups
+// exchange their partial row maxima through shared memory once per tile, so every group uses the same running
+// maximum; the row sums stay partial until the epilogue.  Two warps per scheduler hide each other's TMEM and
+// MUFU latencies.  Then one TMA producer warp (Q, K, V double-buffered) and one warp for TMEM allocation and
 // MMA issue; S is double-buffered in TMEM so that S_{t+1} = Q K^T runs while the softmax of tile t does.
 //   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols [0,128) | [128,256)
 //   P = exp2(S*c - m)  bf16, written over the first 64 columns of its S buffer
@@ -129,18 +132,23 @@ __host__ __device__ constexpr uint32_t idesc_bf16(int n, bool b_mn_major) {
 
 }  // namespace tc5
 
-template <int D>
+template <int D, int NG>
 struct SwaTc5 {
     static constexpr int BLK = 128;
+    static constexpr int GROUPS = NG;                  // softmax column groups (four warps each)
+    static constexpr int GCOLS = BLK / NG;             // S columns per thread
+    static constexpr int OCOLS = D / NG;               // O columns per thread
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
     static constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = 4 * TILE_BYTES, OFF_BAR = 6 * TILE_BYTES;
-    static constexpr int USED_BYTES = OFF_BAR + 256;
+    static constexpr int OFF_XM = OFF_BAR + 256;       // row-max exchange [2][NG][128] floats, then row-sum exchange [NG][128]
+    static constexpr int USED_BYTES = OFF_XM + 3 * NG * BLK * 4;
     // 1 KB slack for manual 1024-byte alignment; more than half an SM's shared memory so that one CTA owns the SM
     // (it allocates all 512 TMEM columns)
     static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
-    static constexpr int THREADS = 192;
+    static constexpr int THREADS = 128 * NG + 64;
+    static constexpr int WARP_TMA = 4 * NG, WARP_MMA = 4 * NG + 1;
     static constexpr int TMEM_COLS = 512;
     static constexpr int COL_S0 = 0, COL_S1 = 128, COL_O = 256;
 };
@@ -158,13 +166,13 @@ struct Tc5Params {
 
 // Persistent: CTA c processes units c, c + gridDim.x, ...  All tiles of all its units form one stream t = 0, 1, ...
 // Shared memory: Q x2 (per unit parity), K x2, V x2 (per tile parity).  TMEM: S0 | S1 | O.
-template <int D>
-__global__ void __launch_bounds__(SwaTc5<D>::THREADS, 1)
+template <int D, int NG>
+__global__ void __launch_bounds__(SwaTc5<D, NG>::THREADS, 1)
 k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
           const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
           const __grid_constant__ CUtensorMap tm_vcur, const Tc5Params p) {
     using namespace tc5;
-    typedef SwaTc5<D> C;
+    typedef SwaTc5<D, NG> C;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
@@ -172,9 +180,12 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     const uint32_t bar0 = s_base + C::OFF_BAR;
     // barrier pairs are indexed [parity]: address = base + 8 * parity
     const uint32_t bar_qf = bar0, bar_qe = bar0 + 16, bar_kf = bar0 + 32, bar_ke = bar0 + 48, bar_vf = bar0 + 64,
-                   bar_ve = bar0 + 80, bar_sf = bar0 + 96, bar_pf = bar0 + 112, bar_pv = bar0 + 128, bar_drain = bar0 + 136;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 160);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 164);
+                   bar_ve = bar0 + 80, bar_sf = bar0 + 96, bar_pf = bar0 + 112, bar_pv = bar0 + 128, bar_drain = bar0 + 136,
+                   bar_mx = bar0 + 144, bar_ep = bar0 + 160;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 176);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 180);
+    float* x_max = reinterpret_cast<float*>(s_gen + C::OFF_XM);          // [2][NG][128]
+    float* x_sum = x_max + 2 * NG * C::BLK;                               // [NG][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int keep = p.keep;
@@ -185,13 +196,14 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_qf + 8 * s, 1); mbar_init(bar_qe + 8 * s, 1); mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1);
-            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1); mbar_init(bar_pf + 8 * s, 128);
+            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1); mbar_init(bar_pf + 8 * s, 128 * NG);
+            mbar_init(bar_mx + 8 * s, 128 * NG);
         }
-        mbar_init(bar_pv, 1); mbar_init(bar_drain, 1);
+        mbar_init(bar_pv, 1); mbar_init(bar_drain, 1); mbar_init(bar_ep, 128 * NG);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
         tmem_relinquish();
     }
@@ -200,7 +212,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == C::WARP_TMA) {
         // ================================================================= TMA producer
         if (lane == 0) {
             int t = 0;
@@ -241,7 +253,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 while (clock64() - t0 < 400000) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == C::WARP_MMA) {
         // ================================================================= MMA issuer
         if (lane == 0) {
             constexpr uint32_t IDESC_S = idesc_bf16(128, false);
@@ -290,9 +302,11 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
     } else {
         // ================================================================= softmax / correction / epilogue
-        const int row = warp * 32 + lane;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        const uint32_t tO = lane_base + C::COL_O;
+        const int grp = warp >> 2;                          // column group
+        const int row = (warp & 3) * 32 + lane;             // query row of the tile = TMEM lane
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        const uint32_t tO = lane_base + C::COL_O + grp * C::OCOLS;
+        constexpr int NC = C::GCOLS / 32;                   // 32-column register chunks of S per thread
         bool ok = true;
         int t = 0;
         for (int n = 0; ok && n < my_units; ++n) {
@@ -301,7 +315,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             const int32_t* my_idx = p.idx + (size_t)u * keep;
             const int q0 = i * C::BLK;
             const int nq = min(C::BLK, p.Tc - q0);
-            float m_used = -INFINITY, l_run = 0.f;
+            float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
             for (int j = 0; j < keep; ++j, ++t) {
                 const int jb = my_idx[j] % p.n_b;
                 const int nv = min(C::BLK, p.Tc - jb * C::BLK);
@@ -310,40 +324,52 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 8));
                 if (!ok) break;
                 fence_after_sync();
-                // ---- the whole S row in registers
-                uint32_t r[4][32];
+                // ---- this thread's share of the S row in registers
+                uint32_t r[NC][32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, r[c]);
+                for (int c = 0; c < NC; ++c) tmem_ld32(tS + grp * C::GCOLS + c * 32, r[c]);
                 tmem_wait_ld();
                 if (nv < C::BLK) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
+                    for (int c = 0; c < NC; ++c)
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
-                            if (c * 32 + e >= nv) r[c][e] = 0xff800000u;   // -inf
+                            if (grp * C::GCOLS + c * 32 + e >= nv) r[c][e] = 0xff800000u;   // -inf
                 }
-                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    mx0 = fmaxf(mx0, __uint_as_float(r[0][e])); mx1 = fmaxf(mx1, __uint_as_float(r[1][e]));
-                    mx2 = fmaxf(mx2, __uint_as_float(r[2][e])); mx3 = fmaxf(mx3, __uint_as_float(r[3][e]));
+                for (int c = 0; c < NC; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(r[c][e]));
+                float mrow = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                if (NG > 1) {
+                    // every group has read its S columns (the P columns written below overlap another group's S)
+                    // and learns the maximum of the whole row
+                    float* xm = x_max + st * NG * C::BLK;
+                    xm[grp * C::BLK + row] = mrow;
+                    mbar_arrive(bar_mx + 8 * st);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 11));
+                    if (!ok) break;
+#pragma unroll
+                    for (int g = 0; g < NG; ++g) mrow = fmaxf(mrow, xm[g * C::BLK + row]);
                 }
-                const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2);
+                const float m_new = fmaxf(m_used, mrow * p.scale_log2);
                 // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
                 if (j == 0) {
                     m_used = m_new;
                 } else {
-                    // every P.V completion is waited for exactly once and in order (parity waits must not skip a phase);
-                    // P.V of the previous tile has normally finished long before this point
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 9));
-                    if (!ok) break;
                     const bool need = (m_new - m_used) > 8.f;
                     if (__any_sync(0xffffffffu, need)) {
+                        // O is rewritten here, so P.V of the previous tile must have landed.  While these threads are in
+                        // tile t, bar_pv has completed t - 1 or t phases (P.V of tile t - 2 precedes S of tile t in the
+                        // tensor pipe; P.V of tile t needs this tile's P), so the parity test below is exact.
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 9));
+                        if (!ok) break;
                         fence_after_sync();
                         const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
                         if (need) { m_used = m_new; l_run *= alpha; }
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
+                        for (int c = 0; c < C::OCOLS / 32; ++c) {
                             uint32_t o[32];
                             tmem_ld32(tO + c * 32, o);
                             tmem_wait_ld();
@@ -353,11 +379,11 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         }
                     }
                 }
-                // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the S columns
+                // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the first half of the S buffer
                 float rs0 = 0.f, rs1 = 0.f;
                 const float neg_m = -m_used;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < NC; ++c) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
@@ -366,7 +392,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         rs0 += p0; rs1 += p1;
                         pk[e >> 1] = pack_bf16(p0, p1);
                     }
-                    tmem_st16(tS + c * 16, pk);
+                    tmem_st16(tS + grp * (C::GCOLS / 2) + c * 16, pk);
                 }
                 l_run += rs0 + rs1;
                 tmem_wait_st();
@@ -375,20 +401,30 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             }
             if (!ok) break;
             // ---- epilogue of the unit: O / l (+ history term), one rounding to bf16
+            if (NG > 1) {
+                x_sum[grp * C::BLK + row] = l_run;
+                mbar_arrive(bar_ep);
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_ep, n & 1, abort_flag, p.dev_status, 12));
+                if (!ok) break;
+                l_run = x_sum[row];
+#pragma unroll
+                for (int g = 1; g < NG; ++g) l_run += x_sum[g * C::BLK + row];
+            }
             ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 10));
             if (!ok) break;
             fence_after_sync();
             const float inv = 1.f / l_run;
-            const size_t g = (size_t)bh * p.Tc + q0 + row;
-            if (row < nq && p.lse) p.lse[g] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+            const size_t g_row = (size_t)bh * p.Tc + q0 + row;
+            if (grp == 0 && row < nq && p.lse) p.lse[g_row] = (m_used + log2f(l_run)) * 0.6931471805599453f;
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < C::OCOLS / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(tO + c * 32, o);
                 tmem_wait_ld();
                 if (row < nq) {
-                    bf16* dst = p.o + g * D + c * 32;
-                    const float* hsrc = p.hist ? p.hist + g * D + c * 32 : nullptr;
+                    const size_t off = g_row * D + grp * C::OCOLS + c * 32;
+                    bf16* dst = p.o + off;
+                    const float* hsrc = p.hist ? p.hist + off : nullptr;
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
                         float x[8];
@@ -414,7 +450,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     }
     fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         fence_after_sync();
         tmem_dealloc(tmem, C::TMEM_COLS);
     }
