@@ -72,6 +72,12 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n .reg .pred P;\n elect.sync _|P, 0xffffffff;\n selp.u32 %0, 1, 0, P;\n}\n" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
@@ -79,16 +85,43 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, bool accumulate) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-                 ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+// One tile's worth of MMAs in a single instruction stream: the descriptors of consecutive k-steps differ only in
+// the address field (low word, 16-byte units), so each step is two adds, two moves and the MMA.
+#define HF_SS_STEP(OFF, PRED)                                                                      \
+    "add.u32 a, %1, " #OFF ";\n add.u32 b, %2, " #OFF ";\n mov.b64 da, {a, %3};\n mov.b64 db, {b, %3};\n" \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, " PRED ";\n"
+// D[tmem] = A[smem] * B[smem] over the whole head dimension (A, B K-major, 128-byte swizzle, 64-column sub-tiles
+// SUB_BYTES = 16 KB apart).  a_lo / b_lo: low descriptor words of the tiles, hi: their common high word.
+template <int D>
+__device__ __forceinline__ void mma_ss_tile(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc) {
+    if constexpr (D == 128) {
+        asm volatile("{\n .reg .pred pt, pf;\n .reg .b64 da, db;\n .reg .b32 a, b;\n"
+                     "setp.eq.u32 pt, %0, %0;\n setp.ne.u32 pf, %0, %0;\n"
+                     HF_SS_STEP(0, "pf") HF_SS_STEP(2, "pt") HF_SS_STEP(4, "pt") HF_SS_STEP(6, "pt")
+                     HF_SS_STEP(1024, "pt") HF_SS_STEP(1026, "pt") HF_SS_STEP(1028, "pt") HF_SS_STEP(1030, "pt")
+                     "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    } else {
+        asm volatile("{\n .reg .pred pt, pf;\n .reg .b64 da, db;\n .reg .b32 a, b;\n"
+                     "setp.eq.u32 pt, %0, %0;\n setp.ne.u32 pf, %0, %0;\n"
+                     HF_SS_STEP(0, "pf") HF_SS_STEP(2, "pt") HF_SS_STEP(4, "pt") HF_SS_STEP(6, "pt")
+                     "}\n" ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc) : "memory");
+    }
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, bool accumulate) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
-                 ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
+#undef HF_SS_STEP
+#define HF_TS_STEP(KS, PRED)                                                                       \
+    "add.u32 a, %1, " #KS " * 8;\n add.u32 b, %2, " #KS " * 128;\n mov.b64 db, {b, %3};\n"          \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, " PRED ";\n"
+// D[tmem] (+)= A[tmem] * B[smem] over 128 keys: A = bf16 P (8 columns per 16 keys), B = V tile, MN-major,
+// 2048 bytes per 16 keys.  accumulate_first: whether the first step adds to D.
+__device__ __forceinline__ void mma_ts_tile(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
+                                            bool accumulate_first) {
+    asm volatile("{\n .reg .pred pt, p0;\n .reg .b64 db;\n .reg .b32 a, b;\n"
+                 "setp.eq.u32 pt, %0, %0;\n setp.ne.b32 p0, %5, 0;\n"
+                 HF_TS_STEP(0, "p0") HF_TS_STEP(1, "pt") HF_TS_STEP(2, "pt") HF_TS_STEP(3, "pt")
+                 HF_TS_STEP(4, "pt") HF_TS_STEP(5, "pt") HF_TS_STEP(6, "pt") HF_TS_STEP(7, "pt")
+                 "}\n" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)accumulate_first) : "memory");
 }
+#undef HF_TS_STEP
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -255,48 +288,56 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         }
     } else if (warp == C::WARP_MMA) {
         // ================================================================= MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t IDESC_S = idesc_bf16(128, false);
-            constexpr uint32_t IDESC_PV = idesc_bf16(D, true);
-            const uint32_t tO = tmem + C::COL_O;
-            bool ok = true;
-            auto issue_s = [&](int t) -> bool {       // S_t = Q_unit(t) K_t^T into S buffer t & 1
-                const int n = t / keep, j = t - n * keep;
-                const int qs = n & 1, st = t & 1;
-                if (j == 0 && !mbar_wait(bar_qf + 8 * qs, (n >> 1) & 1, abort_flag, p.dev_status, 4)) return false;
-                if (!mbar_wait(bar_kf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 5)) return false;
-                fence_after_sync();
+        // The whole warp walks the loop (uniform control flow, so that descriptors and addresses can live in uniform
+        // registers); one elected lane issues the tensor-core instructions.
+        constexpr uint32_t IDESC_S = idesc_bf16(128, false);
+        constexpr uint32_t IDESC_PV = idesc_bf16(D, true);
+        constexpr uint32_t TILE_STEP = C::TILE_BYTES >> 4;      // descriptor address field counts 16-byte units
+        const uint32_t tO = tmem + C::COL_O;
+        const uint64_t dq0 = smem_desc_sw128(sQ, 16, 1024), dk0 = smem_desc_sw128(sK, 16, 1024);
+        const uint64_t dv0 = smem_desc_sw128(sV, C::SUB_BYTES, 1024);
+        const uint32_t q_lo = (uint32_t)dq0, k_lo = (uint32_t)dk0, v_lo = (uint32_t)dv0;
+        const uint32_t qk_hi = (uint32_t)(dq0 >> 32), v_hi = (uint32_t)(dv0 >> 32);
+        bool ok = true;
+        int n_s = 0, j_s = 0;                         // unit and position in its list of the next S tile to issue
+        auto issue_s = [&](int t) -> bool {           // S_t = Q K_t^T into S buffer t & 1
+            const int qs = n_s & 1, st = t & 1;
+            if (j_s == 0 && !__all_sync(0xffffffffu, mbar_wait(bar_qf + 8 * qs, (n_s >> 1) & 1, abort_flag, p.dev_status, 4))) return false;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_kf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 5))) return false;
+            fence_after_sync();
+            if (elect_one()) {
                 const uint32_t tS = tmem + (st ? C::COL_S1 : C::COL_S0);
-                const uint32_t q_base = sQ + qs * C::TILE_BYTES, k_base = sK + st * C::TILE_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * C::SUB_BYTES + (ks & 3) * 32;
-                    mma_ss(tS, smem_desc_sw128(q_base + off, 16, 1024), smem_desc_sw128(k_base + off, 16, 1024), IDESC_S, ks > 0);
-                }
+                mma_ss_tile<D>(tS, q_lo + qs * TILE_STEP, k_lo + st * TILE_STEP, qk_hi, IDESC_S);
                 mma_commit(bar_sf + 8 * st);
                 mma_commit(bar_ke + 8 * st);
-                if (j == keep - 1) mma_commit(bar_qe + 8 * qs);
-                return true;
-            };
-            if (n_tiles > 0) ok = issue_s(0);
-            for (int t = 0; ok && t < n_tiles; ++t) {
-                if (t + 1 < n_tiles && !(ok = issue_s(t + 1))) break;
-                const int st = t & 1;
-                const uint32_t par = (t >> 1) & 1;
-                if (!(ok = mbar_wait(bar_pf + 8 * st, par, abort_flag, p.dev_status, 6))) break;
-                if (!(ok = mbar_wait(bar_vf + 8 * st, par, abort_flag, p.dev_status, 7))) break;
-                fence_after_sync();
+                if (j_s == keep - 1) mma_commit(bar_qe + 8 * qs);
+            }
+            __syncwarp();
+            if (++j_s == keep) { j_s = 0; ++n_s; }
+            return true;
+        };
+        if (n_tiles > 0) ok = issue_s(0);
+        int j_pv = 0;                                 // position of tile t in its unit's list
+        for (int t = 0; ok && t < n_tiles; ++t) {
+            if (t + 1 < n_tiles && !(ok = issue_s(t + 1))) break;
+            const int st = t & 1;
+            const uint32_t par = (t >> 1) & 1;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_pf + 8 * st, par, abort_flag, p.dev_status, 6)))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_vf + 8 * st, par, abort_flag, p.dev_status, 7)))) break;
+            fence_after_sync();
+            if (elect_one()) {
                 const uint32_t tP = tmem + (st ? C::COL_S1 : C::COL_S0);
-                const uint32_t v_base = sV + st * C::TILE_BYTES;
-                const bool first = (t % keep) == 0;
-#pragma unroll
-                for (int ks = 0; ks < C::BLK / 16; ++ks)
-                    mma_ts(tO, tP + ks * 8, smem_desc_sw128(v_base + ks * 2048, C::SUB_BYTES, 1024), IDESC_PV, !first || (ks > 0));
+                mma_ts_tile(tO, tP, v_lo + st * TILE_STEP, v_hi, IDESC_PV, j_pv > 0);
                 mma_commit(bar_pv);
                 mma_commit(bar_ve + 8 * st);
             }
-            // drain: all MMAs issued by this thread have completed before TMEM is freed
-            mma_commit(bar_drain);
+            __syncwarp();
+            if (++j_pv == keep) j_pv = 0;
+        }
+        // drain: all MMAs issued by this warp have completed before TMEM is freed
+        if (elect_one()) mma_commit(bar_drain);
+        __syncwarp();
+        {
             const long long t0 = clock64();
             while (!mbar_try_wait(bar_drain, 0) && clock64() - t0 < WAIT_LIMIT_CYCLES) {}
         }
@@ -316,8 +357,10 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             const int q0 = i * C::BLK;
             const int nq = min(C::BLK, p.Tc - q0);
             float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
+            int blk_next = __ldg(my_idx);                   // block index list read one tile ahead (off the critical path)
             for (int j = 0; j < keep; ++j, ++t) {
-                const int jb = my_idx[j] % p.n_b;
+                const int jb = blk_next % p.n_b;
+                if (j + 1 < keep) blk_next = __ldg(my_idx + j + 1);
                 const int nv = min(C::BLK, p.Tc - jb * C::BLK);
                 const int st = t & 1;
                 const uint32_t tS = lane_base + (st ? C::COL_S1 : C::COL_S0);
