@@ -3,15 +3,19 @@
 // fp32 online softmax with lazy rescaling.  Block size 128, head dim 64 or 128.
 //
 // Persistent kernel, one CTA per SM; a CTA walks its (batch*head, query block) units and their kept key
-// blocks as one stream of tiles.  Softmax warps: NG column groups of four warps; thread (group g, row r) owns
-// columns [g*128/NG, (g+1)*128/NG) of S row r (TMEM lane = row) and the same share of the O columns.  The groups
-// exchange their partial row maxima through shared memory once per tile, so every group uses the same running
-// maximum; the row sums stay partial until the epilogue.  Two warps per scheduler hide each other's TMEM and
-// MUFU latencies.  Then one TMA producer warp (Q, K, V double-buffered) and one warp for TMEM allocation and
-// MMA issue; S is double-buffered in TMEM so that S_{t+1} = Q K^T runs while the softmax of tile t does.
-//   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols [0,128) | [128,256)
+// blocks as one stream of tiles t = 0, 1, ...
+//   softmax warps   NG column groups of four warps; thread (group g, row r) owns columns [g*128/NG, (g+1)*128/NG)
+//                   of S row r (TMEM lane = row) and the same share of the O columns.  The groups exchange their
+//                   partial row maxima through shared memory once per tile, so every group uses the same running
+//                   maximum; the row sums stay partial until the epilogue.
+//   loader warp K   TMA: Q (one buffer, reloaded per unit) and K tiles (ring of three)
+//   loader warp V   TMA: V tiles (ring of two)
+//   MMA warp        TMEM allocation and tcgen05.mma issue.  S lives in three TMEM buffers and is issued two tiles
+//                   ahead of the softmax (S_{t+2} before P_t V_t), so that neither the TMA latency of K nor the
+//                   MMA issue chain sits on the softmax critical path.
+//   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols 128*(t%3)
 //   P = exp2(S*c - m)  bf16, written over the first 64 columns of its S buffer
-//   O += P V_t         A = P (TMEM), B = V_t (smem, MN-major, 128B swizzle)              -> TMEM cols [256,256+D)
+//   O += P V_t         A = P (TMEM), B = V_t (smem, MN-major, 128B swizzle)              -> TMEM cols [384, 384+D)
 // Every wait is bounded (~1 s); on expiry the CTA raises the device status word and leaves through the
 // common exit (drains its copies, frees its TMEM).
 #pragma once
@@ -38,14 +42,29 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait.  Returns false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
-    if (mbar_try_wait(bar, parity)) return true;
+// Same test, but the hardware may park the thread for up to `ns` nanoseconds while the phase is pending: for the
+// roles that wait long and often (loaders, MMA issuer) and would otherwise take issue slots from the softmax warps.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(ns) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.  The polling loop is kept
+// out of line: the common case is a barrier that has already flipped.
+template <bool PARKED>
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
     const long long t0 = clock64();
     for (;;) {
+        if (PARKED) {
 #pragma unroll 1
-        for (int i = 0; i < 32; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
+            for (int i = 0; i < 8; ++i)
+                if (mbar_try_wait_parked(bar, parity, 4000u)) return true;
+        } else {
+#pragma unroll 1
+            for (int i = 0; i < 32; ++i)
+                if (mbar_try_wait(bar, parity)) return true;
+        }
         if (*abort_flag) return false;
         if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
             *abort_flag = 1;
@@ -54,6 +73,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+template <bool PARKED = false>
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow<PARKED>(bar, parity, abort_flag, dev_status, where);
 }
 
 // ----------------------------------------------------------------------------------------- TMA
@@ -174,16 +198,18 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
-    static constexpr int OFF_Q = 0, OFF_K = 2 * TILE_BYTES, OFF_V = 4 * TILE_BYTES, OFF_BAR = 6 * TILE_BYTES;
+    static constexpr int KSTAGES = 3, VSTAGES = 2, SBUFS = 3;
+    static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = OFF_K + KSTAGES * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + VSTAGES * TILE_BYTES;
     static constexpr int OFF_XM = OFF_BAR + 256;       // row-max exchange [2][NG][128] floats, then row-sum exchange [NG][128]
     static constexpr int USED_BYTES = OFF_XM + 3 * NG * BLK * 4;
     // 1 KB slack for manual 1024-byte alignment; more than half an SM's shared memory so that one CTA owns the SM
     // (it allocates all 512 TMEM columns)
     static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
-    static constexpr int THREADS = 128 * NG + 64;
-    static constexpr int WARP_TMA = 4 * NG, WARP_MMA = 4 * NG + 1;
+    static constexpr int THREADS = 128 * NG + 96;
+    static constexpr int WARP_LOAD_K = 4 * NG, WARP_LOAD_V = 4 * NG + 1, WARP_MMA = 4 * NG + 2;
     static constexpr int TMEM_COLS = 512;
-    static constexpr int COL_S0 = 0, COL_S1 = 128, COL_O = 256;
+    static constexpr int COL_O = SBUFS * BLK;          // S buffers at columns 0, 128, 256
 };
 
 struct Tc5Params {
@@ -197,8 +223,15 @@ struct Tc5Params {
     int* dev_status;
 };
 
-// Persistent: CTA c processes units c, c + gridDim.x, ...  All tiles of all its units form one stream t = 0, 1, ...
-// Shared memory: Q x2 (per unit parity), K x2, V x2 (per tile parity).  TMEM: S0 | S1 | O.
+// Ring position of item i in a ring of N stages: stage i % N, completed-phase parity (i / N) & 1, kept incrementally.
+template <int N>
+struct RingPos {
+    int stage = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void advance() { if (++stage == N) { stage = 0; phase ^= 1u; } }
+};
+
+// Persistent: CTA c processes units c, c + gridDim.x, ...
 template <int D, int NG>
 __global__ void __launch_bounds__(SwaTc5<D, NG>::THREADS, 1)
 k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
@@ -211,12 +244,12 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t sQ = s_base + C::OFF_Q, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V;
     const uint32_t bar0 = s_base + C::OFF_BAR;
-    // barrier pairs are indexed [parity]: address = base + 8 * parity
-    const uint32_t bar_qf = bar0, bar_qe = bar0 + 16, bar_kf = bar0 + 32, bar_ke = bar0 + 48, bar_vf = bar0 + 64,
-                   bar_ve = bar0 + 80, bar_sf = bar0 + 96, bar_pf = bar0 + 112, bar_pv = bar0 + 128, bar_drain = bar0 + 136,
-                   bar_mx = bar0 + 144, bar_ep = bar0 + 160;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 176);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 180);
+    // barrier arrays are indexed by stage: address = base + 8 * stage
+    const uint32_t bar_kf = bar0, bar_ke = bar0 + 24, bar_vf = bar0 + 48, bar_ve = bar0 + 64, bar_sf = bar0 + 80,
+                   bar_pf = bar0 + 104, bar_pv = bar0 + 128, bar_mx = bar0 + 160, bar_qf = bar0 + 176, bar_qe = bar0 + 184,
+                   bar_ep = bar0 + 192, bar_drain = bar0 + 200;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 208);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 212);
     float* x_max = reinterpret_cast<float*>(s_gen + C::OFF_XM);          // [2][NG][128]
     float* x_sum = x_max + 2 * NG * C::BLK;                               // [NG][128]
 
@@ -226,13 +259,10 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     const int n_tiles = my_units * keep;
 
     if (threadIdx.x == 0) {
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(bar_qf + 8 * s, 1); mbar_init(bar_qe + 8 * s, 1); mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1);
-            mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1); mbar_init(bar_pf + 8 * s, 128 * NG);
-            mbar_init(bar_mx + 8 * s, 128 * NG);
-        }
-        mbar_init(bar_pv, 1); mbar_init(bar_drain, 1); mbar_init(bar_ep, 128 * NG);
+        for (int s = 0; s < 3; ++s) { mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1); mbar_init(bar_pf + 8 * s, 128 * NG); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_mx + 8 * s, 128 * NG); }
+        for (int s = 0; s < 4; ++s) mbar_init(bar_pv + 8 * s, 1);
+        mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_ep, 128 * NG); mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -245,40 +275,49 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == C::WARP_TMA) {
-        // ================================================================= TMA producer
+    if (warp == C::WARP_LOAD_K || warp == C::WARP_LOAD_V) {
+        // ================================================================= TMA producers
         if (lane == 0) {
-            int t = 0;
+            const bool is_k = (warp == C::WARP_LOAD_K);
             bool ok = true;
+            RingPos<C::KSTAGES> rk;
+            RingPos<C::VSTAGES> rv;
+            int t = 0;
             for (int n = 0; ok && n < my_units; ++n) {
                 const int u = blockIdx.x + n * gridDim.x;
                 const int bh = u / p.Tm, i = u - bh * p.Tm;
                 const int32_t* my_idx = p.idx + (size_t)u * keep;
-                const int qs = n & 1;
-                if (n >= 2 && !(ok = mbar_wait(bar_qe + 8 * qs, ((n >> 1) & 1) ^ 1, abort_flag, p.dev_status, 1))) break;
-                mbar_expect_tx(bar_qf + 8 * qs, C::TILE_BYTES);
+                if (is_k) {   // Q of this unit, once the last S of the previous unit has read the buffer
+                    if (n >= 1 && !(ok = mbar_wait<true>(bar_qe, (n - 1) & 1, abort_flag, p.dev_status, 1))) break;
+                    mbar_expect_tx(bar_qf, C::TILE_BYTES);
 #pragma unroll
-                for (int s = 0; s < C::SUB; ++s)
-                    tma_load_4d(sQ + qs * C::TILE_BYTES + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_qf + 8 * qs);
+                    for (int s = 0; s < C::SUB; ++s)
+                        tma_load_4d(sQ + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_qf);
+                }
                 for (int j = 0; j < keep; ++j, ++t) {
-                    const int blk = my_idx[j];
-                    const int c = blk / p.n_b, jb = blk - c * p.n_b;
+                    const int blk = __ldg(my_idx + j);
+                    int c = 0, jb = blk;
+                    while (jb >= p.n_b) { jb -= p.n_b; ++c; }          // at most HF_MAX_CHUNKS - 1 steps; no XU-pipe division
                     const bool cur = (c == p.n_cached);
-                    const int slot = cur ? 0 : (p.ring_head + c) % p.P;
-                    const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
-                    const CUtensorMap* mv = cur ? &tm_vcur : &tm_vring;
-                    const int st = t & 1;
-                    const uint32_t par_e = ((t >> 1) & 1) ^ 1;
-                    if (t >= 2 && !(ok = mbar_wait(bar_ke + 8 * st, par_e, abort_flag, p.dev_status, 2))) break;
-                    mbar_expect_tx(bar_kf + 8 * st, C::TILE_BYTES);
+                    int slot = cur ? 0 : p.ring_head + c;
+                    if (slot >= p.P) slot -= p.P;
+                    if (is_k) {
+                        const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
+                        if (t >= C::KSTAGES && !(ok = mbar_wait<true>(bar_ke + 8 * rk.stage, rk.phase ^ 1u, abort_flag, p.dev_status, 2))) break;
+                        mbar_expect_tx(bar_kf + 8 * rk.stage, C::TILE_BYTES);
 #pragma unroll
-                    for (int s = 0; s < C::SUB; ++s)
-                        tma_load_4d(sK + st * C::TILE_BYTES + s * C::SUB_BYTES, mk, s * 64, jb * C::BLK, bh, slot, bar_kf + 8 * st);
-                    if (t >= 2 && !(ok = mbar_wait(bar_ve + 8 * st, par_e, abort_flag, p.dev_status, 3))) break;
-                    mbar_expect_tx(bar_vf + 8 * st, C::TILE_BYTES);
+                        for (int s = 0; s < C::SUB; ++s)
+                            tma_load_4d(sK + rk.stage * C::TILE_BYTES + s * C::SUB_BYTES, mk, s * 64, jb * C::BLK, bh, slot, bar_kf + 8 * rk.stage);
+                        rk.advance();
+                    } else {
+                        const CUtensorMap* mv = cur ? &tm_vcur : &tm_vring;
+                        if (t >= C::VSTAGES && !(ok = mbar_wait<true>(bar_ve + 8 * rv.stage, rv.phase ^ 1u, abort_flag, p.dev_status, 3))) break;
+                        mbar_expect_tx(bar_vf + 8 * rv.stage, C::TILE_BYTES);
 #pragma unroll
-                    for (int s = 0; s < C::SUB; ++s)
-                        tma_load_4d(sV + st * C::TILE_BYTES + s * C::SUB_BYTES, mv, s * 64, jb * C::BLK, bh, slot, bar_vf + 8 * st);
+                        for (int s = 0; s < C::SUB; ++s)
+                            tma_load_4d(sV + rv.stage * C::TILE_BYTES + s * C::SUB_BYTES, mv, s * 64, jb * C::BLK, bh, slot, bar_vf + 8 * rv.stage);
+                        rv.advance();
+                    }
                 }
             }
             if (!ok) {   // gave up: let the copies already in flight land before the CTA leaves
@@ -300,38 +339,41 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const uint32_t qk_hi = (uint32_t)(dq0 >> 32), v_hi = (uint32_t)(dv0 >> 32);
         bool ok = true;
         int n_s = 0, j_s = 0;                         // unit and position in its list of the next S tile to issue
-        auto issue_s = [&](int t) -> bool {           // S_t = Q K_t^T into S buffer t & 1
-            const int qs = n_s & 1, st = t & 1;
-            if (j_s == 0 && !__all_sync(0xffffffffu, mbar_wait(bar_qf + 8 * qs, (n_s >> 1) & 1, abort_flag, p.dev_status, 4))) return false;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar_kf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 5))) return false;
+        RingPos<C::KSTAGES> rk;                       // K stage of the next S tile (S buffer ring has the same length)
+        auto issue_s = [&]() -> bool {                // S_t = Q K_t^T into S buffer t % 3
+            if (j_s == 0 && !__all_sync(0xffffffffu, mbar_wait<true>(bar_qf, n_s & 1, abort_flag, p.dev_status, 4))) return false;
+            if (!__all_sync(0xffffffffu, mbar_wait<true>(bar_kf + 8 * rk.stage, rk.phase, abort_flag, p.dev_status, 5))) return false;
             fence_after_sync();
             if (elect_one()) {
-                const uint32_t tS = tmem + (st ? C::COL_S1 : C::COL_S0);
-                mma_ss_tile<D>(tS, q_lo + qs * TILE_STEP, k_lo + st * TILE_STEP, qk_hi, IDESC_S);
-                mma_commit(bar_sf + 8 * st);
-                mma_commit(bar_ke + 8 * st);
-                if (j_s == keep - 1) mma_commit(bar_qe + 8 * qs);
+                mma_ss_tile<D>(tmem + rk.stage * C::BLK, q_lo, k_lo + rk.stage * TILE_STEP, qk_hi, IDESC_S);
+                mma_commit(bar_sf + 8 * rk.stage);
+                mma_commit(bar_ke + 8 * rk.stage);
+                if (j_s == keep - 1) mma_commit(bar_qe);
             }
             __syncwarp();
+            rk.advance();
             if (++j_s == keep) { j_s = 0; ++n_s; }
             return true;
         };
-        if (n_tiles > 0) ok = issue_s(0);
+        static_assert(C::KSTAGES == C::SBUFS, "S buffers and K stages advance together");
+        if (n_tiles > 0) ok = issue_s();
+        if (ok && n_tiles > 1) ok = issue_s();
         int j_pv = 0;                                 // position of tile t in its unit's list
+        RingPos<C::SBUFS> rp;                         // S buffer holding P_t
+        RingPos<C::VSTAGES> rv;
         for (int t = 0; ok && t < n_tiles; ++t) {
-            if (t + 1 < n_tiles && !(ok = issue_s(t + 1))) break;
-            const int st = t & 1;
-            const uint32_t par = (t >> 1) & 1;
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_pf + 8 * st, par, abort_flag, p.dev_status, 6)))) break;
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait(bar_vf + 8 * st, par, abort_flag, p.dev_status, 7)))) break;
+            if (t + 2 < n_tiles && !(ok = issue_s())) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_pf + 8 * rp.stage, rp.phase, abort_flag, p.dev_status, 6)))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_vf + 8 * rv.stage, rv.phase, abort_flag, p.dev_status, 7)))) break;
             fence_after_sync();
             if (elect_one()) {
-                const uint32_t tP = tmem + (st ? C::COL_S1 : C::COL_S0);
-                mma_ts_tile(tO, tP, v_lo + st * TILE_STEP, v_hi, IDESC_PV, j_pv > 0);
-                mma_commit(bar_pv);
-                mma_commit(bar_ve + 8 * st);
+                mma_ts_tile(tO, tmem + rp.stage * C::BLK, v_lo + rv.stage * TILE_STEP, v_hi, IDESC_PV, j_pv > 0);
+                mma_commit(bar_pv + 8 * (t & 3));
+                mma_commit(bar_ve + 8 * rv.stage);
             }
             __syncwarp();
+            rp.advance();
+            rv.advance();
             if (++j_pv == keep) j_pv = 0;
         }
         // drain: all MMAs issued by this warp have completed before TMEM is freed
@@ -350,6 +392,15 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         constexpr int NC = C::GCOLS / 32;                   // 32-column register chunks of S per thread
         bool ok = true;
         int t = 0;
+        RingPos<C::SBUFS> rs;                               // S buffer of tile t
+        // P.V of tile i arrives on bar_pv[i & 3] as that barrier's completion number i >> 2.  When these threads wait for
+        // tile t - 1 they have seen S of tile t - 1 (or later) land, which follows P.V of tile t - 4 in the tensor pipe,
+        // so every earlier completion of that barrier (tiles t - 5, t - 9, ...) has happened; and P.V of tile t + 3
+        // cannot be issued before they have arrived on its P.  The barrier is therefore in completion (t - 1) >> 2 or
+        // one past it, and the parity test is exact.
+        auto wait_pv_prev = [&](int where) -> bool {
+            return __all_sync(0xffffffffu, mbar_wait(bar_pv + 8 * ((t - 1) & 3), ((t - 1) >> 2) & 1, abort_flag, p.dev_status, where));
+        };
         for (int n = 0; ok && n < my_units; ++n) {
             const int u = blockIdx.x + n * gridDim.x;
             const int bh = u / p.Tm, i = u - bh * p.Tm;
@@ -359,13 +410,18 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
             int blk_next = __ldg(my_idx);                   // block index list read one tile ahead (off the critical path)
             for (int j = 0; j < keep; ++j, ++t) {
-                const int jb = blk_next % p.n_b;
+                // a chunk's last block may be short; found without an integer division (those run on the XU pipe and
+                // would queue behind the other warp's exponentials)
+                bool tail = false;
+#pragma unroll
+                for (int c = 1; c <= HF_MAX_CHUNKS; ++c) tail |= (blk_next + 1 == c * p.n_b);
                 if (j + 1 < keep) blk_next = __ldg(my_idx + j + 1);
-                const int nv = min(C::BLK, p.Tc - jb * C::BLK);
+                const int nv = tail ? p.Tc - (p.n_b - 1) * C::BLK : C::BLK;
                 const int st = t & 1;
-                const uint32_t tS = lane_base + (st ? C::COL_S1 : C::COL_S0);
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 8));
+                const uint32_t tS = lane_base + rs.stage * C::BLK;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * rs.stage, rs.phase, abort_flag, p.dev_status, 8));
                 if (!ok) break;
+                rs.advance();
                 fence_after_sync();
                 // ---- this thread's share of the S row in registers
                 uint32_t r[NC][32];
@@ -403,10 +459,8 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 } else {
                     const bool need = (m_new - m_used) > 8.f;
                     if (__any_sync(0xffffffffu, need)) {
-                        // O is rewritten here, so P.V of the previous tile must have landed.  While these threads are in
-                        // tile t, bar_pv has completed t - 1 or t phases (P.V of tile t - 2 precedes S of tile t in the
-                        // tensor pipe; P.V of tile t needs this tile's P), so the parity test below is exact.
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 9));
+                        // O is rewritten here, so P.V of the previous tile must have landed
+                        ok = wait_pv_prev(9);
                         if (!ok) break;
                         fence_after_sync();
                         const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
@@ -440,7 +494,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 l_run += rs0 + rs1;
                 tmem_wait_st();
                 fence_before_sync();
-                mbar_arrive(bar_pf + 8 * st);
+                mbar_arrive(bar_pf + 8 * (rs.stage == 0 ? C::SBUFS - 1 : rs.stage - 1));
             }
             if (!ok) break;
             // ---- epilogue of the unit: O / l (+ history term), one rounding to bf16
@@ -453,7 +507,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                 for (int g = 1; g < NG; ++g) l_run += x_sum[g * C::BLK + row];
             }
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, (t - 1) & 1, abort_flag, p.dev_status, 10));
+            ok = wait_pv_prev(10);
             if (!ok) break;
             fence_after_sync();
             const float inv = 1.f / l_run;
