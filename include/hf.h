@@ -141,7 +141,7 @@ hf_status hf_kv_append_host(hf_ctx* ctx, int layer, const void* k_host, const vo
  * and launches nothing.  All pointers 16-byte aligned (else HF_ERR_INVALID_ARG).
  * The first call on a device looks up the device address of the scratch array and sets a kernel attribute; make
  * that first call outside any stream capture.  No call here uses cudaMalloc, cudaFree or an allocating library routine.
- * All calls on a device share the one array (its bookkeeping words are cleared at the start of every call): two calls
+ * All calls on a device share the one array (each call rewrites the part it reads, so nothing has to be cleared): two calls
  * whose kernels may overlap on the GPU -- different streams, or different threads -- race; keep them stream-ordered. */
 hf_status hf_state_absorb_noalloc(const void* k_ev, const void* v_ev, int batch_heads, int n_tokens, int head_dim,
                                   float* S, float* z, void* stream);

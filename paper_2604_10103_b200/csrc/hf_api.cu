@@ -63,7 +63,6 @@ struct hf_ctx {
     float* pooled_kcur = nullptr;
     float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
     float* partials = nullptr;       // absorb split partials
-    unsigned int* counters = nullptr;
     int nsplit_max = 1;
     bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
     int* dev_status = nullptr;
@@ -134,7 +133,7 @@ void free_all(hf_ctx* c) {
         cudaFree(L.sf_hi); cudaFree(L.sf_lo); cudaFree(L.W); cudaFree(L.bias); cudaFree(L.mask); cudaFree(L.idx);
     }
     cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials);
-    cudaFree(c->counters); cudaFree(c->dev_status);
+    cudaFree(c->dev_status);
     for (auto& s : c->stage) cudaFree(s);
 }
 
@@ -168,21 +167,21 @@ hf_status launch_pool(hf_ctx* c, const PoolJobs& jobs, int njobs, cudaStream_t s
 }
 
 template <int D>
+hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
+    k_reduce_fold<D><<<dim3(D / 8, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, L.has_w ? L.W : nullptr, c->cfg.heads,
+                                                      L.sf_hi, L.sf_lo);
+    return post_launch(c, "k_reduce_fold");
+}
+
+template <int D>
 hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st) {
     typedef AbsorbMma<D> A;
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
     dim3 grid(nsplit, c->BH);
-    k_absorb_mma<D><<<grid, A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, c->partials, c->counters, L.S, L.z);
+    k_absorb_mma<D><<<grid, A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, c->partials);
     HF_TRY(post_launch(c, "k_absorb_mma"));
-    k_fold<D><<<dim3(D / 16, c->BH), D, 0, st>>>(L.S, L.has_w ? L.W : nullptr, c->cfg.heads, L.sf_hi, L.sf_lo);
-    return post_launch(c, "k_fold");
-}
-
-template <int D>
-hf_status launch_fold(hf_ctx* c, LayerState& L, cudaStream_t st) {
-    k_fold<D><<<dim3(D / 16, c->BH), D, 0, st>>>(L.S, L.has_w ? L.W : nullptr, c->cfg.heads, L.sf_hi, L.sf_lo);
-    return post_launch(c, "k_fold");
+    return launch_fold<D>(c, L, nsplit, st);
 }
 
 template <int D>
@@ -355,7 +354,7 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->mask_words = (c->max_Tn + 31) / 32;
     c->chunk_elems = (size_t)c->BH * c->Tc * c->d;
     c->pooled_elems = (size_t)c->BH * c->n_b * c->d;
-    c->nsplit_max = (2 * c->sm_count + c->BH - 1) / c->BH;
+    c->nsplit_max = c->sm_count / c->BH;          // one wave: the absorb kernel runs one thread block per SM
     if (c->nsplit_max > 32) c->nsplit_max = 32;
     if (c->nsplit_max < 1) c->nsplit_max = 1;
     if (cfg->swa_kernel == HF_SWA_TCGEN05 && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the tcgen05 attention kernel needs block == 128"); }
@@ -394,10 +393,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     if (s == HF_OK) s = dmalloc(&c->pooled_kcur, c->pooled_elems);
     if (s == HF_OK) s = dmalloc(&c->hist, c->chunk_elems);
     if (s == HF_OK) s = dmalloc(&c->partials, (size_t)c->BH * c->nsplit_max * ((size_t)c->d * c->d + c->d));
-    if (s == HF_OK) s = dmalloc(&c->counters, (size_t)c->BH);
     if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)4);
     if (s == HF_OK) {
-        cudaMemset(c->counters, 0, (size_t)c->BH * 4);
         cudaMemset(c->dev_status, 0, 16);
         s = set_swa_attr<16, 64>();
         if (s == HF_OK) s = set_swa_attr<16, 128>();
@@ -453,7 +450,7 @@ hf_status hf_set_merge_weights(hf_ctx* c, int layer, const void* W, const void* 
     if (bias) HF_CUDA(cudaMemcpyAsync(L.bias, bias, (size_t)c->cfg.heads * c->d * 2, cudaMemcpyDeviceToDevice, st));
     L.has_w = true;
     L.has_bias = bias != nullptr;
-    return HF_DISPATCH_D(c, launch_fold, c, L, st);
+    return HF_DISPATCH_D(c, launch_fold, c, L, 0, st);
 }
 
 hf_status hf_state_absorb(hf_ctx* c, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream) {

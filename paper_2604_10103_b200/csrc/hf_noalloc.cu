@@ -1,6 +1,6 @@
 // hf_state_absorb_noalloc: the state update (S += phi(K)^T V, z += sum phi(K)) for callers that must not
-// allocate device memory.  The split partials and tickets that hf_state_absorb keeps in buffers of its
-// context live here in one file-scope device array instead.
+// allocate device memory.  The split partials that hf_state_absorb keeps in a buffer of its context live
+// here in one file-scope device array instead.
 #include "../../include/hf.h"
 #include "hf_common.cuh"
 #include "k_state_mma.cuh"
@@ -13,11 +13,11 @@ extern "C" void hf_internal_set_error(const char* text);
 namespace {
 
 constexpr size_t NOALLOC_SCRATCH_BYTES = 16u << 20;     // 16 MiB, held by every device that loads the library
-constexpr size_t NOALLOC_TICKET_BYTES = 4096;           // first 4 KiB: one ticket per (batch, head) -> at most 1024
-constexpr int NOALLOC_MAX_BH = (int)(NOALLOC_TICKET_BYTES / sizeof(unsigned int));
+constexpr size_t NOALLOC_TICKET_BYTES = 4096;           // first 4 KiB: reserved for bookkeeping words
+constexpr int NOALLOC_MAX_BH = 1024;
 constexpr int NOALLOC_MAX_DEVICES = 64;
 
-// Scratch shared by every call on a device: [tickets | split partials].  In host code this name is only a
+// Scratch shared by every call on a device: [reserved 4 KiB | split partials].  In host code this name is only a
 // handle for cudaGetSymbolAddress; it is never passed to a kernel as a pointer.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_SCRATCH_BYTES];
 
@@ -60,13 +60,14 @@ hf_status run(const bf16* k, const bf16* v, int bh, int n_tokens, float* S, floa
     int nsplit = (int)(room / (size_t)bh);
     if (nsplit > 32) nsplit = 32;
     if (nsplit > n_tiles) nsplit = n_tiles;
-    unsigned int* tickets = reinterpret_cast<unsigned int*>(scratch);
     float* partials = reinterpret_cast<float*>(scratch + NOALLOC_TICKET_BYTES);
-    // the array keeps whatever the previous call left: the tickets must start at zero
-    cudaError_t e = cudaMemsetAsync(tickets, 0, (size_t)bh * sizeof(unsigned int), st);
-    if (e != cudaSuccess) return nfail(HF_ERR_CUDA, "cudaMemsetAsync failed with error %lld", (long long)e);
-    k_absorb_mma<D><<<dim3(nsplit, bh), A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, partials, tickets, S, z);
-    e = cudaGetLastError();
+    // the array keeps whatever the previous call left; every partial that is read below is first rewritten in full
+    k_absorb_mma<D><<<dim3(nsplit, bh), A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, partials);
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) {
+        k_reduce_fold<D><<<dim3(D / 8, bh), D, 0, st>>>(partials, nsplit, S, z, nullptr, 1, nullptr, nullptr);
+        e = cudaGetLastError();
+    }
     if (e != cudaSuccess) return nfail(HF_ERR_CUDA, "kernel launch failed with error %lld", (long long)e);
     return HF_OK;
 }

@@ -42,17 +42,32 @@ __global__ void __launch_bounds__(256) k_pool_copy(PoolJobs jobs, int Tc, int bl
     const int n = min(blk, Tc - t0);
     const int r = threadIdx.x >> 4, cv = threadIdx.x & 15;
     const size_t base = ((size_t)bh * Tc + t0) * D + cv * VEC;
+    // all loads of the thread first (up to 8 rows in flight), then the copies, then the chain adds in token order
+    constexpr int MAXR = 8;                       // blk <= 128 -> at most 8 rows per chain
+    V u[MAXR];
+#pragma unroll
+    for (int i = 0; i < MAXR; ++i) {
+        const int t = r + 16 * i;
+        if (t < n) u[i] = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
+    }
+    if (jb.copy_dst) {
+#pragma unroll
+        for (int i = 0; i < MAXR; ++i) {
+            const int t = r + 16 * i;
+            if (t < n) *reinterpret_cast<V*>(jb.copy_dst + base + (size_t)t * D) = u[i];
+        }
+    }
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
-#pragma unroll 4
-    for (int t = r; t < n; t += 16) {
-        V u = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
-        if (jb.copy_dst) *reinterpret_cast<V*>(jb.copy_dst + base + (size_t)t * D) = u;
-        float f[VEC];
-        VecLoad<VEC>::widen(u, f);
 #pragma unroll
-        for (int e = 0; e < VEC; ++e) acc[e] = __fadd_rn(acc[e], f[e]);
+    for (int i = 0; i < MAXR; ++i) {
+        if (r + 16 * i < n) {
+            float f[VEC];
+            VecLoad<VEC>::widen(u[i], f);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = __fadd_rn(acc[e], f[e]);
+        }
     }
     if (jb.pooled == nullptr) return;
     __shared__ float part[16][D];
@@ -83,17 +98,33 @@ __global__ void __launch_bounds__(128) k_select(ChunkTable tab, const float* __r
     const size_t row = (size_t)bh * Tm + i;
     if (threadIdx.x < D) sq[threadIdx.x] = pooled_q[row * D + threadIdx.x];
     __syncthreads();
-    for (int j = warp; j < Tn; j += 4) {
-        const int c = j / n_b, jb = j - c * n_b;
-        const float* kp = tab.pooled[c] + ((size_t)bh * n_b + jb) * D;
-        float acc = __fmul_rn(sq[lane], __ldg(kp + lane));
+    // four scores per pass and warp: the sixteen loads of a lane are issued before any of them is used
+    for (int j0 = warp; j0 < Tn; j0 += 16) {
+        float kv[4][D / 32];
 #pragma unroll
-        for (int m = 1; m < D / 32; ++m) acc = __fadd_rn(acc, __fmul_rn(sq[lane + 32 * m], __ldg(kp + lane + 32 * m)));
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + 4 * u;
+            if (j < Tn) {
+                const int c = j / n_b, jb = j - c * n_b;
+                const float* kp = tab.pooled[c] + ((size_t)bh * n_b + jb) * D;
 #pragma unroll
-        for (int off = 16; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-        if (lane == 0) {
-            sc[j] = acc;
-            if (scores_out) scores_out[row * Tn + j] = acc;
+                for (int m = 0; m < D / 32; ++m) kv[u][m] = __ldg(kp + lane + 32 * m);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int j = j0 + 4 * u;
+            if (j < Tn) {
+                float acc = __fmul_rn(sq[lane], kv[u][0]);
+#pragma unroll
+                for (int m = 1; m < D / 32; ++m) acc = __fadd_rn(acc, __fmul_rn(sq[lane + 32 * m], kv[u][m]));
+#pragma unroll
+                for (int off = 16; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+                if (lane == 0) {
+                    sc[j] = acc;
+                    if (scores_out) scores_out[row * Tn + j] = acc;
+                }
+            }
         }
     }
     __syncthreads();

@@ -1,6 +1,8 @@
 // Linear-attention state kernels on the warp-level tensor path (ldmatrix + mma.sync):
-//   k_absorb_mma   Eq. 3: S += phi(K_ev)^T V_ev, z += sum_t phi(K_ev[t])   (token-split partials + fixed-order reduce)
-//   k_fold         S' = S W^T split into bf16 hi/lo halves (the per-row divisor of Eq. 4 commutes with W)
+//   k_absorb_mma   Eq. 3, first half: per (batch, head) the token range is split over thread blocks, each writing
+//                  its partial phi(K_ev)^T V_ev and sum_t phi(K_ev[t]) to scratch
+//   k_reduce_fold  Eq. 3, second half: S, z += the partials in ascending split order (deterministic), then
+//                  S' = S W^T split into bf16 hi/lo halves (the per-row divisor of Eq. 4 commutes with W)
 //   k_readout_mma  Eq. 4: (phi(Q) S') / (phi(Q).z + eps) + bias
 // phi(K) and phi(Q) are carried as bf16 hi + lo pairs so that the products keep ~16 mantissa bits;
 // accumulation is fp32 throughout.
@@ -13,7 +15,8 @@ struct AbsorbMma {
     static constexpr int TT = 64;                  // tokens per shared-memory tile
     static constexpr int ROW_BYTES = D * 2;
     static constexpr int TILE_BYTES = TT * ROW_BYTES;
-    static constexpr int SMEM_BYTES = 4 * TILE_BYTES;   // 2 stages x (K, V)
+    static constexpr int STAGES = 3;
+    static constexpr int SMEM_BYTES = STAGES * 2 * TILE_BYTES;   // stages x (K, V)
     static constexpr int CHUNKS_PER_ROW = D / 8;
     static constexpr int CHUNKS_PER_THREAD = (TT * CHUNKS_PER_ROW) / THREADS;   // = 4
     static constexpr int PART_FLOATS = D * D + D;  // one partial: S then z
@@ -31,14 +34,11 @@ __device__ __forceinline__ void absorb_load_tile(uint32_t smem_tile, const bf16*
     }
 }
 
-// grid (nsplit, B*H).  k_ev, v_ev: [B*H, n_tokens, D].  partials: [B*H, nsplit, D*D + D] scratch.
-// counters: [B*H] zero-initialised tickets; the last CTA of a (batch, head) adds the partials to S, z in
-// ascending split order (deterministic) and re-arms the ticket.
+// grid (nsplit, B*H).  k_ev, v_ev: [B*H, n_tokens, D].  partials: [B*H, nsplit, D*D + D] scratch, every element
+// of which is written (S part, then z part); k_reduce_fold adds them to the state.
 template <int D>
 __global__ void __launch_bounds__(AbsorbMma<D>::THREADS)
-k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n_tokens,
-             float* __restrict__ partials, unsigned int* __restrict__ counters,
-             float* __restrict__ S, float* __restrict__ z) {
+k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n_tokens, float* __restrict__ partials) {
     typedef AbsorbMma<D> C;
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t s0 = smem_u32(smem);
@@ -53,10 +53,13 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
     const bf16* vb = v_ev + (size_t)bh * n_tokens * D;
 
     auto issue = [&](int tile, int stage) {
-        const int t0 = tile * C::TT;
-        const int nv = min(C::TT, n_tokens - t0);
-        absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES, kb + (size_t)t0 * D, nv);
-        absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES + C::TILE_BYTES, vb + (size_t)t0 * D, nv);
+        if (tile < tile_hi) {
+            const int t0 = tile * C::TT;
+            const int nv = min(C::TT, n_tokens - t0);
+            absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES, kb + (size_t)t0 * D, nv);
+            absorb_load_tile<D>(s0 + stage * 2 * C::TILE_BYTES + C::TILE_BYTES, vb + (size_t)t0 * D, nv);
+        }
+        cp_async_commit();      // one group per call, empty past the end, so that the wait below counts uniformly
     };
 
     float acc[D / 8][4];
@@ -64,14 +67,13 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
     for (int n = 0; n < D / 8; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
     float zs[2] = {0.f, 0.f};
 
-    if (tile_lo < tile_hi) issue(tile_lo, 0);
-    cp_async_commit();
+#pragma unroll
+    for (int s = 0; s < C::STAGES - 1; ++s) issue(tile_lo + s, s);
+    int stage = 0;
     for (int tile = tile_lo; tile < tile_hi; ++tile) {
-        const int stage = (tile - tile_lo) & 1;
-        if (tile + 1 < tile_hi) issue(tile + 1, stage ^ 1);
-        cp_async_commit();
-        cp_async_wait<1>();
-        __syncthreads();
+        cp_async_wait<C::STAGES - 2>();
+        __syncthreads();          // tile landed for every thread; the stage refilled below was read in the previous pass
+        issue(tile + C::STAGES - 1, (stage + C::STAGES - 1) % C::STAGES);
         const uint32_t sK = s0 + stage * 2 * C::TILE_BYTES, sV = sK + C::TILE_BYTES;
         const int nv = min(C::TT, n_tokens - tile * C::TT);
 #pragma unroll
@@ -106,7 +108,7 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
                 mma_bf16(acc[2 * np + 1], alo[0], alo[1], alo[2], alo[3], b2, b3);
             }
         }
-        __syncthreads();
+        stage = (stage + 1) % C::STAGES;
     }
     cp_async_wait<0>();
 
@@ -124,42 +126,51 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
             *reinterpret_cast<float2*>(part + (size_t)a * D + c) = make_float2(acc[n][2 * r], acc[n][2 * r + 1]);
         }
     }
-    // ---- last CTA of this (batch, head) reduces in fixed order
-    __shared__ unsigned int ticket;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) ticket = atomicAdd(&counters[bh], 1u);
-    __syncthreads();
-    if (ticket != (unsigned)(nsplit - 1)) return;
-    __threadfence();
-    const float* base = partials + (size_t)bh * nsplit * C::PART_FLOATS;
-    for (int e = threadIdx.x; e < C::PART_FLOATS; e += C::THREADS) {
-        float sum = __ldcg(base + e);
-        for (int s = 1; s < nsplit; ++s) sum += __ldcg(base + (size_t)s * C::PART_FLOATS + e);
-        if (e < D * D) S[(size_t)bh * D * D + e] += sum;
-        else z[(size_t)bh * D + (e - D * D)] += sum;
-    }
-    if (threadIdx.x == 0) counters[bh] = 0u;
 }
 
-// grid (D/16, B*H), D threads.  Sf = S W_h^T (or S when W == nullptr), written as bf16 hi and lo halves.
+// grid (D/8, B*H), D threads.  Adds the nsplit partials of a (batch, head) to S (rows a0 .. a0+7 per block) and z
+// (block 0) in ascending split order, then folds the updated rows: Sf = S W_h^T (or S when W == nullptr) as bf16
+// hi and lo halves.  nsplit == 0: fold only.  sf_hi == nullptr: state update only.
 template <int D>
 __global__ void __launch_bounds__(D)
-k_fold(const float* __restrict__ S, const bf16* __restrict__ W, int heads,
-       bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
-    __shared__ float rows[16][D];
-    const int a0 = blockIdx.x * 16, bh = blockIdx.y, h = bh % heads;
+k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict__ S, float* __restrict__ z,
+              const bf16* __restrict__ W, int heads, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
+    constexpr int ROWS = 8;
+    constexpr int PART_FLOATS = D * D + D;
+    __shared__ float rows[ROWS][D];
+    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, h = bh % heads;
     const int cp = threadIdx.x;
-    for (int e = threadIdx.x; e < 16 * D; e += D) rows[e / D][e % D] = S[((size_t)bh * D + a0) * D + e];
+    const float* base = partials + (size_t)bh * nsplit * PART_FLOATS;
+    float sum[ROWS];
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) sum[r] = 0.f;
+    for (int s = 0; s < nsplit; ++s) {
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) sum[r] += __ldcg(base + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+    }
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+        float* dst = S + ((size_t)bh * D + a0 + r) * D + cp;
+        const float v = *dst + sum[r];
+        if (nsplit > 0) *dst = v;
+        rows[r][cp] = v;
+    }
+    if (blockIdx.x == 0 && nsplit > 0) {
+        float zsum = 0.f;
+        for (int s = 0; s < nsplit; ++s) zsum += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
+        z[(size_t)bh * D + cp] += zsum;
+    }
+    if (sf_hi == nullptr) return;
     __syncthreads();
-    float out[16];
+    float out[ROWS];
     if (W == nullptr) {
 #pragma unroll
-        for (int r = 0; r < 16; ++r) out[r] = rows[r][cp];
+        for (int r = 0; r < ROWS; ++r) out[r] = rows[r][cp];
     } else {
 #pragma unroll
-        for (int r = 0; r < 16; ++r) out[r] = 0.f;
+        for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
         const bf16* wrow = W + ((size_t)h * D + cp) * D;     // W_h[c'][.]
+#pragma unroll 4
         for (int c = 0; c < D; c += 8) {
             const uint4 u = __ldg(reinterpret_cast<const uint4*>(wrow + c));
             float w[8];
@@ -169,13 +180,13 @@ k_fold(const float* __restrict__ S, const bf16* __restrict__ W, int heads,
             t = unpack_bf16(u.z); w[4] = t.x; w[5] = t.y;
             t = unpack_bf16(u.w); w[6] = t.x; w[7] = t.y;
 #pragma unroll
-            for (int r = 0; r < 16; ++r)
+            for (int r = 0; r < ROWS; ++r)
 #pragma unroll
                 for (int e = 0; e < 8; ++e) out[r] = fmaf(rows[r][c + e], w[e], out[r]);
         }
     }
 #pragma unroll
-    for (int r = 0; r < 16; ++r) {
+    for (int r = 0; r < ROWS; ++r) {
         const __nv_bfloat16 hi = __float2bfloat16_rn(out[r]);
         const size_t o = ((size_t)bh * D + a0 + r) * D + cp;
         sf_hi[o] = hi;
@@ -194,7 +205,7 @@ struct ReadoutMma {
 
 // grid (ceil(T_c/128), B*H).  out_bf16 or out_f32 (exactly one non-null): [B*H, T_c, D].
 template <int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 2)
 k_readout_mma(const bf16* __restrict__ q, const bf16* __restrict__ sf_hi, const bf16* __restrict__ sf_lo,
               const float* __restrict__ z, const bf16* __restrict__ bias, int heads, int Tc, float eps,
               bf16* __restrict__ out_bf16, float* __restrict__ out_f32) {
