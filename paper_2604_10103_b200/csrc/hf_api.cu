@@ -5,6 +5,7 @@
 #include "k_swa_mma.cuh"
 #include "k_swa_tc5.cuh"
 #include "k_state_mma.cuh"
+#include "k_state_tc5.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -49,6 +50,7 @@ struct LayerState {
     unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
     int sel_keep = 0;
     CUtensorMap tm_kring, tm_vring;   // 4-D maps over the whole ring [slot, B*H, T_c, d]
+    CUtensorMap tm_sfhi, tm_sflo;     // folded state halves [B*H, d, d], box = 64 columns x d rows
 };
 
 }  // namespace
@@ -144,8 +146,8 @@ hf_status set_swa_attr() {
 }
 template <int D>
 hf_status set_state_attr() {
-    HF_CUDA(cudaFuncSetAttribute(k_absorb_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbMma<D>::SMEM_BYTES));
-    HF_CUDA(cudaFuncSetAttribute(k_readout_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutMma<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
     return HF_OK;
 }
 
@@ -166,6 +168,28 @@ hf_status launch_pool(hf_ctx* c, const PoolJobs& jobs, int njobs, cudaStream_t s
     return post_launch(c, "k_pool_copy");
 }
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 4-D bf16 map [slots, B*H, rows, d] with a box of box_cols x box_rows, 128-byte swizzle (or none); rows past the end read as zero.
+hf_status make_map_ex(hf_ctx* c, CUtensorMap* m, const void* base, long long rows, int slots, int box_cols, int box_rows, bool swizzle) {
+    const cuuint64_t dims[4] = {(cuuint64_t)c->d, (cuuint64_t)rows, (cuuint64_t)c->BH, (cuuint64_t)slots};
+    const cuuint64_t strides[3] = {(cuuint64_t)c->d * 2, (cuuint64_t)rows * c->d * 2, (cuuint64_t)c->BH * rows * c->d * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1, 1};
+    const cuuint32_t es[4] = {1, 1, 1, 1};
+    CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
+                                                                  strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                                  swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(HF_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
+    return HF_OK;
+}
+// [slots, B*H, T_c, d], box = 64 columns x 128 rows, 128-byte swizzle: the attention kernel's Q / K / V tiles.
+hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
+    return make_map_ex(c, m, base, c->Tc, slots, 64, 128, true);
+}
+
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
     k_reduce_fold<D><<<dim3(D / 8, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, L.has_w ? L.W : nullptr, c->cfg.heads,
@@ -175,22 +199,31 @@ hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
 
 template <int D>
 hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st) {
-    typedef AbsorbMma<D> A;
+    typedef AbsorbTc5<D> A;
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
-    dim3 grid(nsplit, c->BH);
-    k_absorb_mma<D><<<grid, A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, c->partials);
-    HF_TRY(post_launch(c, "k_absorb_mma"));
+    CUtensorMap tk, tv;
+    HF_TRY(make_map_ex(c, &tk, k, n_tokens, 1, D, A::TT, false));
+    HF_TRY(make_map_ex(c, &tv, v, n_tokens, 1, 64, A::TT, true));
+    AbsorbTc5Params p;
+    p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
+    k_absorb_tc5<D><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
+    HF_TRY(post_launch(c, "k_absorb_tc5"));
     return launch_fold<D>(c, L, nsplit, st);
 }
 
 template <int D>
 hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16, float* out_f32, cudaStream_t st) {
-    typedef ReadoutMma<D> R;
-    dim3 grid((c->Tc + R::ROWS - 1) / R::ROWS, c->BH);
-    k_readout_mma<D><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(q, L.sf_hi, L.sf_lo, L.z, L.has_bias ? L.bias : nullptr,
-                                                             c->cfg.heads, c->Tc, c->cfg.eps, out_bf16, out_f32);
-    return post_launch(c, "k_readout_mma");
+    typedef ReadoutTc5<D> R;
+    CUtensorMap tq;
+    HF_TRY(make_map(c, &tq, q, 1));
+    ReadoutTc5Params p;
+    p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr; p.heads = c->cfg.heads; p.Tc = c->Tc;
+    p.Tm = (c->Tc + R::ROWS - 1) / R::ROWS; p.n_units = p.Tm * c->BH; p.eps = c->cfg.eps;
+    p.out_bf16 = out_bf16; p.out_f32 = out_f32; p.dev_status = c->dev_status;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    k_readout_tc5<D><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
+    return post_launch(c, "k_readout_tc5");
 }
 
 ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v_cur) {
@@ -237,23 +270,6 @@ hf_status launch_swa_mma_t(hf_ctx* c, const bf16* q, const ChunkTable& tab, cons
     return post_launch(c, "k_swa_mma");
 }
 
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// 4-D bf16 map [slots, B*H, T_c, d], box = 64 columns x 128 rows, 128-byte swizzle, out-of-range rows read as zero.
-hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
-    const cuuint64_t dims[4] = {(cuuint64_t)c->d, (cuuint64_t)c->Tc, (cuuint64_t)c->BH, (cuuint64_t)slots};
-    const cuuint64_t strides[3] = {(cuuint64_t)c->d * 2, (cuuint64_t)c->Tc * c->d * 2, (cuuint64_t)c->BH * c->Tc * c->d * 2};
-    const cuuint32_t box[4] = {64, 128, 1, 1};
-    const cuuint32_t es[4] = {1, 1, 1, 1};
-    CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims,
-                                                                  strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return fail(HF_ERR_CUDA, "cuTensorMapEncodeTiled failed with %d", (int)r);
-    return HF_OK;
-}
 
 #ifndef HF_TC5_GROUPS
 #define HF_TC5_GROUPS 2   // softmax column groups of the tcgen05 attention kernel
@@ -385,6 +401,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
         if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_kring, L.ring_k, c->P);
         if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_vring, L.ring_v, c->P);
+        if (s == HF_OK) s = make_map_ex(c, &L.tm_sfhi, L.sf_hi, c->d, 1, 64, c->d, true);
+        if (s == HF_OK) s = make_map_ex(c, &L.tm_sflo, L.sf_lo, c->d, 1, 64, c->d, true);
         if (s != HF_OK) break;
         cudaMemset(L.S, 0, dd * 4); cudaMemset(L.z, 0, dz * 4);
         cudaMemset(L.sf_hi, 0, dd * 2); cudaMemset(L.sf_lo, 0, dd * 2);

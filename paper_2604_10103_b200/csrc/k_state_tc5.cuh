@@ -1,0 +1,427 @@
+// Linear-attention state kernels on the Blackwell tensor path (tcgen05.mma, accumulators in tensor memory, TMA loads):
+//   k_absorb_tc5   Eq. 3, first half: per (batch, head) the token range is split over thread blocks, each writing
+//                  its partial phi(K_ev)^T V_ev and sum_t phi(K_ev[t]) to scratch (k_reduce_fold adds them up)
+//   k_readout_tc5  Eq. 4: (phi(Q) S') / (phi(Q).z + eps) + bias with S' = S W^T folded beforehand
+// In both, the phi(.) operand never goes back to shared memory: the thread that owns a row of the A operand
+// (TMEM lane = row) evaluates phi in fp32, splits it into bf16 hi + lo halves (~16 mantissa bits together) and
+// stores them straight into tensor memory, from where the MMA reads A; the other operand comes from shared
+// memory as TMA wrote it.  Accumulation is fp32.  Every wait is bounded (~1 s) and reports through the device
+// status word; nothing traps.
+#pragma once
+#include "tc5_common.cuh"
+
+// ------------------------------------------------------------------------------------------------------------
+// Absorb.  A = phi(K)^T: M = key feature a (lane), K = token.  B = V tile [token][c] (N = c contiguous, MN-major).
+// D[a][c] += sum_t phi(k_t)[a] v_t[c]  over the block's token tiles; z[a] += sum_t phi(k_t)[a] in the lane's register.
+// ------------------------------------------------------------------------------------------------------------
+template <int D>
+struct AbsorbTc5 {
+    static constexpr int TT = 64;                        // tokens per tile
+    static constexpr int NST = 4;                        // K / V stages in flight
+    static constexpr int SUB = D / 64;
+    static constexpr int K_BYTES = TT * D * 2;           // row-major, not swizzled (read column-wise by the lanes)
+    static constexpr int VSUB_BYTES = TT * 128;          // one 64-column sub-tile of V, 128-byte swizzle
+    static constexpr int V_BYTES = SUB * VSUB_BYTES;
+    static constexpr int OFF_K = 0, OFF_V = NST * K_BYTES, OFF_BAR = OFF_V + NST * V_BYTES;
+    static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+    static constexpr int THREADS = 192;                  // warps 0-3: phi / epilogue, warp 4: TMA, warp 5: MMA
+    static constexpr int TMEM_COLS = 256;                // D accumulator [0, D) ; A buffers at 128 + 64 b: hi 32 cols, lo 32 cols
+    static constexpr int COL_A = 128;
+    static constexpr int PART_FLOATS = D * D + D;
+};
+
+struct AbsorbTc5Params {
+    int n_tokens;
+    float* partials;          // [B*H, nsplit, D*D + D]
+    int* dev_status;
+};
+
+// grid (nsplit, B*H).  tm_k: [D, n_tokens, B*H, 1] box {D, 64}, no swizzle.  tm_v: same tensor shape, box {64, 64}, 128B swizzle.
+template <int D>
+__global__ void __launch_bounds__(AbsorbTc5<D>::THREADS, 1)
+k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const AbsorbTc5Params p) {
+    using namespace tc5;
+    typedef AbsorbTc5<D> C;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
+    const uint32_t sK = s_base + C::OFF_K, sV = s_base + C::OFF_V, bar0 = s_base + C::OFF_BAR;
+    const uint32_t bar_full = bar0, bar_kfree = bar0 + 32, bar_vfree = bar0 + 64, bar_afull = bar0 + 96, bar_afree = bar0 + 112,
+                   bar_dfull = bar0 + 128;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 144);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 148);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x, nsplit = gridDim.x, bh = blockIdx.y;
+    const int n_tiles = (p.n_tokens + C::TT - 1) / C::TT;
+    const int tile_lo = (int)(((long long)n_tiles * split) / nsplit);
+    const int tile_hi = (int)(((long long)n_tiles * (split + 1)) / nsplit);
+    const int n_local = tile_hi - tile_lo;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_kfree + 8 * s, D); mbar_init(bar_vfree + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_afull + 8 * s, D); mbar_init(bar_afree + 8 * s, 1); }
+        mbar_init(bar_dfull, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        // ================================================================= TMA producer
+        if (lane == 0) {
+            bool ok = true;
+            for (int i = 0; ok && i < n_local; ++i) {
+                const int s = i % C::NST;
+                const uint32_t par_free = ((i / C::NST) & 1) ^ 1;
+                if (i >= C::NST) {
+                    if (!(ok = mbar_wait<true>(bar_kfree + 8 * s, par_free, abort_flag, p.dev_status, 31))) break;
+                    if (!(ok = mbar_wait<true>(bar_vfree + 8 * s, par_free, abort_flag, p.dev_status, 32))) break;
+                }
+                const int row0 = (tile_lo + i) * C::TT;
+                mbar_expect_tx(bar_full + 8 * s, C::K_BYTES + C::V_BYTES);
+                tma_load_4d(sK + s * C::K_BYTES, &tm_k, 0, row0, bh, 0, bar_full + 8 * s);
+#pragma unroll
+                for (int u = 0; u < C::SUB; ++u)
+                    tma_load_4d(sV + s * C::V_BYTES + u * C::VSUB_BYTES, &tm_v, u * 64, row0, bh, 0, bar_full + 8 * s);
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 400000) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ================================================================= MMA issuer (warp-uniform, one elected lane issues)
+        constexpr uint32_t IDESC = idesc_bf16(D, true);
+        const uint64_t dv0 = smem_desc_sw128(sV, C::VSUB_BYTES, 1024);
+        bool ok = true;
+        for (int i = 0; ok && i < n_local; ++i) {
+            const int s = i % C::NST, ab = i & 1;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_afull + 8 * ab, (i >> 1) & 1, abort_flag, p.dev_status, 33)))) break;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_full + 8 * s, (i / C::NST) & 1, abort_flag, p.dev_status, 34)))) break;
+            fence_after_sync();
+            if (elect_one()) {
+                const uint32_t tA = tmem + C::COL_A + ab * 64;
+                const uint64_t dv = dv0 + (uint64_t)((s * C::V_BYTES) >> 4);
+#pragma unroll
+                for (int ks = 0; ks < C::TT / 16; ++ks) {
+                    const uint64_t db = dv + (uint64_t)(ks * (2048 >> 4));
+                    mma_ts(tmem, tA + ks * 8, db, IDESC, i > 0 || ks > 0);          // hi half
+                    mma_ts(tmem, tA + 32 + ks * 8, db, IDESC, true);                // lo half
+                }
+                mma_commit(bar_afree + 8 * ab);
+                mma_commit(bar_vfree + 8 * s);
+                if (i == n_local - 1) mma_commit(bar_dfull);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ================================================================= phi(K) into tensor memory, then the epilogue
+        const int a = threadIdx.x;                              // key feature = TMEM lane
+        const bool active = a < D;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        float zacc = 0.f;
+        for (int i = 0; ok && i < n_local; ++i) {
+            const int s = i % C::NST, ab = i & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, (i / C::NST) & 1, abort_flag, p.dev_status, 35));
+            if (!ok) break;
+            if (i >= 2) {
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_afree + 8 * ab, ((i >> 1) & 1) ^ 1, abort_flag, p.dev_status, 36));
+                if (!ok) break;
+                fence_after_sync();
+            }
+            if (active) {
+                const int nv = min(C::TT, p.n_tokens - (tile_lo + i) * C::TT);      // rows past the end read as zero: phi(0) = 1 must not count
+                const uint8_t* kt = s_gen + C::OFF_K + s * C::K_BYTES + a * 2;
+                uint32_t hi[C::TT / 2], lo[C::TT / 2];
+#pragma unroll
+                for (int t = 0; t < C::TT; t += 2) {
+                    const float x0 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)t * D * 2)) << 16);
+                    const float x1 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)(t + 1) * D * 2)) << 16);
+                    float f0 = phi_elu1(x0), f1 = phi_elu1(x1);
+                    if (t >= nv) f0 = 0.f;
+                    if (t + 1 >= nv) f1 = 0.f;
+                    zacc += f0 + f1;
+                    const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+                    hi[t >> 1] = pack_bf16(f0, f1);
+                    lo[t >> 1] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                }
+                const uint32_t tA = lane_base + C::COL_A + ab * 64;
+                tmem_st32(tA, hi);
+                tmem_st32(tA + 32, lo);
+                tmem_wait_st();
+                fence_before_sync();
+                mbar_arrive(bar_afull + 8 * ab);
+                mbar_arrive(bar_kfree + 8 * s);
+            }
+        }
+        if (ok) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_dfull, 0, abort_flag, p.dev_status, 37));
+            if (ok && active) {
+                fence_after_sync();
+                float* part = p.partials + ((size_t)bh * nsplit + split) * C::PART_FLOATS;
+                part[D * D + a] = zacc;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(lane_base + c * 32, r);
+                    tmem_wait_ld();
+                    float4* dst = reinterpret_cast<float4*>(part + (size_t)a * D + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                             __uint_as_float(r[4 * v + 3]));
+                }
+            }
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        fence_after_sync();
+        tmem_dealloc(tmem, C::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Read-out.  Unit = (batch*head, tile of 128 query rows).  A = phi(Q): M = query row (lane), K = key feature.
+// B = S' [a][c] (N = c contiguous, MN-major), hi and lo halves.  D = A_hi S'_hi + A_lo S'_hi + A_hi S'_lo.
+// ------------------------------------------------------------------------------------------------------------
+template <int D>
+struct ReadoutTc5 {
+    static constexpr int ROWS = 128;
+    static constexpr int NST = 2;                        // unit stages: {Q tile, S' hi, S' lo}
+    static constexpr int SUB = D / 64;
+    static constexpr int QSUB_BYTES = ROWS * 128, Q_BYTES = SUB * QSUB_BYTES;
+    static constexpr int SSUB_BYTES = D * 128, S_BYTES = SUB * SSUB_BYTES;
+    static constexpr int STAGE_BYTES = Q_BYTES + 2 * S_BYTES;
+    static constexpr int OFF_VEC = NST * STAGE_BYTES;    // per stage: z [D] floats, bias [D] floats
+    static constexpr int OFF_BAR = OFF_VEC + NST * 2 * D * 4;
+    static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
+    static constexpr int THREADS = 192;                  // warps 0-3: phi / epilogue, warp 4: TMA, warp 5: MMA
+    static constexpr int TMEM_COLS = 4 * D;              // D accumulators at D b ; A buffers at 2 D + D b: hi D/2 cols, lo D/2 cols
+};
+
+struct ReadoutTc5Params {
+    const float* z;           // [B*H, D]
+    const bf16* bias;         // [H, D] or nullptr
+    int heads, Tc, Tm, n_units;
+    float eps;
+    bf16* out_bf16;           // exactly one of the two outputs is non-null: [B*H, T_c, D]
+    float* out_f32;
+    int* dev_status;
+};
+
+// Persistent: CTA c processes units c, c + gridDim.x, ...  tm_q: [D, T_c, B*H, 1] box {64, 128};
+// tm_sh, tm_sl: [D, D, B*H, 1] box {64, D}; all 128B swizzle.
+template <int D>
+__global__ void __launch_bounds__(ReadoutTc5<D>::THREADS, 1)
+k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_sh,
+              const __grid_constant__ CUtensorMap tm_sl, const ReadoutTc5Params p) {
+    using namespace tc5;
+    typedef ReadoutTc5<D> C;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
+    const uint32_t bar0 = s_base + C::OFF_BAR;
+    const uint32_t bar_full = bar0, bar_qfree = bar0 + 16, bar_sfree = bar0 + 32, bar_afull = bar0 + 48, bar_afree = bar0 + 64,
+                   bar_dfull = bar0 + 80, bar_dfree = bar0 + 96, bar_vec = bar0 + 112;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 144);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 148);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar_full + 8 * s, 1); mbar_init(bar_qfree + 8 * s, 128); mbar_init(bar_sfree + 8 * s, 1);
+            mbar_init(bar_afull + 8 * s, 128); mbar_init(bar_afree + 8 * s, 1); mbar_init(bar_dfull + 8 * s, 1);
+            mbar_init(bar_dfree + 8 * s, 128); mbar_init(bar_vec + 8 * s, 128);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 5) {
+        tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
+        tmem_relinquish();
+    }
+    fence_before_sync();
+    __syncthreads();
+    fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        // ================================================================= TMA producer
+        if (lane == 0) {
+            bool ok = true;
+            for (int n = 0; ok && n < my_units; ++n) {
+                const int u = blockIdx.x + n * gridDim.x;
+                const int bh = u / p.Tm, i = u - bh * p.Tm;
+                const int s = n & 1;
+                const uint32_t par_free = ((n >> 1) & 1) ^ 1;
+                if (n >= 2) {
+                    if (!(ok = mbar_wait<true>(bar_qfree + 8 * s, par_free, abort_flag, p.dev_status, 41))) break;
+                    if (!(ok = mbar_wait<true>(bar_sfree + 8 * s, par_free, abort_flag, p.dev_status, 42))) break;
+                }
+                const uint32_t st = s_base + s * C::STAGE_BYTES;
+                mbar_expect_tx(bar_full + 8 * s, C::STAGE_BYTES);
+#pragma unroll
+                for (int v = 0; v < C::SUB; ++v) {
+                    tma_load_4d(st + v * C::QSUB_BYTES, &tm_q, v * 64, i * C::ROWS, bh, 0, bar_full + 8 * s);
+                    tma_load_4d(st + C::Q_BYTES + v * C::SSUB_BYTES, &tm_sh, v * 64, 0, bh, 0, bar_full + 8 * s);
+                    tma_load_4d(st + C::Q_BYTES + C::S_BYTES + v * C::SSUB_BYTES, &tm_sl, v * 64, 0, bh, 0, bar_full + 8 * s);
+                }
+            }
+            if (!ok) {
+                const long long t0 = clock64();
+                while (clock64() - t0 < 400000) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ================================================================= MMA issuer (warp-uniform, one elected lane issues)
+        constexpr uint32_t IDESC = idesc_bf16(D, true);
+        bool ok = true;
+        for (int n = 0; ok && n < my_units; ++n) {
+            const int s = n & 1;
+            const uint32_t par = (n >> 1) & 1;
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_afull + 8 * s, par, abort_flag, p.dev_status, 43)))) break;
+            if (n >= 2 && !(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_dfree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 44)))) break;
+            // the unit's S' tiles arrived with its Q tile; this warp takes its own acquire on the barrier the copies
+            // (made by the async proxy) completed on
+            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_full + 8 * s, par, abort_flag, p.dev_status, 45)))) break;
+            fence_after_sync();
+            if (elect_one()) {
+                const uint32_t tD = tmem + s * D, tA = tmem + 2 * D + s * D;
+                const uint32_t st = s_base + s * C::STAGE_BYTES;
+                const uint64_t dsh = smem_desc_sw128(st + C::Q_BYTES, C::SSUB_BYTES, 1024);
+                const uint64_t dsl = smem_desc_sw128(st + C::Q_BYTES + C::S_BYTES, C::SSUB_BYTES, 1024);
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint64_t off = (uint64_t)(ks * (2048 >> 4));
+                    mma_ts(tD, tA + ks * 8, dsh + off, IDESC, ks > 0);              // phi_hi S'_hi
+                    mma_ts(tD, tA + D / 2 + ks * 8, dsh + off, IDESC, true);        // phi_lo S'_hi
+                    mma_ts(tD, tA + ks * 8, dsl + off, IDESC, true);                // phi_hi S'_lo
+                }
+                mma_commit(bar_dfull + 8 * s);
+                mma_commit(bar_afree + 8 * s);
+                mma_commit(bar_sfree + 8 * s);
+            }
+            __syncwarp();
+        }
+    } else {
+        // ================================================================= phi(Q) into tensor memory; epilogue one unit behind
+        const int row = threadIdx.x;                            // query row of the tile = TMEM lane
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        bool ok = true;
+        float den[2] = {0.f, 0.f};
+        auto convert = [&](int n) -> bool {                     // A operand of unit n; den[n & 1] = phi(q_row) . z
+            const int u = blockIdx.x + n * gridDim.x;
+            const int bh = u / p.Tm;
+            const int s = n & 1;
+            const uint32_t par = (n >> 1) & 1;
+            // z and bias of the unit's head, staged by these threads once every thread has left the epilogue that read
+            // the buffer last (two units ago)
+            float* vec = reinterpret_cast<float*>(s_gen + C::OFF_VEC + s * 2 * D * 4);
+            if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_dfree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 50))) return false;
+            if (row < D) {
+                vec[row] = p.z[(size_t)bh * D + row];
+                vec[D + row] = p.bias ? __bfloat162float(p.bias[(size_t)(bh % p.heads) * D + row]) : 0.f;
+            }
+            mbar_arrive(bar_vec + 8 * s);
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_vec + 8 * s, par, abort_flag, p.dev_status, 46))) return false;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, par, abort_flag, p.dev_status, 47))) return false;
+            if (n >= 2) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar_afree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 48))) return false;
+                fence_after_sync();
+            }
+            const uint8_t* qt = s_gen + s * C::STAGE_BYTES + row * 128;
+            const uint32_t tA = lane_base + 2 * D + s * D;
+            float dsum = 0.f;
+#pragma unroll
+            for (int g = 0; g < D / 32; ++g) {                  // 32 features per pass: 16 packed hi + 16 packed lo registers
+                uint32_t hi[16], lo[16];
+#pragma unroll
+                for (int cc = 0; cc < 4; ++cc) {
+                    const int chunk = g * 4 + cc;               // 16-byte chunk of the row (8 features)
+                    const int sub = chunk >> 3, phys = (chunk & 7) ^ (row & 7);
+                    const uint4 w = *reinterpret_cast<const uint4*>(qt + sub * C::QSUB_BYTES + phys * 16);
+                    const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 x = unpack_bf16(ws[e]);
+                        const float f0 = phi_elu1(x.x), f1 = phi_elu1(x.y);
+                        const int feat = chunk * 8 + 2 * e;
+                        dsum = fmaf(f0, vec[feat], fmaf(f1, vec[feat + 1], dsum));
+                        const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
+                        hi[cc * 4 + e] = pack_bf16(f0, f1);
+                        lo[cc * 4 + e] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                    }
+                }
+                tmem_st16(tA + g * 16, hi);
+                tmem_st16(tA + D / 2 + g * 16, lo);
+            }
+            den[s] = dsum;
+            tmem_wait_st();
+            fence_before_sync();
+            mbar_arrive(bar_afull + 8 * s);
+            mbar_arrive(bar_qfree + 8 * s);
+            return true;
+        };
+        auto epilogue = [&](int n) -> bool {
+            const int u = blockIdx.x + n * gridDim.x;
+            const int bh = u / p.Tm, i = u - bh * p.Tm;
+            const int s = n & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar_dfull + 8 * s, (n >> 1) & 1, abort_flag, p.dev_status, 49))) return false;
+            fence_after_sync();
+            const float* vec = reinterpret_cast<const float*>(s_gen + C::OFF_VEC + s * 2 * D * 4);
+            const float inv = 1.f / (den[s] + p.eps);
+            const int r_glob = i * C::ROWS + row;
+            const bool valid = r_glob < p.Tc;
+            const size_t g = ((size_t)bh * p.Tc + r_glob) * D;
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(lane_base + s * D + c * 32, r);
+                tmem_wait_ld();
+                if (valid) {
+                    float x[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) x[e] = fmaf(__uint_as_float(r[e]), inv, vec[D + c * 32 + e]);
+                    if (p.out_f32) {
+                        float4* dst = reinterpret_cast<float4*>(p.out_f32 + g + c * 32);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) dst[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
+                    } else {
+                        uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + g + c * 32);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            dst[v] = make_uint4(pack_bf16(x[8 * v], x[8 * v + 1]), pack_bf16(x[8 * v + 2], x[8 * v + 3]),
+                                                pack_bf16(x[8 * v + 4], x[8 * v + 5]), pack_bf16(x[8 * v + 6], x[8 * v + 7]));
+                    }
+                }
+            }
+            fence_before_sync();
+            mbar_arrive(bar_dfree + 8 * s);
+            return true;
+        };
+        if (my_units > 0) ok = convert(0);
+        for (int n = 0; ok && n < my_units; ++n) {
+            if (n + 1 < my_units && !(ok = convert(n + 1))) break;
+            ok = epilogue(n);
+        }
+    }
+    fence_before_sync();
+    __syncthreads();
+    if (warp == 5) {
+        fence_after_sync();
+        tmem_dealloc(tmem, C::TMEM_COLS);
+    }
+}
