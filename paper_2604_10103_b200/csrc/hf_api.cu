@@ -192,7 +192,7 @@ hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
 
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
-    k_reduce_fold<D><<<dim3(D / 8, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, L.has_w ? L.W : nullptr, c->cfg.heads,
+    k_reduce_fold<D><<<dim3(D / 4, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, L.has_w ? L.W : nullptr, c->cfg.heads,
                                                       L.sf_hi, L.sf_lo);
     return post_launch(c, "k_reduce_fold");
 }

@@ -128,61 +128,72 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
     }
 }
 
-// grid (D/8, B*H), D threads.  Adds the nsplit partials of a (batch, head) to S (rows a0 .. a0+7 per block) and z
+// grid (D/4, B*H), D threads.  Adds the nsplit partials of a (batch, head) to S (rows a0 .. a0+3 per block) and z
 // (block 0) in ascending split order, then folds the updated rows: Sf = S W_h^T (or S when W == nullptr) as bf16
 // hi and lo halves.  nsplit == 0: fold only.  sf_hi == nullptr: state update only.
+// Thread c' owns output column c': its row of W_h is fetched first (all loads in flight while the partials are summed).
 template <int D>
 __global__ void __launch_bounds__(D)
 k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict__ S, float* __restrict__ z,
               const bf16* __restrict__ W, int heads, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
-    constexpr int ROWS = 8;
+    constexpr int ROWS = 4;
     constexpr int PART_FLOATS = D * D + D;
     __shared__ float rows[ROWS][D];
     const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, h = bh % heads;
     const int cp = threadIdx.x;
+    const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr;
+    uint4 wq[D / 8];
+    if (with_w) {
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + ((size_t)h * D + cp) * D);     // W_h[c'][.]
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
+    }
     const float* base = partials + (size_t)bh * nsplit * PART_FLOATS;
     float sum[ROWS];
 #pragma unroll
-    for (int r = 0; r < ROWS; ++r) sum[r] = 0.f;
-    for (int s = 0; s < nsplit; ++s) {
+    for (int r = 0; r < ROWS; ++r) sum[r] = S[((size_t)bh * D + a0 + r) * D + cp];
+    float zsum = 0.f;
+    const bool do_z = blockIdx.x == 0 && nsplit > 0;
+    if (do_z) zsum = z[(size_t)bh * D + cp];
+#pragma unroll 8
+    for (int s = 0; s < nsplit; ++s) {      // ascending split order per element; several splits' loads in flight
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) sum[r] += __ldcg(base + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+        if (do_z) zsum += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
     }
+    if (nsplit > 0) {
 #pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-        float* dst = S + ((size_t)bh * D + a0 + r) * D + cp;
-        const float v = *dst + sum[r];
-        if (nsplit > 0) *dst = v;
-        rows[r][cp] = v;
+        for (int r = 0; r < ROWS; ++r) S[((size_t)bh * D + a0 + r) * D + cp] = sum[r];
+        if (do_z) z[(size_t)bh * D + cp] = zsum;
     }
-    if (blockIdx.x == 0 && nsplit > 0) {
-        float zsum = 0.f;
-        for (int s = 0; s < nsplit; ++s) zsum += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
-        z[(size_t)bh * D + cp] += zsum;
-    }
-    if (sf_hi == nullptr) return;
-    __syncthreads();
+    if (!fold) return;
     float out[ROWS];
-    if (W == nullptr) {
+    if (!with_w) {
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) out[r] = rows[r][cp];
+        for (int r = 0; r < ROWS; ++r) out[r] = sum[r];
     } else {
 #pragma unroll
+        for (int r = 0; r < ROWS; ++r) rows[r][cp] = sum[r];
+        __syncthreads();
+#pragma unroll
         for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
-        const bf16* wrow = W + ((size_t)h * D + cp) * D;     // W_h[c'][.]
-#pragma unroll 4
-        for (int c = 0; c < D; c += 8) {
-            const uint4 u = __ldg(reinterpret_cast<const uint4*>(wrow + c));
+#pragma unroll
+        for (int i = 0; i < D / 8; ++i) {
             float w[8];
             float2 t;
-            t = unpack_bf16(u.x); w[0] = t.x; w[1] = t.y;
-            t = unpack_bf16(u.y); w[2] = t.x; w[3] = t.y;
-            t = unpack_bf16(u.z); w[4] = t.x; w[5] = t.y;
-            t = unpack_bf16(u.w); w[6] = t.x; w[7] = t.y;
+            t = unpack_bf16(wq[i].x); w[0] = t.x; w[1] = t.y;
+            t = unpack_bf16(wq[i].y); w[2] = t.x; w[3] = t.y;
+            t = unpack_bf16(wq[i].z); w[4] = t.x; w[5] = t.y;
+            t = unpack_bf16(wq[i].w); w[6] = t.x; w[7] = t.y;
 #pragma unroll
-            for (int r = 0; r < ROWS; ++r)
-#pragma unroll
-                for (int e = 0; e < 8; ++e) out[r] = fmaf(rows[r][c + e], w[e], out[r]);
+            for (int r = 0; r < ROWS; ++r) {
+                const float4 s0 = *reinterpret_cast<const float4*>(&rows[r][i * 8]);
+                const float4 s1 = *reinterpret_cast<const float4*>(&rows[r][i * 8 + 4]);
+                out[r] = fmaf(s0.x, w[0], out[r]); out[r] = fmaf(s0.y, w[1], out[r]);
+                out[r] = fmaf(s0.z, w[2], out[r]); out[r] = fmaf(s0.w, w[3], out[r]);
+                out[r] = fmaf(s1.x, w[4], out[r]); out[r] = fmaf(s1.y, w[5], out[r]);
+                out[r] = fmaf(s1.z, w[6], out[r]); out[r] = fmaf(s1.w, w[7], out[r]);
+            }
         }
     }
 #pragma unroll

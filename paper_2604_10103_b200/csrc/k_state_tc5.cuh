@@ -23,8 +23,13 @@ struct AbsorbTc5 {
     static constexpr int VSUB_BYTES = TT * 128;          // one 64-column sub-tile of V, 128-byte swizzle
     static constexpr int V_BYTES = SUB * VSUB_BYTES;
     static constexpr int OFF_K = 0, OFF_V = NST * K_BYTES, OFF_BAR = OFF_V + NST * V_BYTES;
-    static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
-    static constexpr int THREADS = 192;                  // warps 0-3: phi / epilogue, warp 4: TMA, warp 5: MMA
+    static constexpr int NQ = 4;                         // phi warps per TMEM lane quadrant: each converts TT / NQ tokens of a tile
+    static constexpr int OFF_Z = OFF_BAR + 256;          // z partials of the warps of a quadrant, [NQ][D] floats
+    static constexpr int SMEM_BYTES = OFF_Z + NQ * D * 4 + 1024;
+    static constexpr int THREADS = 128 * NQ + 64;        // phi / epilogue warps, then one TMA warp and one MMA warp
+    static constexpr int WARP_TMA = 4 * NQ, WARP_MMA = 4 * NQ + 1;
+    static constexpr int OUT_STRIDE = D + 4;             // floats; padded row of the epilogue's staging tile (reuses the K / V stages)
+    static_assert(D * OUT_STRIDE * 4 <= OFF_BAR, "staging tile must fit in the pipeline stages");
     static constexpr int TMEM_COLS = 256;                // D accumulator [0, D) ; A buffers at 128 + 64 b: hi 32 cols, lo 32 cols
     static constexpr int COL_A = 128;
     static constexpr int PART_FLOATS = D * D + D;
@@ -47,9 +52,10 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t sK = s_base + C::OFF_K, sV = s_base + C::OFF_V, bar0 = s_base + C::OFF_BAR;
     const uint32_t bar_full = bar0, bar_kfree = bar0 + 32, bar_vfree = bar0 + 64, bar_afull = bar0 + 96, bar_afree = bar0 + 112,
-                   bar_dfull = bar0 + 128;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 144);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 148);
+                   bar_dfull = bar0 + 128, bar_z = bar0 + 136, bar_st = bar0 + 152;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 160);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 164);
+    float* z_x = reinterpret_cast<float*>(s_gen + C::OFF_Z);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int split = blockIdx.x, nsplit = gridDim.x, bh = blockIdx.y;
@@ -59,13 +65,13 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
     const int n_local = tile_hi - tile_lo;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_kfree + 8 * s, D); mbar_init(bar_vfree + 8 * s, 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(bar_afull + 8 * s, D); mbar_init(bar_afree + 8 * s, 1); }
-        mbar_init(bar_dfull, 1);
+        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_kfree + 8 * s, C::NQ * D); mbar_init(bar_vfree + 8 * s, 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(bar_afull + 8 * s, C::NQ * D); mbar_init(bar_afree + 8 * s, 1); }
+        mbar_init(bar_dfull, 1); mbar_init(bar_z, C::NQ * D); mbar_init(bar_st, 128 * C::NQ);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
         tmem_relinquish();
     }
@@ -74,7 +80,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == C::WARP_TMA) {
         // ================================================================= TMA producer
         if (lane == 0) {
             bool ok = true;
@@ -97,7 +103,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
                 while (clock64() - t0 < 400000) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == C::WARP_MMA) {
         // ================================================================= MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t IDESC = idesc_bf16(D, true);
         const uint64_t dv0 = smem_desc_sw128(sV, C::VSUB_BYTES, 1024);
@@ -124,9 +130,13 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
         }
     } else {
         // ================================================================= phi(K) into tensor memory, then the epilogue
-        const int a = threadIdx.x;                              // key feature = TMEM lane
+        // NQ warps per TMEM lane quadrant: warps w, w + 4, ... own the same 32 key features (lanes) and convert
+        // consecutive groups of TT / NQ tokens of a tile.
+        const int part = warp >> 2;
+        const int a = (warp & 3) * 32 + lane;                   // key feature = TMEM lane
         const bool active = a < D;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        constexpr int HT = C::TT / C::NQ;                       // tokens per thread and tile
         bool ok = true;
         float zacc = 0.f;
         for (int i = 0; ok && i < n_local; ++i) {
@@ -139,53 +149,81 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
                 fence_after_sync();
             }
             if (active) {
-                const int nv = min(C::TT, p.n_tokens - (tile_lo + i) * C::TT);      // rows past the end read as zero: phi(0) = 1 must not count
-                const uint8_t* kt = s_gen + C::OFF_K + s * C::K_BYTES + a * 2;
-                uint32_t hi[C::TT / 2], lo[C::TT / 2];
+                // rows past the end of the tensor read as zero: phi(0) = 1 must not count
+                const int nv = min(C::TT, p.n_tokens - (tile_lo + i) * C::TT) - part * HT;
+                const uint8_t* kt = s_gen + C::OFF_K + s * C::K_BYTES + (size_t)(part * HT) * D * 2 + a * 2;
+                uint32_t hi[HT / 2], lo[HT / 2];
 #pragma unroll
-                for (int t = 0; t < C::TT; t += 2) {
+                for (int t = 0; t < HT; t += 2) {
                     const float x0 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)t * D * 2)) << 16);
                     const float x1 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)(t + 1) * D * 2)) << 16);
                     float f0 = phi_elu1(x0), f1 = phi_elu1(x1);
-                    if (t >= nv) f0 = 0.f;
-                    if (t + 1 >= nv) f1 = 0.f;
+                    if (nv < HT) {                              // only the tensor's last tile
+                        if (t >= nv) f0 = 0.f;
+                        if (t + 1 >= nv) f1 = 0.f;
+                    }
                     zacc += f0 + f1;
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
-                    hi[t >> 1] = pack_bf16(f0, f1);
-                    lo[t >> 1] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                    const uint32_t hp = pack_bf16(f0, f1);
+                    const float2 hf = unpack_bf16(hp);
+                    hi[t >> 1] = hp;
+                    lo[t >> 1] = pack_bf16(f0 - hf.x, f1 - hf.y);
                 }
-                const uint32_t tA = lane_base + C::COL_A + ab * 64;
-                tmem_st32(tA, hi);
-                tmem_st32(tA + 32, lo);
+                const uint32_t tA = lane_base + C::COL_A + ab * 64 + part * (HT / 2);
+                tmem_st8(tA, hi);
+                tmem_st8(tA + 32, lo);
                 tmem_wait_st();
                 fence_before_sync();
                 mbar_arrive(bar_afull + 8 * ab);
                 mbar_arrive(bar_kfree + 8 * s);
             }
         }
+        // ---- epilogue: the accumulator goes through a padded staging tile in shared memory (the pipeline stages are
+        // idle by now: every TMA copy has been consumed) so that the partial is written with coalesced stores
+        if (ok && active) {
+            z_x[part * D + a] = zacc;
+            mbar_arrive(bar_z);
+        }
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_dfull, 0, abort_flag, p.dev_status, 37));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_z, 0, abort_flag, p.dev_status, 38));
+        float* stage_out = reinterpret_cast<float*>(s_gen);
+        if (ok && active) {
+            fence_after_sync();
+            constexpr int CW = D / C::NQ;                       // accumulator columns staged by this warp
+            static_assert(CW % 16 == 0, "column share must be a multiple of 16");
+#pragma unroll
+            for (int c = 0; c < CW / 16; ++c) {
+                const int col = part * CW + c * 16;
+                uint32_t r[16];
+                tmem_ld16(lane_base + col, r);
+                tmem_wait_ld();
+                float4* dst = reinterpret_cast<float4*>(stage_out + (size_t)a * C::OUT_STRIDE + col);
+#pragma unroll
+                for (int v = 0; v < 4; ++v)
+                    dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                         __uint_as_float(r[4 * v + 3]));
+            }
+        }
+        // all phi warps (active or not) meet before the staged tile is read back
+        mbar_arrive(bar_st);
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_st, 0, abort_flag, p.dev_status, 39));
         if (ok) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_dfull, 0, abort_flag, p.dev_status, 37));
-            if (ok && active) {
-                fence_after_sync();
-                float* part = p.partials + ((size_t)bh * nsplit + split) * C::PART_FLOATS;
-                part[D * D + a] = zacc;
+            float* part_out = p.partials + ((size_t)bh * nsplit + split) * C::PART_FLOATS;
+            const int tid = threadIdx.x;                        // 0 .. 128 NQ - 1
+            for (int e = tid; e < D * D / 4; e += 128 * C::NQ) {
+                const int rrow = e / (D / 4), c4 = e - rrow * (D / 4);
+                reinterpret_cast<float4*>(part_out)[e] = *reinterpret_cast<const float4*>(stage_out + (size_t)rrow * C::OUT_STRIDE + c4 * 4);
+            }
+            if (tid < D) {
+                float zs = z_x[tid];
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(lane_base + c * 32, r);
-                    tmem_wait_ld();
-                    float4* dst = reinterpret_cast<float4*>(part + (size_t)a * D + c * 32);
-#pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
-                                             __uint_as_float(r[4 * v + 3]));
-                }
+                for (int q = 1; q < C::NQ; ++q) zs += z_x[q * D + tid];
+                part_out[D * D + tid] = zs;
             }
         }
     }
     fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         fence_after_sync();
         tmem_dealloc(tmem, C::TMEM_COLS);
     }
@@ -194,19 +232,23 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
 // ------------------------------------------------------------------------------------------------------------
 // Read-out.  Unit = (batch*head, tile of 128 query rows).  A = phi(Q): M = query row (lane), K = key feature.
 // B = S' [a][c] (N = c contiguous, MN-major), hi and lo halves.  D = A_hi S'_hi + A_lo S'_hi + A_hi S'_lo.
+// A thread block takes a contiguous run of units, so that S' is fetched once per (batch, head) it touches
+// ("epoch"), into one of two buffers.
 // ------------------------------------------------------------------------------------------------------------
 template <int D>
 struct ReadoutTc5 {
     static constexpr int ROWS = 128;
-    static constexpr int NST = 2;                        // unit stages: {Q tile, S' hi, S' lo}
+    static constexpr int NST = 2;                        // Q stages; S' {hi, lo} buffers likewise two
     static constexpr int SUB = D / 64;
     static constexpr int QSUB_BYTES = ROWS * 128, Q_BYTES = SUB * QSUB_BYTES;
     static constexpr int SSUB_BYTES = D * 128, S_BYTES = SUB * SSUB_BYTES;
-    static constexpr int STAGE_BYTES = Q_BYTES + 2 * S_BYTES;
-    static constexpr int OFF_VEC = NST * STAGE_BYTES;    // per stage: z [D] floats, bias [D] floats
-    static constexpr int OFF_BAR = OFF_VEC + NST * 2 * D * 4;
+    static constexpr int OFF_Q = 0, OFF_S = NST * Q_BYTES;   // S' buffer e at OFF_S + e * 2 * S_BYTES: hi then lo
+    static constexpr int OFF_VEC = OFF_S + 2 * 2 * S_BYTES;  // per stage: z [D] floats, bias [D] floats
+    static constexpr int OFF_DEN = OFF_VEC + NST * 2 * D * 4;   // per stage: denominator partials [2][128] floats
+    static constexpr int OFF_BAR = OFF_DEN + NST * 2 * ROWS * 4;
     static constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;
-    static constexpr int THREADS = 192;                  // warps 0-3: phi / epilogue, warp 4: TMA, warp 5: MMA
+    static constexpr int THREADS = 320;                  // warps 0-7: phi / epilogue (two per TMEM lane quadrant), warp 8: TMA, warp 9: MMA
+    static constexpr int WARP_TMA = 8, WARP_MMA = 9;
     static constexpr int TMEM_COLS = 4 * D;              // D accumulators at D b ; A buffers at 2 D + D b: hi D/2 cols, lo D/2 cols
 };
 
@@ -220,7 +262,7 @@ struct ReadoutTc5Params {
     int* dev_status;
 };
 
-// Persistent: CTA c processes units c, c + gridDim.x, ...  tm_q: [D, T_c, B*H, 1] box {64, 128};
+// CTA c processes units [c * upc, (c + 1) * upc), upc = ceil(n_units / gridDim.x).  tm_q: [D, T_c, B*H, 1] box {64, 128};
 // tm_sh, tm_sl: [D, D, B*H, 1] box {64, D}; all 128B swizzle.
 template <int D>
 __global__ void __launch_bounds__(ReadoutTc5<D>::THREADS, 1)
@@ -233,23 +275,25 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t bar0 = s_base + C::OFF_BAR;
     const uint32_t bar_full = bar0, bar_qfree = bar0 + 16, bar_sfree = bar0 + 32, bar_afull = bar0 + 48, bar_afree = bar0 + 64,
-                   bar_dfull = bar0 + 80, bar_dfree = bar0 + 96, bar_vec = bar0 + 112;
+                   bar_dfull = bar0 + 80, bar_dfree = bar0 + 96, bar_vec = bar0 + 112, bar_sfull = bar0 + 128;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 144);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 148);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int upc = (p.n_units + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int u0 = min((int)blockIdx.x * upc, p.n_units);
+    const int my_units = min(upc, p.n_units - u0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar_full + 8 * s, 1); mbar_init(bar_qfree + 8 * s, 128); mbar_init(bar_sfree + 8 * s, 1);
-            mbar_init(bar_afull + 8 * s, 128); mbar_init(bar_afree + 8 * s, 1); mbar_init(bar_dfull + 8 * s, 1);
-            mbar_init(bar_dfree + 8 * s, 128); mbar_init(bar_vec + 8 * s, 128);
+            mbar_init(bar_full + 8 * s, 1); mbar_init(bar_qfree + 8 * s, 256); mbar_init(bar_sfree + 8 * s, 1);
+            mbar_init(bar_afull + 8 * s, 256); mbar_init(bar_afree + 8 * s, 1); mbar_init(bar_dfull + 8 * s, 1);
+            mbar_init(bar_dfree + 8 * s, 256); mbar_init(bar_vec + 8 * s, 256); mbar_init(bar_sfull + 8 * s, 1);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
         tmem_relinquish();
     }
@@ -258,51 +302,61 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == C::WARP_TMA) {
         // ================================================================= TMA producer
         if (lane == 0) {
             bool ok = true;
+            int epoch = -1, bh_prev = -1;
             for (int n = 0; ok && n < my_units; ++n) {
-                const int u = blockIdx.x + n * gridDim.x;
+                const int u = u0 + n;
                 const int bh = u / p.Tm, i = u - bh * p.Tm;
                 const int s = n & 1;
-                const uint32_t par_free = ((n >> 1) & 1) ^ 1;
-                if (n >= 2) {
-                    if (!(ok = mbar_wait<true>(bar_qfree + 8 * s, par_free, abort_flag, p.dev_status, 41))) break;
-                    if (!(ok = mbar_wait<true>(bar_sfree + 8 * s, par_free, abort_flag, p.dev_status, 42))) break;
-                }
-                const uint32_t st = s_base + s * C::STAGE_BYTES;
-                mbar_expect_tx(bar_full + 8 * s, C::STAGE_BYTES);
+                if (bh != bh_prev) {                 // new (batch, head): its folded state, hi and lo halves
+                    bh_prev = bh; ++epoch;
+                    const int e = epoch & 1;
+                    if (epoch >= 2 && !(ok = mbar_wait<true>(bar_sfree + 8 * e, ((epoch >> 1) & 1) ^ 1, abort_flag, p.dev_status, 42))) break;
+                    const uint32_t sb = s_base + C::OFF_S + e * 2 * C::S_BYTES;
+                    mbar_expect_tx(bar_sfull + 8 * e, 2 * C::S_BYTES);
 #pragma unroll
-                for (int v = 0; v < C::SUB; ++v) {
-                    tma_load_4d(st + v * C::QSUB_BYTES, &tm_q, v * 64, i * C::ROWS, bh, 0, bar_full + 8 * s);
-                    tma_load_4d(st + C::Q_BYTES + v * C::SSUB_BYTES, &tm_sh, v * 64, 0, bh, 0, bar_full + 8 * s);
-                    tma_load_4d(st + C::Q_BYTES + C::S_BYTES + v * C::SSUB_BYTES, &tm_sl, v * 64, 0, bh, 0, bar_full + 8 * s);
+                    for (int v = 0; v < C::SUB; ++v) {
+                        tma_load_4d(sb + v * C::SSUB_BYTES, &tm_sh, v * 64, 0, bh, 0, bar_sfull + 8 * e);
+                        tma_load_4d(sb + C::S_BYTES + v * C::SSUB_BYTES, &tm_sl, v * 64, 0, bh, 0, bar_sfull + 8 * e);
+                    }
                 }
+                if (n >= 2 && !(ok = mbar_wait<true>(bar_qfree + 8 * s, ((n >> 1) & 1) ^ 1, abort_flag, p.dev_status, 41))) break;
+                const uint32_t st = s_base + C::OFF_Q + s * C::Q_BYTES;
+                mbar_expect_tx(bar_full + 8 * s, C::Q_BYTES);
+#pragma unroll
+                for (int v = 0; v < C::SUB; ++v)
+                    tma_load_4d(st + v * C::QSUB_BYTES, &tm_q, v * 64, i * C::ROWS, bh, 0, bar_full + 8 * s);
             }
             if (!ok) {
                 const long long t0 = clock64();
                 while (clock64() - t0 < 400000) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == C::WARP_MMA) {
         // ================================================================= MMA issuer (warp-uniform, one elected lane issues)
         constexpr uint32_t IDESC = idesc_bf16(D, true);
         bool ok = true;
+        int epoch = -1, bh_prev = -1;
         for (int n = 0; ok && n < my_units; ++n) {
             const int s = n & 1;
             const uint32_t par = (n >> 1) & 1;
+            const int bh = (u0 + n) / p.Tm;
+            if (bh != bh_prev) {
+                bh_prev = bh; ++epoch;
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_sfull + 8 * (epoch & 1), (epoch >> 1) & 1, abort_flag, p.dev_status, 45)))) break;
+            }
+            const bool last_of_epoch = (n + 1 == my_units) || ((u0 + n + 1) / p.Tm != bh);
             if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_afull + 8 * s, par, abort_flag, p.dev_status, 43)))) break;
             if (n >= 2 && !(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_dfree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 44)))) break;
-            // the unit's S' tiles arrived with its Q tile; this warp takes its own acquire on the barrier the copies
-            // (made by the async proxy) completed on
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_full + 8 * s, par, abort_flag, p.dev_status, 45)))) break;
             fence_after_sync();
             if (elect_one()) {
                 const uint32_t tD = tmem + s * D, tA = tmem + 2 * D + s * D;
-                const uint32_t st = s_base + s * C::STAGE_BYTES;
-                const uint64_t dsh = smem_desc_sw128(st + C::Q_BYTES, C::SSUB_BYTES, 1024);
-                const uint64_t dsl = smem_desc_sw128(st + C::Q_BYTES + C::S_BYTES, C::SSUB_BYTES, 1024);
+                const uint32_t sb = s_base + C::OFF_S + (epoch & 1) * 2 * C::S_BYTES;
+                const uint64_t dsh = smem_desc_sw128(sb, C::SSUB_BYTES, 1024);
+                const uint64_t dsl = smem_desc_sw128(sb + C::S_BYTES, C::SSUB_BYTES, 1024);
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint64_t off = (uint64_t)(ks * (2048 >> 4));
@@ -312,28 +366,33 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
                 mma_commit(bar_dfull + 8 * s);
                 mma_commit(bar_afree + 8 * s);
-                mma_commit(bar_sfree + 8 * s);
+                if (last_of_epoch) mma_commit(bar_sfree + 8 * (epoch & 1));
             }
             __syncwarp();
         }
     } else {
         // ================================================================= phi(Q) into tensor memory; epilogue one unit behind
-        const int row = threadIdx.x;                            // query row of the tile = TMEM lane
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        // Two warps per TMEM lane quadrant: warp w and w + 4 own the same 32 query rows (lanes); the lower one converts
+        // key features [0, D/2) and stores output columns [0, D/2), the upper one the other halves.  Loops over 32-wide
+        // chunks are kept rolled: the code stays small enough for the instruction cache.
+        const int half = warp >> 2;
+        const int row = (warp & 3) * 32 + lane;                 // query row of the tile = TMEM lane
+        const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
+        constexpr int PASSES = D / 64;                          // 32-feature (and 32-column) passes per thread
         bool ok = true;
-        float den[2] = {0.f, 0.f};
-        auto convert = [&](int n) -> bool {                     // A operand of unit n; den[n & 1] = phi(q_row) . z
-            const int u = blockIdx.x + n * gridDim.x;
+        auto convert = [&](int n) -> bool {                     // A operand of unit n; denominator partial of the half
+            const int u = u0 + n;
             const int bh = u / p.Tm;
             const int s = n & 1;
             const uint32_t par = (n >> 1) & 1;
             // z and bias of the unit's head, staged by these threads once every thread has left the epilogue that read
-            // the buffer last (two units ago)
+            // the stage's buffers last (two units ago)
             float* vec = reinterpret_cast<float*>(s_gen + C::OFF_VEC + s * 2 * D * 4);
+            float* den_x = reinterpret_cast<float*>(s_gen + C::OFF_DEN + s * 2 * C::ROWS * 4);
             if (n >= 2 && !__all_sync(0xffffffffu, mbar_wait(bar_dfree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 50))) return false;
-            if (row < D) {
-                vec[row] = p.z[(size_t)bh * D + row];
-                vec[D + row] = p.bias ? __bfloat162float(p.bias[(size_t)(bh % p.heads) * D + row]) : 0.f;
+            if (threadIdx.x < D) {
+                vec[threadIdx.x] = p.z[(size_t)bh * D + threadIdx.x];
+                vec[D + threadIdx.x] = p.bias ? __bfloat162float(p.bias[(size_t)(bh % p.heads) * D + threadIdx.x]) : 0.f;
             }
             mbar_arrive(bar_vec + 8 * s);
             if (!__all_sync(0xffffffffu, mbar_wait(bar_vec + 8 * s, par, abort_flag, p.dev_status, 46))) return false;
@@ -342,11 +401,12 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 if (!__all_sync(0xffffffffu, mbar_wait(bar_afree + 8 * s, par ^ 1u, abort_flag, p.dev_status, 48))) return false;
                 fence_after_sync();
             }
-            const uint8_t* qt = s_gen + s * C::STAGE_BYTES + row * 128;
+            const uint8_t* qt = s_gen + C::OFF_Q + s * C::Q_BYTES + row * 128;
             const uint32_t tA = lane_base + 2 * D + s * D;
             float dsum = 0.f;
-#pragma unroll
-            for (int g = 0; g < D / 32; ++g) {                  // 32 features per pass: 16 packed hi + 16 packed lo registers
+#pragma unroll 1
+            for (int gi = 0; gi < PASSES; ++gi) {               // 32 features per pass: 16 packed hi + 16 packed lo registers
+                const int g = half * PASSES + gi;
                 uint32_t hi[16], lo[16];
 #pragma unroll
                 for (int cc = 0; cc < 4; ++cc) {
@@ -360,15 +420,16 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         const float f0 = phi_elu1(x.x), f1 = phi_elu1(x.y);
                         const int feat = chunk * 8 + 2 * e;
                         dsum = fmaf(f0, vec[feat], fmaf(f1, vec[feat + 1], dsum));
-                        const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
-                        hi[cc * 4 + e] = pack_bf16(f0, f1);
-                        lo[cc * 4 + e] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
+                        const uint32_t hp = pack_bf16(f0, f1);
+                        const float2 hf = unpack_bf16(hp);
+                        hi[cc * 4 + e] = hp;
+                        lo[cc * 4 + e] = pack_bf16(f0 - hf.x, f1 - hf.y);
                     }
                 }
                 tmem_st16(tA + g * 16, hi);
                 tmem_st16(tA + D / 2 + g * 16, lo);
             }
-            den[s] = dsum;
+            den_x[half * C::ROWS + row] = dsum;
             tmem_wait_st();
             fence_before_sync();
             mbar_arrive(bar_afull + 8 * s);
@@ -376,31 +437,35 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             return true;
         };
         auto epilogue = [&](int n) -> bool {
-            const int u = blockIdx.x + n * gridDim.x;
+            const int u = u0 + n;
             const int bh = u / p.Tm, i = u - bh * p.Tm;
             const int s = n & 1;
+            // the accumulator is complete; its MMAs were issued after every phi thread of the unit had arrived (and
+            // published its denominator partial), so the partials of both halves are visible here
             if (!__all_sync(0xffffffffu, mbar_wait(bar_dfull + 8 * s, (n >> 1) & 1, abort_flag, p.dev_status, 49))) return false;
             fence_after_sync();
             const float* vec = reinterpret_cast<const float*>(s_gen + C::OFF_VEC + s * 2 * D * 4);
-            const float inv = 1.f / (den[s] + p.eps);
+            const float* den_x = reinterpret_cast<const float*>(s_gen + C::OFF_DEN + s * 2 * C::ROWS * 4);
+            const float inv = 1.f / (den_x[row] + den_x[C::ROWS + row] + p.eps);
             const int r_glob = i * C::ROWS + row;
             const bool valid = r_glob < p.Tc;
             const size_t g = ((size_t)bh * p.Tc + r_glob) * D;
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+#pragma unroll 1
+            for (int ci = 0; ci < PASSES; ++ci) {
+                const int col = half * (D / 2) + ci * 32;
                 uint32_t r[32];
-                tmem_ld32(lane_base + s * D + c * 32, r);
+                tmem_ld32(lane_base + s * D + col, r);
                 tmem_wait_ld();
                 if (valid) {
                     float x[32];
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) x[e] = fmaf(__uint_as_float(r[e]), inv, vec[D + c * 32 + e]);
+                    for (int e = 0; e < 32; ++e) x[e] = fmaf(__uint_as_float(r[e]), inv, vec[D + col + e]);
                     if (p.out_f32) {
-                        float4* dst = reinterpret_cast<float4*>(p.out_f32 + g + c * 32);
+                        float4* dst = reinterpret_cast<float4*>(p.out_f32 + g + col);
 #pragma unroll
                         for (int v = 0; v < 8; ++v) dst[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
                     } else {
-                        uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + g + c * 32);
+                        uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + g + col);
 #pragma unroll
                         for (int v = 0; v < 4; ++v)
                             dst[v] = make_uint4(pack_bf16(x[8 * v], x[8 * v + 1]), pack_bf16(x[8 * v + 2], x[8 * v + 3]),
@@ -420,7 +485,7 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     fence_before_sync();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == C::WARP_MMA) {
         fence_after_sync();
         tmem_dealloc(tmem, C::TMEM_COLS);
     }
