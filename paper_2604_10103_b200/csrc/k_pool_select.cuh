@@ -98,34 +98,35 @@ __global__ void __launch_bounds__(128) k_select(ChunkTable tab, const float* __r
     const size_t row = (size_t)bh * Tm + i;
     if (threadIdx.x < D) sq[threadIdx.x] = pooled_q[row * D + threadIdx.x];
     __syncthreads();
-    // four scores per pass and warp: the sixteen loads of a lane are issued before any of them is used
-    for (int j0 = warp; j0 < Tn; j0 += 16) {
-        float kv[4][D / 32];
+    // One thread per key block: the 32 partials and the butterfly of the canonical order are formed by that thread
+    // alone.  The shuffle butterfly p[l] + p[l ^ off] gives both partners the same value (IEEE addition commutes), so
+    // folding the upper half onto the lower half level by level yields lane 0's result bit for bit.
+    for (int j = threadIdx.x; j < Tn; j += 128) {
+        const int c = j / n_b, jb = j - c * n_b;
+        const float4* kp = reinterpret_cast<const float4*>(tab.pooled[c] + ((size_t)bh * n_b + jb) * D);
+        float pl[32];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + 4 * u;
-            if (j < Tn) {
-                const int c = j / n_b, jb = j - c * n_b;
-                const float* kp = tab.pooled[c] + ((size_t)bh * n_b + jb) * D;
+        for (int m = 0; m < D / 32; ++m) {
+            float4 kv[8];
 #pragma unroll
-                for (int m = 0; m < D / 32; ++m) kv[u][m] = __ldg(kp + lane + 32 * m);
-            }
-        }
+            for (int i = 0; i < 8; ++i) kv[i] = __ldg(kp + m * 8 + i);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int j = j0 + 4 * u;
-            if (j < Tn) {
-                float acc = __fmul_rn(sq[lane], kv[u][0]);
+            for (int i = 0; i < 8; ++i) {
+                const float kk[4] = {kv[i].x, kv[i].y, kv[i].z, kv[i].w};
 #pragma unroll
-                for (int m = 1; m < D / 32; ++m) acc = __fadd_rn(acc, __fmul_rn(sq[lane + 32 * m], kv[u][m]));
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-                if (lane == 0) {
-                    sc[j] = acc;
-                    if (scores_out) scores_out[row * Tn + j] = acc;
+                for (int e = 0; e < 4; ++e) {
+                    const int l = 4 * i + e;
+                    const float pr = __fmul_rn(sq[l + 32 * m], kk[e]);
+                    pl[l] = (m == 0) ? pr : __fadd_rn(pl[l], pr);
                 }
             }
         }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+            for (int l = 0; l < off; ++l) pl[l] = __fadd_rn(pl[l], pl[l + off]);
+        sc[j] = pl[0];
+        if (scores_out) scores_out[row * Tn + j] = pl[0];
     }
     __syncthreads();
     for (int j = threadIdx.x; j < Tn; j += 128) {
