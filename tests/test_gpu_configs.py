@@ -1,0 +1,115 @@
+"""GPU parity at the workload level: the long stream (state drift), the full-depth stack and a subset of the
+sweep grid, all at the 832x480 latent shape (1560 tokens per latent frame, 3-frame chunks).  The oracle is
+evaluated on sampled query blocks where a full evaluation would take minutes; masks are compared in full."""
+import numpy as np
+import pytest
+
+from paper_2604_10103_b200 import inputs as gen
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+
+f64 = gen.bf16_bits_to_f64
+
+
+def check_forward(gpu, ora, w, layer, chunk, step, q_blocks, what):
+    """Select + forward of one denoising step on both sides; masks in full, outputs on q_blocks."""
+    qb, kb, vb = gen.qkv(w, layer, chunk, step)
+    q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+    m_gpu, _, sc_gpu = gpu.select(q, k)
+    m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+    assert np.array_equal(sc_gpu, sc_ref), f"{what}: scores differ in {np.sum(sc_gpu != sc_ref)} places"
+    assert np.array_equal(m_gpu, m_ref), f"{what}: masks differ"
+    o_ref = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, q_blocks=q_blocks)
+    return hz.assert_close_out(gpu.forward(q, k, v), o_ref, what)
+
+
+def test_stream_200_chunks_state_drift():
+    """200 consecutive chunks of one layer, one 3-frame chunk evicted into the state per chunk once the window is
+    full: final (S, z) within rel-L2 1e-4 of the fp64 recurrence; outputs and masks checked every 25th chunk."""
+    w = gen.stream_832x480(chunks=200)
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        worst = 0.0
+        for c in range(w.chunks):
+            if c % 25 == 24 or c == w.chunks - 1:
+                _, rl = check_forward(gpu, ora, w, 0, c, 0, [0, 36], f"chunk {c}")
+                worst = max(worst, rl)
+                S, z = gpu.state()
+                assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2, f"chunk {c}: S rel-L2 {hz.rel_l2(S, ora.S):.3e}"
+                assert hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc))
+            ora.append(f64(kc), f64(vc))
+        S, z = gpu.state()
+        assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_ABSORBED_TOKENS) == ora.absorbed_tokens == 198 * w.chunk_tokens
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2, f"final S rel-L2 {hz.rel_l2(S, ora.S):.3e}"
+        assert hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2, f"final z rel-L2 {hz.rel_l2(z, ora.z):.3e}"
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
+
+
+def test_full_depth_stack_three_layers_verified():
+    """30 layer states in one context, 4 denoising-step forwards and one cache commit per chunk; layers are
+    independent, so three of them (first, middle, last) are followed by the oracle through 4 chunks and every
+    step of the last chunk is compared."""
+    w = gen.full_depth_832x480(layers=30, steps=4, chunks=4)
+    layers = [0, 14, 29]
+    from paper_2604_10103_b200 import binding as hf
+    base = hz.GpuStream(w, layer=layers[0], layers=w.layers)      # one context holds all 30 layer states
+    oras = {l: hz.make_oracle(w, layer=l) for l in layers}
+    try:
+        for l in layers[1:]:
+            Wb, bb = gen.merge_weights(w, l)
+            base.ctx.hf_set_merge_weights(l, hf.bits_to_cuda(Wb), hf.bits_to_cuda(bb))
+        filler_k, filler_v = (base.up(t) for t in gen.clean_kv(w, 999, 0))
+        for c in range(w.chunks):
+            for l in range(w.layers):
+                if l in layers:
+                    base.layer = l
+                    if c == w.chunks - 1:
+                        for s in range(w.steps):
+                            check_forward(base, oras[l], w, l, c, s, [5, 36], f"layer {l} chunk {c} step {s}")
+                    kc, vc = gen.clean_kv(w, l, c)
+                    base.ctx.hf_kv_append(l, base.up(kc), base.up(vc))
+                    oras[l].append(f64(kc), f64(vc))
+                else:       # the other layers only carry their share of the cache traffic
+                    base.ctx.hf_kv_append(l, filler_k, filler_v)
+        for l in layers:
+            base.layer = l
+            S, z = base.state()
+            assert hz.rel_l2(S, oras[l].S) <= hz.STATE_REL_L2 and hz.rel_l2(z, oras[l].z) <= hz.STATE_REL_L2
+            assert base.ctx.hf_query(l, hf.HF_Q_ABSORBED_TOKENS) == oras[l].absorbed_tokens
+        assert base.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        base.close()
+
+
+SWEEP_SUBSET = [
+    # keep permille, window frames, head_dim, block, batch
+    (100, 3, 64, 64, 4),      # window == chunk: every committed chunk goes straight into the state
+    (500, 21, 128, 128, 1),   # longest window: six cached chunks
+    (1000, 9, 64, 128, 1),    # everything kept: dense attention over the window, head_dim 64 on the tcgen05 path
+    (250, 9, 128, 64, 4),     # 64-token blocks (warp-level tensor path), batch 4
+    (100, 9, 128, 128, 1),    # sparsest setting of the grid
+]
+
+
+@pytest.mark.parametrize("permille,window,d,blk,batch", SWEEP_SUBSET)
+def test_sweep_subset(permille, window, d, blk, batch):
+    w = gen.layer_832x480().with_(name="sweep", keep_permille=permille, window_frames=window, head_dim=d, block=blk,
+                                  batch=batch, heads=12 if batch == 1 else 3, seed=5)
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        n_prime = w.past_chunks + 2            # window full and at least two chunks in the state
+        for c in range(n_prime):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        last = w.blocks_per_chunk - 1
+        check_forward(gpu, ora, w, 0, n_prime, 0, [1, last], f"sweep point {permille}/{window}/{d}/{blk}/{batch}")
+        S, z = gpu.state()
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2 and hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
