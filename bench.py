@@ -27,9 +27,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2604_10103_b200 import inputs as gen  # noqa: E402
+from paper_2604_10103_b200 import inputs as gen, replicas  # noqa: E402
 
 METRIC = "hybrid-attn latent frames/s at 832x480 shape"
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_swa_tc5 launch at this workload's layer shape, from the ncu
+# capture summarised in profiles/k_swa_tc5_layer_832x480.md; None when the kernel has changed since that capture.
+SWA_DRAM_BYTES_PER_LAUNCH = None
 UNIT = "latent frames/s"
 
 
@@ -166,7 +169,7 @@ def run_ours(args, w):
     ctx = hf.Context(hf.make_config(w), device=local)
     L, P = w.layers, w.past_chunks
     shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
-    g = torch.Generator(device="cuda"); g.manual_seed(1234 + rank)
+    g = torch.Generator(device="cuda"); g.manual_seed(replicas.replica_seed(1234, rank))
     rn = lambda: torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
     q = [rn() for _ in range(L)]; k = [rn() for _ in range(L)]; v = [rn() for _ in range(L)]
     kc = [rn() for _ in range(L)]; vc = [rn() for _ in range(L)]
@@ -206,10 +209,9 @@ def run_ours(args, w):
     ms = e0.elapsed_time(e1)
     launches = ctx.hf_launch_count() - n0
     clocks = sampler.stop() if rank == 0 else None
-    if world > 1:
-        t = torch.tensor([ms], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); ms = float(t.item())
+    ms, frames = replicas.aggregate(ms, args.steps * w.chunk_frames * w.batch)     # slowest rank, frames of all ranks
     ms_per_step = ms / args.steps
-    value = world * w.chunk_frames * w.batch / (ms_per_step * 1e-3)
+    value = replicas.throughput(frames, ms)
 
     # ---- per-stage split and the dominant kernel's launch time (CUDA events around batches of single-stage calls)
     def timed(fn, reps):
@@ -252,7 +254,8 @@ def run_ours(args, w):
         peak = peaks["bf16_tflops_sustained"]
         roof = {"bound": "tensor", "kernel": "sparse_swa", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
                 "peak_source": f"{peaks['source']} (sustained cuBLAS bf16; burst {peaks['bf16_tflops']})",
-                "frac_of_burst": ach / peaks["bf16_tflops"], "flops_per_launch": flops, "traffic": None}
+                "frac_of_burst": ach / peaks["bf16_tflops"], "frac_of_datasheet_2250": ach / 2250.0,
+                "flops_per_launch": flops, "traffic": SWA_DRAM_BYTES_PER_LAUNCH}
         bytes_absorb = 2 * w.batch * w.heads * w.chunk_tokens * w.head_dim * 2
         stage["absorb_gbs"] = bytes_absorb / (stage["absorb_us"] * 1e-6) / 1e9
         stage["absorb_frac_hbm"] = stage["absorb_gbs"] / peaks["hbm_gbs"]
@@ -278,10 +281,9 @@ def run_ours(args, w):
         step_host()
     barrier()
     t_e2e = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([t_e2e], device="cuda"); dist.all_reduce(t, op=dist.ReduceOp.MAX); t_e2e = float(t.item())
+    t_e2e_ms, frames_e2e = replicas.aggregate(t_e2e * 1e3, e2e_steps * w.chunk_frames * w.batch)
     nbytes = hq.numel() * 2
-    e2e = {"value": world * w.chunk_frames * w.batch * e2e_steps / t_e2e, "unit": UNIT,
+    e2e = {"value": replicas.throughput(frames_e2e, t_e2e_ms), "unit": UNIT,
            "h2d_bytes_per_step": L * (w.steps * 3 + 2) * nbytes, "d2h_bytes_per_step": L * w.steps * nbytes, "steps": e2e_steps}
     flags, detail = ctx.hf_get_device_status()
 
@@ -307,8 +309,8 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=30)
     ap.add_argument("--denoise-steps", type=int, default=4)

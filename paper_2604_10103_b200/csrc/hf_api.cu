@@ -272,13 +272,17 @@ hf_status launch_swa_mma_t(hf_ctx* c, const bf16* q, const ChunkTable& tab, cons
 
 
 #ifndef HF_TC5_GROUPS
-#define HF_TC5_GROUPS 2   // softmax column groups of the tcgen05 attention kernel
+#define HF_TC5_GROUPS 2   // softmax column groups of the tcgen05 attention kernel at head_dim 64
 #endif
+#ifndef HF_TC5_GROUPS_128
+#define HF_TC5_GROUPS_128 2   // ... and at head_dim 128
+#endif
+template <int D> struct Tc5Groups { static constexpr int N = (D == 128) ? HF_TC5_GROUPS_128 : HF_TC5_GROUPS; };
 
 template <int D>
 hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
                            int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
-    typedef SwaTc5<D, HF_TC5_GROUPS> C;
+    typedef SwaTc5<D, Tc5Groups<D>::N> C;
     CUtensorMap tq, tk, tv;
     HF_TRY(make_map(c, &tq, q, 1));
     HF_TRY(make_map(c, &tk, k_cur, 1));
@@ -292,7 +296,7 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
-    k_swa_tc5<D, HF_TC5_GROUPS><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    k_swa_tc5<D, Tc5Groups<D>::N><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
     return post_launch(c, "k_swa_tc5");
 }
 
@@ -420,8 +424,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = set_swa_attr<64, 128>();
         if (s == HF_OK) s = set_swa_attr<128, 64>();
         if (s == HF_OK) s = set_swa_attr<128, 128>();
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, HF_TC5_GROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, HF_TC5_GROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, HF_TC5_GROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, HF_TC5_GROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, Tc5Groups<64>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, Tc5Groups<64>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }
