@@ -68,6 +68,8 @@ struct hf_ctx {
     int nsplit_max = 1;
     bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
     int* dev_status = nullptr;
+    cudaStream_t side = nullptr;     // hf_hybrid_forward runs the history read-out here, beside pooling + selection
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     long long launches = 0;
     int swa_kernel = HF_SWA_MMA;
     void* encode_tiled = nullptr;    // cuTensorMapEncodeTiled, resolved through the runtime (no link against libcuda)
@@ -136,6 +138,9 @@ void free_all(hf_ctx* c) {
     }
     cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials);
     cudaFree(c->dev_status);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
     for (auto& s : c->stage) cudaFree(s);
 }
 
@@ -416,6 +421,10 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     if (s == HF_OK) s = dmalloc(&c->hist, c->chunk_elems);
     if (s == HF_OK) s = dmalloc(&c->partials, (size_t)c->BH * c->nsplit_max * ((size_t)c->d * c->d + c->d));
     if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)4);
+    if (s == HF_OK && (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+                       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                       cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
+        s = fail(HF_ERR_CUDA, "could not create the context's side stream / events");
     if (s == HF_OK) {
         cudaMemset(c->dev_status, 0, 16);
         s = set_swa_attr<16, 64>();
@@ -560,8 +569,16 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     HF_TRY(check_ptr(o, "o"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
+    // The history term depends on q and the state only: it runs on the context's side stream while pooling and
+    // selection run on the caller's stream; the attention kernel, which adds it in its epilogue, waits for both.
+    // (The fork event also orders this read-out after the previous call's attention kernel, which read the same
+    // scratch buffer.)
+    HF_CUDA(cudaEventRecord(c->ev_fork, st));
+    HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+    HF_TRY(HF_DISPATCH_D(c, launch_readout, c, L, (const bf16*)q, (bf16*)nullptr, c->hist, c->side));
+    HF_CUDA(cudaEventRecord(c->ev_join, c->side));
     HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
-    HF_TRY(HF_DISPATCH_D(c, launch_readout, c, L, (const bf16*)q, (bf16*)nullptr, c->hist, st));
+    HF_CUDA(cudaStreamWaitEvent(st, c->ev_join, 0));
     return launch_swa(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, c->hist, (bf16*)o, nullptr, st);
 }
 
