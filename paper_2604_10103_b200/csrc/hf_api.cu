@@ -202,8 +202,11 @@ hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
     return post_launch(c, "k_reduce_fold");
 }
 
+// fold_on_side: the reduce/fold kernel goes to the context's side stream (the caller has more work for `st` that only
+// needs the partials kernel to be done, and joins with ev_join afterwards).
 template <int D>
-hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st) {
+hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st,
+                        bool fold_on_side = false) {
     typedef AbsorbTc5<D> A;
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
@@ -214,7 +217,12 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
     k_absorb_tc5<D><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
     HF_TRY(post_launch(c, "k_absorb_tc5"));
-    return launch_fold<D>(c, L, nsplit, st);
+    if (!fold_on_side) return launch_fold<D>(c, L, nsplit, st);
+    HF_CUDA(cudaEventRecord(c->ev_fork, st));
+    HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+    HF_TRY(launch_fold<D>(c, L, nsplit, c->side));
+    HF_CUDA(cudaEventRecord(c->ev_join, c->side));
+    return HF_OK;
 }
 
 template <int D>
@@ -508,10 +516,14 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
         return HF_OK;
     }
     int slot;
+    bool evicted = false;
     if (L.n_cached == c->P) {   // cache full: the state is updated before the evicted chunk's slot is reused
         slot = L.head;
+        // the slot may be overwritten as soon as the partials kernel has read it; adding the partials to the state and
+        // folding it runs beside the copy, on the side stream
         HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)slot * c->chunk_elems,
-                             L.ring_v + (size_t)slot * c->chunk_elems, c->Tc, st));
+                             L.ring_v + (size_t)slot * c->chunk_elems, c->Tc, st, true));
+        evicted = true;
         L.absorbed += c->Tc;
         L.head = (L.head + 1) % c->P;
     } else {
@@ -524,6 +536,7 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     jobs.job[0].pooled = L.pooled_k + (size_t)slot * c->pooled_elems;
     jobs.job[1].src = (const bf16*)v; jobs.job[1].copy_dst = L.ring_v + (size_t)slot * c->chunk_elems;
     HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
+    if (evicted) HF_CUDA(cudaStreamWaitEvent(st, c->ev_join, 0));
     L.cache_epoch++;
     return HF_OK;
 }
