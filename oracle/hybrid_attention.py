@@ -20,6 +20,7 @@ What follows which passage:
   sparse_attention        Eq. 6 as its plain definition: softmax over the kept keys
   sparse_attention_tiled  Alg. 3 inner loops (running max / sum / rescale), step by step
   absorb                  Eq. 3 (state update) without the rotation
+  absorb_frame_mean       Eq. 3 with H accumulated as printed: per evicted frame the mean of phi(K) over its tokens
   linear_readout          Eq. 4 without the rotation: Linear(phi(Q) L / (phi(Q) H))
   HybridStream            Alg. 2 cache protocol (evict -> update state -> append) around Alg. 3, Eq. 7 sum
 
@@ -217,6 +218,18 @@ def absorb(S: np.ndarray, z: np.ndarray, k_ev, v_ev):
     return S + f.T @ np.asarray(v_ev, np.float64), z + f.sum(axis=0)
 
 
+def absorb_frame_mean(S: np.ndarray, z: np.ndarray, k_ev, v_ev, frame_tokens: int):
+    """Eq. 3 read literally for H: S as in absorb(); z += sum over the evicted latent frames of the MEAN over that
+    frame's tokens of phi(K) (the paper prints "mean" inside the sum).  k_ev must hold whole frames."""
+    f = phi(k_ev)
+    n = f.shape[0]
+    assert n % frame_tokens == 0, "evicted tokens must be whole frames"
+    zinc = np.zeros_like(z)
+    for fr in range(n // frame_tokens):
+        zinc = zinc + f[fr * frame_tokens:(fr + 1) * frame_tokens].mean(axis=0)
+    return S + f.T @ np.asarray(v_ev, np.float64), z + zinc
+
+
 def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6) -> np.ndarray:
     """O_history (Eq. 4): h = phi(q) S / (phi(q) . z + eps) per query row, then Linear: y = W h + bias."""
     f = phi(q)
@@ -239,8 +252,9 @@ class HybridStream:
     """
 
     def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
-                 W=None, bias=None, eps=1e-6):
+                 W=None, bias=None, eps=1e-6, z_frame_tokens=None):
         self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
+        self.z_frame_tokens = z_frame_tokens     # None: z is the plain sum of phi(K); n: per-frame means of n tokens (Eq. 3 literal)
         self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
         self.W = None if W is None else np.asarray(W, np.float64)        # [H, d, d]
         self.bias = None if bias is None else np.asarray(bias, np.float64)  # [H, d]
@@ -256,7 +270,11 @@ class HybridStream:
             k_ev, v_ev = self.past.pop(0)
             for bi in range(self.B):
                 for h in range(self.H):
-                    self.S[bi, h], self.z[bi, h] = absorb(self.S[bi, h], self.z[bi, h], k_ev[bi, h], v_ev[bi, h])
+                    if self.z_frame_tokens is None:
+                        self.S[bi, h], self.z[bi, h] = absorb(self.S[bi, h], self.z[bi, h], k_ev[bi, h], v_ev[bi, h])
+                    else:
+                        self.S[bi, h], self.z[bi, h] = absorb_frame_mean(self.S[bi, h], self.z[bi, h], k_ev[bi, h],
+                                                                         v_ev[bi, h], self.z_frame_tokens)
             self.absorbed_tokens += k_ev.shape[2]
 
     # -- Eq. 5 + top-K

@@ -66,6 +66,7 @@ struct hf_ctx {
     float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
     float* partials = nullptr;       // absorb split partials
     int nsplit_max = 1;
+    float z_scale = 1.f;             // 1 (z = sum of phi(K)) or 1 / tokens_per_frame (per-frame means)
     bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
     int* dev_status = nullptr;
     cudaStream_t side = nullptr;     // hf_hybrid_forward runs the history read-out here, beside pooling + selection
@@ -112,6 +113,7 @@ hf_status validate(const hf_config& g) {
     if (g.merge != HF_MERGE_IDENTITY && g.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_UNSUPPORTED, "merge %d unsupported", g.merge);
     if (!(g.eps >= 0.f)) return fail(HF_ERR_SHAPE, "eps must be >= 0");
     if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
+    if (g.z_mode != HF_Z_SUM && g.z_mode != HF_Z_FRAME_MEAN) return fail(HF_ERR_UNSUPPORTED, "z_mode %d unknown", g.z_mode);
     const long long Tc = (long long)g.tokens_per_frame * g.chunk_frames;
     const long long n_b = (Tc + g.block - 1) / g.block;
     if (Tc > (1 << 20)) return fail(HF_ERR_SHAPE, "chunk of %lld tokens too large", Tc);
@@ -197,7 +199,7 @@ hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
 
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
-    k_reduce_fold<D><<<dim3(D / 4, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, L.has_w ? L.W : nullptr, c->cfg.heads,
+    k_reduce_fold<D><<<dim3(D / 4, c->BH), D, 0, st>>>(c->partials, nsplit, L.S, L.z, c->z_scale, L.has_w ? L.W : nullptr, c->cfg.heads,
                                                       L.sf_hi, L.sf_lo);
     return post_launch(c, "k_reduce_fold");
 }
@@ -387,6 +389,7 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->mask_words = (c->max_Tn + 31) / 32;
     c->chunk_elems = (size_t)c->BH * c->Tc * c->d;
     c->pooled_elems = (size_t)c->BH * c->n_b * c->d;
+    c->z_scale = cfg->z_mode == HF_Z_FRAME_MEAN ? 1.f / (float)cfg->tokens_per_frame : 1.f;
     c->nsplit_max = c->sm_count / c->BH;          // one wave: the absorb kernel runs one thread block per SM
     if (c->nsplit_max > 32) c->nsplit_max = 32;
     if (c->nsplit_max < 1) c->nsplit_max = 1;
@@ -497,6 +500,8 @@ hf_status hf_state_absorb(hf_ctx* c, int layer, const void* k_ev, const void* v_
     HF_TRY(check_ptr(k_ev, "k_ev"));
     HF_TRY(check_ptr(v_ev, "v_ev"));
     if (n_tokens < 1) return fail(HF_ERR_SHAPE, "n_tokens must be >= 1");
+    if (c->cfg.z_mode == HF_Z_FRAME_MEAN && n_tokens % c->cfg.tokens_per_frame != 0)
+        return fail(HF_ERR_SHAPE, "with HF_Z_FRAME_MEAN n_tokens must be a multiple of tokens_per_frame (%d)", c->cfg.tokens_per_frame);
     LayerState& L = c->layers[layer];
     HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, (const bf16*)k_ev, (const bf16*)v_ev, n_tokens, (cudaStream_t)stream));
     L.absorbed += n_tokens;

@@ -130,11 +130,12 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
 
 // grid (D/4, B*H), D threads.  Adds the nsplit partials of a (batch, head) to S (rows a0 .. a0+3 per block) and z
 // (block 0) in ascending split order, then folds the updated rows: Sf = S W_h^T (or S when W == nullptr) as bf16
-// hi and lo halves.  nsplit == 0: fold only.  sf_hi == nullptr: state update only.
+// hi and lo halves.  nsplit == 0: fold only.  sf_hi == nullptr: state update only.  z_scale: 1 for z = sum of phi(K)
+// rows, 1 / tokens-per-frame for the per-frame-mean reading of Eq. 3.
 // Thread c' owns output column c': its row of W_h is fetched first (all loads in flight while the partials are summed).
 template <int D>
 __global__ void __launch_bounds__(D)
-k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict__ S, float* __restrict__ z,
+k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict__ S, float* __restrict__ z, float z_scale,
               const bf16* __restrict__ W, int heads, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
     constexpr int ROWS = 4;
     constexpr int PART_FLOATS = D * D + D;
@@ -152,9 +153,8 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
     float sum[ROWS];
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) sum[r] = S[((size_t)bh * D + a0 + r) * D + cp];
-    float zsum = 0.f;
+    float zsum = 0.f;           // this call's sum of phi(K) rows; enters z scaled (1, or 1 / tokens per frame)
     const bool do_z = blockIdx.x == 0 && nsplit > 0;
-    if (do_z) zsum = z[(size_t)bh * D + cp];
 #pragma unroll 8
     for (int s = 0; s < nsplit; ++s) {      // ascending split order per element; several splits' loads in flight
 #pragma unroll
@@ -164,7 +164,7 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
     if (nsplit > 0) {
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) S[((size_t)bh * D + a0 + r) * D + cp] = sum[r];
-        if (do_z) z[(size_t)bh * D + cp] = zsum;
+        if (do_z) z[(size_t)bh * D + cp] += zsum * z_scale;
     }
     if (!fold) return;
     float out[ROWS];

@@ -224,3 +224,31 @@ def test_layer_832x480_single_forward():
         assert hz.rel_l2(oh[ok], oh_ref[ok]) <= hz.REL_L2
     finally:
         gpu.close()
+
+
+def test_frame_mean_reading_of_the_state_denominator():
+    """HF_Z_FRAME_MEAN: z accumulates per-frame means of phi(K) (Eq. 3 as printed); outputs and state against the oracle
+    run the same way; a token count that is not whole frames is refused."""
+    import torch
+    w = gen.Workload("zmean", batch=1, heads=3, head_dim=128, tokens_per_frame=96, chunk_frames=2, window_frames=4,
+                     block=64, topk=0, keep_permille=500, seed=14)
+    gpu = hz.GpuStream(w, z_frame_mean=True); ora = hz.make_oracle(w, z_frame_mean=True)
+    try:
+        for c in range(4):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        S, z = gpu.state()
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2 and hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        qb, kb, vb = gen.qkv(w, 0, 4, 0)
+        o_ref, _, oh_ref = ora.forward(f64(qb), f64(kb), f64(vb), parts=True)
+        # with per-frame means the history term is T_f = 96 times larger (|O| up to ~10 here): the absolute bound is
+        # widened by the bf16 half-ulp of the largest output, the relative bound stays
+        o = gpu.forward(gpu.up(qb), gpu.up(kb), gpu.up(vb))
+        assert hz.rel_l2(o, o_ref) <= hz.REL_L2
+        assert hz.max_abs(o, o_ref) <= hz.MAX_ABS + 2.0 ** -8 * np.abs(o_ref).max()
+        assert hz.rel_l2(gpu.linear(gpu.up(qb)), oh_ref) <= hz.REL_L2
+        bad = torch.zeros((1, 3, 100, 128), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_SHAPE"):
+            gpu.ctx.hf_state_absorb(0, bad, bad, 100)
+    finally:
+        gpu.close()

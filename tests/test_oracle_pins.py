@@ -371,3 +371,38 @@ def test_pins_catch_planted_mistakes(monkeypatch):
             self.P += 1
     monkeypatch.setattr(oa.HybridStream, "append", early)
     assert fails(test_recurrent_state_equals_from_scratch_sum_and_partition, 2)
+
+
+# ----------------------------------------------------------------------------- Eq. 3 as printed: per-frame means in H
+def test_frame_mean_state_brute_force_and_scaling_identity():
+    """absorb_frame_mean against token-by-token loops, and the identity that makes the two readings of H
+    interchangeable up to a learned scale: with whole frames of T_f tokens, z_mean = z_sum / T_f, so the
+    normalised read-out (eps = 0) is exactly T_f times larger."""
+    tf, frames, d = 5, 3, 8
+    k = rnd((tf * frames, d), 41); v = rnd((tf * frames, d), 42); q = rnd((7, d), 43)
+    S, z = oa.absorb_frame_mean(np.zeros((d, d)), np.zeros(d), k, v, tf)
+    z_ref = np.zeros(d); S_ref = np.zeros((d, d))
+    for fr in range(frames):
+        acc = np.zeros(d)
+        for t in range(fr * tf, (fr + 1) * tf):
+            f = np.array([x + 1.0 if x > 0 else math.exp(x) for x in k[t]])
+            acc += f
+            S_ref += np.outer(f, v[t])
+        z_ref += acc / tf
+    assert np.allclose(S, S_ref, rtol=0, atol=1e-12) and np.allclose(z, z_ref, rtol=0, atol=1e-13)
+    S2, z2 = oa.absorb(np.zeros((d, d)), np.zeros(d), k, v)
+    assert np.allclose(S, S2, rtol=0, atol=1e-12) and np.allclose(z * tf, z2, rtol=1e-14, atol=0)
+    h_mean = oa.linear_readout(q, S, z, eps=0.0); h_sum = oa.linear_readout(q, S2, z2, eps=0.0)
+    assert np.allclose(h_mean, tf * h_sum, rtol=1e-12, atol=0)
+    with pytest.raises(AssertionError):
+        oa.absorb_frame_mean(np.zeros((d, d)), np.zeros(d), k[:-1], v[:-1], tf)
+
+
+def test_stream_with_frame_mean_matches_one_shot():
+    st = oa.HybridStream(1, 1, 8, 4, 1, topk=1, z_frame_tokens=4)
+    ks = [rnd((1, 1, 8, 8), 50 + i) for i in range(4)]; vs = [rnd((1, 1, 8, 8), 60 + i) for i in range(4)]
+    for kk, vv in zip(ks, vs):
+        st.append(kk, vv)
+    ev = np.concatenate([x[0, 0] for x in ks[:3]])
+    z_ref = sum(oa.phi(ev[i * 4:(i + 1) * 4]).mean(axis=0) for i in range(6))
+    assert np.allclose(st.z[0, 0], z_ref, rtol=0, atol=1e-13) and st.absorbed_tokens == 24
