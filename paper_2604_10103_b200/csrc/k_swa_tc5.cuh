@@ -272,7 +272,8 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                 for (int c = 0; c < NC; ++c)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) mx[e & 3] = fmaxf(mx[e & 3], __uint_as_float(r[c][e]));
+                    for (int e = 0; e < 32; e += 2)         // three-input maximum: two values per instruction
+                        mx[(e >> 1) & 3] = fmax3(mx[(e >> 1) & 3], __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]));
                 float mrow = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
                 if (NG > 1) {
                     // every group has read its S columns (the P columns written below overlap another group's S)
@@ -310,21 +311,22 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     }
                 }
                 // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the first half of the S buffer
-                float rs0 = 0.f, rs1 = 0.f;
-                const float neg_m = -m_used;
+                // (packed fp32: the scale-and-shift and the row sum handle two columns per instruction)
+                float2 rsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), negm2 = make_float2(-m_used, -m_used);
 #pragma unroll
                 for (int c = 0; c < NC; ++c) {
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[c][e]), p.scale_log2, neg_m));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[c][e + 1]), p.scale_log2, neg_m));
-                        rs0 += p0; rs1 += p1;
-                        pk[e >> 1] = pack_bf16(p0, p1);
+                        const float2 x = ffma2(make_float2(__uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1])), scale2, negm2);
+                        const float2 pe = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        rsum[(e >> 1) & 1] = fadd2(rsum[(e >> 1) & 1], pe);
+                        pk[e >> 1] = pack_bf16(pe.x, pe.y);
                     }
                     tmem_st16(tS + grp * (C::GCOLS / 2) + c * 16, pk);
                 }
-                l_run += rs0 + rs1;
+                l_run += (rsum[0].x + rsum[0].y) + (rsum[1].x + rsum[1].y);
                 tmem_wait_st();
                 fence_before_sync();
                 mbar_arrive(bar_pf + 8 * (rs.stage == 0 ? C::SBUFS - 1 : rs.stage - 1));
