@@ -41,7 +41,7 @@ typedef enum {
 
 enum { HF_PHI_ELU1 = 0 };                                /* phi(x) = elu(x) + 1                 */
 enum { HF_MERGE_IDENTITY = 0, HF_MERGE_PER_HEAD = 1 };   /* "Linear" of Eq. 4: none | W[H,d,d]  */
-enum { HF_SWA_AUTO = 0, HF_SWA_MMA = 1, HF_SWA_TCGEN05 = 2 }; /* sparse-attention kernel choice */
+enum { HF_SWA_AUTO = 0, HF_SWA_MMA = 1, HF_SWA_TCGEN05 = 2, HF_SWA_TCGEN05_PINGPONG = 3 }; /* sparse-attention kernel choice */
 enum { HF_Z_SUM = 0, HF_Z_FRAME_MEAN = 1 };              /* z of Eq. 3: sum of phi(K) rows | per-frame means */
 
 typedef struct {
@@ -57,7 +57,7 @@ typedef struct {
     int phi;                         /* HF_PHI_ELU1                                                     */
     float eps;                       /* added to the denominator phi(q).z of Eq. 4                      */
     int merge;                       /* HF_MERGE_IDENTITY | HF_MERGE_PER_HEAD                           */
-    int swa_kernel;                  /* HF_SWA_AUTO | HF_SWA_MMA | HF_SWA_TCGEN05                       */
+    int swa_kernel;                  /* HF_SWA_AUTO | HF_SWA_MMA | HF_SWA_TCGEN05 | HF_SWA_TCGEN05_PINGPONG */
     int z_mode;                      /* HF_Z_SUM: z += sum_t phi(K_ev[t]) (default).  HF_Z_FRAME_MEAN: Eq. 3 as printed,
                                         z += sum over evicted latent frames of the mean of phi(K) over the frame's
                                         tokens; absorbed token counts must then be multiples of tokens_per_frame      */

@@ -4,6 +4,7 @@
 #include "k_pool_select.cuh"
 #include "k_swa_mma.cuh"
 #include "k_swa_tc5.cuh"
+#include "k_swa_tc5p.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
 
@@ -112,7 +113,7 @@ hf_status validate(const hf_config& g) {
     if (g.phi != HF_PHI_ELU1) return fail(HF_ERR_UNSUPPORTED, "phi %d unsupported", g.phi);
     if (g.merge != HF_MERGE_IDENTITY && g.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_UNSUPPORTED, "merge %d unsupported", g.merge);
     if (!(g.eps >= 0.f)) return fail(HF_ERR_SHAPE, "eps must be >= 0");
-    if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
+    if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05_PINGPONG) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
     if (g.z_mode != HF_Z_SUM && g.z_mode != HF_Z_FRAME_MEAN) return fail(HF_ERR_UNSUPPORTED, "z_mode %d unknown", g.z_mode);
     const long long Tc = (long long)g.tokens_per_frame * g.chunk_frames;
     const long long n_b = (Tc + g.block - 1) / g.block;
@@ -315,8 +316,33 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     return post_launch(c, "k_swa_tc5");
 }
 
+template <int D>
+hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
+                            int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    typedef SwaTc5P<D> C;
+    CUtensorMap tq, tk, tv;
+    HF_TRY(make_map(c, &tq, q, 1));
+    HF_TRY(make_map(c, &tk, k_cur, 1));
+    HF_TRY(make_map(c, &tv, v_cur, 1));
+    Tc5Params p;
+    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head;
+    p.P = c->P > 0 ? c->P : 1;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+    p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
+    const CUtensorMap& rk = c->P > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
+    p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    k_swa_tc5p<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    return post_launch(c, "k_swa_tc5p");
+}
+
 hf_status launch_swa(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
                      int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    if (c->swa_kernel == HF_SWA_TCGEN05_PINGPONG) {
+        if (c->d == 128) return launch_swa_tc5p_t<128>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+        return launch_swa_tc5p_t<64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+    }
     if (c->swa_kernel == HF_SWA_TCGEN05) {
         if (c->d == 128) return launch_swa_tc5_t<128>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
         return launch_swa_tc5_t<64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
@@ -393,8 +419,9 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->nsplit_max = c->sm_count / c->BH;          // one wave: the absorb kernel runs one thread block per SM
     if (c->nsplit_max > 32) c->nsplit_max = 32;
     if (c->nsplit_max < 1) c->nsplit_max = 1;
-    if (cfg->swa_kernel == HF_SWA_TCGEN05 && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the tcgen05 attention kernel needs block == 128"); }
-    c->swa_kernel = (cfg->swa_kernel == HF_SWA_MMA || cfg->block != 128) ? HF_SWA_MMA : HF_SWA_TCGEN05;
+    if ((cfg->swa_kernel == HF_SWA_TCGEN05 || cfg->swa_kernel == HF_SWA_TCGEN05_PINGPONG) && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the tcgen05 attention kernels need block == 128"); }
+    c->swa_kernel = (cfg->swa_kernel == HF_SWA_MMA || cfg->block != 128) ? HF_SWA_MMA
+                    : (cfg->swa_kernel == HF_SWA_TCGEN05_PINGPONG ? HF_SWA_TCGEN05_PINGPONG : HF_SWA_TCGEN05);
     {
         cudaDriverEntryPointQueryResult qres;
         e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &c->encode_tiled, cudaEnableDefault, &qres);
@@ -446,6 +473,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = set_swa_attr<128, 128>();
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, Tc5Groups<64>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, Tc5Groups<64>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<64>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<64>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<128>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<128>) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }

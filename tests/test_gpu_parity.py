@@ -252,3 +252,26 @@ def test_frame_mean_reading_of_the_state_denominator():
             gpu.ctx.hf_state_absorb(0, bad, bad, 100)
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,tpf,wf,permille", [
+    (128, 300, 2, 400),     # several 128-tiles + 44-token tail, one cached chunk
+    (64, 129, 3, 1000),     # head_dim 64, 1-token tail block, everything kept
+    (128, 200, 1, 1000),    # window == chunk: two key blocks per row
+    (128, 520, 3, 100),     # sparse: few tiles per row (odd counts leave one group with fewer tiles)
+])
+def test_pingpong_attention_kernel(d, tpf, wf, permille):
+    """The tile-alternating tcgen05 kernel against the oracle (same stream as the other kernels), including rows whose
+    kept list gives the two softmax groups unequal numbers of tiles."""
+    from paper_2604_10103_b200 import binding as hf
+    w = gen.Workload("pp", batch=2, heads=2, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=wf,
+                     block=128, topk=0, keep_permille=permille, seed=15)
+    stream_compare(w, wf + 2, swa_kernel=hf.HF_SWA_TCGEN05_PINGPONG)
+
+
+def test_pingpong_single_kept_block_and_lse():
+    """k = 1: the second softmax group has no tile at all and must drop out of the merge."""
+    from paper_2604_10103_b200 import binding as hf
+    w = gen.Workload("pp1", batch=1, heads=2, head_dim=128, tokens_per_frame=256, chunk_frames=1, window_frames=3,
+                     block=128, topk=1, keep_permille=0, seed=16)
+    stream_compare(w, 4, swa_kernel=hf.HF_SWA_TCGEN05_PINGPONG)
