@@ -316,10 +316,14 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     return post_launch(c, "k_swa_tc5");
 }
 
+#ifndef HF_TC5P_COLGROUPS
+#define HF_TC5P_COLGROUPS 1   // column groups per tile group of the ping-pong attention kernel
+#endif
+
 template <int D>
 hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
                             int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
-    typedef SwaTc5P<D> C;
+    typedef SwaTc5P<D, HF_TC5P_COLGROUPS> C;
     CUtensorMap tq, tk, tv;
     HF_TRY(make_map(c, &tq, q, 1));
     HF_TRY(make_map(c, &tk, k_cur, 1));
@@ -333,7 +337,7 @@ hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16*
     const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
-    k_swa_tc5p<D><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    k_swa_tc5p<D, HF_TC5P_COLGROUPS><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
     return post_launch(c, "k_swa_tc5p");
 }
 
@@ -473,8 +477,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = set_swa_attr<128, 128>();
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, Tc5Groups<64>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, Tc5Groups<64>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<64>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<64>) failed");
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<128>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<128>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<64, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<64, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<64>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<128, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<128, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<128>) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }

@@ -8,15 +8,20 @@
 //   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols 128 (t & 1)
 //   P = exp2(S*c - m)  bf16, written over the first 64 columns of its S buffer
 //   O_g += P V_t       A = P (TMEM), B = V_t (smem, MN-major, 128B swizzle)              -> TMEM cols 256 + D (t & 1)
-// Loader warps (Q + three-stage K ring; two-stage V ring) and the MMA warp as in k_swa_tc5.  A row of S is read
-// from tensor memory twice, 64 columns at a time (maximum, then exponentials), so that a thread never holds more
-// than 64 of its 128 values.  Every wait is bounded (~1 s) and reports through the device status word.
+// Loader warps (Q + three-stage K ring; two-stage V ring) and the MMA warp as in k_swa_tc5.  Each tile group may be
+// split further into CG column groups of four warps (thread = one row, 128 / CG columns; the column groups of a
+// tile group exchange their row maxima through shared memory once per tile, as in k_swa_tc5), which puts 4 CG
+// softmax warps of two different tiles on every scheduler.  A row share of S is read from tensor memory twice,
+// 32 columns at a time (maximum, then exponentials), so that a thread holds 32 values at a time.  Every wait is
+// bounded (~1 s) and reports through the device status word.
 #pragma once
 #include "tc5_common.cuh"
 #include "k_swa_tc5.cuh"      // Tc5Params, RingPos
 
-template <int D>
+template <int D, int CG>
 struct SwaTc5P {
+    static constexpr int NCOL = 128 / CG;              // S columns per thread
+    static constexpr int NSM = 256 * CG;               // softmax threads
     static constexpr int BLK = 128;
     static constexpr int SUB = D / 64;
     static constexpr int SUB_BYTES = BLK * 128;
@@ -24,22 +29,23 @@ struct SwaTc5P {
     static constexpr int KSTAGES = 3, VSTAGES = 2;
     static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = OFF_K + KSTAGES * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_V + VSTAGES * TILE_BYTES;
-    static constexpr int OFF_X = OFF_BAR + 256;        // per group and row: (m, l) of the unit, [2][128] float2
-    static constexpr int USED_BYTES = OFF_X + 2 * BLK * 8;
+    static constexpr int OFF_X = OFF_BAR + 256;        // per tile group, column group and row: (m, l) of the unit, [2][CG][128] float2
+    static constexpr int OFF_XM = OFF_X + 2 * CG * BLK * 8;   // row-max exchange [2 tile groups][2 parities][CG][128] floats
+    static constexpr int USED_BYTES = OFF_XM + 4 * CG * BLK * 4;
     static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
-    static constexpr int THREADS = 256 + 96;
-    static constexpr int WARP_LOAD_K = 8, WARP_LOAD_V = 9, WARP_MMA = 10;
+    static constexpr int THREADS = NSM + 96;
+    static constexpr int WARP_LOAD_K = NSM / 32, WARP_LOAD_V = NSM / 32 + 1, WARP_MMA = NSM / 32 + 2;
     static constexpr int TMEM_COLS = 512;
     static constexpr int COL_O = 2 * BLK;              // O_A at 256, O_B at 256 + D
 };
 
-template <int D>
-__global__ void __launch_bounds__(SwaTc5P<D>::THREADS, 1)
+template <int D, int CG>
+__global__ void __launch_bounds__(SwaTc5P<D, CG>::THREADS, 1)
 k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
            const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
            const __grid_constant__ CUtensorMap tm_vcur, const Tc5Params p) {
     using namespace tc5;
-    typedef SwaTc5P<D> C;
+    typedef SwaTc5P<D, CG> C;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
@@ -47,10 +53,11 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const uint32_t bar0 = s_base + C::OFF_BAR;
     const uint32_t bar_kf = bar0, bar_ke = bar0 + 24, bar_vf = bar0 + 48, bar_ve = bar0 + 64, bar_sf = bar0 + 80,
                    bar_pf = bar0 + 96, bar_pv = bar0 + 112, bar_qf = bar0 + 128, bar_qe = bar0 + 136, bar_ep = bar0 + 144,
-                   bar_ep2 = bar0 + 152, bar_drain = bar0 + 160;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 176);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 180);
-    float2* x_ml = reinterpret_cast<float2*>(s_gen + C::OFF_X);           // [2][128]
+                   bar_ep2 = bar0 + 152, bar_drain = bar0 + 160, bar_mx = bar0 + 168, bar_mx2 = bar0 + 200;   // bar_mx*, [tile group][parity]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 240);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 244);
+    float2* x_ml = reinterpret_cast<float2*>(s_gen + C::OFF_X);           // [2][CG][128]
+    float* x_max = reinterpret_cast<float*>(s_gen + C::OFF_XM);           // [2][2][CG][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int keep = p.keep;
@@ -61,9 +68,11 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         for (int s = 0; s < 3; ++s) { mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1); }
         for (int s = 0; s < 2; ++s) {
             mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_sf + 8 * s, 1);
-            mbar_init(bar_pf + 8 * s, 128); mbar_init(bar_pv + 8 * s, 1);
+            mbar_init(bar_pf + 8 * s, 128 * CG); mbar_init(bar_pv + 8 * s, 1);
+            mbar_init(bar_mx + 16 * s, 128 * CG); mbar_init(bar_mx + 16 * s + 8, 128 * CG);
+            mbar_init(bar_mx2 + 16 * s, 128 * CG); mbar_init(bar_mx2 + 16 * s + 8, 128 * CG);
         }
-        mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_ep, 256); mbar_init(bar_ep2, 256); mbar_init(bar_drain, 1);
+        mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_ep, C::NSM); mbar_init(bar_ep2, C::NSM); mbar_init(bar_drain, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -184,13 +193,18 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
     } else {
         // ================================================================= softmax groups / merge / epilogue
-        const int g = warp >> 2;                            // group: tiles with stream index t & 1 == g
+        const int g = warp / (4 * CG);                      // tile group: tiles with stream index t & 1 == g
+        const int cg = (warp >> 2) % CG;                    // column group inside the tile group
         const int row = (warp & 3) * 32 + lane;             // query row of the tile = TMEM lane
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         const uint32_t tS = lane_base + g * C::BLK;
-        const uint32_t tO_mine = lane_base + C::COL_O + g * D;
+        constexpr int OC = D / CG;                          // accumulator columns this thread rescales
+        const uint32_t tO_mine = lane_base + C::COL_O + g * D + cg * OC;
         const int tail_cols = p.Tc - (p.n_b - 1) * C::BLK;
+        constexpr int NCH = C::NCOL / 32;                   // 32-column chunks of this thread's S share
+        const int col0 = cg * C::NCOL;
         bool ok = true;
+        int n_mine = 0;                                     // tiles this group has processed (exchange barrier phases)
         for (int n = 0; ok && n < my_units; ++n) {
             const int u = blockIdx.x + n * gridDim.x;
             const int bh = u / p.Tm, i = u - bh * p.Tm;
@@ -198,16 +212,16 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int q0 = i * C::BLK;
             const int nq = min(C::BLK, p.Tc - q0);
             const int t0 = n * keep;                        // stream index of the unit's first tile
-            float m_used = -INFINITY, l_run = 0.f;
+            float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
             bool first = true;
             int j = (t0 & 1) == g ? 0 : 1;                  // this group's first position in the unit
             int blk_next = j < keep ? __ldg(my_idx + j) : 0;
             if (n >= 1) {
-                // both groups have read both accumulators of the previous unit before either is started afresh
+                // every softmax thread has read both accumulators of the previous unit before either is started afresh
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_ep2, (n - 1) & 1, abort_flag, p.dev_status, 14));
                 if (!ok) break;
             }
-            for (; j < keep; j += 2) {
+            for (; j < keep; j += 2, ++n_mine) {
                 const int t = t0 + j;
                 bool tail = false;
 #pragma unroll
@@ -218,27 +232,37 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * g, (t >> 1) & 1, abort_flag, p.dev_status, 8));
                 if (!ok) break;
                 fence_after_sync();
-                // ---- pass 1: row maximum, 64 columns at a time
+                // ---- pass 1: maximum of this thread's share of the row, 32 columns at a time
                 float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r[2][32];
-                    tmem_ld32(tS + h * 64, r[0]);
-                    tmem_ld32(tS + h * 64 + 32, r[1]);
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tS + col0 + c * 32, r);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 2; ++c)
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float v0 = __uint_as_float(r[c][e]), v1 = __uint_as_float(r[c][e + 1]);
-                            if (nv < C::BLK) {
-                                if (h * 64 + c * 32 + e >= nv) v0 = -INFINITY;
-                                if (h * 64 + c * 32 + e + 1 >= nv) v1 = -INFINITY;
-                            }
-                            mx[(e >> 1) & 3] = fmax3(mx[(e >> 1) & 3], v0, v1);
+                    for (int e = 0; e < 32; e += 2) {
+                        float v0 = __uint_as_float(r[e]), v1 = __uint_as_float(r[e + 1]);
+                        if (nv < C::BLK) {
+                            if (col0 + c * 32 + e >= nv) v0 = -INFINITY;
+                            if (col0 + c * 32 + e + 1 >= nv) v1 = -INFINITY;
                         }
+                        mx[(e >> 1) & 3] = fmax3(mx[(e >> 1) & 3], v0, v1);
+                    }
                 }
-                const float m_new = fmaxf(m_used, fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2);
+                float mrow = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                if (CG > 1) {
+                    // the column groups of this tile group learn the maximum of the whole row; the exchange also tells
+                    // them that this thread has finished pass 1 (P columns written in pass 2 overlap other groups' S)
+                    const int par = n_mine & 1;
+                    float* xm = x_max + ((g * 2 + par) * CG) * C::BLK;
+                    xm[cg * C::BLK + row] = mrow;
+                    mbar_arrive(bar_mx + 16 * g + 8 * par);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 16 * g + 8 * par, (n_mine >> 1) & 1, abort_flag, p.dev_status, 11));
+                    if (!ok) break;
+#pragma unroll
+                    for (int q = 0; q < CG; ++q) mrow = fmaxf(mrow, xm[q * C::BLK + row]);
+                }
+                const float m_new = fmaxf(m_used, mrow * p.scale_log2);
                 // ---- lazy rescale of this group's accumulator: only when some row of the warp moved its maximum by more than 2^8
                 if (first) {
                     m_used = m_new;
@@ -249,7 +273,7 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
                         if (need) { m_used = m_new; l_run *= alpha; }
 #pragma unroll 1
-                        for (int c = 0; c < D / 32; ++c) {
+                        for (int c = 0; c < OC / 32; ++c) {
                             uint32_t o[32];
                             tmem_ld32(tO_mine + c * 32, o);
                             tmem_wait_ld();
@@ -259,32 +283,39 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         }
                     }
                 }
-                // ---- pass 2: P = exp2(S*c - m), row sum, bf16 pairs over the first 64 columns of the S buffer.  The
-                // columns a half overwrites (32 h .. 32 h + 31) were read by this or an earlier half.
+                // ---- pass 2: P = exp2(S*c - m), row sum, bf16 pairs over the first 64 columns of the S buffer.  With one
+                // column group a chunk of P overwrites columns this thread has already read.  With several, a group's P
+                // columns overlap another group's S columns: every thread first turns its whole share into packed P in
+                // registers, the groups meet (second exchange barrier), then all store.
                 float2 rsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), negm2 = make_float2(-m_used, -m_used);
-#pragma unroll 1
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t r[2][32];
-                    tmem_ld32(tS + h * 64, r[0]);
-                    tmem_ld32(tS + h * 64 + 32, r[1]);
+                uint32_t pk[NCH][16];
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                    uint32_t r[32];
+                    tmem_ld32(tS + col0 + c * 32, r);
                     tmem_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        uint32_t pk[16];
-#pragma unroll
-                        for (int e = 0; e < 32; e += 2) {
-                            float2 x = ffma2(make_float2(__uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1])), scale2, negm2);
-                            if (nv < C::BLK) {
-                                if (h * 64 + c * 32 + e >= nv) x.x = -INFINITY;
-                                if (h * 64 + c * 32 + e + 1 >= nv) x.y = -INFINITY;
-                            }
-                            const float2 pe = make_float2(fast_exp2(x.x), fast_exp2(x.y));
-                            rsum[(e >> 1) & 1] = fadd2(rsum[(e >> 1) & 1], pe);
-                            pk[e >> 1] = pack_bf16(pe.x, pe.y);
+                    for (int e = 0; e < 32; e += 2) {
+                        float2 x = ffma2(make_float2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), scale2, negm2);
+                        if (nv < C::BLK) {
+                            if (col0 + c * 32 + e >= nv) x.x = -INFINITY;
+                            if (col0 + c * 32 + e + 1 >= nv) x.y = -INFINITY;
                         }
-                        tmem_st16(tS + h * 32 + c * 16, pk);
+                        const float2 pe = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        rsum[(e >> 1) & 1] = fadd2(rsum[(e >> 1) & 1], pe);
+                        pk[c][e >> 1] = pack_bf16(pe.x, pe.y);
                     }
+                    if (CG == 1) tmem_st16(tS + c * 16, pk[c]);
+                }
+                if (CG > 1) {
+                    // all column groups have read their S values of this tile: P may now overwrite the buffer's first half
+                    const int par = n_mine & 1;
+                    mbar_arrive(bar_mx2 + 16 * g + 8 * par);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_mx2 + 16 * g + 8 * par, (n_mine >> 1) & 1, abort_flag, p.dev_status, 15));
+                    if (!ok) break;
+#pragma unroll
+                    for (int c = 0; c < NCH; ++c) tmem_st16(tS + col0 / 2 + c * 16, pk[c]);
                 }
                 l_run += (rsum[0].x + rsum[0].y) + (rsum[1].x + rsum[1].y);
                 tmem_wait_st();
@@ -292,16 +323,18 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 mbar_arrive(bar_pf + 8 * g);
             }
             if (!ok) break;
-            // ---- merge of the two groups and epilogue: O / l (+ history term), one rounding to bf16
-            x_ml[g * C::BLK + row] = make_float2(m_used, l_run);
+            // ---- merge of the two tile groups and epilogue: O / l (+ history term), one rounding to bf16
+            x_ml[(g * CG + cg) * C::BLK + row] = make_float2(m_used, l_run);
             mbar_arrive(bar_ep);
             ok = __all_sync(0xffffffffu, mbar_wait(bar_ep, n & 1, abort_flag, p.dev_status, 12));
             if (!ok) break;
-            const float2 mlA = x_ml[row], mlB = x_ml[C::BLK + row];
-            const float m = fmaxf(mlA.x, mlB.x);
-            const float fA = mlA.y > 0.f ? fast_exp2(mlA.x - m) : 0.f;
-            const float fB = mlB.y > 0.f ? fast_exp2(mlB.x - m) : 0.f;
-            const float l = mlA.y * fA + mlB.y * fB;
+            float mA = x_ml[row].x, lA = 0.f, mB = x_ml[CG * C::BLK + row].x, lB = 0.f;
+#pragma unroll
+            for (int q = 0; q < CG; ++q) { lA += x_ml[q * C::BLK + row].y; lB += x_ml[(CG + q) * C::BLK + row].y; }
+            const float m = fmaxf(mA, mB);
+            const float fA = lA > 0.f ? fast_exp2(mA - m) : 0.f;
+            const float fB = lB > 0.f ? fast_exp2(mB - m) : 0.f;
+            const float l = lA * fA + lB * fB;
             // last P V of each group in this unit: stream index of the last tile with that parity
             const int t_last = t0 + keep - 1;
 #pragma unroll
@@ -317,20 +350,23 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const float inv = 1.f / l;
             const float wA = fA * inv, wB = fB * inv;
             const size_t g_row = (size_t)bh * p.Tc + q0 + row;
-            if (g == 0 && row < nq && p.lse) p.lse[g_row] = (m + log2f(l)) * 0.6931471805599453f;
+            if (g == 0 && cg == 0 && row < nq && p.lse) p.lse[g_row] = (m + log2f(l)) * 0.6931471805599453f;
+            constexpr int EC = D / (2 * CG);                // output columns per thread: the 2 CG warps of a row quadrant split the row
+            static_assert(EC % 16 == 0, "output share must be a multiple of 16 columns");
+            const int ecol0 = (g * CG + cg) * EC;
 #pragma unroll 1
-            for (int c = 0; c < D / 64; ++c) {              // this group stores output columns [g D/2, (g+1) D/2)
-                const int col = g * (D / 2) + c * 32;
-                uint32_t oa[32], ob[32];
-                tmem_ld32(lane_base + C::COL_O + col, oa);
-                tmem_ld32(lane_base + C::COL_O + D + col, ob);
+            for (int c = 0; c < EC / 16; ++c) {
+                const int col = ecol0 + c * 16;
+                uint32_t oa[16], ob[16];
+                tmem_ld16(lane_base + C::COL_O + col, oa);
+                tmem_ld16(lane_base + C::COL_O + D + col, ob);
                 tmem_wait_ld();
                 if (row < nq) {
                     const size_t off = g_row * D + col;
                     bf16* dst = p.o + off;
                     const float* hsrc = p.hist ? p.hist + off : nullptr;
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
+                    for (int v = 0; v < 2; ++v) {
                         float x[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
