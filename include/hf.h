@@ -61,17 +61,22 @@ typedef struct {
     int z_mode;                      /* HF_Z_SUM: z += sum_t phi(K_ev[t]) (default).  HF_Z_FRAME_MEAN: Eq. 3 as printed,
                                         z += sum over evicted latent frames of the mean of phi(K) over the frame's
                                         tokens; absorbed token counts must then be multiples of tokens_per_frame      */
+    int sink_frames;                 /* latent frames at the start of the stream kept visible for ever (attention sink):
+                                        a multiple of chunk_frames; those first chunks go to slots of their own, as the oldest
+                                        logical key blocks, and are never evicted nor folded into the state.  Sink chunks +
+                                        window chunks may not exceed 8                                                   */
 } hf_config;
 
 /* Fields of hf_query(). */
 enum {
-    HF_Q_CACHED_CHUNKS = 0,   /* clean chunks now in the rolling cache of the layer                   */
-    HF_Q_KEY_BLOCKS = 1,      /* T_n a forward would see now: (cached + 1) * blocks per chunk          */
+    HF_Q_CACHED_CHUNKS = 0,   /* clean chunks now in the rolling cache of the layer (sink chunks not counted) */
+    HF_Q_KEY_BLOCKS = 1,      /* T_n a forward would see now: (sink + cached + 1) * blocks per chunk   */
     HF_Q_KEPT_BLOCKS = 2,     /* k_eff = min(k, T_n) for that T_n                                      */
     HF_Q_ABSORBED_TOKENS = 3, /* tokens folded into (S, z) so far (per batch*head)                     */
     HF_Q_QUERY_BLOCKS = 4,    /* T_m = ceil(T_c / block)                                               */
     HF_Q_MASK_WORDS = 5,      /* uint32 words per mask row = ceil(max T_n / 32)                        */
-    HF_Q_SWA_KERNEL = 6       /* kernel hf_sparse_swa resolves to (HF_SWA_MMA | HF_SWA_TCGEN05)        */
+    HF_Q_SWA_KERNEL = 6,      /* kernel hf_sparse_swa resolves to (HF_SWA_MMA | HF_SWA_TCGEN05 | ..._PINGPONG) */
+    HF_Q_SINK_CHUNKS = 7      /* sink chunks held so far                                               */
 };
 
 /* Create a context on CUDA device `device` (allocates all persistent buffers, zero state).

@@ -249,15 +249,19 @@ class HybridStream:
     is appended and whatever then exceeds P chunks is popped from the front and folded into (S, z) --
     the state is updated before the evicted K/V are dropped.  With P >= 1 this is the paper's
     "if full: pop(0), update state; append"; with P = 0 a committed chunk goes straight into the state.
+    Sink (Eq. 1's first-frame term): the first sink_chunks committed chunks are kept outside that rotation, as the
+    oldest logical key blocks of every later window; they are never evicted and never folded into the state.
     """
 
     def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
-                 W=None, bias=None, eps=1e-6, z_frame_tokens=None):
+                 W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0):
         self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
         self.z_frame_tokens = z_frame_tokens     # None: z is the plain sum of phi(K); n: per-frame means of n tokens (Eq. 3 literal)
         self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
         self.W = None if W is None else np.asarray(W, np.float64)        # [H, d, d]
         self.bias = None if bias is None else np.asarray(bias, np.float64)  # [H, d]
+        self.sink_chunks = sink_chunks   # the first chunks of the stream stay visible for ever ("sink"): never evicted, never absorbed
+        self.sink = []                                                   # list of (k, v) like self.past, oldest first
         self.past = []                                                   # list of (k [B,H,n,d], v) fp64
         self.S = np.zeros((batch, heads, d, d))
         self.z = np.zeros((batch, heads, d))
@@ -265,6 +269,9 @@ class HybridStream:
 
     # -- Alg. 2, cache commit
     def append(self, k_clean, v_clean):
+        if len(self.sink) < self.sink_chunks:
+            self.sink.append((np.asarray(k_clean, np.float64), np.asarray(v_clean, np.float64)))
+            return
         self.past.append((np.asarray(k_clean, np.float64), np.asarray(v_clean, np.float64)))
         while len(self.past) > self.P:
             k_ev, v_ev = self.past.pop(0)
@@ -279,7 +286,7 @@ class HybridStream:
 
     # -- Eq. 5 + top-K
     def n_key_blocks(self, n_cur: int) -> int:
-        return sum(-(-kp.shape[2] // self.b) for kp, _ in self.past) + -(-n_cur // self.b)
+        return sum(-(-kp.shape[2] // self.b) for kp, _ in self.sink + self.past) + -(-n_cur // self.b)
 
     def select(self, q, k_cur, exact: bool = False):
         """Masks [B, H, T_m, T_n].  exact=False: canonical float32 scores (the bit-exact contract);
@@ -292,13 +299,13 @@ class HybridStream:
             for h in range(H):
                 if exact:
                     qm = block_means(q[bi, h], self.b)
-                    km = np.concatenate([block_means(kp[bi, h], self.b) for kp, _ in self.past]
+                    km = np.concatenate([block_means(kp[bi, h], self.b) for kp, _ in self.sink + self.past]
                                         + [block_means(k_cur[bi, h], self.b)])
                     a = block_scores(qm, km)
                 else:
                     as32 = lambda x: np.asarray(x, np.float64).astype(F32)   # exact: values are bf16
                     qm = block_means_f32(as32(q[bi, h]), self.b)
-                    km = np.concatenate([block_means_f32(as32(kp[bi, h]), self.b) for kp, _ in self.past]
+                    km = np.concatenate([block_means_f32(as32(kp[bi, h]), self.b) for kp, _ in self.sink + self.past]
                                         + [block_means_f32(as32(k_cur[bi, h]), self.b)])
                     a = block_scores_f32(qm, km)
                 scores.append(a)
@@ -316,8 +323,8 @@ class HybridStream:
         o_loc = np.empty_like(q); o_hist = np.empty_like(q)
         for bi in range(self.B):
             for h in range(self.H):
-                kc = [kp[bi, h] for kp, _ in self.past] + [k_cur[bi, h]]
-                vc = [vp[bi, h] for _, vp in self.past] + [v_cur[bi, h]]
+                kc = [kp[bi, h] for kp, _ in self.sink + self.past] + [k_cur[bi, h]]
+                vc = [vp[bi, h] for _, vp in self.sink + self.past] + [v_cur[bi, h]]
                 o_loc[bi, h] = sparse_attention(q[bi, h], kc, vc, self.b, mask[bi, h], q_blocks)
                 o_hist[bi, h] = linear_readout(q[bi, h], self.S[bi, h], self.z[bi, h],
                                                None if self.W is None else self.W[h],

@@ -20,7 +20,7 @@ HF_MERGE_IDENTITY, HF_MERGE_PER_HEAD = 0, 1
 HF_SWA_AUTO, HF_SWA_MMA, HF_SWA_TCGEN05, HF_SWA_TCGEN05_PINGPONG = 0, 1, 2, 3
 HF_Z_SUM, HF_Z_FRAME_MEAN = 0, 1
 (HF_Q_CACHED_CHUNKS, HF_Q_KEY_BLOCKS, HF_Q_KEPT_BLOCKS, HF_Q_ABSORBED_TOKENS, HF_Q_QUERY_BLOCKS,
- HF_Q_MASK_WORDS, HF_Q_SWA_KERNEL) = range(7)
+ HF_Q_MASK_WORDS, HF_Q_SWA_KERNEL, HF_Q_SINK_CHUNKS) = range(8)
 
 # every symbol include/hf.h declares
 EXPORTS = [
@@ -35,7 +35,7 @@ class hf_config(C.Structure):
     _fields_ = [("batch", C.c_int), ("heads", C.c_int), ("head_dim", C.c_int),
                 ("tokens_per_frame", C.c_int), ("chunk_frames", C.c_int), ("window_frames", C.c_int),
                 ("block", C.c_int), ("topk", C.c_int), ("keep_permille", C.c_int), ("layers", C.c_int),
-                ("phi", C.c_int), ("eps", C.c_float), ("merge", C.c_int), ("swa_kernel", C.c_int), ("z_mode", C.c_int)]
+                ("phi", C.c_int), ("eps", C.c_float), ("merge", C.c_int), ("swa_kernel", C.c_int), ("z_mode", C.c_int), ("sink_frames", C.c_int)]
 
 
 class HFError(RuntimeError):
@@ -100,12 +100,13 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def make_config(w, merge: int = HF_MERGE_PER_HEAD, swa_kernel: int = HF_SWA_AUTO, z_mode: int = HF_Z_SUM) -> hf_config:
+def make_config(w, merge: int = HF_MERGE_PER_HEAD, swa_kernel: int = HF_SWA_AUTO, z_mode: int = HF_Z_SUM,
+                sink_frames: int = 0) -> hf_config:
     """hf_config from an inputs.Workload."""
     return hf_config(batch=w.batch, heads=w.heads, head_dim=w.head_dim, tokens_per_frame=w.tokens_per_frame,
                      chunk_frames=w.chunk_frames, window_frames=w.window_frames, block=w.block, topk=w.topk,
                      keep_permille=w.keep_permille, layers=w.layers, phi=HF_PHI_ELU1, eps=w.eps, merge=merge,
-                     swa_kernel=swa_kernel, z_mode=z_mode)
+                     swa_kernel=swa_kernel, z_mode=z_mode, sink_frames=sink_frames)
 
 
 class Context:

@@ -47,6 +47,7 @@ struct LayerState {
     uint32_t* mask = nullptr;    // last selection [B*H, T_m, mask_words]
     int32_t* idx = nullptr;      // [B*H, T_m, keep]
     int n_cached = 0, head = 0;  // head = slot of the oldest cached chunk
+    int n_sink = 0;              // sink chunks held (slots P, P + 1, ...)
     long long absorbed = 0;
     unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
     int sel_keep = 0;
@@ -60,6 +61,7 @@ struct hf_ctx {
     hf_config cfg;
     int device = 0, sm_count = 0;
     int BH = 0, Tc = 0, n_b = 0, P = 0, Tm = 0, max_Tn = 0, mask_words = 0, d = 0;
+    int n_sink_max = 0;              // sink chunks of the configuration; ring and sink share one allocation of P + n_sink_max slots
     size_t chunk_elems = 0, pooled_elems = 0;
     std::vector<LayerState> layers;
     float* pooled_q = nullptr;
@@ -115,11 +117,15 @@ hf_status validate(const hf_config& g) {
     if (!(g.eps >= 0.f)) return fail(HF_ERR_SHAPE, "eps must be >= 0");
     if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05_PINGPONG) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
     if (g.z_mode != HF_Z_SUM && g.z_mode != HF_Z_FRAME_MEAN) return fail(HF_ERR_UNSUPPORTED, "z_mode %d unknown", g.z_mode);
+    if (g.sink_frames < 0 || g.sink_frames % g.chunk_frames != 0) return fail(HF_ERR_SHAPE, "sink_frames must be a non-negative multiple of chunk_frames");
+    if (g.sink_frames / g.chunk_frames + g.window_frames / g.chunk_frames > HF_MAX_CHUNKS)
+        return fail(HF_ERR_SHAPE, "sink chunks + window chunks exceed %d", HF_MAX_CHUNKS);
     const long long Tc = (long long)g.tokens_per_frame * g.chunk_frames;
     const long long n_b = (Tc + g.block - 1) / g.block;
     if (Tc > (1 << 20)) return fail(HF_ERR_SHAPE, "chunk of %lld tokens too large", Tc);
-    if (n_b * (g.window_frames / g.chunk_frames) > HF_MAX_TN)
-        return fail(HF_ERR_SHAPE, "window spans %lld key blocks, more than %d", n_b * (g.window_frames / g.chunk_frames), HF_MAX_TN);
+    if (n_b * (g.window_frames / g.chunk_frames + g.sink_frames / g.chunk_frames) > HF_MAX_TN)
+        return fail(HF_ERR_SHAPE, "window and sink span %lld key blocks, more than %d",
+                    n_b * (g.window_frames / g.chunk_frames + g.sink_frames / g.chunk_frames), HF_MAX_TN);
     if ((long long)g.batch * g.heads > 65535) return fail(HF_ERR_SHAPE, "batch*heads exceeds 65535");
     return HF_OK;
 }
@@ -245,16 +251,17 @@ hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16
 ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v_cur) {
     ChunkTable t;
     memset(&t, 0, sizeof(t));
-    for (int i = 0; i < L.n_cached; ++i) {
-        const int slot = (L.head + i) % c->P;
+    const int n_old = L.n_sink + L.n_cached;
+    for (int i = 0; i < n_old; ++i) {       // sink chunks first, then the cached chunks oldest first
+        const int slot = i < L.n_sink ? c->P + i : (L.head + i - L.n_sink) % c->P;
         t.k[i] = L.ring_k + (size_t)slot * c->chunk_elems;
         t.v[i] = L.ring_v + (size_t)slot * c->chunk_elems;
         t.pooled[i] = L.pooled_k + (size_t)slot * c->pooled_elems;
     }
-    t.k[L.n_cached] = k_cur;
-    t.v[L.n_cached] = v_cur;
-    t.pooled[L.n_cached] = c->pooled_kcur;
-    t.n_chunks = L.n_cached + 1;
+    t.k[n_old] = k_cur;
+    t.v[n_old] = v_cur;
+    t.pooled[n_old] = c->pooled_kcur;
+    t.n_chunks = n_old + 1;
     return t;
 }
 
@@ -266,7 +273,7 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     jobs.job[0].src = q;     jobs.job[0].pooled = c->pooled_q;
     jobs.job[1].src = k_cur; jobs.job[1].pooled = c->pooled_kcur;
     HF_TRY(launch_pool<D>(c, jobs, 2, st));
-    const int Tn = (L.n_cached + 1) * c->n_b;
+    const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     const int keep = keep_for(c, Tn);
     ChunkTable tab = make_table(c, L, k_cur, nullptr);
     k_select<D><<<dim3(c->Tm, c->BH), 128, 0, st>>>(tab, c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
@@ -304,12 +311,12 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     HF_TRY(make_map(c, &tk, k_cur, 1));
     HF_TRY(make_map(c, &tv, v_cur, 1));
     Tc5Params p;
-    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head;
-    p.P = c->P > 0 ? c->P : 1;
+    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.n_sink = L.n_sink;
+    p.P = c->P;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
-    const CUtensorMap& rk = c->P > 0 ? L.tm_kring : tk;
-    const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
+    const CUtensorMap& rk = c->P + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     k_swa_tc5<D, Tc5Groups<D>::N><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
@@ -329,12 +336,12 @@ hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16*
     HF_TRY(make_map(c, &tk, k_cur, 1));
     HF_TRY(make_map(c, &tv, v_cur, 1));
     Tc5Params p;
-    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head;
-    p.P = c->P > 0 ? c->P : 1;
+    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.n_sink = L.n_sink;
+    p.P = c->P;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
-    const CUtensorMap& rk = c->P > 0 ? L.tm_kring : tk;
-    const CUtensorMap& rv = c->P > 0 ? L.tm_vring : tv;
+    const CUtensorMap& rk = c->P + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     k_swa_tc5p<D, HF_TC5P_COLGROUPS><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
@@ -415,7 +422,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->n_b = (c->Tc + cfg->block - 1) / cfg->block;
     c->Tm = c->n_b;
     c->P = cfg->window_frames / cfg->chunk_frames - 1;
-    c->max_Tn = (c->P + 1) * c->n_b;
+    c->n_sink_max = cfg->sink_frames / cfg->chunk_frames;
+    c->max_Tn = (c->P + c->n_sink_max + 1) * c->n_b;
     c->mask_words = (c->max_Tn + 31) / 32;
     c->chunk_elems = (size_t)c->BH * c->Tc * c->d;
     c->pooled_elems = (size_t)c->BH * c->n_b * c->d;
@@ -439,9 +447,10 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->layers.resize(cfg->layers);
     const size_t dd = (size_t)c->BH * c->d * c->d, dz = (size_t)c->BH * c->d;
     for (auto& L : c->layers) {
-        if (s == HF_OK) s = dmalloc(&L.ring_k, (size_t)c->P * c->chunk_elems);
-        if (s == HF_OK) s = dmalloc(&L.ring_v, (size_t)c->P * c->chunk_elems);
-        if (s == HF_OK) s = dmalloc(&L.pooled_k, (size_t)c->P * c->pooled_elems);
+        const size_t slots = (size_t)c->P + c->n_sink_max;      // ring slots, then sink slots
+        if (s == HF_OK) s = dmalloc(&L.ring_k, slots * c->chunk_elems);
+        if (s == HF_OK) s = dmalloc(&L.ring_v, slots * c->chunk_elems);
+        if (s == HF_OK) s = dmalloc(&L.pooled_k, slots * c->pooled_elems);
         if (s == HF_OK) s = dmalloc(&L.S, dd);
         if (s == HF_OK) s = dmalloc(&L.z, dz);
         if (s == HF_OK) s = dmalloc(&L.sf_hi, dd);
@@ -450,8 +459,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
         if (s == HF_OK) s = dmalloc(&L.mask, (size_t)c->BH * c->Tm * c->mask_words);
         if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
-        if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_kring, L.ring_k, c->P);
-        if (s == HF_OK && c->P > 0) s = make_map(c, &L.tm_vring, L.ring_v, c->P);
+        if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_kring, L.ring_k, (int)slots);
+        if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_vring, L.ring_v, (int)slots);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sfhi, L.sf_hi, c->d, 1, 64, c->d, true);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sflo, L.sf_lo, c->d, 1, 64, c->d, true);
         if (s != HF_OK) break;
@@ -509,7 +518,7 @@ hf_status hf_reset(hf_ctx* c, int layer, void* stream) {
         HF_CUDA(cudaMemsetAsync(L.z, 0, dz * 4, st));
         HF_CUDA(cudaMemsetAsync(L.sf_hi, 0, dd * 2, st));
         HF_CUDA(cudaMemsetAsync(L.sf_lo, 0, dd * 2, st));
-        L.n_cached = 0; L.head = 0; L.absorbed = 0; L.cache_epoch++; L.sel_epoch = ~0ull;
+        L.n_cached = 0; L.head = 0; L.n_sink = 0; L.absorbed = 0; L.cache_epoch++; L.sel_epoch = ~0ull;
     }
     return HF_OK;
 }
@@ -547,6 +556,18 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     HF_TRY(check_ptr(v, "v"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
+    if (L.n_sink < c->n_sink_max) {   // the stream's first chunks are the attention sink: kept in slots of their own for good
+        const int slot = c->P + L.n_sink;
+        PoolJobs jobs;
+        memset(&jobs, 0, sizeof(jobs));
+        jobs.job[0].src = (const bf16*)k; jobs.job[0].copy_dst = L.ring_k + (size_t)slot * c->chunk_elems;
+        jobs.job[0].pooled = L.pooled_k + (size_t)slot * c->pooled_elems;
+        jobs.job[1].src = (const bf16*)v; jobs.job[1].copy_dst = L.ring_v + (size_t)slot * c->chunk_elems;
+        HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
+        L.n_sink++;
+        L.cache_epoch++;
+        return HF_OK;
+    }
     if (c->P == 0) {   // window == chunk: a committed chunk leaves the window at once
         HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, (const bf16*)k, (const bf16*)v, c->Tc, st));
         L.absorbed += c->Tc;
@@ -596,7 +617,7 @@ hf_status hf_sparse_swa(hf_ctx* c, int layer, const void* q, const void* k_cur, 
     HF_TRY(check_ptr(v_cur, "v_cur"));
     HF_TRY(check_ptr(o_local, "o_local"));
     LayerState& L = c->layers[layer];
-    const int keep = keep_for(c, (L.n_cached + 1) * c->n_b);
+    const int keep = keep_for(c, (L.n_sink + L.n_cached + 1) * c->n_b);
     if (idx == nullptr) {
         if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
         idx = L.idx;
@@ -675,7 +696,7 @@ hf_status hf_query(hf_ctx* c, int layer, int what, int64_t* value) {
     HF_TRY(check_layer(c, layer));
     if (value == nullptr) return fail(HF_ERR_INVALID_ARG, "value is null");
     LayerState& L = c->layers[layer];
-    const int Tn = (L.n_cached + 1) * c->n_b;
+    const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     switch (what) {
         case HF_Q_CACHED_CHUNKS: *value = L.n_cached; break;
         case HF_Q_KEY_BLOCKS: *value = Tn; break;
@@ -684,6 +705,7 @@ hf_status hf_query(hf_ctx* c, int layer, int what, int64_t* value) {
         case HF_Q_QUERY_BLOCKS: *value = c->Tm; break;
         case HF_Q_MASK_WORDS: *value = c->mask_words; break;
         case HF_Q_SWA_KERNEL: *value = c->swa_kernel; break;
+        case HF_Q_SINK_CHUNKS: *value = L.n_sink; break;
         default: return fail(HF_ERR_INVALID_ARG, "unknown query %d", what);
     }
     return HF_OK;

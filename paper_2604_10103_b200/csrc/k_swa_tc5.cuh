@@ -47,7 +47,8 @@ struct SwaTc5 {
 
 struct Tc5Params {
     const int32_t* idx;      // [B*H, T_m, keep]
-    int keep, Tc, n_b, n_cached, ring_head, P;
+    int keep, Tc, n_b, n_cached, ring_head, P;   // P: ring slots (the cache's past chunks); the sink slots follow them
+    int n_sink;              // sink chunks held (logical chunks 0 .. n_sink - 1)
     int Tm, n_units;         // units = (batch*head, query block) pairs, unit u = bh * Tm + i
     float scale_log2;
     const float* hist;       // optional fp32 [B*H, T_c, D]
@@ -131,9 +132,13 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     const int blk = __ldg(my_idx + j);
                     int c = 0, jb = blk;
                     while (jb >= p.n_b) { jb -= p.n_b; ++c; }          // at most HF_MAX_CHUNKS - 1 steps; no XU-pipe division
-                    const bool cur = (c == p.n_cached);
-                    int slot = cur ? 0 : p.ring_head + c;
-                    if (slot >= p.P) slot -= p.P;
+                    // logical chunk order: sink chunks (slots P, P + 1, ...), cached chunks oldest first (ring), current chunk
+                    const bool cur = (c == p.n_sink + p.n_cached);
+                    int slot = 0;
+                    if (!cur) {
+                        if (c < p.n_sink) slot = p.P + c;
+                        else { slot = p.ring_head + c - p.n_sink; if (slot >= p.P) slot -= p.P; }
+                    }
                     if (is_k) {
                         const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
                         if (t >= C::KSTAGES && !(ok = mbar_wait<true>(bar_ke + 8 * rk.stage, rk.phase ^ 1u, abort_flag, p.dev_status, 2))) break;

@@ -108,9 +108,13 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     const int blk = __ldg(my_idx + j);
                     int c = 0, jb = blk;
                     while (jb >= p.n_b) { jb -= p.n_b; ++c; }          // at most HF_MAX_CHUNKS - 1 steps; no XU-pipe division
-                    const bool cur = (c == p.n_cached);
-                    int slot = cur ? 0 : p.ring_head + c;
-                    if (slot >= p.P) slot -= p.P;
+                    // logical chunk order: sink chunks (slots P, P + 1, ...), cached chunks oldest first (ring), current chunk
+                    const bool cur = (c == p.n_sink + p.n_cached);
+                    int slot = 0;
+                    if (!cur) {
+                        if (c < p.n_sink) slot = p.P + c;
+                        else { slot = p.ring_head + c - p.n_sink; if (slot >= p.P) slot -= p.P; }
+                    }
                     if (is_k) {
                         const CUtensorMap* mk = cur ? &tm_kcur : &tm_kring;
                         if (t >= C::KSTAGES && !(ok = mbar_wait<true>(bar_ke + 8 * rk.stage, rk.phase ^ 1u, abort_flag, p.dev_status, 2))) break;

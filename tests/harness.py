@@ -21,7 +21,8 @@ def max_abs(a, b):
     return float(np.abs(np.asarray(a, np.float64) - np.asarray(b, np.float64)).max())
 
 
-def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, z_frame_mean: bool = False):
+def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, z_frame_mean: bool = False,
+                sink_chunks: int = 0):
     W = b = None
     if merge:
         Wb, bb = gen.merge_weights(w, layer, with_bias=bias)
@@ -29,7 +30,7 @@ def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool 
         b = None if bb is None else gen.bf16_bits_to_f64(bb)
     return oa.HybridStream(w.batch, w.heads, w.head_dim, w.block, w.past_chunks, topk=w.topk,
                            keep_permille=w.keep_permille, W=W, bias=b, eps=w.eps,
-                           z_frame_tokens=w.tokens_per_frame if z_frame_mean else None)
+                           z_frame_tokens=w.tokens_per_frame if z_frame_mean else None, sink_chunks=sink_chunks)
 
 
 from paper_2604_10103_b200.binding import unpack_mask  # noqa: E402,F401
@@ -39,13 +40,14 @@ class GpuStream:
     """The library side of a one-layer stream (torch only for memory)."""
 
     def __init__(self, w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, swa_kernel: int = 0,
-                 layers: int | None = None, z_frame_mean: bool = False):
+                 layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0):
         import torch
         from paper_2604_10103_b200 import binding as hf
         self.torch, self.hf, self.w, self.layer = torch, hf, w, layer
         cfg = hf.make_config(w.with_(layers=layers or max(w.layers, layer + 1)),
                              merge=hf.HF_MERGE_PER_HEAD if merge else hf.HF_MERGE_IDENTITY, swa_kernel=swa_kernel,
-                             z_mode=hf.HF_Z_FRAME_MEAN if z_frame_mean else hf.HF_Z_SUM)
+                             z_mode=hf.HF_Z_FRAME_MEAN if z_frame_mean else hf.HF_Z_SUM,
+                             sink_frames=sink_chunks * w.chunk_frames)
         self.ctx = hf.Context(cfg)
         if merge:
             Wb, bb = gen.merge_weights(w, layer, with_bias=bias)

@@ -275,3 +275,37 @@ def test_pingpong_single_kept_block_and_lse():
     w = gen.Workload("pp1", batch=1, heads=2, head_dim=128, tokens_per_frame=256, chunk_frames=1, window_frames=3,
                      block=128, topk=1, keep_permille=0, seed=16)
     stream_compare(w, 4, swa_kernel=hf.HF_SWA_TCGEN05_PINGPONG)
+
+
+@pytest.mark.parametrize("d,b,tpf,wf,sink,kernel", [
+    (128, 128, 300, 2, 1, 0),    # tcgen05 path, one sink chunk + one cached chunk
+    (128, 128, 260, 3, 2, 3),    # ping-pong kernel, two sink chunks
+    (64, 16, 64, 3, 1, 0),       # small blocks (warp-level tensor path)
+    (128, 128, 200, 1, 1, 0),    # window == chunk: no rolling cache at all, only sink + current + state
+])
+def test_sink_chunks(d, b, tpf, wf, sink, kernel):
+    """Attention sink: the first chunks of the stream stay visible as the oldest key blocks, are never evicted and
+    never reach the state (cache bookkeeping, masks, outputs and state against the oracle run the same way)."""
+    w = gen.Workload("sink", batch=1, heads=3, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=wf,
+                     block=b, topk=0, keep_permille=500, seed=17)
+    gpu = hz.GpuStream(w, sink_chunks=sink, swa_kernel=kernel); ora = hz.make_oracle(w, sink_chunks=sink)
+    try:
+        for c in range(sink + wf + 2):
+            qb, kb, vb = gen.qkv(w, 0, c, 0)
+            q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+            m_gpu, _, sc_gpu = gpu.select(q, k)
+            m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+            assert np.array_equal(sc_gpu, sc_ref) and np.array_equal(m_gpu, m_ref), f"chunk {c}"
+            o_ref = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref)
+            hz.assert_close_out(gpu.forward(q, k, v), o_ref, f"chunk {c} hybrid O with sink")
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+            assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_SINK_CHUNKS) == len(ora.sink)
+            assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_CACHED_CHUNKS) == len(ora.past)
+            assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_ABSORBED_TOKENS) == ora.absorbed_tokens
+        S, z = gpu.state()
+        assert ora.absorbed_tokens > 0
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2 and hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()

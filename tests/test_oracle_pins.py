@@ -406,3 +406,44 @@ def test_stream_with_frame_mean_matches_one_shot():
     ev = np.concatenate([x[0, 0] for x in ks[:3]])
     z_ref = sum(oa.phi(ev[i * 4:(i + 1) * 4]).mean(axis=0) for i in range(6))
     assert np.allclose(st.z[0, 0], z_ref, rtol=0, atol=1e-13) and st.absorbed_tokens == 24
+
+
+# ----------------------------------------------------------------------------- attention sink (first chunks kept for ever)
+def test_sink_chunks_partition_and_brute_force():
+    """With s sink chunks the first s committed chunks stay visible as the oldest key blocks, are never evicted and
+    never absorbed: window tokens, sink tokens and absorbed tokens partition everything committed so far; the
+    forward equals a token-level masked softmax over [sink | cached | current] plus the read-out of a state built
+    from the absorbed chunks alone."""
+    B, H, d, b, P, s, n = 1, 1, 32, 4, 1, 1, 8
+    st = oa.HybridStream(B, H, d, b, P, topk=2, sink_chunks=s)
+    ks = [rnd((B, H, n, d), 70 + i) for i in range(5)]; vs = [rnd((B, H, n, d), 80 + i) for i in range(5)]
+    for c in range(5):
+        st.append(ks[c], vs[c])
+        n_abs = max(0, c + 1 - s - P)
+        assert len(st.sink) == min(c + 1, s) and len(st.past) == min(max(c + 1 - s, 0), P)
+        assert st.absorbed_tokens == n_abs * n
+    # after 5 appends with s = 1, P = 1: sink = {0}, cached = {4}, absorbed = {1, 2, 3}
+    S_ref, z_ref = np.zeros((d, d)), np.zeros(d)
+    for c in (1, 2, 3):
+        S_ref, z_ref = oa.absorb(S_ref, z_ref, ks[c][0, 0], vs[c][0, 0])
+    assert np.allclose(st.S[0, 0], S_ref, atol=1e-12) and np.allclose(st.z[0, 0], z_ref, atol=1e-12)
+    assert st.sink[0][0] is not None and np.array_equal(st.sink[0][0], ks[0]) and np.array_equal(st.past[0][0], ks[4])
+    q = rnd((B, H, n, d), 90); kc = rnd((B, H, n, d), 91); vc = rnd((B, H, n, d), 92)
+    mask, _ = st.select(q, kc)
+    assert mask.shape == (B, H, 2, 6)      # 2 query blocks x (2 sink + 2 cached + 2 current) key blocks
+    o, ol, oh = st.forward(q, kc, vc, mask=mask, parts=True)
+    kall = np.concatenate([ks[0][0, 0], ks[4][0, 0], kc[0, 0]]); vall = np.concatenate([vs[0][0, 0], vs[4][0, 0], vc[0, 0]])
+    for r in range(n):
+        keep_cols = np.repeat(mask[0, 0, r // b], b)
+        sc = np.array([q[0, 0, r] @ kall[c] / math.sqrt(d) if keep_cols[c] else -np.inf for c in range(3 * n)])
+        w = np.exp(sc - sc.max()); w /= w.sum()
+        assert np.allclose(ol[0, 0, r], w @ vall, atol=1e-12)
+    assert np.allclose(oh[0, 0], oa.linear_readout(q[0, 0], S_ref, z_ref), atol=1e-12)
+
+
+def test_no_sink_is_the_default_protocol():
+    a = oa.HybridStream(1, 1, 8, 4, 1, topk=1); b_ = oa.HybridStream(1, 1, 8, 4, 1, topk=1, sink_chunks=0)
+    for i in range(3):
+        k = rnd((1, 1, 8, 8), 95 + i); v = rnd((1, 1, 8, 8), 98 + i)
+        a.append(k, v); b_.append(k, v)
+    assert np.array_equal(a.S, b_.S) and a.absorbed_tokens == b_.absorbed_tokens == 16 and not b_.sink
