@@ -92,6 +92,15 @@ hf_status hf_reset(hf_ctx* ctx, int layer, void* stream);
  * or NULL.  Copied into the context.  HF_ERR_STATE if the context was created with HF_MERGE_IDENTITY. */
 hf_status hf_set_merge_weights(hf_ctx* ctx, int layer, const void* W, const void* bias, void* stream);
 
+/* Rotation inside the linear branch (Eq. 3: RoPE(phi(K))^T V in the state; Eq. 4: RoPE(phi(Q)) in the numerator only, the
+ * normaliser never rotates).  The rotation acts on feature pairs (2i, 2i+1); the angles are the caller's: device float
+ * tables cos / sin [T_c, d/2], one row per token of a chunk, shared by batch, heads and layers (e.g. built from the
+ * capped relative temporal index of Eq. 8 and the spatial coordinates).  cos_q / sin_q rotate the queries of every later
+ * hf_linear_attn / hf_hybrid_forward; cos_k / sin_k rotate the keys of every chunk folded into the state from now on
+ * (they are applied when the chunk is absorbed).  The tables are copied into the context.  A NULL pair switches that
+ * rotation off (the default).  With key tables set, hf_state_absorb accepts at most T_c tokens per call. */
+hf_status hf_set_rope(hf_ctx* ctx, const float* cos_q, const float* sin_q, const float* cos_k, const float* sin_k, void* stream);
+
 /* Alg. 2, cache commit of a clean chunk: k, v bf16 [B,H,T_c,d].  If the cache already holds P chunks the oldest
  * is first folded into the state (Eq. 3: S += phi(K_ev)^T V_ev, z += sum phi(K_ev)) and its slot reused; the
  * chunk's K, V are copied in and its per-block K means stored.  With P = 0 the chunk goes straight into the

@@ -21,7 +21,9 @@ What follows which passage:
   sparse_attention_tiled  Alg. 3 inner loops (running max / sum / rescale), step by step
   absorb                  Eq. 3 (state update) without the rotation
   absorb_frame_mean       Eq. 3 with H accumulated as printed: per evicted frame the mean of phi(K) over its tokens
-  linear_readout          Eq. 4 without the rotation: Linear(phi(Q) L / (phi(Q) H))
+  linear_readout          Eq. 4: Linear(phi(Q) L / (phi(Q) H)), optionally with RoPE(phi(Q)) in the numerator
+  rotate_pairs, absorb_rope        the rotation of Eq. 3 / Eq. 4 on feature pairs (2i, 2i+1); angles are inputs
+  relative_temporal_indices        Eq. 8 (capped relative temporal index)
   HybridStream            Alg. 2 cache protocol (evict -> update state -> append) around Alg. 3, Eq. 7 sum
 
 Readings taken where the paper is silent or inconsistent (all listed again in the
@@ -230,10 +232,39 @@ def absorb_frame_mean(S: np.ndarray, z: np.ndarray, k_ev, v_ev, frame_tokens: in
     return S + f.T @ np.asarray(v_ev, np.float64), z + zinc
 
 
-def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6) -> np.ndarray:
-    """O_history (Eq. 4): h = phi(q) S / (phi(q) . z + eps) per query row, then Linear: y = W h + bias."""
+def rotate_pairs(x, cos, sin) -> np.ndarray:
+    """RoPE on feature pairs (2i, 2i+1): x [T, d], cos / sin [T, d/2] (one angle per token and pair).
+    out[2i] = x[2i] cos_i - x[2i+1] sin_i,  out[2i+1] = x[2i] sin_i + x[2i+1] cos_i."""
+    x = np.asarray(x, np.float64); cos = np.asarray(cos, np.float64); sin = np.asarray(sin, np.float64)
+    out = np.empty_like(x)
+    out[:, 0::2] = x[:, 0::2] * cos - x[:, 1::2] * sin
+    out[:, 1::2] = x[:, 0::2] * sin + x[:, 1::2] * cos
+    return out
+
+
+def absorb_rope(S: np.ndarray, z: np.ndarray, k_ev, v_ev, cos_k, sin_k, frame_tokens=None):
+    """Eq. 3 with its rotation: S += RoPE(phi(K_ev))^T V_ev; the normaliser keeps the unrotated phi(K_ev)
+    (sum over tokens, or per-frame means when frame_tokens is given)."""
+    f = phi(k_ev)
+    S = S + rotate_pairs(f, cos_k, sin_k).T @ np.asarray(v_ev, np.float64)
+    if frame_tokens is None:
+        return S, z + f.sum(axis=0)
+    _, z2 = absorb_frame_mean(np.zeros_like(S), z, k_ev, np.zeros_like(np.asarray(v_ev, np.float64)), frame_tokens)
+    return S, z2
+
+
+def relative_temporal_indices(i: int, t0: int):
+    """Eq. 8: temporal RoPE indices of the three frames of the chunk that ends at (1-based) frame i, capped at the
+    largest index T_0 the pretrained model has seen."""
+    return [i - 2, i - 1, i] if i <= t0 else [t0 - 2, t0 - 1, t0]
+
+
+def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6, cos_q=None, sin_q=None) -> np.ndarray:
+    """O_history (Eq. 4): h = phi(q) S / (phi(q) . z + eps) per query row, then Linear: y = W h + bias.
+    With cos_q / sin_q [T, d/2] the numerator uses RoPE(phi(q)) (Eq. 4 as printed); the denominator never rotates."""
     f = phi(q)
-    h = (f @ S) / (f @ z + eps)[:, None]
+    fn = f if cos_q is None else rotate_pairs(f, cos_q, sin_q)      # Eq. 4: rotation in the numerator only
+    h = (fn @ S) / (f @ z + eps)[:, None]
     if W is not None:
         h = h @ np.asarray(W, np.float64).T
     if bias is not None:
@@ -254,12 +285,13 @@ class HybridStream:
     """
 
     def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
-                 W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0):
+                 W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0, rope_q=None, rope_k=None):
         self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
         self.z_frame_tokens = z_frame_tokens     # None: z is the plain sum of phi(K); n: per-frame means of n tokens (Eq. 3 literal)
         self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
         self.W = None if W is None else np.asarray(W, np.float64)        # [H, d, d]
         self.bias = None if bias is None else np.asarray(bias, np.float64)  # [H, d]
+        self.rope_q, self.rope_k = rope_q, rope_k    # (cos, sin) tables [T_c, d/2] of the linear branch, or None
         self.sink_chunks = sink_chunks   # the first chunks of the stream stay visible for ever ("sink"): never evicted, never absorbed
         self.sink = []                                                   # list of (k, v) like self.past, oldest first
         self.past = []                                                   # list of (k [B,H,n,d], v) fp64
@@ -277,7 +309,10 @@ class HybridStream:
             k_ev, v_ev = self.past.pop(0)
             for bi in range(self.B):
                 for h in range(self.H):
-                    if self.z_frame_tokens is None:
+                    if self.rope_k is not None:
+                        self.S[bi, h], self.z[bi, h] = absorb_rope(self.S[bi, h], self.z[bi, h], k_ev[bi, h], v_ev[bi, h],
+                                                                   self.rope_k[0], self.rope_k[1], self.z_frame_tokens)
+                    elif self.z_frame_tokens is None:
                         self.S[bi, h], self.z[bi, h] = absorb(self.S[bi, h], self.z[bi, h], k_ev[bi, h], v_ev[bi, h])
                     else:
                         self.S[bi, h], self.z[bi, h] = absorb_frame_mean(self.S[bi, h], self.z[bi, h], k_ev[bi, h],
@@ -328,7 +363,9 @@ class HybridStream:
                 o_loc[bi, h] = sparse_attention(q[bi, h], kc, vc, self.b, mask[bi, h], q_blocks)
                 o_hist[bi, h] = linear_readout(q[bi, h], self.S[bi, h], self.z[bi, h],
                                                None if self.W is None else self.W[h],
-                                               None if self.bias is None else self.bias[h], self.eps)
+                                               None if self.bias is None else self.bias[h], self.eps,
+                                               None if self.rope_q is None else self.rope_q[0],
+                                               None if self.rope_q is None else self.rope_q[1])
         if parts:
             return o_loc + o_hist, o_loc, o_hist
         return o_loc + o_hist

@@ -27,7 +27,7 @@ EXPORTS = [
     "hf_create", "hf_destroy", "hf_reset", "hf_set_merge_weights", "hf_kv_append", "hf_state_absorb",
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
-    "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc",
+    "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope",
 ]
 
 
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
     L.hf_destroy.argtypes = [vp]
     L.hf_reset.argtypes = [vp, ip, vp]
     L.hf_set_merge_weights.argtypes = [vp, ip, vp, vp, vp]
+    L.hf_set_rope.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hf_kv_append.argtypes = [vp, ip, vp, vp, vp]
     L.hf_state_absorb.argtypes = [vp, ip, vp, vp, ip, vp]
     L.hf_block_select.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp]
@@ -134,6 +135,10 @@ class Context:
 
     def hf_set_merge_weights(self, layer, W, bias=None):
         _check(lib().hf_set_merge_weights(self._h, layer, _ptr(W), _ptr(bias), _stream()))
+
+    def hf_set_rope(self, cos_q=None, sin_q=None, cos_k=None, sin_k=None):
+        """float32 CUDA tensors [T_c, d/2] (or None) -- see include/hf.h."""
+        _check(lib().hf_set_rope(self._h, _ptr(cos_q), _ptr(sin_q), _ptr(cos_k), _ptr(sin_k), _stream()))
 
     def hf_kv_append(self, layer, k, v):
         _check(lib().hf_kv_append(self._h, layer, _ptr(k), _ptr(v), _stream()))

@@ -72,6 +72,9 @@ struct hf_ctx {
     float z_scale = 1.f;             // 1 (z = sum of phi(K)) or 1 / tokens_per_frame (per-frame means)
     bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
     int* dev_status = nullptr;
+    float* rope_q[2] = {nullptr, nullptr};   // cos / sin tables [T_c, d/2] of Eq. 4's numerator (nullptr: no rotation)
+    float* rope_k[2] = {nullptr, nullptr};   // ... of Eq. 3, applied to a chunk when it is absorbed
+    bool has_rope_q = false, has_rope_k = false;
     cudaStream_t side = nullptr;     // hf_hybrid_forward runs the history read-out here, beside pooling + selection
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     long long launches = 0;
@@ -147,6 +150,7 @@ void free_all(hf_ctx* c) {
     }
     cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials);
     cudaFree(c->dev_status);
+    cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
@@ -160,8 +164,10 @@ hf_status set_swa_attr() {
 }
 template <int D>
 hf_status set_state_attr() {
-    HF_CUDA(cudaFuncSetAttribute(k_absorb_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbTc5<D>::SMEM_BYTES));
-    HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_tc5<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_tc5<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
     return HF_OK;
 }
 
@@ -224,7 +230,9 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     HF_TRY(make_map_ex(c, &tv, v, n_tokens, 1, 64, A::TT, true));
     AbsorbTc5Params p;
     p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
-    k_absorb_tc5<D><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
+    p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc;
+    if (c->has_rope_k) k_absorb_tc5<D, true><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
+    else k_absorb_tc5<D, false><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
     HF_TRY(post_launch(c, "k_absorb_tc5"));
     if (!fold_on_side) return launch_fold<D>(c, L, nsplit, st);
     HF_CUDA(cudaEventRecord(c->ev_fork, st));
@@ -240,11 +248,13 @@ hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16
     CUtensorMap tq;
     HF_TRY(make_map(c, &tq, q, 1));
     ReadoutTc5Params p;
+    p.cos_q = c->rope_q[0]; p.sin_q = c->rope_q[1];
     p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr; p.heads = c->cfg.heads; p.Tc = c->Tc;
     p.Tm = (c->Tc + R::ROWS - 1) / R::ROWS; p.n_units = p.Tm * c->BH; p.eps = c->cfg.eps;
     p.out_bf16 = out_bf16; p.out_f32 = out_f32; p.dev_status = c->dev_status;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
-    k_readout_tc5<D><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
+    if (c->has_rope_q) k_readout_tc5<D, true><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
+    else k_readout_tc5<D, false><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
     return post_launch(c, "k_readout_tc5");
 }
 
@@ -537,11 +547,32 @@ hf_status hf_set_merge_weights(hf_ctx* c, int layer, const void* W, const void* 
     return HF_DISPATCH_D(c, launch_fold, c, L, 0, st);
 }
 
+hf_status hf_set_rope(hf_ctx* c, const float* cos_q, const float* sin_q, const float* cos_k, const float* sin_k, void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    if ((cos_q == nullptr) != (sin_q == nullptr) || (cos_k == nullptr) != (sin_k == nullptr))
+        return fail(HF_ERR_INVALID_ARG, "cos and sin tables come in pairs");
+    const float* src[4] = {cos_q, sin_q, cos_k, sin_k};
+    float** dst[4] = {&c->rope_q[0], &c->rope_q[1], &c->rope_k[0], &c->rope_k[1]};
+    const size_t count = (size_t)c->Tc * (c->d / 2);
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int i = 0; i < 4; ++i) {
+        if (src[i] == nullptr) continue;
+        HF_TRY(check_ptr(src[i], "rotation table"));
+        if (*dst[i] == nullptr) HF_TRY(dmalloc(dst[i], count));
+        HF_CUDA(cudaMemcpyAsync(*dst[i], src[i], count * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    }
+    c->has_rope_q = cos_q != nullptr;
+    c->has_rope_k = cos_k != nullptr;
+    return HF_OK;
+}
+
 hf_status hf_state_absorb(hf_ctx* c, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream) {
     HF_TRY(check_layer(c, layer));
     HF_TRY(check_ptr(k_ev, "k_ev"));
     HF_TRY(check_ptr(v_ev, "v_ev"));
     if (n_tokens < 1) return fail(HF_ERR_SHAPE, "n_tokens must be >= 1");
+    if (c->has_rope_k && n_tokens > c->Tc)
+        return fail(HF_ERR_SHAPE, "with rotation tables set, n_tokens may not exceed the chunk length (%d)", c->Tc);
     if (c->cfg.z_mode == HF_Z_FRAME_MEAN && n_tokens % c->cfg.tokens_per_frame != 0)
         return fail(HF_ERR_SHAPE, "with HF_Z_FRAME_MEAN n_tokens must be a multiple of tokens_per_frame (%d)", c->cfg.tokens_per_frame);
     LayerState& L = c->layers[layer];

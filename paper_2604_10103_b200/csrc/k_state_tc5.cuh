@@ -36,13 +36,16 @@ struct AbsorbTc5 {
 };
 
 struct AbsorbTc5Params {
+    const float* cos_k;       // rotation tables of Eq. 3, [rope_rows, D/2] each (used by the ROPE instantiation only)
+    const float* sin_k;
+    int rope_rows;
     int n_tokens;
     float* partials;          // [B*H, nsplit, D*D + D]
     int* dev_status;
 };
 
 // grid (nsplit, B*H).  tm_k: [D, n_tokens, B*H, 1] box {D, 64}, no swizzle.  tm_v: same tensor shape, box {64, 64}, 128B swizzle.
-template <int D>
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(AbsorbTc5<D>::THREADS, 1)
 k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const AbsorbTc5Params p) {
     using namespace tc5;
@@ -162,7 +165,18 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
                         if (t >= nv) f0 = 0.f;
                         if (t + 1 >= nv) f1 = 0.f;
                     }
-                    zacc += f0 + f1;
+                    zacc += f0 + f1;                            // the normaliser keeps the unrotated values
+                    if (ROPE) {
+                        // feature pairs (2i, 2i+1) sit in neighbouring lanes; the pair's angle belongs to the token
+                        const float g0 = __shfl_xor_sync(0xffffffffu, f0, 1), g1 = __shfl_xor_sync(0xffffffffu, f1, 1);
+                        const int tok = (tile_lo + i) * C::TT + part * HT + t;     // rows past the tables belong to masked tokens
+                        const size_t o0 = (size_t)min(tok, p.rope_rows - 1) * (D / 2) + (a >> 1);
+                        const size_t o1 = (size_t)min(tok + 1, p.rope_rows - 1) * (D / 2) + (a >> 1);
+                        const float c0 = __ldg(p.cos_k + o0), s0 = __ldg(p.sin_k + o0);
+                        const float c1 = __ldg(p.cos_k + o1), s1 = __ldg(p.sin_k + o1);
+                        f0 = (a & 1) ? fmaf(g0, s0, f0 * c0) : fmaf(-g0, s0, f0 * c0);
+                        f1 = (a & 1) ? fmaf(g1, s1, f1 * c1) : fmaf(-g1, s1, f1 * c1);
+                    }
                     const uint32_t hp = pack_bf16(f0, f1);
                     const float2 hf = unpack_bf16(hp);
                     hi[t >> 1] = hp;
@@ -253,6 +267,8 @@ struct ReadoutTc5 {
 };
 
 struct ReadoutTc5Params {
+    const float* cos_q;       // rotation tables of Eq. 4's numerator, [T_c, D/2] each (ROPE instantiation only)
+    const float* sin_q;
     const float* z;           // [B*H, D]
     const bf16* bias;         // [H, D] or nullptr
     int heads, Tc, Tm, n_units;
@@ -264,7 +280,7 @@ struct ReadoutTc5Params {
 
 // CTA c processes units [c * upc, (c + 1) * upc), upc = ceil(n_units / gridDim.x).  tm_q: [D, T_c, B*H, 1] box {64, 128};
 // tm_sh, tm_sl: [D, D, B*H, 1] box {64, D}; all 128B swizzle.
-template <int D>
+template <int D, bool ROPE>
 __global__ void __launch_bounds__(ReadoutTc5<D>::THREADS, 1)
 k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_sh,
               const __grid_constant__ CUtensorMap tm_sl, const ReadoutTc5Params p) {
@@ -385,6 +401,7 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const int bh = u / p.Tm;
             const int s = n & 1;
             const uint32_t par = (n >> 1) & 1;
+            const int r_tab = min((u - bh * p.Tm) * C::ROWS + row, p.Tc - 1);     // row of the rotation tables
             // z and bias of the unit's head, staged by these threads once every thread has left the epilogue that read
             // the stage's buffers last (two units ago)
             float* vec = reinterpret_cast<float*>(s_gen + C::OFF_VEC + s * 2 * D * 4);
@@ -414,12 +431,23 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const int sub = chunk >> 3, phys = (chunk & 7) ^ (row & 7);
                     const uint4 w = *reinterpret_cast<const uint4*>(qt + sub * C::QSUB_BYTES + phys * 16);
                     const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+                    float cs[4] = {1.f, 1.f, 1.f, 1.f}, sn[4] = {0.f, 0.f, 0.f, 0.f};
+                    if (ROPE) {
+                        const float4 c4 = __ldg(reinterpret_cast<const float4*>(p.cos_q + (size_t)r_tab * (D / 2)) + chunk);
+                        const float4 s4 = __ldg(reinterpret_cast<const float4*>(p.sin_q + (size_t)r_tab * (D / 2)) + chunk);
+                        cs[0] = c4.x; cs[1] = c4.y; cs[2] = c4.z; cs[3] = c4.w;
+                        sn[0] = s4.x; sn[1] = s4.y; sn[2] = s4.z; sn[3] = s4.w;
+                    }
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const float2 x = unpack_bf16(ws[e]);
-                        const float f0 = phi_elu1(x.x), f1 = phi_elu1(x.y);
+                        float f0 = phi_elu1(x.x), f1 = phi_elu1(x.y);
                         const int feat = chunk * 8 + 2 * e;
-                        dsum = fmaf(f0, vec[feat], fmaf(f1, vec[feat + 1], dsum));
+                        dsum = fmaf(f0, vec[feat], fmaf(f1, vec[feat + 1], dsum));     // denominator: unrotated
+                        if (ROPE) {
+                            const float r0 = fmaf(-f1, sn[e], f0 * cs[e]), r1 = fmaf(f0, sn[e], f1 * cs[e]);
+                            f0 = r0; f1 = r1;
+                        }
                         const uint32_t hp = pack_bf16(f0, f1);
                         const float2 hf = unpack_bf16(hp);
                         hi[cc * 4 + e] = hp;

@@ -18,7 +18,7 @@ from dataclasses import dataclass, replace
 import numpy as np
 
 # tensor ids used in seeds
-T_Q, T_K, T_V, T_KCLEAN, T_VCLEAN, T_W, T_BIAS = range(7)
+T_Q, T_K, T_V, T_KCLEAN, T_VCLEAN, T_W, T_BIAS, T_ANGLE_Q, T_ANGLE_K = range(9)
 
 
 @dataclass(frozen=True)
@@ -147,3 +147,10 @@ def merge_weights(w: Workload, layer: int, with_bias: bool = True):
     W = normal_bf16((w.heads, d, d), w.seed, layer, 0, 0, T_W, scale=d ** -0.5)
     b = normal_bf16((w.heads, d), w.seed, layer, 0, 0, T_BIAS, scale=0.1) if with_bias else None
     return W, b
+
+
+def rotation_tables(w: Workload, which: int):
+    """(cos, sin) float32 tables [T_c, d/2] of seeded angles ~ U(0, 2 pi): stand-ins for the position angles a model
+    would supply to the linear branch's rotation.  `which`: T_ANGLE_Q or T_ANGLE_K."""
+    th = _rng(w.seed, 0, 0, 0, which).uniform(0.0, 2.0 * np.pi, size=(w.chunk_tokens, w.head_dim // 2))
+    return np.cos(th).astype(np.float32), np.sin(th).astype(np.float32)

@@ -22,7 +22,7 @@ def max_abs(a, b):
 
 
 def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, z_frame_mean: bool = False,
-                sink_chunks: int = 0):
+                sink_chunks: int = 0, rope: bool = False):
     W = b = None
     if merge:
         Wb, bb = gen.merge_weights(w, layer, with_bias=bias)
@@ -30,7 +30,9 @@ def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool 
         b = None if bb is None else gen.bf16_bits_to_f64(bb)
     return oa.HybridStream(w.batch, w.heads, w.head_dim, w.block, w.past_chunks, topk=w.topk,
                            keep_permille=w.keep_permille, W=W, bias=b, eps=w.eps,
-                           z_frame_tokens=w.tokens_per_frame if z_frame_mean else None, sink_chunks=sink_chunks)
+                           z_frame_tokens=w.tokens_per_frame if z_frame_mean else None, sink_chunks=sink_chunks,
+                           rope_q=gen.rotation_tables(w, gen.T_ANGLE_Q) if rope else None,
+                           rope_k=gen.rotation_tables(w, gen.T_ANGLE_K) if rope else None)
 
 
 from paper_2604_10103_b200.binding import unpack_mask  # noqa: E402,F401
@@ -40,7 +42,7 @@ class GpuStream:
     """The library side of a one-layer stream (torch only for memory)."""
 
     def __init__(self, w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, swa_kernel: int = 0,
-                 layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0):
+                 layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0, rope: bool = False):
         import torch
         from paper_2604_10103_b200 import binding as hf
         self.torch, self.hf, self.w, self.layer = torch, hf, w, layer
@@ -52,6 +54,11 @@ class GpuStream:
         if merge:
             Wb, bb = gen.merge_weights(w, layer, with_bias=bias)
             self.ctx.hf_set_merge_weights(layer, hf.bits_to_cuda(Wb), None if bb is None else hf.bits_to_cuda(bb))
+        if rope:
+            to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+            cq, sq = gen.rotation_tables(w, gen.T_ANGLE_Q); ck, sk = gen.rotation_tables(w, gen.T_ANGLE_K)
+            self.ctx.hf_set_rope(to_dev(cq), to_dev(sq), to_dev(ck), to_dev(sk))
+            torch.cuda.synchronize()
         self.shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
 
     def up(self, bits):

@@ -309,3 +309,37 @@ def test_sink_chunks(d, b, tpf, wf, sink, kernel):
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,b,tpf,cf,wf,zmean", [
+    (128, 128, 150, 2, 4, False),   # 300-token chunks (ragged tiles), one cached chunk
+    (64, 64, 100, 1, 2, True),      # head_dim 64, per-frame-mean normaliser, odd tile tails
+])
+def test_rotation_inside_the_linear_branch(d, b, tpf, cf, wf, zmean):
+    """hf_set_rope: RoPE(phi(K)) in the state (Eq. 3), RoPE(phi(Q)) in the numerator only (Eq. 4), seeded angle
+    tables as inputs; state, read-out and hybrid output against the oracle run the same way."""
+    w = gen.Workload("rope", batch=1, heads=3, head_dim=d, tokens_per_frame=tpf, chunk_frames=cf, window_frames=wf,
+                     block=b, topk=0, keep_permille=500, seed=18)
+    gpu = hz.GpuStream(w, rope=True, z_frame_mean=zmean); ora = hz.make_oracle(w, rope=True, z_frame_mean=zmean)
+    try:
+        for c in range(wf // cf + 2):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert ora.absorbed_tokens == 3 * w.chunk_tokens
+        S, z = gpu.state()
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2, f"S rel-L2 {hz.rel_l2(S, ora.S):.3e}"
+        assert hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        qb, kb, vb = gen.qkv(w, 0, 9, 0)
+        o_ref, _, oh_ref = ora.forward(f64(qb), f64(kb), f64(vb), parts=True)
+        assert hz.rel_l2(gpu.linear(gpu.up(qb)), oh_ref) <= hz.REL_L2
+        o = gpu.forward(gpu.up(qb), gpu.up(kb), gpu.up(vb))
+        assert hz.rel_l2(o, o_ref) <= hz.REL_L2
+        assert hz.max_abs(o, o_ref) <= hz.MAX_ABS + 2.0 ** -8 * np.abs(o_ref).max()
+        # the rotation matters: without the tables the state differs
+        plain = hz.make_oracle(w, z_frame_mean=zmean)
+        for c in range(wf // cf + 2):
+            kc, vc = gen.clean_kv(w, 0, c)
+            plain.append(f64(kc), f64(vc))
+        assert hz.rel_l2(S, plain.S) > 0.1
+    finally:
+        gpu.close()

@@ -447,3 +447,51 @@ def test_no_sink_is_the_default_protocol():
         k = rnd((1, 1, 8, 8), 95 + i); v = rnd((1, 1, 8, 8), 98 + i)
         a.append(k, v); b_.append(k, v)
     assert np.array_equal(a.S, b_.S) and a.absorbed_tokens == b_.absorbed_tokens == 16 and not b_.sink
+
+
+# ----------------------------------------------------------------------------- rotation inside the linear branch (Eq. 3 / Eq. 4 / Eq. 8)
+def _angles(shape, seed):
+    th = np.random.default_rng(seed).uniform(0, 2 * np.pi, size=shape)
+    return np.cos(th), np.sin(th), th
+
+
+def test_rotate_pairs_is_a_plane_rotation():
+    x = rnd((6, 8), 101); cos, sin, th = _angles((6, 4), 1)
+    y = oa.rotate_pairs(x, cos, sin)
+    for t in range(6):
+        for i in range(4):
+            R = np.array([[math.cos(th[t, i]), -math.sin(th[t, i])], [math.sin(th[t, i]), math.cos(th[t, i])]])
+            assert np.allclose(y[t, 2 * i:2 * i + 2], R @ x[t, 2 * i:2 * i + 2], atol=1e-14)
+    assert np.allclose(np.linalg.norm(y, axis=1), np.linalg.norm(x, axis=1), rtol=1e-14)
+    assert np.array_equal(oa.rotate_pairs(x, np.ones((6, 4)), np.zeros((6, 4))), x)      # zero angle: identity
+
+
+def test_rotated_state_and_readout_against_token_sum_and_relative_angle():
+    """Numerator of Eq. 4 with Eq. 3's state = sum_j (R_q phi(q)) . (R_j phi(k_j)) v_j, and each term depends on the
+    angles only through their difference (the point of a rotary embedding); the denominator ignores the angles."""
+    n, d = 9, 8
+    k = rnd((n, d), 111); v = rnd((n, d), 112); q = rnd((4, d), 113)
+    ck, sk, thk = _angles((n, d // 2), 2); cq, sq, thq = _angles((4, d // 2), 3)
+    S, z = oa.absorb_rope(np.zeros((d, d)), np.zeros(d), k, v, ck, sk)
+    h = oa.linear_readout(q, S, z, eps=0.0, cos_q=cq, sin_q=sq)
+    fq, fk = oa.phi(q), oa.phi(k)
+    for r in range(4):
+        num = np.zeros(d); den = 0.0
+        for j in range(n):
+            w = 0.0
+            for i in range(d // 2):      # pair i: phi(q)_i^T R(theta_k - theta_q) phi(k)_i
+                dth = thk[j, i] - thq[r, i]
+                a, b = fq[r, 2 * i], fq[r, 2 * i + 1]; c_, e_ = fk[j, 2 * i], fk[j, 2 * i + 1]
+                w += math.cos(dth) * (a * c_ + b * e_) + math.sin(dth) * (b * c_ - a * e_)
+            num += w * v[j]; den += fq[r] @ fk[j]
+        assert np.allclose(h[r], num / den, atol=1e-12)
+    S0, z0 = oa.absorb(np.zeros((d, d)), np.zeros(d), k, v)
+    assert np.allclose(z, z0, atol=1e-14)                       # normaliser unrotated
+    S1, _ = oa.absorb_rope(np.zeros((d, d)), np.zeros(d), k, v, np.ones((n, d // 2)), np.zeros((n, d // 2)))
+    assert np.allclose(S1, S0, atol=1e-14)                      # zero angles: Eq. 3 without rotation
+
+
+def test_relative_temporal_indices_eq8():
+    assert oa.relative_temporal_indices(3, 21) == [1, 2, 3]
+    assert oa.relative_temporal_indices(21, 21) == [19, 20, 21]
+    assert oa.relative_temporal_indices(22, 21) == [19, 20, 21] and oa.relative_temporal_indices(600, 21) == [19, 20, 21]
