@@ -32,7 +32,7 @@ from paper_2604_10103_b200 import inputs as gen, replicas  # noqa: E402
 METRIC = "hybrid-attn latent frames/s at 832x480 shape"
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_swa_tc5 launch at this workload's layer shape, from the ncu
 # capture summarised in profiles/k_swa_tc5_layer_832x480.md; None when the kernel has changed since that capture.
-SWA_DRAM_BYTES_PER_LAUNCH = 137.3e6
+SWA_DRAM_BYTES_PER_LAUNCH = 137.4e6
 UNIT = "latent frames/s"
 
 
