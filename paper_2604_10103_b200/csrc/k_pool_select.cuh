@@ -82,6 +82,37 @@ __global__ void __launch_bounds__(256) k_pool_copy(PoolJobs jobs, int Tc, int bl
     }
 }
 
+// A[i][j] = Mean(q_i) . Mean(k_j) in the canonical order, formed by one thread: 32 partials (partial l = columns l,
+// l + 32, ... ascending, product and sum rounded separately), then the butterfly.  The shuffle butterfly
+// p[l] + p[l ^ off] gives both partners the same value (IEEE addition commutes), so folding the upper half onto the
+// lower half level by level yields lane 0's result bit for bit.  sq: the pooled query row (shared memory), kp: the
+// pooled key row.
+template <int D>
+__device__ __forceinline__ float canonical_score(const float* sq, const float4* __restrict__ kp) {
+    float pl[32];
+#pragma unroll
+    for (int m = 0; m < D / 32; ++m) {
+        float4 kv[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) kv[i] = __ldg(kp + m * 8 + i);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float kk[4] = {kv[i].x, kv[i].y, kv[i].z, kv[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int l = 4 * i + e;
+                const float pr = __fmul_rn(sq[l + 32 * m], kk[e]);
+                pl[l] = (m == 0) ? pr : __fadd_rn(pl[l], pr);
+            }
+        }
+    }
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1)
+#pragma unroll
+        for (int l = 0; l < off; ++l) pl[l] = __fadd_rn(pl[l], pl[l + off]);
+    return pl[0];
+}
+
 // grid (T_m, B*H), 128 threads.  One query-block row: T_n scores, rank-based top-K under the total order
 // (score descending, block index ascending), bit mask + ascending index list.
 template <int D>
@@ -98,35 +129,12 @@ __global__ void __launch_bounds__(128) k_select(ChunkTable tab, const float* __r
     const size_t row = (size_t)bh * Tm + i;
     if (threadIdx.x < D) sq[threadIdx.x] = pooled_q[row * D + threadIdx.x];
     __syncthreads();
-    // One thread per key block: the 32 partials and the butterfly of the canonical order are formed by that thread
-    // alone.  The shuffle butterfly p[l] + p[l ^ off] gives both partners the same value (IEEE addition commutes), so
-    // folding the upper half onto the lower half level by level yields lane 0's result bit for bit.
+    // One thread per key block (see canonical_score).
     for (int j = threadIdx.x; j < Tn; j += 128) {
         const int c = j / n_b, jb = j - c * n_b;
-        const float4* kp = reinterpret_cast<const float4*>(tab.pooled[c] + ((size_t)bh * n_b + jb) * D);
-        float pl[32];
-#pragma unroll
-        for (int m = 0; m < D / 32; ++m) {
-            float4 kv[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) kv[i] = __ldg(kp + m * 8 + i);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float kk[4] = {kv[i].x, kv[i].y, kv[i].z, kv[i].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int l = 4 * i + e;
-                    const float pr = __fmul_rn(sq[l + 32 * m], kk[e]);
-                    pl[l] = (m == 0) ? pr : __fadd_rn(pl[l], pr);
-                }
-            }
-        }
-#pragma unroll
-        for (int off = 16; off >= 1; off >>= 1)
-#pragma unroll
-            for (int l = 0; l < off; ++l) pl[l] = __fadd_rn(pl[l], pl[l + off]);
-        sc[j] = pl[0];
-        if (scores_out) scores_out[row * Tn + j] = pl[0];
+        const float s = canonical_score<D>(sq, reinterpret_cast<const float4*>(tab.pooled[c] + ((size_t)bh * n_b + jb) * D));
+        sc[j] = s;
+        if (scores_out) scores_out[row * Tn + j] = s;
     }
     __syncthreads();
     for (int j = threadIdx.x; j < Tn; j += 128) {
