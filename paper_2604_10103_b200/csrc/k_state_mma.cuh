@@ -1,11 +1,10 @@
-// Linear-attention state kernels on the warp-level tensor path (ldmatrix + mma.sync):
-//   k_absorb_mma   Eq. 3, first half: per (batch, head) the token range is split over thread blocks, each writing
-//                  its partial phi(K_ev)^T V_ev and sum_t phi(K_ev[t]) to scratch
+// Linear-attention state kernels off the tcgen05 path:
+//   k_absorb_mma   Eq. 3, first half, on the warp-level tensor path (ldmatrix + mma.sync): per (batch, head) the token
+//                  range is split over thread blocks, each writing its partial phi(K_ev)^T V_ev and sum_t phi(K_ev[t])
+//                  to scratch.  Used by the entry point that may not allocate; the context's path is k_absorb_tc5.
 //   k_reduce_fold  Eq. 3, second half: S, z += the partials in ascending split order (deterministic), then
 //                  S' = S W^T split into bf16 hi/lo halves (the per-row divisor of Eq. 4 commutes with W)
-//   k_readout_mma  Eq. 4: (phi(Q) S') / (phi(Q).z + eps) + bias
-// phi(K) and phi(Q) are carried as bf16 hi + lo pairs so that the products keep ~16 mantissa bits;
-// accumulation is fp32 throughout.
+// phi(K) is carried as a bf16 hi + lo pair so that the products keep ~16 mantissa bits; accumulation is fp32.
 #pragma once
 #include "hf_common.cuh"
 
@@ -202,99 +201,5 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
         const size_t o = ((size_t)bh * D + a0 + r) * D + cp;
         sf_hi[o] = hi;
         sf_lo[o] = __float2bfloat16_rn(out[r] - __bfloat162float(hi));
-    }
-}
-
-template <int D>
-struct ReadoutMma {
-    static constexpr int ROWS = 128, THREADS = 256;
-    static constexpr int ROW_BYTES = D * 2;
-    static constexpr int Q_BYTES = ROWS * ROW_BYTES, S_BYTES = D * ROW_BYTES;
-    static constexpr int SMEM_BYTES = Q_BYTES + 2 * S_BYTES + 2 * D * 4;   // Q, Sf hi, Sf lo, z, bias
-    static constexpr int CHUNKS_PER_ROW = D / 8;
-};
-
-// grid (ceil(T_c/128), B*H).  out_bf16 or out_f32 (exactly one non-null): [B*H, T_c, D].
-template <int D>
-__global__ void __launch_bounds__(256, 2)
-k_readout_mma(const bf16* __restrict__ q, const bf16* __restrict__ sf_hi, const bf16* __restrict__ sf_lo,
-              const float* __restrict__ z, const bf16* __restrict__ bias, int heads, int Tc, float eps,
-              bf16* __restrict__ out_bf16, float* __restrict__ out_f32) {
-    typedef ReadoutMma<D> C;
-    extern __shared__ __align__(128) uint8_t smem[];
-    const uint32_t sQ = smem_u32(smem), sHi = sQ + C::Q_BYTES, sLo = sHi + C::S_BYTES;
-    float* sz = reinterpret_cast<float*>(smem + C::Q_BYTES + 2 * C::S_BYTES);
-    float* sb = sz + D;
-    const int bh = blockIdx.y, h = bh % heads;
-    const int r0 = blockIdx.x * C::ROWS;
-    const int nq = min(C::ROWS, Tc - r0);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    for (int id = threadIdx.x; id < C::ROWS * C::CHUNKS_PER_ROW; id += C::THREADS) {
-        const int row = id / C::CHUNKS_PER_ROW, ch = id % C::CHUNKS_PER_ROW;
-        const bool ok = row < nq;
-        cp_async16(sQ + swz<C::ROW_BYTES>(row, ch), q + ((size_t)bh * Tc + r0 + (ok ? row : 0)) * D + ch * 8, ok);
-    }
-    for (int id = threadIdx.x; id < D * C::CHUNKS_PER_ROW; id += C::THREADS) {
-        const int row = id / C::CHUNKS_PER_ROW, ch = id % C::CHUNKS_PER_ROW;
-        cp_async16(sHi + swz<C::ROW_BYTES>(row, ch), sf_hi + ((size_t)bh * D + row) * D + ch * 8, true);
-        cp_async16(sLo + swz<C::ROW_BYTES>(row, ch), sf_lo + ((size_t)bh * D + row) * D + ch * 8, true);
-    }
-    cp_async_commit();
-    if (threadIdx.x < D) {
-        sz[threadIdx.x] = z[(size_t)bh * D + threadIdx.x];
-        sb[threadIdx.x] = bias ? __bfloat162float(bias[(size_t)h * D + threadIdx.x]) : 0.f;
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-
-    float acc[D / 8][4];
-#pragma unroll
-    for (int n = 0; n < D / 8; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
-    float den[2] = {0.f, 0.f};
-#pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) {
-        uint32_t r[4];
-        ldsm_x4(sQ + swz<C::ROW_BYTES>(warp * 16 + (lane & 15), ks * 2 + (lane >> 4)), r[0], r[1], r[2], r[3]);
-        uint32_t ahi[4], alo[4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x) {
-            const float2 qv = unpack_bf16(r[x]);
-            const float f0 = phi_elu1(qv.x), f1 = phi_elu1(qv.y);
-            const int a = ks * 16 + 2 * (lane & 3) + ((x >> 1) << 3);      // key-feature column of f0
-            den[x & 1] = fmaf(f0, sz[a], fmaf(f1, sz[a + 1], den[x & 1]));
-            const __nv_bfloat16 h0 = __float2bfloat16_rn(f0), h1 = __float2bfloat16_rn(f1);
-            ahi[x] = pack_bf16(f0, f1);
-            alo[x] = pack_bf16(f0 - __bfloat162float(h0), f1 - __bfloat162float(h1));
-        }
-#pragma unroll
-        for (int np = 0; np < D / 16; ++np) {
-            const int row = ks * 16 + (lane & 7) + (((lane >> 3) & 1) << 3), ch = np * 2 + (lane >> 4);
-            uint32_t b0, b1, b2, b3, c0, c1, c2, c3;
-            ldsm_x4_t(sHi + swz<C::ROW_BYTES>(row, ch), b0, b1, b2, b3);
-            ldsm_x4_t(sLo + swz<C::ROW_BYTES>(row, ch), c0, c1, c2, c3);
-            mma_bf16(acc[2 * np], ahi[0], ahi[1], ahi[2], ahi[3], b0, b1);
-            mma_bf16(acc[2 * np], alo[0], alo[1], alo[2], alo[3], b0, b1);
-            mma_bf16(acc[2 * np], ahi[0], ahi[1], ahi[2], ahi[3], c0, c1);
-            mma_bf16(acc[2 * np + 1], ahi[0], ahi[1], ahi[2], ahi[3], b2, b3);
-            mma_bf16(acc[2 * np + 1], alo[0], alo[1], alo[2], alo[3], b2, b3);
-            mma_bf16(acc[2 * np + 1], ahi[0], ahi[1], ahi[2], ahi[3], c2, c3);
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 1);
-        den[r] += __shfl_xor_sync(0xffffffffu, den[r], 2);
-        const int row = warp * 16 + (lane >> 2) + r * 8;
-        if (row >= nq) continue;
-        const float inv = 1.f / (den[r] + eps);
-        const size_t g = ((size_t)bh * Tc + r0 + row) * D;
-#pragma unroll
-        for (int n = 0; n < D / 8; ++n) {
-            const int col = n * 8 + 2 * (lane & 3);
-            const float x0 = fmaf(acc[n][2 * r], inv, sb[col]), x1 = fmaf(acc[n][2 * r + 1], inv, sb[col + 1]);
-            if (out_f32) *reinterpret_cast<float2*>(out_f32 + g + col) = make_float2(x0, x1);
-            else *reinterpret_cast<uint32_t*>(out_bf16 + g + col) = pack_bf16(x0, x1);
-        }
     }
 }

@@ -343,3 +343,40 @@ def test_rotation_inside_the_linear_branch(d, b, tpf, cf, wf, zmean):
         assert hz.rel_l2(S, plain.S) > 0.1
     finally:
         gpu.close()
+
+
+def test_maximum_number_of_key_blocks_per_row():
+    """The largest selection row the library accepts: 8 chunks x 128 blocks = 1024 key blocks (16-token blocks)."""
+    w = gen.Workload("maxtn", batch=1, heads=1, head_dim=64, tokens_per_frame=2048, chunk_frames=1, window_frames=8,
+                     block=16, topk=0, keep_permille=30, seed=19)
+    gpu = hz.GpuStream(w, merge=False); ora = hz.make_oracle(w, merge=False)
+    try:
+        for c in range(8):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        qb, kb, vb = gen.qkv(w, 0, 8, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        assert gpu.ctx.hf_query(0, gpu.hf.HF_Q_KEY_BLOCKS) == 1024 and gpu.ctx.hf_query(0, gpu.hf.HF_Q_KEPT_BLOCKS) == 31
+        m_gpu, idx_gpu, sc_gpu = gpu.select(q, k)
+        m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+        assert m_ref.shape == (1, 1, 128, 1024)
+        assert np.array_equal(sc_gpu, sc_ref) and np.array_equal(m_gpu, m_ref)
+        qbl = [0, 63, 127]
+        o_ref = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, q_blocks=qbl)
+        hz.assert_close_out(gpu.forward(q, k, v), o_ref, "1024 key blocks")
+    finally:
+        gpu.close()
+
+
+def test_empty_token_range_is_refused_without_a_launch():
+    import torch
+    w = gen.tiny()
+    gpu = hz.GpuStream(w)
+    try:
+        t = torch.zeros((1, 2, 64, 64), dtype=torch.bfloat16, device="cuda")
+        n0 = gpu.ctx.hf_launch_count()
+        with pytest.raises(gpu.hf.HFError, match="HF_ERR_SHAPE"):
+            gpu.ctx.hf_state_absorb(0, t, t, 0)
+        assert gpu.ctx.hf_launch_count() == n0
+    finally:
+        gpu.close()
