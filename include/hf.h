@@ -167,6 +167,25 @@ hf_status hf_state_absorb_noalloc(const void* k_ev, const void* v_ev, int batch_
 /* Copy the state out: S float [B,H,d,d] (row = key feature, column = value dim), z float [B,H,d]; either may be NULL. */
 hf_status hf_get_state(hf_ctx* ctx, int layer, float* S, float* z, void* stream);
 
+/* Checkpoint of the whole streaming state of the method (the rolling cache and the linear state, which is all the
+ * memory the method carries from chunk to chunk -- Sec. 3.3; Alg. 2's KV and LN), for every layer of the context, into
+ * ONE host buffer: per layer the sink chunks and the cached clean chunks (K, V and their pooled block sums, oldest
+ * first -- the physical rotation of the ring is not kept), S, z and the absorbed-token count.  Merge weights and
+ * rotation tables are parameters, not state: they are not in the image.
+ *   host_buf == NULL : *bytes receives the size the image would have now; nothing is copied.
+ *   host_buf != NULL : *bytes holds the capacity of host_buf on entry and the bytes written on return;
+ *                      HF_ERR_SHAPE (and the needed size in *bytes) if the capacity is too small.
+ * Synchronises the device.  The image is only meaningful to hf_state_import of this library version. */
+hf_status hf_state_export(hf_ctx* ctx, void* host_buf, size_t* bytes);
+
+/* Load an image written by hf_state_export into a context created with the same configuration (every field that
+ * fixes a shape or the arithmetic of the state must match: HF_ERR_SHAPE otherwise; HF_ERR_INVALID_ARG for a buffer
+ * that is not an image or is cut short).  All layers are replaced; the folded state is rebuilt from S and the merge
+ * weights the context holds at that moment (weights set later refold it again).  A stream that continues after the
+ * import produces bit-for-bit what the uninterrupted stream produces.  Synchronises the device.  Nothing is changed
+ * when the image is rejected. */
+hf_status hf_state_import(hf_ctx* ctx, const void* host_buf, size_t bytes);
+
 /* Host-side bookkeeping values (HF_Q_*). */
 hf_status hf_query(hf_ctx* ctx, int layer, int what, int64_t* value);
 

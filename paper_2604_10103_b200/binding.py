@@ -27,7 +27,7 @@ EXPORTS = [
     "hf_create", "hf_destroy", "hf_reset", "hf_set_merge_weights", "hf_kv_append", "hf_state_absorb",
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
-    "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope",
+    "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
 ]
 
 
@@ -72,6 +72,8 @@ def lib() -> C.CDLL:
     L.hf_hybrid_forward_host.argtypes = [vp, ip, vp, vp, vp, vp, vp]
     L.hf_kv_append_host.argtypes = [vp, ip, vp, vp, vp]
     L.hf_get_state.argtypes = [vp, ip, vp, vp, vp]
+    L.hf_state_export.argtypes = [vp, vp, C.POINTER(C.c_size_t)]
+    L.hf_state_import.argtypes = [vp, vp, C.c_size_t]
     L.hf_query.argtypes = [vp, ip, ip, C.POINTER(C.c_int64)]
     L.hf_get_device_status.argtypes = [vp, C.POINTER(ip), C.POINTER(ip)]
     L.hf_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
@@ -169,6 +171,19 @@ class Context:
 
     def hf_get_state(self, layer, S=None, z=None):
         _check(lib().hf_get_state(self._h, layer, _ptr(S), _ptr(z), _stream()))
+
+    def hf_state_export(self):
+        """The checkpoint image of all layers as a numpy uint8 array (size asked for first, then filled)."""
+        import numpy as np
+        n = C.c_size_t(0)
+        _check(lib().hf_state_export(self._h, None, C.byref(n)))
+        buf = np.empty(n.value, dtype=np.uint8)
+        _check(lib().hf_state_export(self._h, C.c_void_p(buf.ctypes.data), C.byref(n)))
+        return buf[:n.value]
+
+    def hf_state_import(self, image):
+        """image: contiguous numpy uint8 array written by hf_state_export."""
+        _check(lib().hf_state_import(self._h, C.c_void_p(image.ctypes.data), image.nbytes))
 
     def hf_query(self, layer, what) -> int:
         v = C.c_int64()

@@ -723,6 +723,124 @@ hf_status hf_get_state(hf_ctx* c, int layer, float* S, float* z, void* stream) {
     return HF_OK;
 }
 
+// ---- checkpoint image: header, then per layer {counts, S, z, held chunks in logical order (K, V, pooled sums)}
+namespace {
+constexpr uint64_t IMAGE_MAGIC = 0x3145544154534648ull;   // "HFSTATE1"
+constexpr uint32_t IMAGE_VERSION = 1;
+struct ImageHeader {
+    uint64_t magic;
+    uint32_t version, header_bytes;
+    int32_t batch, heads, head_dim, tokens_per_frame, chunk_frames, window_frames, block, layers, phi, z_mode, sink_frames, reserved;
+    uint64_t total_bytes;
+};
+struct ImageLayer {
+    int32_t n_sink, n_cached;
+    int64_t absorbed;
+};
+size_t image_chunk_bytes(const hf_ctx* c) { return 2 * c->chunk_elems * sizeof(bf16) + c->pooled_elems * sizeof(float); }
+size_t image_state_bytes(const hf_ctx* c) { return ((size_t)c->BH * c->d * c->d + (size_t)c->BH * c->d) * sizeof(float); }
+ImageHeader image_header(const hf_ctx* c) {
+    ImageHeader h;
+    memset(&h, 0, sizeof(h));
+    h.magic = IMAGE_MAGIC; h.version = IMAGE_VERSION; h.header_bytes = (uint32_t)sizeof(ImageHeader);
+    h.batch = c->cfg.batch; h.heads = c->cfg.heads; h.head_dim = c->cfg.head_dim; h.tokens_per_frame = c->cfg.tokens_per_frame;
+    h.chunk_frames = c->cfg.chunk_frames; h.window_frames = c->cfg.window_frames; h.block = c->cfg.block;
+    h.layers = c->cfg.layers; h.phi = c->cfg.phi; h.z_mode = c->cfg.z_mode; h.sink_frames = c->cfg.sink_frames;
+    return h;
+}
+int held_slot(const hf_ctx* c, const LayerState& L, int i) {   // slot of the i-th held chunk in logical order
+    return i < L.n_sink ? c->P + i : (L.head + i - L.n_sink) % c->P;
+}
+}  // namespace
+
+hf_status hf_state_export(hf_ctx* c, void* host_buf, size_t* bytes) {
+    if (c == nullptr || bytes == nullptr) return fail(HF_ERR_INVALID_ARG, "null argument");
+    size_t need = sizeof(ImageHeader);
+    for (const LayerState& L : c->layers)
+        need += sizeof(ImageLayer) + image_state_bytes(c) + (size_t)(L.n_sink + L.n_cached) * image_chunk_bytes(c);
+    if (host_buf == nullptr) { *bytes = need; return HF_OK; }
+    if (*bytes < need) {
+        const size_t have = *bytes;
+        *bytes = need;
+        return fail(HF_ERR_SHAPE, "image needs %zu bytes, buffer holds %zu", need, have);
+    }
+    HF_CUDA(cudaSetDevice(c->device));
+    HF_CUDA(cudaDeviceSynchronize());
+    uint8_t* out = (uint8_t*)host_buf;
+    ImageHeader h = image_header(c);
+    h.total_bytes = need;
+    memcpy(out, &h, sizeof(h));
+    out += sizeof(h);
+    const size_t dd = (size_t)c->BH * c->d * c->d * sizeof(float), dz = (size_t)c->BH * c->d * sizeof(float);
+    const size_t kv = c->chunk_elems * sizeof(bf16), pl = c->pooled_elems * sizeof(float);
+    for (const LayerState& L : c->layers) {
+        ImageLayer il;
+        il.n_sink = L.n_sink; il.n_cached = L.n_cached; il.absorbed = L.absorbed;
+        memcpy(out, &il, sizeof(il)); out += sizeof(il);
+        HF_CUDA(cudaMemcpy(out, L.S, dd, cudaMemcpyDeviceToHost)); out += dd;
+        HF_CUDA(cudaMemcpy(out, L.z, dz, cudaMemcpyDeviceToHost)); out += dz;
+        for (int i = 0; i < L.n_sink + L.n_cached; ++i) {
+            const int slot = held_slot(c, L, i);
+            HF_CUDA(cudaMemcpy(out, L.ring_k + (size_t)slot * c->chunk_elems, kv, cudaMemcpyDeviceToHost)); out += kv;
+            HF_CUDA(cudaMemcpy(out, L.ring_v + (size_t)slot * c->chunk_elems, kv, cudaMemcpyDeviceToHost)); out += kv;
+            HF_CUDA(cudaMemcpy(out, L.pooled_k + (size_t)slot * c->pooled_elems, pl, cudaMemcpyDeviceToHost)); out += pl;
+        }
+    }
+    *bytes = need;
+    return HF_OK;
+}
+
+hf_status hf_state_import(hf_ctx* c, const void* host_buf, size_t bytes) {
+    if (c == nullptr || host_buf == nullptr) return fail(HF_ERR_INVALID_ARG, "null argument");
+    if (bytes < sizeof(ImageHeader)) return fail(HF_ERR_INVALID_ARG, "buffer is shorter than an image header");
+    const uint8_t* in = (const uint8_t*)host_buf;
+    ImageHeader h;
+    memcpy(&h, in, sizeof(h));
+    if (h.magic != IMAGE_MAGIC || h.version != IMAGE_VERSION || h.header_bytes != sizeof(ImageHeader))
+        return fail(HF_ERR_INVALID_ARG, "buffer is not a state image of this library version");
+    const ImageHeader mine = image_header(c);
+    if (h.batch != mine.batch || h.heads != mine.heads || h.head_dim != mine.head_dim ||
+        h.tokens_per_frame != mine.tokens_per_frame || h.chunk_frames != mine.chunk_frames ||
+        h.window_frames != mine.window_frames || h.block != mine.block || h.layers != mine.layers || h.phi != mine.phi ||
+        h.z_mode != mine.z_mode || h.sink_frames != mine.sink_frames)
+        return fail(HF_ERR_SHAPE, "the image was written by a context with another configuration");
+    if (h.total_bytes > bytes) return fail(HF_ERR_INVALID_ARG, "image is cut short: %zu of %zu bytes", bytes, (size_t)h.total_bytes);
+    // first pass: every count in range and the sizes add up; nothing is touched before the image is known to be whole
+    size_t off = sizeof(ImageHeader);
+    for (int l = 0; l < c->cfg.layers; ++l) {
+        if (off + sizeof(ImageLayer) > h.total_bytes) return fail(HF_ERR_INVALID_ARG, "image ends inside layer %d", l);
+        ImageLayer il;
+        memcpy(&il, in + off, sizeof(il));
+        if (il.n_sink < 0 || il.n_sink > c->n_sink_max || il.n_cached < 0 || il.n_cached > c->P || il.absorbed < 0 ||
+            (il.n_cached > 0 && il.n_sink < c->n_sink_max))
+            return fail(HF_ERR_INVALID_ARG, "layer %d of the image holds counts this configuration cannot have", l);
+        off += sizeof(ImageLayer) + image_state_bytes(c) + (size_t)(il.n_sink + il.n_cached) * image_chunk_bytes(c);
+    }
+    if (off != h.total_bytes) return fail(HF_ERR_INVALID_ARG, "image size does not match its contents");
+    HF_CUDA(cudaSetDevice(c->device));
+    HF_CUDA(cudaDeviceSynchronize());
+    const size_t dd = (size_t)c->BH * c->d * c->d * sizeof(float), dz = (size_t)c->BH * c->d * sizeof(float);
+    const size_t kv = c->chunk_elems * sizeof(bf16), pl = c->pooled_elems * sizeof(float);
+    in += sizeof(ImageHeader);
+    for (LayerState& L : c->layers) {
+        ImageLayer il;
+        memcpy(&il, in, sizeof(il)); in += sizeof(il);
+        HF_CUDA(cudaMemcpy(L.S, in, dd, cudaMemcpyHostToDevice)); in += dd;
+        HF_CUDA(cudaMemcpy(L.z, in, dz, cudaMemcpyHostToDevice)); in += dz;
+        L.n_sink = il.n_sink; L.n_cached = il.n_cached; L.head = 0; L.absorbed = il.absorbed;
+        L.cache_epoch++; L.sel_epoch = ~0ull;
+        for (int i = 0; i < L.n_sink + L.n_cached; ++i) {
+            const int slot = held_slot(c, L, i);
+            HF_CUDA(cudaMemcpy(L.ring_k + (size_t)slot * c->chunk_elems, in, kv, cudaMemcpyHostToDevice)); in += kv;
+            HF_CUDA(cudaMemcpy(L.ring_v + (size_t)slot * c->chunk_elems, in, kv, cudaMemcpyHostToDevice)); in += kv;
+            HF_CUDA(cudaMemcpy(L.pooled_k + (size_t)slot * c->pooled_elems, in, pl, cudaMemcpyHostToDevice)); in += pl;
+        }
+        HF_TRY(HF_DISPATCH_D(c, launch_fold, c, L, 0, (cudaStream_t)0));   // S W^T halves from the restored S
+    }
+    HF_CUDA(cudaDeviceSynchronize());
+    return HF_OK;
+}
+
 hf_status hf_query(hf_ctx* c, int layer, int what, int64_t* value) {
     HF_TRY(check_layer(c, layer));
     if (value == nullptr) return fail(HF_ERR_INVALID_ARG, "value is null");
