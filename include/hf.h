@@ -123,7 +123,11 @@ hf_status hf_block_select(hf_ctx* ctx, int layer, const void* q, const void* k_c
 /* Eq. 6 / Alg. 3 inner loops: o_local[r] = softmax_c(q_r . k_c / sqrt(d)) V over the tokens c of the kept key
  * blocks of r's query block.  idx: int32 [B,H,T_m,k_eff] ascending block indices, or NULL = the context's last
  * selection for this layer (HF_ERR_STATE if none or if the cache changed since).  o_local: bf16 [B,H,T_c,d].
- * lse: float [B,H,T_c] natural-log sum of exp of the scaled logits, or NULL. */
+ * lse: float [B,H,T_c] natural-log sum of exp of the scaled logits, or NULL.
+ * The list lives on the device, so the host cannot look at it: the kernel checks every entry against [0, T_n), reads
+ * block 0 in place of an entry outside it (no address is ever formed from such an entry) and sets flag 2 of the
+ * device status word; the rows of that query block are then meaningless and hf_get_device_status reports
+ * HF_ERR_INVALID_ARG. */
 hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur,
                         const int32_t* idx, void* o_local, float* lse, void* stream);
 
@@ -189,8 +193,10 @@ hf_status hf_state_import(hf_ctx* ctx, const void* host_buf, size_t bytes);
 /* Host-side bookkeeping values (HF_Q_*). */
 hf_status hf_query(hf_ctx* ctx, int layer, int what, int64_t* value);
 
-/* Synchronises the device and reports the device status word: flags != 0 means a bounded wait inside a kernel
- * ran out (detail = where); the result of that launch is invalid, the context stays usable. */
+/* Synchronises the device and reports the device status word.  Flag 1: a bounded wait inside a kernel ran out
+ * (detail = where), HF_ERR_DEVICE_TIMEOUT.  Flag 2: a caller's index list held a block index outside [0, T_n)
+ * (detail = batch*head and query block of the row, as one number), HF_ERR_INVALID_ARG.  Either way the result of that
+ * launch is invalid, the word is cleared and the context stays usable. */
 hf_status hf_get_device_status(hf_ctx* ctx, int* flags, int* detail);
 
 /* Number of kernels the library has launched since the context was created. */

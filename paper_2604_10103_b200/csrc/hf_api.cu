@@ -299,7 +299,7 @@ hf_status launch_swa_mma_t(hf_ctx* c, const bf16* q, const ChunkTable& tab, cons
                            const float* hist, bf16* o, float* lse, cudaStream_t st) {
     typedef SwaMma<BLK, D> C;
     const float scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
-    k_swa_mma<BLK, D><<<dim3(c->Tm, c->BH), C::THREADS, C::SMEM_BYTES, st>>>(q, tab, idx, keep, c->Tc, c->n_b, scale_log2, hist, o, lse);
+    k_swa_mma<BLK, D><<<dim3(c->Tm, c->BH), C::THREADS, C::SMEM_BYTES, st>>>(q, tab, idx, keep, c->Tc, c->n_b, scale_log2, hist, o, lse, c->dev_status);
     return post_launch(c, "k_swa_mma");
 }
 
@@ -869,7 +869,10 @@ hf_status hf_get_device_status(hf_ctx* c, int* flags, int* detail) {
     if (detail) *detail = h[1];
     if (h[0] != 0) {
         HF_CUDA(cudaMemset(c->dev_status, 0, 16));
-        return fail(HF_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (flags %d, detail %d)", h[0], h[1]);
+        if (h[0] & HF_DEV_TIMEOUT_FLAG)
+            return fail(HF_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (flags %d, detail %d)", h[0], h[1]);
+        return fail(HF_ERR_INVALID_ARG, "an index list held a block index outside [0, T_n) (unit %d); block 0 was read in its place",
+                    h[1]);
     }
     return HF_OK;
 }

@@ -18,7 +18,18 @@ struct ChunkTable {
 };
 
 // Device status word layout (int[4]): [0] flags, [1] detail, [2..3] reserved.
-enum { HF_DEV_TIMEOUT_FLAG = 1 };
+enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2 };
+
+// A kept-block index read from a caller's list: inside [0, Tn) it is returned as it is; anything else is replaced by
+// block 0 (so that every address formed from it stays inside the cache) and recorded in the status word.
+__device__ __forceinline__ int checked_block(int j, int Tn, int* dev_status, int unit) {
+    if ((unsigned)j < (unsigned)Tn) return j;
+    if (dev_status) {
+        atomicOr(dev_status, HF_DEV_BAD_INDEX_FLAG);
+        atomicExch(dev_status + 1, unit);
+    }
+    return 0;
+}
 
 // ---------------------------------------------------------------------------------------------
 // small PTX helpers (legacy tensor path: ldmatrix + mma.sync, cp.async)

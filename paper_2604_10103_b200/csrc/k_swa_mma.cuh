@@ -36,7 +36,7 @@ template <int BLK, int D>
 __global__ void __launch_bounds__(SwaMma<BLK, D>::THREADS)
 k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict__ idx, int keep,
           int Tc, int n_b, float scale_log2, const float* __restrict__ hist,
-          bf16* __restrict__ o, float* __restrict__ lse) {
+          bf16* __restrict__ o, float* __restrict__ lse, int* dev_status) {
     typedef SwaMma<BLK, D> C;
     extern __shared__ __align__(128) uint8_t smem[];
     const uint32_t sQ = smem_u32(smem);
@@ -48,8 +48,9 @@ k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict_
     const int nq = min(BLK, Tc - q0);
     const int32_t* my_idx = idx + ((size_t)bh * gridDim.x + i) * keep;
 
+    const int Tn = tab.n_chunks * n_b;
     auto issue = [&](int it, int stage) {
-        const int j = my_idx[it];
+        const int j = checked_block(my_idx[it], Tn, dev_status, bh * gridDim.x + i);
         const int c = j / n_b, jb = j - c * n_b;
         const int nv = min(BLK, Tc - jb * BLK);
         const size_t off = ((size_t)bh * Tc + (size_t)jb * BLK) * D;
@@ -74,7 +75,7 @@ k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict_
         cp_async_wait<1>();
         __syncthreads();
 
-        const int j = my_idx[it];
+        const int j = checked_block(my_idx[it], Tn, nullptr, 0);
         const int jb = j % n_b;
         const int nv = min(BLK, Tc - jb * BLK);
         const uint32_t sK = sKV + stage * 2 * C::TILE_BYTES, sV = sK + C::TILE_BYTES;

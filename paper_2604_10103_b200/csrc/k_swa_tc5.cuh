@@ -117,6 +117,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             RingPos<C::KSTAGES> rk;
             RingPos<C::VSTAGES> rv;
             int t = 0;
+            const int Tn = (p.n_sink + p.n_cached + 1) * p.n_b;
             for (int n = 0; ok && n < my_units; ++n) {
                 const int u = blockIdx.x + n * gridDim.x;
                 const int bh = u / p.Tm, i = u - bh * p.Tm;
@@ -129,7 +130,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         tma_load_4d(sQ + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_qf);
                 }
                 for (int j = 0; j < keep; ++j, ++t) {
-                    const int blk = __ldg(my_idx + j);
+                    const int blk = checked_block(__ldg(my_idx + j), Tn, is_k ? p.dev_status : nullptr, u);
                     int c = 0, jb = blk;
                     while (jb >= p.n_b) { jb -= p.n_b; ++c; }          // at most HF_MAX_CHUNKS - 1 steps; no XU-pipe division
                     // logical chunk order: sink chunks (slots P, P + 1, ...), cached chunks oldest first (ring), current chunk
@@ -246,14 +247,15 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             const int q0 = i * C::BLK;
             const int nq = min(C::BLK, p.Tc - q0);
             float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
-            int blk_next = __ldg(my_idx);                   // block index list read one tile ahead (off the critical path)
+            const int Tn = (p.n_sink + p.n_cached + 1) * p.n_b;
+            int blk_next = checked_block(__ldg(my_idx), Tn, nullptr, 0);   // block index list read one tile ahead (off the critical path)
             for (int j = 0; j < keep; ++j, ++t) {
                 // a chunk's last block may be short; found without an integer division (those run on the XU pipe and
                 // would queue behind the other warp's exponentials)
                 bool tail = false;
 #pragma unroll
                 for (int c = 1; c <= HF_MAX_CHUNKS; ++c) tail |= (blk_next + 1 == c * p.n_b);
-                if (j + 1 < keep) blk_next = __ldg(my_idx + j + 1);
+                if (j + 1 < keep) blk_next = checked_block(__ldg(my_idx + j + 1), Tn, nullptr, 0);
                 const int nv = tail ? p.Tc - (p.n_b - 1) * C::BLK : C::BLK;
                 const int st = t & 1;
                 const uint32_t tS = lane_base + rs.stage * C::BLK;

@@ -93,6 +93,7 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             RingPos<C::KSTAGES> rk;
             RingPos<C::VSTAGES> rv;
             int t = 0;
+            const int Tn = (p.n_sink + p.n_cached + 1) * p.n_b;
             for (int n = 0; ok && n < my_units; ++n) {
                 const int u = blockIdx.x + n * gridDim.x;
                 const int bh = u / p.Tm, i = u - bh * p.Tm;
@@ -105,7 +106,7 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         tma_load_4d(sQ + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_qf);
                 }
                 for (int j = 0; j < keep; ++j, ++t) {
-                    const int blk = __ldg(my_idx + j);
+                    const int blk = checked_block(__ldg(my_idx + j), Tn, is_k ? p.dev_status : nullptr, u);
                     int c = 0, jb = blk;
                     while (jb >= p.n_b) { jb -= p.n_b; ++c; }          // at most HF_MAX_CHUNKS - 1 steps; no XU-pipe division
                     // logical chunk order: sink chunks (slots P, P + 1, ...), cached chunks oldest first (ring), current chunk
@@ -219,7 +220,8 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
             bool first = true;
             int j = (t0 & 1) == g ? 0 : 1;                  // this group's first position in the unit
-            int blk_next = j < keep ? __ldg(my_idx + j) : 0;
+            const int Tn = (p.n_sink + p.n_cached + 1) * p.n_b;
+            int blk_next = j < keep ? checked_block(__ldg(my_idx + j), Tn, nullptr, 0) : 0;
             if (n >= 1) {
                 // every softmax thread has read both accumulators of the previous unit before either is started afresh
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_ep2, (n - 1) & 1, abort_flag, p.dev_status, 14));
@@ -230,7 +232,7 @@ k_swa_tc5p(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 bool tail = false;
 #pragma unroll
                 for (int c = 1; c <= HF_MAX_CHUNKS; ++c) tail |= (blk_next + 1 == c * p.n_b);
-                if (j + 2 < keep) blk_next = __ldg(my_idx + j + 2);
+                if (j + 2 < keep) blk_next = checked_block(__ldg(my_idx + j + 2), Tn, nullptr, 0);
                 const int nv = tail ? tail_cols : C::BLK;
                 // S of this tile has landed; so has P V of this group's previous tile (it precedes this S in the tensor pipe)
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sf + 8 * g, (t >> 1) & 1, abort_flag, p.dev_status, 8));

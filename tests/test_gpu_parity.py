@@ -380,3 +380,34 @@ def test_empty_token_range_is_refused_without_a_launch():
         assert gpu.ctx.hf_launch_count() == n0
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,b,tpf,kernel", [(64, 16, 64, 0), (128, 128, 200, 0), (128, 128, 200, 3)])
+def test_block_indices_outside_the_cache_are_caught_on_the_device(d, b, tpf, kernel):
+    """An index list is device memory the host never sees: every kernel checks each entry against [0, T_n), reads block 0
+    in its place and reports through the status word; the next call with a valid list is right again."""
+    import torch
+    w = gen.Workload("badidx", batch=1, heads=2, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=3,
+                     block=b, topk=2, keep_permille=0, seed=23)
+    gpu = hz.GpuStream(w, swa_kernel=kernel); ora = hz.make_oracle(w)
+    try:
+        for c in range(3):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        qb, kb, vb = gen.qkv(w, 0, 3, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        m_gpu, idx, _ = gpu.select(q, k)
+        tn = gpu.ctx.hf_query(0, gpu.hf.HF_Q_KEY_BLOCKS)
+        for bad in (tn, -1, 2 ** 30, -2 ** 31):
+            wrong = idx.copy()
+            wrong[0, 1, -1, 1] = bad
+            gpu.swa(q, k, v, idx=torch.from_numpy(wrong).cuda())
+            with pytest.raises(gpu.hf.HFError, match="HF_ERR_INVALID_ARG"):
+                gpu.ctx.hf_get_device_status()
+            assert gpu.ctx.hf_get_device_status() == (0, 0)      # the word was cleared
+        m_ref, _ = ora.select(f64(qb), f64(kb))
+        _, ol_ref, _ = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, parts=True)
+        hz.assert_close_out(gpu.swa(q, k, v, idx=torch.from_numpy(idx).cuda()), ol_ref, "O_local after the refused lists")
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
