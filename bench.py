@@ -322,6 +322,79 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Stage times and roofline fractions over the grid keep in {10,25,50,100} % x window in {3,9,21} frames x head_dim
+    in {64,128} x block in {64,128} x batch in {1,4} at 1560 tokens per latent frame, 12 heads, 3-frame chunks: one JSON
+    line per grid point (layer calls rotate over several layer contexts so that the inputs exceed L2)."""
+    import torch
+    from paper_2604_10103_b200 import binding as hf, build as hfbuild
+    hfbuild.build()
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    out = open(args.sweep_out, "w") if args.sweep_out else sys.stdout
+
+    def timed(fn, reps):
+        for r in range(3):
+            fn(r)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for r in range(reps):
+            fn(r)
+        b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps * 1e3
+
+    for batch in (1, 4):
+        for d in (64, 128):
+            for blk in (64, 128):
+                for win in (3, 9, 21):
+                    for permille in (100, 250, 500, 1000):
+                        L = 4 if batch == 1 else 2
+                        w = gen.layer_832x480().with_(name="sweep", batch=batch, head_dim=d, block=blk, window_frames=win,
+                                                      keep_permille=permille, topk=0, layers=L)
+                        ctx = hf.Context(hf.make_config(w))
+                        shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
+                        g = torch.Generator(device="cuda"); g.manual_seed(4321)
+                        rn = lambda: torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+                        q = [rn() for _ in range(L)]; k = [rn() for _ in range(L)]; v = [rn() for _ in range(L)]
+                        o = torch.empty(shape, dtype=torch.bfloat16, device="cuda")
+                        for l in range(L):
+                            Wb, bb = gen.merge_weights(w, l)
+                            ctx.hf_set_merge_weights(l, hf.bits_to_cuda(Wb), hf.bits_to_cuda(bb))
+                            for c in range(w.past_chunks + 1):
+                                ctx.hf_kv_append(l, k[(l + c) % L], v[(l + c) % L])
+                        reps = 4 * L
+                        st = {"select_us": timed(lambda r: ctx.hf_block_select(r % L, q[r % L], k[r % L]), reps)}
+                        st["sparse_swa_us"] = timed(lambda r: ctx.hf_sparse_swa(r % L, q[r % L], k[r % L], v[r % L], o), reps)
+                        st["linear_us"] = timed(lambda r: ctx.hf_linear_attn(r % L, q[r % L], o), reps)
+                        st["forward_us"] = timed(lambda r: ctx.hf_hybrid_forward(r % L, q[r % L], k[r % L], v[r % L], o), reps)
+                        st["absorb_us"] = timed(lambda r: ctx.hf_state_absorb(r % L, k[r % L], v[r % L], w.chunk_tokens), reps)
+                        st["append_us"] = timed(lambda r: ctx.hf_kv_append(r % L, k[r % L], v[r % L]), reps)
+                        tn = ctx.hf_query(0, hf.HF_Q_KEY_BLOCKS); tm = ctx.hf_query(0, hf.HF_Q_QUERY_BLOCKS)
+                        mw = ctx.hf_query(0, hf.HF_Q_MASK_WORDS)
+                        mask = torch.zeros((w.batch, w.heads, tm, mw), dtype=torch.int32, device="cuda")
+                        ctx.hf_block_select(0, q[0], k[0], mask)
+                        torch.cuda.synchronize()
+                        flops = kept_flops(hf.unpack_mask(mask.cpu().numpy().view(np.uint32), tn), w)
+                        tf = flops / (st["sparse_swa_us"] * 1e-6) / 1e12
+                        nbytes = 2 * w.batch * w.heads * w.chunk_tokens * w.head_dim * 2
+                        flags, _ = ctx.hf_get_device_status()
+                        line = {"batch": batch, "head_dim": d, "block": blk, "window_frames": win, "keep_permille": permille,
+                                "key_blocks": tn, "kept_blocks": ctx.hf_query(0, hf.HF_Q_KEPT_BLOCKS),
+                                "swa_kernel": {1: "mma.sync", 2: "tcgen05", 3: "tcgen05 ping-pong"}.get(ctx.hf_query(0, hf.HF_Q_SWA_KERNEL)),
+                                **{k_: round(v_, 2) for k_, v_ in st.items()},
+                                "swa_tflops": round(tf, 1), "swa_frac_of_burst_peak": round(tf / peaks["bf16_tflops"], 3),
+                                "absorb_frac_hbm": round(nbytes / (st["absorb_us"] * 1e-6) / 1e9 / peaks["hbm_gbs"], 3),
+                                "append_frac_hbm": round((3 * nbytes if w.past_chunks else nbytes) / (st["append_us"] * 1e-6) / 1e9 / peaks["hbm_gbs"], 3),
+                                "device_status": flags}
+                        out.write(json.dumps(line) + "\n"); out.flush()
+                        ctx.close()
+                        del q, k, v, o
+                        torch.cuda.empty_cache()
+    if out is not sys.stdout:
+        out.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -333,9 +406,15 @@ def main():
     ap.add_argument("--no-extras", action="store_true",
                     help="run only the warm-up and the timed step loop (no stage split, end-to-end leg or CPU baseline): "
                          "the command profilers are pointed at")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the benchmark line: per-stage times over the keep x window x head_dim x block x batch grid, "
+                         "one JSON line per point (1 GPU)")
+    ap.add_argument("--sweep-out", default=None, help="file for the sweep's JSON lines (default: stdout)")
     args = ap.parse_args()
     w = gen.full_depth_832x480(layers=args.layers, steps=args.denoise_steps)
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

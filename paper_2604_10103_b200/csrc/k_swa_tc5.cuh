@@ -247,15 +247,16 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             const int q0 = i * C::BLK;
             const int nq = min(C::BLK, p.Tc - q0);
             float m_used = -INFINITY, l_run = 0.f;          // l_run: this thread's share of the row sum
-            const int Tn = (p.n_sink + p.n_cached + 1) * p.n_b;
-            int blk_next = checked_block(__ldg(my_idx), Tn, nullptr, 0);   // block index list read one tile ahead (off the critical path)
+            // block index list read one tile ahead (off the critical path); an entry outside [0, T_n) -- the loader reads
+            // block 0 for it and reports it -- is simply no tail here, so the loaded value is not touched until its tile comes
+            int blk_next = __ldg(my_idx);
             for (int j = 0; j < keep; ++j, ++t) {
                 // a chunk's last block may be short; found without an integer division (those run on the XU pipe and
                 // would queue behind the other warp's exponentials)
                 bool tail = false;
 #pragma unroll
                 for (int c = 1; c <= HF_MAX_CHUNKS; ++c) tail |= (blk_next + 1 == c * p.n_b);
-                if (j + 1 < keep) blk_next = checked_block(__ldg(my_idx + j + 1), Tn, nullptr, 0);
+                if (j + 1 < keep) blk_next = __ldg(my_idx + j + 1);
                 const int nv = tail ? p.Tc - (p.n_b - 1) * C::BLK : C::BLK;
                 const int st = t & 1;
                 const uint32_t tS = lane_base + rs.stage * C::BLK;
