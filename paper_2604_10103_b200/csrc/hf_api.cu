@@ -314,22 +314,32 @@ template <int D> struct Tc5Groups { static constexpr int N = (D == 128) ? HF_TC5
 
 template <int D>
 hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
-                           int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+                           int keep, const float* hist, bf16* o, float* lse, cudaStream_t st, bool fuse_history = false) {
     typedef SwaTc5<D, Tc5Groups<D>::N> C;
-    CUtensorMap tq, tk, tv;
+    CUtensorMap tq, tk, tv, to;
     HF_TRY(make_map(c, &tq, q, 1));
     HF_TRY(make_map(c, &tk, k_cur, 1));
     HF_TRY(make_map(c, &tv, v_cur, 1));
+    HF_TRY(make_map_ex(c, &to, o, c->Tc, 1, 64, 32, true));      // output: one warp's 32 rows x 64 columns per store
     Tc5Params p;
     p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.n_sink = L.n_sink;
     p.P = c->P;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
+    p.heads = c->cfg.heads; p.eps = c->cfg.eps;
+    p.q = q; p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr;
     const CUtensorMap& rk = c->P + c->n_sink_max > 0 ? L.tm_kring : tk;
     const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
-    k_swa_tc5<D, Tc5Groups<D>::N><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
+    if constexpr (C::FUSE) {
+        if (fuse_history) {
+            k_swa_tc5<D, Tc5Groups<D>::N, true><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p);
+            return post_launch(c, "k_swa_tc5 (history term inside)");
+        }
+    }
+    if (fuse_history) return fail(HF_ERR_UNSUPPORTED, "the attention kernel of this configuration cannot form the history term");
+    k_swa_tc5<D, Tc5Groups<D>::N, false><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p);
     return post_launch(c, "k_swa_tc5");
 }
 
@@ -494,8 +504,10 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = set_swa_attr<64, 128>();
         if (s == HF_OK) s = set_swa_attr<128, 64>();
         if (s == HF_OK) s = set_swa_attr<128, 128>();
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, Tc5Groups<64>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, Tc5Groups<64>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
-        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<64, Tc5Groups<64>::N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, Tc5Groups<64>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<64>) failed");
+        if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128>) failed");
+        if constexpr (SwaTc5<128, Tc5Groups<128>::N>::FUSE)
+            if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128, history>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<64, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<64, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<64>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<128, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<128, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<128>) failed");
         if (s == HF_OK) s = set_state_attr<64>();
@@ -672,7 +684,15 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     HF_TRY(check_ptr(o, "o"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
-    // The history term depends on q and the state only: it runs on the context's side stream while pooling and
+    // At head_dim 128 the tcgen05 attention kernel forms the history term itself (three more tensor-core products per
+    // query block against the folded state, which it keeps in shared memory): no read-out kernel, no scratch buffer.
+    // The rotated variant of Eq. 4 (numerator and denominator see different phi(Q)) keeps the separate read-out.
+    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q) {
+        HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
+        return launch_swa_tc5_t<128>(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, nullptr, (bf16*)o,
+                                     nullptr, st, true);
+    }
+    // Otherwise the history term depends on q and the state only: it runs on the context's side stream while pooling and
     // selection run on the caller's stream; the attention kernel, which adds it in its epilogue, waits for both.
     // (The fork event also orders this read-out after the previous call's attention kernel, which read the same
     // scratch buffer.)

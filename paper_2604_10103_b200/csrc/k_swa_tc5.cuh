@@ -31,14 +31,21 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
-    static constexpr int KSTAGES = 3, VSTAGES = 2, SBUFS = 3;
+    static constexpr int KSTAGES = (D == 128) ? 2 : 3, VSTAGES = 2, SBUFS = 3;   // (a K tile is free again as soon as its S is done)
+    // The history term (Eq. 4) can be formed inside this kernel at head_dim 128 with two column groups: the folded
+    // state S W^T (bf16 hi and lo halves, one operand tile each) then sits in shared memory beside the K / V rings.
+    static constexpr bool FUSE = (D == 128 && NG == 2);
     static constexpr int OFF_Q = 0, OFF_K = TILE_BYTES, OFF_V = OFF_K + KSTAGES * TILE_BYTES;
-    static constexpr int OFF_BAR = OFF_V + VSTAGES * TILE_BYTES;
-    static constexpr int OFF_XM = OFF_BAR + 256;       // row-max exchange [2][NG][128] floats, then row-sum exchange [NG][128]
-    static constexpr int USED_BYTES = OFF_XM + 3 * NG * BLK * 4;
-    // 1 KB slack for manual 1024-byte alignment; more than half an SM's shared memory so that one CTA owns the SM
-    // (it allocates all 512 TMEM columns)
-    static constexpr int SMEM_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
+    static constexpr int OFF_H = OFF_V + VSTAGES * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_H + (FUSE ? 2 * TILE_BYTES : 0);
+    static constexpr int OFF_XM = OFF_BAR + 320;       // exchange between the column groups: [2][NG][128] floats
+    static constexpr int USED_BYTES = OFF_XM + 2 * NG * BLK * 4;
+    static constexpr int MAX_SMEM = 232448;            // 227 KB: the most one thread block can have
+    // Slack for the manual 1024-byte alignment of the operand tiles (the kernel checks that it was enough); more than
+    // half an SM's shared memory so that one CTA owns the SM (it allocates all 512 TMEM columns)
+    static constexpr int WANT_BYTES = (USED_BYTES + 1024) > 120 * 1024 ? (USED_BYTES + 1024) : 120 * 1024;
+    static constexpr int SMEM_BYTES = WANT_BYTES < MAX_SMEM ? WANT_BYTES : MAX_SMEM;
+    static_assert(USED_BYTES <= MAX_SMEM, "shared memory layout does not fit");
     static constexpr int THREADS = 128 * NG + 96;
     static constexpr int WARP_LOAD_K = 4 * NG, WARP_LOAD_V = 4 * NG + 1, WARP_MMA = 4 * NG + 2;
     static constexpr int TMEM_COLS = 512;
@@ -51,7 +58,14 @@ struct Tc5Params {
     int n_sink;              // sink chunks held (logical chunks 0 .. n_sink - 1)
     int Tm, n_units;         // units = (batch*head, query block) pairs, unit u = bh * Tm + i
     float scale_log2;
-    const float* hist;       // optional fp32 [B*H, T_c, D]
+    const float* hist;       // optional fp32 [B*H, T_c, D]: history term formed by another kernel, added in the epilogue
+    // History term formed in the kernel (its HIST instantiation): q as the kernel's own tensor map sees it, z [B*H, D],
+    // bias [H, D] or nullptr, eps of Eq. 4's denominator
+    int heads;
+    float eps;
+    const bf16* q;
+    const float* z;
+    const bf16* bias;
     bf16* o;
     float* lse;
     int* dev_status;
@@ -66,26 +80,37 @@ struct RingPos {
 };
 
 // Persistent: CTA c processes units c, c + gridDim.x, ...
-template <int D, int NG>
+// HIST: the history term is formed here (needs SwaTc5::FUSE and the tensor maps of S W^T); otherwise p.hist, if any, is added.
+template <int D, int NG, bool HIST>
 __global__ void __launch_bounds__(SwaTc5<D, NG>::THREADS, 1)
 k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
           const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
-          const __grid_constant__ CUtensorMap tm_vcur, const Tc5Params p) {
+          const __grid_constant__ CUtensorMap tm_vcur, const __grid_constant__ CUtensorMap tm_sh,
+          const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ CUtensorMap tm_o, const Tc5Params p) {
     using namespace tc5;
     typedef SwaTc5<D, NG> C;
-    extern __shared__ uint8_t smem_raw[];
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
     const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    if (s_base - smem_u32(smem_raw) + C::USED_BYTES > C::SMEM_BYTES) {   // the window started too far off a 1 KB boundary
+        if (threadIdx.x == 0) { atomicOr(p.dev_status, HF_DEV_TIMEOUT_FLAG); atomicExch(p.dev_status + 1, 99); }
+        return;
+    }
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
-    const uint32_t sQ = s_base + C::OFF_Q, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V;
+    const uint32_t sQ = s_base + C::OFF_Q, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V, sH = s_base + C::OFF_H;
+    static_assert(!HIST || C::FUSE, "no room for the folded state in this configuration");
+    constexpr bool fuse = HIST;
     const uint32_t bar0 = s_base + C::OFF_BAR;
     // barrier arrays are indexed by stage: address = base + 8 * stage
     const uint32_t bar_kf = bar0, bar_ke = bar0 + 24, bar_vf = bar0 + 48, bar_ve = bar0 + 64, bar_sf = bar0 + 80,
                    bar_pf = bar0 + 104, bar_pv = bar0 + 128, bar_mx = bar0 + 160, bar_qf = bar0 + 176, bar_qe = bar0 + 184,
-                   bar_ep = bar0 + 192, bar_drain = bar0 + 200;
+                   bar_ep = bar0 + 192, bar_drain = bar0 + 200,
+                   // history term: every thread has read the last tile's maxima / S W^T loaded / ... free again /
+                   // phi(Q) operand written / the unit's accumulator complete
+                   bar_rd = bar0 + 216, bar_hf = bar0 + 224, bar_he = bar0 + 232, bar_af = bar0 + 240, bar_ud = bar0 + 248,
+                   bar_h2 = bar0 + 256;                    // ... and its hi tile loaded (after the copy of Q has been read)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 208);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 212);
     float* x_max = reinterpret_cast<float*>(s_gen + C::OFF_XM);          // [2][NG][128]
-    float* x_sum = x_max + 2 * NG * C::BLK;                               // [NG][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int keep = p.keep;
@@ -97,6 +122,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         for (int s = 0; s < 2; ++s) { mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); mbar_init(bar_mx + 8 * s, 128 * NG); }
         for (int s = 0; s < 4; ++s) mbar_init(bar_pv + 8 * s, 1);
         mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_ep, 128 * NG); mbar_init(bar_drain, 1);
+        mbar_init(bar_rd, 128 * NG); mbar_init(bar_hf, 1); mbar_init(bar_he, 4 * NG); mbar_init(bar_af, 128 * NG); mbar_init(bar_ud, 1); mbar_init(bar_h2, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -158,6 +184,19 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         rv.advance();
                     }
                 }
+                if (ok && fuse && is_k) {
+                    // For the history term at the unit's end: the lo tile of the head's folded state, and a second copy of
+                    // the unit's Q tile where the hi tile will go (the softmax threads take phi(Q) from it; the Q buffer
+                    // proper belongs to the next unit by then).  The buffer is free once the previous unit's output,
+                    // which was staged in it, has been read by the bulk stores.
+                    if (n >= 1 && !(ok = mbar_wait<true>(bar_he, (n - 1) & 1, abort_flag, p.dev_status, 13))) break;
+                    mbar_expect_tx(bar_hf, 2 * C::TILE_BYTES);
+#pragma unroll
+                    for (int s = 0; s < C::SUB; ++s) {
+                        tma_load_4d(sH + s * C::SUB_BYTES, &tm_q, s * 64, i * C::BLK, bh, 0, bar_hf);
+                        tma_load_4d(sH + C::TILE_BYTES + s * C::SUB_BYTES, &tm_sl, s * 64, 0, bh, 0, bar_hf);
+                    }
+                }
             }
             if (!ok) {   // gave up: let the copies already in flight land before the CTA leaves
                 const long long t0 = clock64();
@@ -174,34 +213,39 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         const uint32_t tO = tmem + C::COL_O;
         const uint64_t dq0 = smem_desc_sw128(sQ, 16, 1024), dk0 = smem_desc_sw128(sK, 16, 1024);
         const uint64_t dv0 = smem_desc_sw128(sV, C::SUB_BYTES, 1024);
-        const uint32_t q_lo = (uint32_t)dq0, k_lo = (uint32_t)dk0, v_lo = (uint32_t)dv0;
+        const uint64_t dh0 = smem_desc_sw128(sH, C::SUB_BYTES, 1024);     // S W^T tiles: laid out like a V tile (rows = contraction index)
+        const uint32_t q_lo = (uint32_t)dq0, k_lo = (uint32_t)dk0, v_lo = (uint32_t)dv0, h_lo = (uint32_t)dh0;
         const uint32_t qk_hi = (uint32_t)(dq0 >> 32), v_hi = (uint32_t)(dv0 >> 32);
         bool ok = true;
         int n_s = 0, j_s = 0;                         // unit and position in its list of the next S tile to issue
-        RingPos<C::KSTAGES> rk;                       // K stage of the next S tile (S buffer ring has the same length)
+        RingPos<C::KSTAGES> rk;                       // K stage of the next S tile
+        RingPos<C::SBUFS> rb;                         // ... and its S buffer
         auto issue_s = [&]() -> bool {                // S_t = Q K_t^T into S buffer t % 3
             if (j_s == 0 && !__all_sync(0xffffffffu, mbar_wait<true>(bar_qf, n_s & 1, abort_flag, p.dev_status, 4))) return false;
             if (!__all_sync(0xffffffffu, mbar_wait<true>(bar_kf + 8 * rk.stage, rk.phase, abort_flag, p.dev_status, 5))) return false;
             fence_after_sync();
             if (elect_one()) {
-                mma_ss_tile<D>(tmem + rk.stage * C::BLK, q_lo, k_lo + rk.stage * TILE_STEP, qk_hi, IDESC_S);
-                mma_commit(bar_sf + 8 * rk.stage);
+                mma_ss_tile<D>(tmem + rb.stage * C::BLK, q_lo, k_lo + rk.stage * TILE_STEP, qk_hi, IDESC_S);
+                mma_commit(bar_sf + 8 * rb.stage);
                 mma_commit(bar_ke + 8 * rk.stage);
                 if (j_s == keep - 1) mma_commit(bar_qe);
             }
             __syncwarp();
             rk.advance();
+            rb.advance();
             if (++j_s == keep) { j_s = 0; ++n_s; }
             return true;
         };
-        static_assert(C::KSTAGES == C::SBUFS, "S buffers and K stages advance together");
         if (n_tiles > 0) ok = issue_s();
         if (ok && n_tiles > 1) ok = issue_s();
-        int j_pv = 0;                                 // position of tile t in its unit's list
+        int j_pv = 0, n_pv = 0;                       // position of tile t in its unit's list; the unit
         RingPos<C::SBUFS> rp;                         // S buffer holding P_t
         RingPos<C::VSTAGES> rv;
         for (int t = 0; ok && t < n_tiles; ++t) {
-            if (t + 2 < n_tiles && !(ok = issue_s())) break;
+            // With the history term formed here, the S buffer two tiles on takes the phi(Q) operand at a unit's last tile:
+            // its S is issued after the history products instead of before this tile's P V.
+            const bool last = fuse && (j_pv == keep - 1);
+            if (t + 2 < n_tiles && !last && !(ok = issue_s())) break;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_pf + 8 * rp.stage, rp.phase, abort_flag, p.dev_status, 6)))) break;
             if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_vf + 8 * rv.stage, rv.phase, abort_flag, p.dev_status, 7)))) break;
             fence_after_sync();
@@ -211,9 +255,30 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 mma_commit(bar_ve + 8 * rv.stage);
             }
             __syncwarp();
+            if (last) {
+                // O += (l / den) phi(Q) S W^T: A = hi (64 columns) and lo (64 columns) halves in S buffer (t + 2) % 3,
+                // B = the hi and lo tiles of S W^T; three products, the lo x lo one is below fp32 resolution
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_hf, n_pv & 1, abort_flag, p.dev_status, 14)))) break;
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_af, n_pv & 1, abort_flag, p.dev_status, 15)))) break;
+                fence_after_sync();
+                const int sb = rp.stage + 2 >= C::SBUFS ? rp.stage + 2 - C::SBUFS : rp.stage + 2;
+                const uint32_t tA = tmem + sb * C::BLK;
+                if (elect_one()) mma_ts_tile(tO, tA, h_lo + TILE_STEP, v_hi, IDESC_PV, true);         // hi x lo
+                __syncwarp();
+                // the hi tile was fetched over the copy of Q once every thread had taken its row from it
+                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_h2, n_pv & 1, abort_flag, p.dev_status, 20)))) break;
+                fence_after_sync();
+                if (elect_one()) {
+                    mma_ts_tile(tO, tA, h_lo, v_hi, IDESC_PV, true);                                  // hi x hi
+                    mma_ts_tile(tO, tA + D / 2, h_lo, v_hi, IDESC_PV, true);                          // lo x hi
+                    mma_commit(bar_ud);
+                }
+                __syncwarp();
+                if (t + 2 < n_tiles && !(ok = issue_s())) break;
+            }
             rp.advance();
             rv.advance();
-            if (++j_pv == keep) j_pv = 0;
+            if (++j_pv == keep) { j_pv = 0; ++n_pv; }
         }
         // drain: all MMAs issued by this warp have completed before TMEM is freed
         if (elect_one()) mma_commit(bar_drain);
@@ -287,12 +352,25 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     // every group has read its S columns (the P columns written below overlap another group's S)
                     // and learns the maximum of the whole row
                     float* xm = x_max + st * NG * C::BLK;
+                    if (fuse && j == 0 && n >= 1 && lane == 0) {
+                        // the output tile of the previous unit was staged where S W^T lives: the loader may refill the
+                        // buffer once every warp's bulk store has read its part
+                        bulk_wait_read();
+                        mbar_arrive(bar_he);
+                    }
+                    if (fuse && j == 0 && n >= 1) {
+                        // the previous unit used both exchange buffers for its row sums and denominators: every thread
+                        // has read them once it has arrived with its phi(Q) operand
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_af, (n - 1) & 1, abort_flag, p.dev_status, 16));
+                        if (!ok) break;
+                    }
                     xm[grp * C::BLK + row] = mrow;
                     mbar_arrive(bar_mx + 8 * st);
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 11));
                     if (!ok) break;
 #pragma unroll
                     for (int g = 0; g < NG; ++g) mrow = fmaxf(mrow, xm[g * C::BLK + row]);
+                    if (j == keep - 1) mbar_arrive(bar_rd);     // the unit's last maxima are out of the buffers
                 }
                 const float m_new = fmaxf(m_used, mrow * p.scale_log2);
                 // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
@@ -346,22 +424,153 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 mbar_arrive(bar_pf + 8 * (rs.stage == 0 ? C::SBUFS - 1 : rs.stage - 1));
             }
             if (!ok) break;
-            // ---- epilogue of the unit: O / l (+ history term), one rounding to bf16
+            // ---- end of the unit.  The exchange buffers of the row maxima carry the groups' row sums (and, with the
+            // history term formed here, their shares of Eq. 4's denominator) once every thread has read the last maxima.
+            float inv;
             if (NG > 1) {
-                x_sum[grp * C::BLK + row] = l_run;
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_rd, n & 1, abort_flag, p.dev_status, 17));
+                if (!ok) break;
+            }
+            float* x_l = x_max + ((t - 1) & 1) * NG * C::BLK;     // buffer of the unit's last tile: next written two tiles on
+            float* x_d = x_max + (t & 1) * NG * C::BLK;           // buffer of the next tile: see the wait at a unit's first tile
+            if constexpr (fuse) {
+                // ---- history term (Eq. 4): A = (l / den) phi(q) as bf16 hi + lo, this group's 64 features of the row,
+                // read from global memory (the Q tile in shared memory already belongs to the next unit)
+                constexpr int FPT = D / NG;                         // features per thread
+                const int feat0 = grp * FPT;
+                uint4 qv[FPT / 8];
+                {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_hf, n & 1, abort_flag, p.dev_status, 21));
+                    if (!ok) break;
+                    // this group's 64-column sub-tile of the copy, 128-byte swizzle (rows past the chunk's end: zero fill)
+                    const uint8_t* qrow = s_gen + C::OFF_H + grp * C::SUB_BYTES + row * 128;
+#pragma unroll
+                    for (int c = 0; c < FPT / 8; ++c) qv[c] = *reinterpret_cast<const uint4*>(qrow + ((c ^ (row & 7)) << 4));
+                }
+                float f[FPT];
+                float dsum = 0.f;
+                const float4* zsrc = reinterpret_cast<const float4*>(p.z + (size_t)bh * D + feat0);
+#pragma unroll
+                for (int c = 0; c < FPT / 8; ++c) {
+                    const float4 z0 = __ldg(zsrc + 2 * c), z1 = __ldg(zsrc + 2 * c + 1);
+                    const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+                    const uint32_t ws[4] = {qv[c].x, qv[c].y, qv[c].z, qv[c].w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 x = unpack_bf16(ws[e]);
+                        const float f0 = phi_elu1(x.x), f1 = phi_elu1(x.y);
+                        f[c * 8 + 2 * e] = f0; f[c * 8 + 2 * e + 1] = f1;
+                        dsum = fmaf(f0, zz[2 * e], fmaf(f1, zz[2 * e + 1], dsum));
+                    }
+                }
+                x_l[grp * C::BLK + row] = l_run;
+                x_d[grp * C::BLK + row] = dsum;
                 mbar_arrive(bar_ep);
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_ep, n & 1, abort_flag, p.dev_status, 12));
                 if (!ok) break;
-                l_run = x_sum[row];
+                if (warp == 0 && lane == 0) {
+                    // every thread has taken its row of the Q copy (it arrived above only after that): the hi tile of the
+                    // folded state can come in over it
+                    mbar_expect_tx(bar_h2, C::TILE_BYTES);
 #pragma unroll
-                for (int g = 1; g < NG; ++g) l_run += x_sum[g * C::BLK + row];
+                    for (int s = 0; s < C::SUB; ++s) tma_load_4d(sH + s * C::SUB_BYTES, &tm_sh, s * 64, 0, bh, 0, bar_h2);
+                }
+                float den = p.eps;
+                l_run = 0.f;
+#pragma unroll
+                for (int g = 0; g < NG; ++g) { l_run += x_l[g * C::BLK + row]; den += x_d[g * C::BLK + row]; }
+                inv = 1.f / l_run;
+                const float fac = l_run / den;                      // O is divided by l at the end: pre-multiply the history term
+                // the S buffer two tiles on held P of the tile before the unit's last one: its P V must have read it
+                if (t >= 2) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_pv + 8 * ((t - 2) & 3), ((t - 2) >> 2) & 1, abort_flag, p.dev_status, 18));
+                    if (!ok) break;
+                    fence_after_sync();
+                }
+                const int sb = rs.stage + 1 >= C::SBUFS ? rs.stage + 1 - C::SBUFS : rs.stage + 1;   // rs: buffer of tile t; + 1 = (t_last + 2) % 3
+                const uint32_t tA = lane_base + sb * C::BLK + feat0 / 2;
+#pragma unroll
+                for (int h = 0; h < FPT / 32; ++h) {
+                    uint32_t hi[16], lo[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const float a0 = f[h * 32 + 2 * e] * fac, a1 = f[h * 32 + 2 * e + 1] * fac;
+                        const uint32_t hp = pack_bf16(a0, a1);
+                        const float2 hf = unpack_bf16(hp);
+                        hi[e] = hp;
+                        lo[e] = pack_bf16(a0 - hf.x, a1 - hf.y);
+                    }
+                    tmem_st16(tA + h * 16, hi);
+                    tmem_st16(tA + D / 2 + h * 16, lo);
+                }
+                tmem_wait_st();
+                fence_before_sync();
+                mbar_arrive(bar_af);
+                // the unit's accumulator: its last P V and the three history products
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_ud, n & 1, abort_flag, p.dev_status, 19));
+                if (!ok) break;
+                fence_after_sync();
+            } else {
+                if (NG > 1) {
+                    x_l[grp * C::BLK + row] = l_run;
+                    mbar_arrive(bar_ep);
+                    ok = __all_sync(0xffffffffu, mbar_wait(bar_ep, n & 1, abort_flag, p.dev_status, 12));
+                    if (!ok) break;
+                    l_run = x_l[row];
+#pragma unroll
+                    for (int g = 1; g < NG; ++g) l_run += x_l[g * C::BLK + row];
+                }
+                ok = wait_pv_prev(10);
+                if (!ok) break;
+                fence_after_sync();
+                inv = 1.f / l_run;
             }
-            ok = wait_pv_prev(10);
-            if (!ok) break;
-            fence_after_sync();
-            const float inv = 1.f / l_run;
+            const bf16* bias_row = (fuse && p.bias) ? p.bias + (size_t)(bh % p.heads) * D : nullptr;
             const size_t g_row = (size_t)bh * p.Tc + q0 + row;
             if (grp == 0 && row < nq && p.lse) p.lse[g_row] = (m_used + log2f(l_run)) * 0.6931471805599453f;
+            if constexpr (C::FUSE) {
+                // Output through shared memory and one bulk tensor store per warp (32 rows x 64 columns): row-per-thread
+                // global stores would touch 32 lines per instruction.  The staging tile is the S W^T buffer (free: the
+                // history products have completed, or were never asked for); layout = the 128-byte swizzle of the map.
+                uint8_t* stage = s_gen + C::OFF_H + grp * C::SUB_BYTES + (warp & 3) * 4096 + lane * 128;
+                if (lane == 0) bulk_wait_read();            // this warp's previous store has read its part
+                __syncwarp();
+#pragma unroll
+                for (int c = 0; c < C::OCOLS / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
+                    const float* hsrc = p.hist ? p.hist + g_row * D + grp * C::OCOLS + c * 32 : nullptr;
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        float x[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) x[e] = __uint_as_float(o[v * 8 + e]) * inv;
+                        if (hsrc && row < nq) {
+                            const float4 h0 = *reinterpret_cast<const float4*>(hsrc + v * 8);
+                            const float4 h1 = *reinterpret_cast<const float4*>(hsrc + v * 8 + 4);
+                            x[0] += h0.x; x[1] += h0.y; x[2] += h0.z; x[3] += h0.w;
+                            x[4] += h1.x; x[5] += h1.y; x[6] += h1.z; x[7] += h1.w;
+                        }
+                        if (bias_row) {     // Eq. 4's Linear: its matrix is folded into the state, its bias is added here
+                            const uint4 bw = __ldg(reinterpret_cast<const uint4*>(bias_row + grp * C::OCOLS + c * 32 + v * 8));
+                            const float2 b0 = unpack_bf16(bw.x), b1 = unpack_bf16(bw.y), b2 = unpack_bf16(bw.z), b3 = unpack_bf16(bw.w);
+                            x[0] += b0.x; x[1] += b0.y; x[2] += b1.x; x[3] += b1.y;
+                            x[4] += b2.x; x[5] += b2.y; x[6] += b3.x; x[7] += b3.y;
+                        }
+                        uint4 w;
+                        w.x = pack_bf16(x[0], x[1]); w.y = pack_bf16(x[2], x[3]);
+                        w.z = pack_bf16(x[4], x[5]); w.w = pack_bf16(x[6], x[7]);
+                        *reinterpret_cast<uint4*>(stage + (((c * 4 + v) ^ (lane & 7)) << 4)) = w;
+                    }
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0 && q0 + (warp & 3) * 32 < p.Tc) {     // rows past the chunk's end are clipped by the map
+                    tma_store_4d(&tm_o, s_base + C::OFF_H + grp * C::SUB_BYTES + (warp & 3) * 4096, grp * 64, q0 + (warp & 3) * 32, bh, 0);
+                    bulk_commit();
+                }
+            } else {
 #pragma unroll
             for (int c = 0; c < C::OCOLS / 32; ++c) {
                 uint32_t o[32];
@@ -389,11 +598,13 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     }
                 }
             }
+            }
             // the next unit's first P.V overwrites O: it is gated by p_full of that tile, which these threads
             // arrive on only after this epilogue
             fence_before_sync();
         }
     }
+    if (C::FUSE && warp < 4 * NG && lane == 0) bulk_wait_all();     // output tiles still on their way out of shared memory
     fence_before_sync();
     __syncthreads();
     if (warp == C::WARP_MMA) {
