@@ -286,7 +286,7 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     const int keep = keep_for(c, Tn);
     ChunkTable tab = make_table(c, L, k_cur, nullptr);
-    k_select<D><<<dim3(c->Tm, c->BH), 128, 0, st>>>(tab, c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+    k_select<D><<<dim3(c->Tm, c->BH), 256, 0, st>>>(tab, c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
                                                    L.mask, L.idx, mask_out, idx_out, scores_out);
     HF_TRY(post_launch(c, "k_select"));
     L.sel_epoch = L.cache_epoch;

@@ -82,62 +82,55 @@ __global__ void __launch_bounds__(256) k_pool_copy(PoolJobs jobs, int Tc, int bl
     }
 }
 
-// A[i][j] = Mean(q_i) . Mean(k_j) in the canonical order, formed by one thread: 32 partials (partial l = columns l,
-// l + 32, ... ascending, product and sum rounded separately), then the butterfly.  The shuffle butterfly
-// p[l] + p[l ^ off] gives both partners the same value (IEEE addition commutes), so folding the upper half onto the
-// lower half level by level yields lane 0's result bit for bit.  sq: the pooled query row (shared memory), kp: the
-// pooled key row.
-template <int D>
-__device__ __forceinline__ float canonical_score(const float* sq, const float4* __restrict__ kp) {
-    float pl[32];
-#pragma unroll
-    for (int m = 0; m < D / 32; ++m) {
-        float4 kv[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) kv[i] = __ldg(kp + m * 8 + i);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float kk[4] = {kv[i].x, kv[i].y, kv[i].z, kv[i].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int l = 4 * i + e;
-                const float pr = __fmul_rn(sq[l + 32 * m], kk[e]);
-                pl[l] = (m == 0) ? pr : __fadd_rn(pl[l], pr);
-            }
-        }
-    }
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1)
-#pragma unroll
-        for (int l = 0; l < off; ++l) pl[l] = __fadd_rn(pl[l], pl[l + off]);
-    return pl[0];
-}
-
-// grid (T_m, B*H), 128 threads.  One query-block row: T_n scores, rank-based top-K under the total order
+// A[i][j] = Mean(q_i) . Mean(k_j) in the canonical order, formed by one warp: 32 partials (partial l = columns l,
+// l + 32, ... ascending, product and sum rounded separately; lane l holds partial l, so the loads of a key row are
+// coalesced), then the butterfly p[l] + p[l ^ off], off = 16 .. 1: both partners get the same value (IEEE addition
+// commutes), so lane 0 ends with the fold of the upper half onto the lower half level by level, bit for bit.
+// grid (T_m, B*H), 256 threads.  One query-block row: T_n scores, rank-based top-K under the total order
 // (score descending, block index ascending), bit mask + ascending index list.
 template <int D>
-__global__ void __launch_bounds__(128) k_select(ChunkTable tab, const float* __restrict__ pooled_q,
+__global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __restrict__ pooled_q,
                                                 int n_b, int Tm, int Tn, int keep, int mask_words,
                                                 uint32_t* __restrict__ mask, int32_t* __restrict__ idx,
                                                 uint32_t* __restrict__ mask_out, int32_t* __restrict__ idx_out,
                                                 float* __restrict__ scores_out) {
-    __shared__ float sq[D];
     __shared__ float sc[HF_MAX_TN];
     __shared__ uint8_t keepf[HF_MAX_TN];
     const int i = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const size_t row = (size_t)bh * Tm + i;
-    if (threadIdx.x < D) sq[threadIdx.x] = pooled_q[row * D + threadIdx.x];
-    __syncthreads();
-    // One thread per key block (see canonical_score).
-    for (int j = threadIdx.x; j < Tn; j += 128) {
-        const int c = j / n_b, jb = j - c * n_b;
-        const float s = canonical_score<D>(sq, reinterpret_cast<const float4*>(tab.pooled[c] + ((size_t)bh * n_b + jb) * D));
-        sc[j] = s;
-        if (scores_out) scores_out[row * Tn + j] = s;
+    // One warp per score, lane l = partial l.  All loads of a pass (the lane's columns of the query row and of sixteen key
+    // rows) are issued before the first use: one trip to memory per pass, and one pass covers 128 key blocks.
+    constexpr int NW = 8, PER = 16, M = D / 32;
+    float qv[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) qv[m] = __ldg(pooled_q + row * D + lane + 32 * m);
+    for (int base = 0; base < Tn; base += NW * PER) {
+        float kv[PER][M];
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            const int j = min(base + warp + NW * u, Tn - 1);
+            const int c = j / n_b, jb = j - c * n_b;
+            const float* kp = tab.pooled[c] + ((size_t)bh * n_b + jb) * D + lane;
+#pragma unroll
+            for (int m = 0; m < M; ++m) kv[u][m] = __ldg(kp + 32 * m);
+        }
+#pragma unroll
+        for (int u = 0; u < PER; ++u) {
+            float p = __fmul_rn(qv[0], kv[u][0]);
+#pragma unroll
+            for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[m], kv[u][m]));
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, off));
+            const int j = base + warp + NW * u;
+            if (lane == 0 && j < Tn) {
+                sc[j] = p;
+                if (scores_out) scores_out[row * Tn + j] = p;
+            }
+        }
     }
     __syncthreads();
-    for (int j = threadIdx.x; j < Tn; j += 128) {
+    for (int j = threadIdx.x; j < Tn; j += 256) {
         const float s = sc[j];
         int rank = 0;
         for (int jj = 0; jj < Tn; ++jj) {
