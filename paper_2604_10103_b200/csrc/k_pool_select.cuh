@@ -33,40 +33,45 @@ struct PoolJobs { PoolJob job[3]; };
 
 // grid (n_b, B*H, jobs), 256 threads: 16 threads per token row, 16 rows per pass.
 template <int D>
-__global__ void __launch_bounds__(256) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
+__global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
     constexpr int VEC = D / 16;
     typedef typename VecLoad<VEC>::T V;
-    const PoolJob jb = jobs.job[blockIdx.z];
+    const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
     const int b_idx = blockIdx.x, bh = blockIdx.y;
     const int t0 = b_idx * blk;
     const int n = min(blk, Tc - t0);
     const int r = threadIdx.x >> 4, cv = threadIdx.x & 15;
     const size_t base = ((size_t)bh * Tc + t0) * D + cv * VEC;
-    // all loads of the thread first (up to 8 rows in flight), then the copies, then the chain adds in token order
-    constexpr int MAXR = 8;                       // blk <= 128 -> at most 8 rows per chain
-    V u[MAXR];
-#pragma unroll
-    for (int i = 0; i < MAXR; ++i) {
-        const int t = r + 16 * i;
-        if (t < n) u[i] = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
-    }
-    if (jb.copy_dst) {
-#pragma unroll
-        for (int i = 0; i < MAXR; ++i) {
-            const int t = r + 16 * i;
-            if (t < n) *reinterpret_cast<V*>(jb.copy_dst + base + (size_t)t * D) = u[i];
-        }
-    }
+    // Two batches of four rows: the loads of a batch first, then its copies, then its chain adds in token order.  (Four
+    // 16-byte loads in flight per thread at six thread blocks per SM keep ~100 KB in flight per SM; eight would cost the
+    // registers that the sixth block needs.)
+    constexpr int MAXR = 8, BATCH = 4;            // blk <= 128 -> at most 8 rows per chain
     float acc[VEC];
 #pragma unroll
     for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
 #pragma unroll
-    for (int i = 0; i < MAXR; ++i) {
-        if (r + 16 * i < n) {
-            float f[VEC];
-            VecLoad<VEC>::widen(u[i], f);
+    for (int i0 = 0; i0 < MAXR; i0 += BATCH) {
+        V u[BATCH];
 #pragma unroll
-            for (int e = 0; e < VEC; ++e) acc[e] = __fadd_rn(acc[e], f[e]);
+        for (int i = 0; i < BATCH; ++i) {
+            const int t = r + 16 * (i0 + i);
+            if (t < n) u[i] = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
+        }
+        if (jb.copy_dst) {
+#pragma unroll
+            for (int i = 0; i < BATCH; ++i) {
+                const int t = r + 16 * (i0 + i);
+                if (t < n) *reinterpret_cast<V*>(jb.copy_dst + base + (size_t)t * D) = u[i];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+            if (r + 16 * (i0 + i) < n) {
+                float f[VEC];
+                VecLoad<VEC>::widen(u[i], f);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc[e] = __fadd_rn(acc[e], f[e]);
+            }
         }
     }
     if (jb.pooled == nullptr) return;
