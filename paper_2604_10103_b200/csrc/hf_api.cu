@@ -173,6 +173,20 @@ hf_status set_state_attr() {
 
 #define HF_DISPATCH_D(c, FN, ...) ((c)->d == 128 ? FN<128>(__VA_ARGS__) : FN<64>(__VA_ARGS__))
 
+// Launch configuration of a kernel that may start while the kernel before it in the stream still runs (programmatic
+// dependent launch); the kernel calls pdl_wait() before it touches anything that kernel wrote.
+struct PdlLaunch {
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    PdlLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool overlap) {
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = overlap ? 1 : 0;
+    }
+};
+
 hf_status post_launch(hf_ctx* c, const char* what, int n = 1) {
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(HF_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
@@ -286,8 +300,9 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     const int keep = keep_for(c, Tn);
     ChunkTable tab = make_table(c, L, k_cur, nullptr);
-    k_select<D><<<dim3(c->Tm, c->BH), 256, 0, st>>>(tab, c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
-                                                   L.mask, L.idx, mask_out, idx_out, scores_out);
+    PdlLaunch pl(dim3(c->Tm, c->BH), dim3(256), 0, st, true);      // follows the pooling kernel launched above
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+                               L.mask, L.idx, mask_out, idx_out, scores_out));
     HF_TRY(post_launch(c, "k_select"));
     L.sel_epoch = L.cache_epoch;
     L.sel_keep = keep;
@@ -314,7 +329,8 @@ template <int D> struct Tc5Groups { static constexpr int N = (D == 128) ? HF_TC5
 
 template <int D>
 hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
-                           int keep, const float* hist, bf16* o, float* lse, cudaStream_t st, bool fuse_history = false) {
+                           int keep, const float* hist, bf16* o, float* lse, cudaStream_t st, bool fuse_history = false,
+                           bool overlap_prev = false) {
     typedef SwaTc5<D, Tc5Groups<D>::N> C;
     CUtensorMap tq, tk, tv, to;
     HF_TRY(make_map(c, &tq, q, 1));
@@ -332,14 +348,15 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, overlap_prev);
     if constexpr (C::FUSE) {
         if (fuse_history) {
-            k_swa_tc5<D, Tc5Groups<D>::N, true><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p);
+            HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_tc5<D, Tc5Groups<D>::N, true>, tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p));
             return post_launch(c, "k_swa_tc5 (history term inside)");
         }
     }
     if (fuse_history) return fail(HF_ERR_UNSUPPORTED, "the attention kernel of this configuration cannot form the history term");
-    k_swa_tc5<D, Tc5Groups<D>::N, false><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_tc5<D, Tc5Groups<D>::N, false>, tq, rk, rv, tk, tv, L.tm_sfhi, L.tm_sflo, to, p));
     return post_launch(c, "k_swa_tc5");
 }
 
@@ -690,7 +707,7 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q) {
         HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
         return launch_swa_tc5_t<128>(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, nullptr, (bf16*)o,
-                                     nullptr, st, true);
+                                     nullptr, st, true, true);       // may start under the selection kernel's tail
     }
     // Otherwise the history term depends on q and the state only: it runs on the context's side stream while pooling and
     // selection run on the caller's stream; the attention kernel, which adds it in its epilogue, waits for both.

@@ -20,6 +20,12 @@ struct ChunkTable {
 // Device status word layout (int[4]): [0] flags, [1] detail, [2..3] reserved.
 enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2 };
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its predecessor
+// in the stream still runs (once every block of the predecessor has called pdl_trigger or exited); pdl_wait returns when the
+// predecessor has completed and its writes are visible.  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
 // A kept-block index read from a caller's list: inside [0, Tn) it is returned as it is; anything else is replaced by
 // block 0 (so that every address formed from it stays inside the cache) and recorded in the status word.
 __device__ __forceinline__ int checked_block(int j, int Tn, int* dev_status, int unit) {

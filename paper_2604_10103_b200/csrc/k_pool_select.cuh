@@ -36,6 +36,7 @@ template <int D>
 __global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
     constexpr int VEC = D / 16;
     typedef typename VecLoad<VEC>::T V;
+    pdl_trigger();              // a dependent kernel (the selection) may be made resident; it waits for this grid itself
     const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
     const int b_idx = blockIdx.x, bh = blockIdx.y;
     const int t0 = b_idx * blk;
@@ -104,6 +105,8 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
     const int i = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const size_t row = (size_t)bh * Tm + i;
+    pdl_trigger();              // the attention kernel may be made resident as blocks of this grid leave
+    pdl_wait();                 // the pooled rows of the query and of the current chunk come from the kernel before
     // One warp per score, lane l = partial l.  All loads of a pass (the lane's columns of the query row and of sixteen key
     // rows) are issued before the first use: one trip to memory per pass, and one pass covers 128 key blocks.
     constexpr int NW = 8, PER = 16, M = D / 32;

@@ -134,6 +134,9 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     __syncthreads();
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
+    // Everything above (barriers, tensor memory) may overlap the tail of the kernel before this one in the stream when the
+    // launch allows it; the index list it wrote is read from here on.
+    pdl_wait();
 
     if (warp == C::WARP_LOAD_K || warp == C::WARP_LOAD_V) {
         // ================================================================= TMA producers
