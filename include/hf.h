@@ -134,6 +134,14 @@ hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur
 /* Eq. 4 without rotation: o_hist[r] = W (phi(q_r) S / (phi(q_r) . z + eps)) + bias, bf16 [B,H,T_c,d]. */
 hf_status hf_linear_attn(hf_ctx* ctx, int layer, const void* q, void* o_hist, void* stream);
 
+/* Eq. 6 + Eq. 4 + Eq. 7 for a selection that is already made (idx as for hf_sparse_swa; NULL = the context's last
+ * selection): o = o_local + o_history, rounded once to bf16 [B,H,T_c,d].  hf_hybrid_forward is hf_block_select followed
+ * by this call.  With 128-token blocks at head_dim 128 and no rotation tables it is ONE kernel: the attention kernel
+ * forms the history term on the tensor cores at the end of each query block; otherwise the read-out kernel runs first
+ * and the attention kernel adds its result. */
+hf_status hf_sparse_swa_merged(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
+                               void* o, void* stream);
+
 /* Alg. 3 + Eq. 7 for one denoising step: selection, sparse attention and history read-out of q against the
  * cache + (k, v), o = o_local + o_history rounded once to bf16 [B,H,T_c,d]. */
 hf_status hf_hybrid_forward(hf_ctx* ctx, int layer, const void* q, const void* k, const void* v, void* o, void* stream);

@@ -28,6 +28,7 @@ EXPORTS = [
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
     "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
+    "hf_sparse_swa_merged",
 ]
 
 
@@ -68,6 +69,7 @@ def lib() -> C.CDLL:
     L.hf_block_select.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp]
     L.hf_sparse_swa.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp, vp]
     L.hf_linear_attn.argtypes = [vp, ip, vp, vp, vp]
+    L.hf_sparse_swa_merged.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp]
     L.hf_hybrid_forward.argtypes = [vp, ip, vp, vp, vp, vp, vp]
     L.hf_hybrid_forward_host.argtypes = [vp, ip, vp, vp, vp, vp, vp]
     L.hf_kv_append_host.argtypes = [vp, ip, vp, vp, vp]
@@ -155,6 +157,9 @@ class Context:
     def hf_sparse_swa(self, layer, q, k_cur, v_cur, o_local, idx=None, lse=None):
         _check(lib().hf_sparse_swa(self._h, layer, _ptr(q), _ptr(k_cur), _ptr(v_cur), _ptr(idx), _ptr(o_local),
                                    _ptr(lse), _stream()))
+
+    def hf_sparse_swa_merged(self, layer, q, k_cur, v_cur, o, idx=None):
+        _check(lib().hf_sparse_swa_merged(self._h, layer, _ptr(q), _ptr(k_cur), _ptr(v_cur), _ptr(idx), _ptr(o), _stream()))
 
     def hf_linear_attn(self, layer, q, o_hist):
         _check(lib().hf_linear_attn(self._h, layer, _ptr(q), _ptr(o_hist), _stream()))

@@ -693,6 +693,37 @@ hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void
     return HF_DISPATCH_D(c, launch_readout, c, c->layers[layer], (const bf16*)q, (bf16*)o_hist, (float*)nullptr, (cudaStream_t)stream);
 }
 
+// Eq. 6 + Eq. 4 + Eq. 7 for a selection that is already made.  after_select: the call follows launch_select in the same
+// stream directly, so the attention kernel may be launched under its tail.
+static hf_status attend_merge(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k, const bf16* v, const int32_t* idx, int keep,
+                              bf16* o, cudaStream_t st, bool after_select) {
+    // At head_dim 128 the tcgen05 attention kernel forms the history term itself (three more tensor-core products per
+    // query block against the folded state, which it keeps in shared memory): no read-out kernel, no scratch buffer.
+    // The rotated variant of Eq. 4 (numerator and denominator see different phi(Q)) keeps the separate read-out.
+    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q)
+        return launch_swa_tc5_t<128>(c, L, q, k, v, idx, keep, nullptr, o, nullptr, st, true, after_select);
+    // Otherwise the read-out kernel writes the history term to the context's scratch buffer and the attention kernel adds
+    // it in its epilogue.
+    HF_TRY(HF_DISPATCH_D(c, launch_readout, c, L, q, (bf16*)nullptr, c->hist, st));
+    return launch_swa(c, L, q, k, v, idx, keep, c->hist, o, nullptr, st);
+}
+
+hf_status hf_sparse_swa_merged(hf_ctx* c, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
+                               void* o, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q"));
+    HF_TRY(check_ptr(k_cur, "k_cur"));
+    HF_TRY(check_ptr(v_cur, "v_cur"));
+    HF_TRY(check_ptr(o, "o"));
+    LayerState& L = c->layers[layer];
+    const int keep = keep_for(c, (L.n_sink + L.n_cached + 1) * c->n_b);
+    if (idx == nullptr) {
+        if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
+        idx = L.idx;
+    }
+    return attend_merge(c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, (bf16*)o, (cudaStream_t)stream, false);
+}
+
 hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, const void* v, void* o, void* stream) {
     HF_TRY(check_layer(c, layer));
     HF_TRY(check_ptr(q, "q"));
@@ -701,13 +732,10 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     HF_TRY(check_ptr(o, "o"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
-    // At head_dim 128 the tcgen05 attention kernel forms the history term itself (three more tensor-core products per
-    // query block against the folded state, which it keeps in shared memory): no read-out kernel, no scratch buffer.
-    // The rotated variant of Eq. 4 (numerator and denominator see different phi(Q)) keeps the separate read-out.
-    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q) {
+    const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q;
+    if (one_kernel) {
         HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
-        return launch_swa_tc5_t<128>(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, nullptr, (bf16*)o,
-                                     nullptr, st, true, true);       // may start under the selection kernel's tail
+        return attend_merge(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, (bf16*)o, st, true);
     }
     // Otherwise the history term depends on q and the state only: it runs on the context's side stream while pooling and
     // selection run on the caller's stream; the attention kernel, which adds it in its epilogue, waits for both.

@@ -411,3 +411,34 @@ def test_block_indices_outside_the_cache_are_caught_on_the_device(d, b, tpf, ker
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,b,tpf", [(128, 128, 200), (64, 16, 64)])
+def test_attention_with_history_for_a_given_selection(d, b, tpf):
+    """hf_sparse_swa_merged on the context's last selection gives the bits hf_hybrid_forward gives (one kernel at
+    head_dim 128 with 128-token blocks, read-out + attention otherwise), and the oracle's output."""
+    import torch
+    w = gen.Workload("merged", batch=1, heads=2, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=3,
+                     block=b, topk=2, keep_permille=0, seed=29)
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        for c in range(4):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        qb, kb, vb = gen.qkv(w, 0, 4, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        o_fwd = gpu.forward(q, k, v)
+        m_gpu, idx, _ = gpu.select(q, k)
+        o = torch.empty(gpu.shape, dtype=torch.bfloat16, device="cuda")
+        gpu.ctx.hf_sparse_swa_merged(0, q, k, v, o)
+        torch.cuda.synchronize()
+        assert np.array_equal(gpu.f64(o), o_fwd)
+        o2 = torch.empty_like(o)
+        gpu.ctx.hf_sparse_swa_merged(0, q, k, v, o2, idx=torch.from_numpy(idx).cuda())
+        torch.cuda.synchronize()
+        assert np.array_equal(gpu.f64(o2), o_fwd)
+        m_ref, _ = ora.select(f64(qb), f64(kb))
+        hz.assert_close_out(o_fwd, ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref), "merged output")
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
