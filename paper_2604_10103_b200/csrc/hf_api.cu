@@ -198,7 +198,8 @@ hf_status post_launch(hf_ctx* c, const char* what, int n = 1) {
 template <int D>
 hf_status launch_pool(hf_ctx* c, const PoolJobs& jobs, int njobs, cudaStream_t st) {
     dim3 grid(c->n_b, c->BH, njobs);
-    k_pool_copy<D><<<grid, 256, 0, st>>>(jobs, c->Tc, c->cfg.block, c->n_b);
+    PdlLaunch pl(grid, dim3(256), 0, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_pool_copy<D>, jobs, c->Tc, c->cfg.block, c->n_b));
     return post_launch(c, "k_pool_copy");
 }
 
@@ -245,8 +246,9 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     AbsorbTc5Params p;
     p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
     p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc;
-    if (c->has_rope_k) k_absorb_tc5<D, true><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
-    else k_absorb_tc5<D, false><<<dim3(nsplit, c->BH), A::THREADS, A::SMEM_BYTES, st>>>(tk, tv, p);
+    PdlLaunch pl(dim3(nsplit, c->BH), dim3(A::THREADS), A::SMEM_BYTES, st, true);
+    if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, true>, tk, tv, p));
+    else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, false>, tk, tv, p));
     HF_TRY(post_launch(c, "k_absorb_tc5"));
     if (!fold_on_side) return launch_fold<D>(c, L, nsplit, st);
     HF_CUDA(cudaEventRecord(c->ev_fork, st));

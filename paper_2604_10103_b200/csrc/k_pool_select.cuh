@@ -36,6 +36,7 @@ template <int D>
 __global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
     constexpr int VEC = D / 16;
     typedef typename VecLoad<VEC>::T V;
+    pdl_wait();                 // launched under the tail of the kernel before it: that kernel's reads and writes are done from here on
     pdl_trigger();              // a dependent kernel (the selection) may be made resident; it waits for this grid itself
     const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
     const int b_idx = blockIdx.x, bh = blockIdx.y;

@@ -82,6 +82,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
     __syncthreads();
     fence_after_sync();
     const uint32_t tmem = *tmem_slot;
+    pdl_wait();                 // (set-up above may overlap the tail of the kernel before this one in the stream)
 
     if (warp == C::WARP_TMA) {
         // ================================================================= TMA producer

@@ -137,6 +137,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // Everything above (barriers, tensor memory) may overlap the tail of the kernel before this one in the stream when the
     // launch allows it; the index list it wrote is read from here on.
     pdl_wait();
+    pdl_trigger();              // the next kernel in the stream may be made resident on SMs this grid has left; it waits itself
 
     if (warp == C::WARP_LOAD_K || warp == C::WARP_LOAD_V) {
         // ================================================================= TMA producers
