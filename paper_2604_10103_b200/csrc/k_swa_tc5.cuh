@@ -319,6 +319,18 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             // block index list read one tile ahead (off the critical path); an entry outside [0, T_n) -- the loader reads
             // block 0 for it and reports it -- is simply no tail here, so the loaded value is not touched until its tile comes
             int blk_next = __ldg(my_idx);
+            if (fuse && n >= 1) {
+                // The output tile of the previous unit was staged where S W^T lives: the loader may refill the buffer once
+                // every warp's bulk store has read its part.  And that unit used both exchange buffers for its row sums and
+                // denominators: every thread has read them once it has arrived with its phi(Q) operand.
+                if (lane == 0) {
+                    bulk_wait_read();
+                    mbar_arrive(bar_he);
+                }
+                __syncwarp();
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_af, (n - 1) & 1, abort_flag, p.dev_status, 16));
+                if (!ok) break;
+            }
             for (int j = 0; j < keep; ++j, ++t) {
                 // a chunk's last block may be short; found without an integer division (those run on the XU pipe and
                 // would queue behind the other warp's exponentials)
@@ -356,18 +368,6 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                     // every group has read its S columns (the P columns written below overlap another group's S)
                     // and learns the maximum of the whole row
                     float* xm = x_max + st * NG * C::BLK;
-                    if (fuse && j == 0 && n >= 1 && lane == 0) {
-                        // the output tile of the previous unit was staged where S W^T lives: the loader may refill the
-                        // buffer once every warp's bulk store has read its part
-                        bulk_wait_read();
-                        mbar_arrive(bar_he);
-                    }
-                    if (fuse && j == 0 && n >= 1) {
-                        // the previous unit used both exchange buffers for its row sums and denominators: every thread
-                        // has read them once it has arrived with its phi(Q) operand
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar_af, (n - 1) & 1, abort_flag, p.dev_status, 16));
-                        if (!ok) break;
-                    }
                     xm[grp * C::BLK + row] = mrow;
                     mbar_arrive(bar_mx + 8 * st);
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 11));
