@@ -442,3 +442,14 @@ def test_attention_with_history_for_a_given_selection(d, b, tpf):
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("topk,wf", [(1, 3), (2, 2), (3, 1)])
+def test_one_kernel_forward_with_few_kept_blocks_and_several_units_per_cta(topk, wf):
+    """The attention kernel with the history term inside, in the corners of its unit bookkeeping: one, two or three
+    kept tiles per query block (the S buffer taken for the phi(Q) operand is then the previous unit's), more
+    (head, query block) units than SMs, so that thread blocks walk several units, and a short last block."""
+    w = gen.Workload("fewkept", batch=2, heads=8, head_dim=128, tokens_per_frame=1300, chunk_frames=1, window_frames=wf,
+                     block=128, topk=topk, keep_permille=0, seed=31)
+    assert w.batch * w.heads * w.blocks_per_chunk > 148
+    stream_compare(w, wf + 2, check_parts=False)
