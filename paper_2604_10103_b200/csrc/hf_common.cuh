@@ -18,7 +18,7 @@ struct ChunkTable {
 };
 
 // Device status word layout (int[4]): [0] flags, [1] detail, [2..3] reserved.
-enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2 };
+enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2, HF_DEV_RANGE_FLAG = 4 };
 
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its predecessor
 // in the stream still runs (once every block of the predecessor has called pdl_trigger or exited); pdl_wait returns when the

@@ -31,6 +31,7 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
+    static constexpr float HEADROOM = 40.f;           // log2 distance of the softmax reference above the first tile's row maximum
     static constexpr int KSTAGES = (D == 128) ? 2 : 3, VSTAGES = 2, SBUFS = 3;   // (a K tile is free again as soon as its S is done)
     // The history term (Eq. 4) can be formed inside this kernel at head_dim 128 with two column groups: the folded
     // state S W^T (bf16 hi and lo halves, one operand tile each) then sits in shared memory beside the K / V rings.
@@ -254,7 +255,9 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
             if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_vf + 8 * rv.stage, rv.phase, abort_flag, p.dev_status, 7)))) break;
             fence_after_sync();
             if (elect_one()) {
-                mma_ts_tile(tO, tmem + rp.stage * C::BLK, v_lo + rv.stage * TILE_STEP, v_hi, IDESC_PV, j_pv > 0);
+                // P of keys 0..63 at the buffer's columns 0..31, of keys 64..127 where the second column group left them
+                mma_ts_tile_split(tO, tmem + rp.stage * C::BLK, tmem + rp.stage * C::BLK + (NG > 1 ? C::GCOLS : 32),
+                                  v_lo + rv.stage * TILE_STEP, v_hi, IDESC_PV, j_pv > 0);
                 mma_commit(bar_pv + 8 * (t & 3));
                 mma_commit(bar_ve + 8 * rv.stage);
             }
@@ -357,50 +360,33 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         for (int e = 0; e < 32; ++e)
                             if (grp * C::GCOLS + c * 32 + e >= nv) r[c][e] = 0xff800000u;   // -inf
                 }
-                float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int c = 0; c < NC; ++c)
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2)         // three-input maximum: two values per instruction
-                        mx[(e >> 1) & 3] = fmax3(mx[(e >> 1) & 3], __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]));
-                float mrow = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                if (NG > 1) {
-                    // every group has read its S columns (the P columns written below overlap another group's S)
-                    // and learns the maximum of the whole row
-                    float* xm = x_max + st * NG * C::BLK;
-                    xm[grp * C::BLK + row] = mrow;
-                    mbar_arrive(bar_mx + 8 * st);
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 8 * st, (t >> 1) & 1, abort_flag, p.dev_status, 11));
-                    if (!ok) break;
-#pragma unroll
-                    for (int g = 0; g < NG; ++g) mrow = fmaxf(mrow, xm[g * C::BLK + row]);
-                    if (j == keep - 1) mbar_arrive(bar_rd);     // the unit's last maxima are out of the buffers
-                }
-                const float m_new = fmaxf(m_used, mrow * p.scale_log2);
-                // ---- lazy rescale: only when some row of the warp moved its maximum by more than 2^8
                 if (j == 0) {
-                    m_used = m_new;
-                } else {
-                    const bool need = (m_new - m_used) > 8.f;
-                    if (__any_sync(0xffffffffu, need)) {
-                        // O is rewritten here, so P.V of the previous tile must have landed
-                        ok = wait_pv_prev(9);
+                    // ---- the reference exponent of the row for the whole unit: the maximum of its first kept tile plus
+                    // HEADROOM.  No running maximum, no rescaling and no exchange between the column groups after this: a
+                    // later tile may exceed the first one by 2^HEADROOM .. 2^(HEADROOM + ~85) before fp32 overflows, which
+                    // the end of the unit detects and reports (row sum not finite or beyond 2^100).  Scale invariance of
+                    // floating point makes the result the same as with the exact running maximum otherwise.
+                    float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int c = 0; c < NC; ++c)
+#pragma unroll
+                        for (int e = 0; e < 32; e += 2)     // three-input maximum: two values per instruction
+                            mx[(e >> 1) & 3] = fmax3(mx[(e >> 1) & 3], __uint_as_float(r[c][e]), __uint_as_float(r[c][e + 1]));
+                    float mrow = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    if (NG > 1) {
+                        float* xm = x_max + (n & 1) * NG * C::BLK;
+                        xm[grp * C::BLK + row] = mrow;
+                        mbar_arrive(bar_mx + 8 * (n & 1));
+                        ok = __all_sync(0xffffffffu, mbar_wait(bar_mx + 8 * (n & 1), (n >> 1) & 1, abort_flag, p.dev_status, 11));
                         if (!ok) break;
-                        fence_after_sync();
-                        const float alpha = need ? fast_exp2(m_used - m_new) : 1.f;
-                        if (need) { m_used = m_new; l_run *= alpha; }
 #pragma unroll
-                        for (int c = 0; c < C::OCOLS / 32; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tO + c * 32, o);
-                            tmem_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                            tmem_st32(tO + c * 32, o);
-                        }
+                        for (int g = 0; g < NG; ++g) mrow = fmaxf(mrow, xm[g * C::BLK + row]);
+                        mbar_arrive(bar_rd);                // this thread is done with the buffer
                     }
+                    m_used = fmaf(mrow, p.scale_log2, C::HEADROOM);
                 }
-                // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the first half of the S buffer
+                // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the thread's own S columns (group g: key columns
+                // 64 g .. 64 g + 63 -> columns 64 g .. 64 g + 31 of the buffer; no group writes where another one reads)
                 // (packed fp32: the scale-and-shift and the row sum handle two columns per instruction)
                 float2 rsum[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                 const float2 scale2 = make_float2(p.scale_log2, p.scale_log2), negm2 = make_float2(-m_used, -m_used);
@@ -420,7 +406,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                         for (int u = 0; u < 4; ++u) pk[(e0 >> 1) + u] = pack_bf16(pe[u].x, pe[u].y);
                     }
-                    tmem_st16(tS + grp * (C::GCOLS / 2) + c * 16, pk);
+                    tmem_st16(tS + grp * C::GCOLS + c * 16, pk);
                 }
                 l_run += ((rsum[0].x + rsum[0].y) + (rsum[1].x + rsum[1].y)) + ((rsum[2].x + rsum[2].y) + (rsum[3].x + rsum[3].y));
                 tmem_wait_st();
@@ -435,8 +421,8 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_rd, n & 1, abort_flag, p.dev_status, 17));
                 if (!ok) break;
             }
-            float* x_l = x_max + ((t - 1) & 1) * NG * C::BLK;     // buffer of the unit's last tile: next written two tiles on
-            float* x_d = x_max + (t & 1) * NG * C::BLK;           // buffer of the next tile: see the wait at a unit's first tile
+            float* x_l = x_max + (n & 1) * NG * C::BLK;           // this unit's buffer: next written two units on
+            float* x_d = x_max + ((n + 1) & 1) * NG * C::BLK;     // the next unit's buffer: see the wait at a unit's start
             if constexpr (fuse) {
                 // ---- history term (Eq. 4): A = (l / den) phi(q) as bf16 hi + lo, this group's 64 features of the row,
                 // read from global memory (the Q tile in shared memory already belongs to the next unit)
@@ -484,6 +470,10 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                 for (int g = 0; g < NG; ++g) { l_run += x_l[g * C::BLK + row]; den += x_d[g * C::BLK + row]; }
                 inv = 1.f / l_run;
+                if (!(l_run < 1e30f)) {     // overflow (or NaN): a later tile rose too far above the first one
+                    atomicOr(p.dev_status, HF_DEV_RANGE_FLAG);
+                    atomicExch(p.dev_status + 1, u);
+                }
                 const float fac = l_run / den;                      // O is divided by l at the end: pre-multiply the history term
                 // the S buffer two tiles on held P of the tile before the unit's last one: its P V must have read it
                 if (t >= 2) {
@@ -528,6 +518,10 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 if (!ok) break;
                 fence_after_sync();
                 inv = 1.f / l_run;
+                if (!(l_run < 1e30f)) {     // overflow (or NaN): a later tile rose too far above the first one
+                    atomicOr(p.dev_status, HF_DEV_RANGE_FLAG);
+                    atomicExch(p.dev_status + 1, u);
+                }
             }
             const bf16* bias_row = (fuse && p.bias) ? p.bias + (size_t)(bh % p.heads) * D : nullptr;
             const size_t g_row = (size_t)bh * p.Tc + q0 + row;

@@ -139,6 +139,20 @@ __device__ __forceinline__ void mma_ts_tile(uint32_t d_tmem, uint32_t a_tmem, ui
                  "}\n" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)accumulate_first) : "memory");
 }
 #undef HF_TS_STEP
+// The same product with the A operand in two pieces: keys 0..63 at a_tmem (32 columns), keys 64..127 at a_tmem_hi.
+#define HF_TS2_STEP(KS, AOP, AOFF, PRED)                                                            \
+    "add.u32 a, " AOP ", " #AOFF " * 8;\n add.u32 b, %2, " #KS " * 128;\n mov.b64 db, {b, %3};\n" \
+    "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], db, %4, " PRED ";\n"
+__device__ __forceinline__ void mma_ts_tile_split(uint32_t d_tmem, uint32_t a_tmem, uint32_t a_tmem_hi, uint32_t b_lo, uint32_t b_hi,
+                                                  uint32_t idesc, bool accumulate_first) {
+    asm volatile("{\n .reg .pred pt, p0;\n .reg .b64 db;\n .reg .b32 a, b;\n"
+                 "setp.eq.u32 pt, %0, %0;\n setp.ne.b32 p0, %5, 0;\n"
+                 HF_TS2_STEP(0, "%1", 0, "p0") HF_TS2_STEP(1, "%1", 1, "pt") HF_TS2_STEP(2, "%1", 2, "pt") HF_TS2_STEP(3, "%1", 3, "pt")
+                 HF_TS2_STEP(4, "%6", 0, "pt") HF_TS2_STEP(5, "%6", 1, "pt") HF_TS2_STEP(6, "%6", 2, "pt") HF_TS2_STEP(7, "%6", 3, "pt")
+                 "}\n" ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"((uint32_t)accumulate_first), "r"(a_tmem_hi)
+                 : "memory");
+}
+#undef HF_TS2_STEP
 // 32 lanes x 32 consecutive 32-bit columns: thread t of the warp gets lane (base lane + t)
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
