@@ -203,8 +203,12 @@ hf_status hf_query(hf_ctx* ctx, int layer, int what, int64_t* value);
 
 /* Synchronises the device and reports the device status word.  Flag 1: a bounded wait inside a kernel ran out
  * (detail = where), HF_ERR_DEVICE_TIMEOUT.  Flag 2: a caller's index list held a block index outside [0, T_n)
- * (detail = batch*head and query block of the row, as one number), HF_ERR_INVALID_ARG.  Either way the result of that
- * launch is invalid, the word is cleared and the context stays usable. */
+ * (detail = batch*head and query block of the row, as one number), HF_ERR_INVALID_ARG.  Flag 4: the tcgen05 attention
+ * kernel (HF_SWA_TCGEN05) fixes a query row's softmax reference at the row maximum of its first kept key block times
+ * 2^60 and keeps no running maximum; a row whose later blocks rise more than about 100 natural-log units above the first
+ * one would overflow fp32 and is reported instead (detail = the query block), HF_ERR_UNSUPPORTED: HF_SWA_TCGEN05_PINGPONG
+ * and HF_SWA_MMA keep a running maximum and take any input.  In every case the result of that launch is invalid, the
+ * word is cleared and the context stays usable. */
 hf_status hf_get_device_status(hf_ctx* ctx, int* flags, int* detail);
 
 /* Number of kernels the library has launched since the context was created. */

@@ -939,7 +939,7 @@ hf_status hf_get_device_status(hf_ctx* c, int* flags, int* detail) {
         if (h[0] & HF_DEV_TIMEOUT_FLAG)
             return fail(HF_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (flags %d, detail %d)", h[0], h[1]);
         if (h[0] & HF_DEV_RANGE_FLAG)
-            return fail(HF_ERR_UNSUPPORTED, "attention logits of a query row rose by more than ~85 (natural log units) above those of "
+            return fail(HF_ERR_UNSUPPORTED, "attention logits of a query row rose by more than ~100 (natural log units) above those of "
                         "its first kept block (unit %d): beyond the fixed-reference softmax of the tcgen05 kernel; "
                         "HF_SWA_TCGEN05_PINGPONG and HF_SWA_MMA keep a running maximum", h[1]);
         return fail(HF_ERR_INVALID_ARG, "an index list held a block index outside [0, T_n) (unit %d); block 0 was read in its place",

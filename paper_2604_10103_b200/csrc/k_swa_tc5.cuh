@@ -31,7 +31,7 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
-    static constexpr float HEADROOM = 40.f;           // log2 distance of the softmax reference above the first tile's row maximum
+    static constexpr float HEADROOM = 60.f;           // log2 distance of the softmax reference above the first tile's row maximum
     static constexpr int KSTAGES = (D == 128) ? 2 : 3, VSTAGES = 2, SBUFS = 3;   // (a K tile is free again as soon as its S is done)
     // The history term (Eq. 4) can be formed inside this kernel at head_dim 128 with two column groups: the folded
     // state S W^T (bf16 hi and lo halves, one operand tile each) then sits in shared memory beside the K / V rings.
@@ -362,10 +362,12 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 }
                 if (j == 0) {
                     // ---- the reference exponent of the row for the whole unit: the maximum of its first kept tile plus
-                    // HEADROOM.  No running maximum, no rescaling and no exchange between the column groups after this: a
-                    // later tile may exceed the first one by 2^HEADROOM .. 2^(HEADROOM + ~85) before fp32 overflows, which
-                    // the end of the unit detects and reports (row sum not finite or beyond 2^100).  Scale invariance of
-                    // floating point makes the result the same as with the exact running maximum otherwise.
+                    // HEADROOM (2^60).  No running maximum, no rescaling and no exchange between the column groups after
+                    // this.  P of the first tile is <= 2^-60; a later tile may rise above the first one by a factor of up to
+                    // ~2^150 (about 100 natural-log units) before the row sum passes 2^100, which the end of the unit
+                    // detects and reports (fp32 overflows at 2^128; rows that fall below the first tile lose nothing: what
+                    // flushes to zero is 2^-66 of the largest term).  Floating point is scale invariant, so the result is
+                    // the one the exact running maximum gives.
                     float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int c = 0; c < NC; ++c)
