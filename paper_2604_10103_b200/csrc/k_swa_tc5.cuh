@@ -31,6 +31,10 @@ struct SwaTc5 {
     static constexpr int SUB = D / 64;                 // 64-column (128-byte) sub-tiles per operand tile
     static constexpr int SUB_BYTES = BLK * 128;        // 16 KB
     static constexpr int TILE_BYTES = SUB * SUB_BYTES;
+#ifndef HF_TC5_SKEW_CLK
+#define HF_TC5_SKEW_CLK 500
+#endif
+    static constexpr long long SKEW_CLK = HF_TC5_SKEW_CLK;   // offset between the column groups, in clocks (see the softmax warps)
     static constexpr float HEADROOM = 60.f;           // log2 distance of the softmax reference above the first tile's row maximum
     static constexpr int KSTAGES = (D == 128) ? 2 : 3, VSTAGES = 2, SBUFS = 3;   // (a K tile is free again as soon as its S is done)
     // The history term (Eq. 4) can be formed inside this kernel at head_dim 128 with two column groups: the folded
@@ -386,6 +390,15 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                         mbar_arrive(bar_rd);                // this thread is done with the buffer
                     }
                     m_used = fmaf(mrow, p.scale_log2, C::HEADROOM);
+                    if (NG > 1 && grp > 0) {
+                        // The exchange above has put the column groups in step.  The two warps that share a scheduler
+                        // (same rows, different column groups) then run their exponentials at the same time and their
+                        // waits at the same time, and the special-function unit idles through the latter; set back by part
+                        // of a tile, one group's waits fall into the other's exponentials.  Nothing couples the groups
+                        // until the end of the unit, so the offset stays.
+                        const long long t_skew = clock64();
+                        while (clock64() - t_skew < C::SKEW_CLK * grp) {}
+                    }
                 }
                 // ---- P = exp2(S*c - m), row sum, bf16 pairs written over the thread's own S columns (group g: key columns
                 // 64 g .. 64 g + 63 -> columns 64 g .. 64 g + 31 of the buffer; no group writes where another one reads)
