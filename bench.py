@@ -33,7 +33,7 @@ METRIC = "hybrid-attn latent frames/s at 832x480 shape"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention kernel (history term inside) at this
 # workload's layer shape, from the ncu capture summarised in profiles/k_swa_tc5_layer_832x480.md; None when the kernel
 # has changed since that capture.
-SWA_DRAM_BYTES_PER_LAUNCH = 109.3e6
+SWA_DRAM_BYTES_PER_LAUNCH = 108.6e6
 UNIT = "latent frames/s"
 
 
