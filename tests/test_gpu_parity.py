@@ -485,3 +485,34 @@ def test_logit_range_beyond_the_fixed_softmax_reference_is_reported_and_the_othe
                 assert gpu.ctx.hf_get_device_status() == (0, 0)
         finally:
             gpu.close()
+
+
+def test_lse_output_of_the_tcgen05_kernel():
+    """Natural-log sum of exponentials per query row from the fixed-reference kernel (reference exponent + log2 of the
+    row sum, which is of the order 2^-60 there)."""
+    w = gen.Workload("lse128", batch=1, heads=2, head_dim=128, tokens_per_frame=200, chunk_frames=1, window_frames=2,
+                     block=128, topk=2, keep_permille=0, seed=43)
+    gpu = hz.GpuStream(w)
+    try:
+        kc, vc = gen.clean_kv(w, 0, 0)
+        gpu.append(gpu.up(kc), gpu.up(vc))
+        qb, kb, vb = gen.qkv(w, 0, 1, 0)
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        m, idx, _ = gpu.select(q, k)
+        o, lse = gpu.swa(q, k, v, want_lse=True)
+        qf = f64(qb); keys = np.concatenate([f64(kc), f64(kb)], axis=2)       # logical order: cached chunk, current chunk
+        nb = w.blocks_per_chunk
+        for h in range(2):
+            for i in range(nb):
+                cols = []
+                for j in idx[0, h, i]:
+                    c, jb = divmod(int(j), nb)
+                    lo = c * w.chunk_tokens + jb * 128
+                    cols.append(np.arange(lo, min(lo + 128, (c + 1) * w.chunk_tokens)))
+                cols = np.concatenate(cols)
+                rows = slice(i * 128, min((i + 1) * 128, w.chunk_tokens))
+                s = qf[0, h, rows] @ keys[0, h, cols].T / np.sqrt(128.0)
+                ref = np.log(np.exp(s - s.max(axis=1, keepdims=True)).sum(axis=1)) + s.max(axis=1)
+                assert np.abs(lse[0, h, rows] - ref).max() < 2e-3
+    finally:
+        gpu.close()
