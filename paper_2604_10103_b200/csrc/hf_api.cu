@@ -47,7 +47,7 @@ struct LayerState {
     uint32_t* mask = nullptr;    // last selection [B*H, T_m, mask_words]
     int32_t* idx = nullptr;      // [B*H, T_m, keep]
     int n_cached = 0, head = 0;  // head = slot of the oldest cached chunk
-    int n_sink = 0;              // sink chunks held (slots P, P + 1, ...)
+    int n_sink = 0;              // sink chunks held (slots R, R + 1, ...)
     long long absorbed = 0;
     unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
     int sel_keep = 0;
@@ -60,8 +60,8 @@ struct LayerState {
 struct hf_ctx {
     hf_config cfg;
     int device = 0, sm_count = 0;
-    int BH = 0, Tc = 0, n_b = 0, P = 0, Tm = 0, max_Tn = 0, mask_words = 0, d = 0;
-    int n_sink_max = 0;              // sink chunks of the configuration; ring and sink share one allocation of P + n_sink_max slots
+    int BH = 0, Tc = 0, n_b = 0, P = 0, R = 0, Tm = 0, max_Tn = 0, mask_words = 0, d = 0;
+    int n_sink_max = 0;              // sink chunks of the configuration; ring (R = P + 1 slots: the window's P past chunks and a spare) and sink share one allocation
     size_t chunk_elems = 0, pooled_elems = 0;
     std::vector<LayerState> layers;
     float* pooled_q = nullptr;
@@ -232,11 +232,11 @@ hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
     return post_launch(c, "k_reduce_fold");
 }
 
-// fold_on_side: the reduce/fold kernel goes to the context's side stream (the caller has more work for `st` that only
-// needs the partials kernel to be done, and joins with ev_join afterwards).
+// on_side: both kernels go to the context's side stream, ordered after what `st` holds so far (the caller has
+// independent work for `st` and joins with ev_join afterwards).
 template <int D>
 hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st,
-                        bool fold_on_side = false) {
+                        bool on_side = false) {
     typedef AbsorbTc5<D> A;
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
@@ -246,15 +246,18 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     AbsorbTc5Params p;
     p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
     p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc;
-    PdlLaunch pl(dim3(nsplit, c->BH), dim3(A::THREADS), A::SMEM_BYTES, st, true);
+    cudaStream_t run = st;
+    if (on_side) {
+        HF_CUDA(cudaEventRecord(c->ev_fork, st));
+        HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        run = c->side;
+    }
+    PdlLaunch pl(dim3(nsplit, c->BH), dim3(A::THREADS), A::SMEM_BYTES, run, !on_side);   // (an event wait sits before it on the side stream)
     if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, true>, tk, tv, p));
     else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, false>, tk, tv, p));
     HF_TRY(post_launch(c, "k_absorb_tc5"));
-    if (!fold_on_side) return launch_fold<D>(c, L, nsplit, st);
-    HF_CUDA(cudaEventRecord(c->ev_fork, st));
-    HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
-    HF_TRY(launch_fold<D>(c, L, nsplit, c->side));
-    HF_CUDA(cudaEventRecord(c->ev_join, c->side));
+    HF_TRY(launch_fold<D>(c, L, nsplit, run));
+    if (on_side) HF_CUDA(cudaEventRecord(c->ev_join, c->side));
     return HF_OK;
 }
 
@@ -279,7 +282,7 @@ ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v
     memset(&t, 0, sizeof(t));
     const int n_old = L.n_sink + L.n_cached;
     for (int i = 0; i < n_old; ++i) {       // sink chunks first, then the cached chunks oldest first
-        const int slot = i < L.n_sink ? c->P + i : (L.head + i - L.n_sink) % c->P;
+        const int slot = i < L.n_sink ? c->R + i : (L.head + i - L.n_sink) % c->R;
         t.k[i] = L.ring_k + (size_t)slot * c->chunk_elems;
         t.v[i] = L.ring_v + (size_t)slot * c->chunk_elems;
         t.pooled[i] = L.pooled_k + (size_t)slot * c->pooled_elems;
@@ -341,13 +344,13 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     HF_TRY(make_map_ex(c, &to, o, c->Tc, 1, 64, 32, true));      // output: one warp's 32 rows x 64 columns per store
     Tc5Params p;
     p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.n_sink = L.n_sink;
-    p.P = c->P;
+    p.P = c->R;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
     p.heads = c->cfg.heads; p.eps = c->cfg.eps;
     p.q = q; p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr;
-    const CUtensorMap& rk = c->P + c->n_sink_max > 0 ? L.tm_kring : tk;
-    const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
+    const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, overlap_prev);
@@ -376,11 +379,11 @@ hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16*
     HF_TRY(make_map(c, &tv, v_cur, 1));
     Tc5Params p;
     p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.n_sink = L.n_sink;
-    p.P = c->P;
+    p.P = c->R;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
-    const CUtensorMap& rk = c->P + c->n_sink_max > 0 ? L.tm_kring : tk;
-    const CUtensorMap& rv = c->P + c->n_sink_max > 0 ? L.tm_vring : tv;
+    const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     k_swa_tc5p<D, HF_TC5P_COLGROUPS><<<grid, C::THREADS, C::SMEM_BYTES, st>>>(tq, rk, rv, tk, tv, p);
@@ -461,6 +464,7 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->n_b = (c->Tc + cfg->block - 1) / cfg->block;
     c->Tm = c->n_b;
     c->P = cfg->window_frames / cfg->chunk_frames - 1;
+    c->R = c->P > 0 ? c->P + 1 : 0;
     c->n_sink_max = cfg->sink_frames / cfg->chunk_frames;
     c->max_Tn = (c->P + c->n_sink_max + 1) * c->n_b;
     c->mask_words = (c->max_Tn + 31) / 32;
@@ -486,7 +490,7 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->layers.resize(cfg->layers);
     const size_t dd = (size_t)c->BH * c->d * c->d, dz = (size_t)c->BH * c->d;
     for (auto& L : c->layers) {
-        const size_t slots = (size_t)c->P + c->n_sink_max;      // ring slots, then sink slots
+        const size_t slots = (size_t)c->R + c->n_sink_max;      // ring slots, then sink slots
         if (s == HF_OK) s = dmalloc(&L.ring_k, slots * c->chunk_elems);
         if (s == HF_OK) s = dmalloc(&L.ring_v, slots * c->chunk_elems);
         if (s == HF_OK) s = dmalloc(&L.pooled_k, slots * c->pooled_elems);
@@ -619,7 +623,7 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
     if (L.n_sink < c->n_sink_max) {   // the stream's first chunks are the attention sink: kept in slots of their own for good
-        const int slot = c->P + L.n_sink;
+        const int slot = c->R + L.n_sink;
         PoolJobs jobs;
         memset(&jobs, 0, sizeof(jobs));
         jobs.job[0].src = (const bf16*)k; jobs.job[0].copy_dst = L.ring_k + (size_t)slot * c->chunk_elems;
@@ -636,19 +640,20 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
         L.cache_epoch++;
         return HF_OK;
     }
-    int slot;
+    // The ring has one slot more than the window holds, so the new chunk never lands on the chunk that leaves: the state
+    // update (Eq. 3) of the evicted chunk runs on the side stream beside the copy of the new one (the copy kernel's thread
+    // blocks fit on the SMs next to the absorb kernel's), and the call joins the two before it returns to the caller's
+    // stream.  The state is still updated before anything can overwrite the evicted chunk: the slot it sits in is the
+    // target of the NEXT commit, which is ordered after this call's join.
+    const int slot = (L.head + L.n_cached) % c->R;
     bool evicted = false;
-    if (L.n_cached == c->P) {   // cache full: the state is updated before the evicted chunk's slot is reused
-        slot = L.head;
-        // the slot may be overwritten as soon as the partials kernel has read it; adding the partials to the state and
-        // folding it runs beside the copy, on the side stream
-        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)slot * c->chunk_elems,
-                             L.ring_v + (size_t)slot * c->chunk_elems, c->Tc, st, true));
+    if (L.n_cached == c->P) {
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)L.head * c->chunk_elems,
+                             L.ring_v + (size_t)L.head * c->chunk_elems, c->Tc, st, true));
         evicted = true;
         L.absorbed += c->Tc;
-        L.head = (L.head + 1) % c->P;
+        L.head = (L.head + 1) % c->R;
     } else {
-        slot = (L.head + L.n_cached) % c->P;
         L.n_cached++;
     }
     PoolJobs jobs;
@@ -816,7 +821,7 @@ ImageHeader image_header(const hf_ctx* c) {
     return h;
 }
 int held_slot(const hf_ctx* c, const LayerState& L, int i) {   // slot of the i-th held chunk in logical order
-    return i < L.n_sink ? c->P + i : (L.head + i - L.n_sink) % c->P;
+    return i < L.n_sink ? c->R + i : (L.head + i - L.n_sink) % c->R;
 }
 }  // namespace
 
