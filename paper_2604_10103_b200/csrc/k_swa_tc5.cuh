@@ -1,21 +1,29 @@
 // Block-sparse sliding-window attention (Eq. 6; Alg. 3 inner loops) on the Blackwell tensor path:
-// TMA loads addressed by the kept-block index list, tcgen05.mma with S / P / O in tensor memory,
-// fp32 online softmax with lazy rescaling.  Block size 128, head dim 64 or 128.
+// TMA loads addressed by the kept-block index list, tcgen05.mma with S / P / O in tensor memory, fp32 softmax
+// against a reference exponent fixed per query block.  Block size 128, head dim 64 or 128.  The HIST instantiation
+// (head dim 128) also forms the history term of Eq. 4 and adds it (Eq. 7) before the one rounding to bf16.
 //
 // Persistent kernel, one CTA per SM; a CTA walks its (batch*head, query block) units and their kept key
 // blocks as one stream of tiles t = 0, 1, ...
 //   softmax warps   NG column groups of four warps; thread (group g, row r) owns columns [g*128/NG, (g+1)*128/NG)
-//                   of S row r (TMEM lane = row) and the same share of the O columns.  The groups exchange their
-//                   partial row maxima through shared memory once per tile, so every group uses the same running
-//                   maximum; the row sums stay partial until the epilogue.
-//   loader warp K   TMA: Q (one buffer, reloaded per unit) and K tiles (ring of three)
+//                   of S row r (TMEM lane = row) and the same share of the O columns.  At a unit's first tile the
+//                   groups exchange their row maxima through shared memory; that maximum times 2^HEADROOM is the
+//                   reference exponent m of the row for the whole unit (softmax does not depend on m; what m must do is
+//                   keep exp2(S c - m) inside fp32, which the end of the unit checks).  After that tile the groups do not
+//                   meet until the unit ends: no running maximum, no rescaling of O, row sums partial until then.
+//   loader warp K   TMA: Q (one buffer, reloaded per unit), K tiles (ring of two at head dim 128, three at 64); HIST:
+//                   per unit the lo tile of the head's folded state and a second copy of the Q tile
 //   loader warp V   TMA: V tiles (ring of two)
 //   MMA warp        TMEM allocation and tcgen05.mma issue.  S lives in three TMEM buffers and is issued two tiles
 //                   ahead of the softmax (S_{t+2} before P_t V_t), so that neither the TMA latency of K nor the
 //                   MMA issue chain sits on the softmax critical path.
 //   S = Q K_t^T        A = Q (smem, K-major, 128B swizzle), B = K_t (smem, K-major)     -> TMEM cols 128*(t%3)
-//   P = exp2(S*c - m)  bf16, written over the first 64 columns of its S buffer
-//   O += P V_t         A = P (TMEM), B = V_t (smem, MN-major, 128B swizzle)              -> TMEM cols [384, 384+D)
+//   P = exp2(S*c - m)  bf16, written over the writing thread's own S columns (group g: columns 64 g .. 64 g + 31)
+//   O += P V_t         A = P (TMEM, two pieces), B = V_t (smem, MN-major, 128B swizzle)  -> TMEM cols [384, 384+D)
+//   HIST, unit end     A = (l / den) phi(Q) as bf16 hi + lo in the free S buffer (phi(Q) from the shared-memory copy of
+//                      Q, den = phi(q).z + eps exchanged between the groups with the row sums l);
+//                      O += A_hi S'_lo + A_hi S'_hi + A_lo S'_hi, S' = the folded state S W^T (hi tile loaded over the
+//                      Q copy once it has been read); then O / l (+ bias) -> bf16 -> shared memory -> bulk tensor store
 // Every wait is bounded (~1 s); on expiry the CTA raises the device status word and leaves through the
 // common exit (drains its copies, frees its TMEM).
 #pragma once
