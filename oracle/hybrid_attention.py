@@ -272,6 +272,18 @@ def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6, cos_q=None, si
     return h
 
 
+def merge_full_width(h: np.ndarray, W_full, bias_full=None) -> np.ndarray:
+    """Eq. 4's "Linear" read as ONE projection over the model width (the paper gives no shape; the per-head reading is the
+    default): h [H, T, d] of one batch element, per token x = concat_h h[h, t, :] (head-major), y = W_full x + bias_full,
+    W_full [H d, H d] (row = output feature), split back into heads.  Returns [H, T, d]."""
+    H, T, d = h.shape
+    x = np.transpose(np.asarray(h, np.float64), (1, 0, 2)).reshape(T, H * d)
+    y = x @ np.asarray(W_full, np.float64).T
+    if bias_full is not None:
+        y = y + np.asarray(bias_full, np.float64)[None, :]
+    return np.transpose(y.reshape(T, H, d), (1, 0, 2))
+
+
 # --------------------------------------------------------------------------- Alg. 2 + Alg. 3
 class HybridStream:
     """Streaming state of one layer (all batches and heads) and the per-chunk forward.
@@ -285,12 +297,17 @@ class HybridStream:
     """
 
     def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
-                 W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0, rope_q=None, rope_k=None):
+                 W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0, rope_q=None, rope_k=None,
+                 W_full=None, bias_full=None):
         self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
         self.z_frame_tokens = z_frame_tokens     # None: z is the plain sum of phi(K); n: per-frame means of n tokens (Eq. 3 literal)
         self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
         self.W = None if W is None else np.asarray(W, np.float64)        # [H, d, d]
         self.bias = None if bias is None else np.asarray(bias, np.float64)  # [H, d]
+        # the full-width reading of "Linear" (one [H d, H d] matrix over all heads) replaces the per-head one
+        self.W_full = None if W_full is None else np.asarray(W_full, np.float64)
+        self.bias_full = None if bias_full is None else np.asarray(bias_full, np.float64)
+        assert self.W_full is None or self.W is None
         self.rope_q, self.rope_k = rope_q, rope_k    # (cos, sin) tables [T_c, d/2] of the linear branch, or None
         self.sink_chunks = sink_chunks   # the first chunks of the stream stay visible for ever ("sink"): never evicted, never absorbed
         self.sink = []                                                   # list of (k, v) like self.past, oldest first
@@ -366,6 +383,8 @@ class HybridStream:
                                                None if self.bias is None else self.bias[h], self.eps,
                                                None if self.rope_q is None else self.rope_q[0],
                                                None if self.rope_q is None else self.rope_q[1])
+            if self.W_full is not None:     # o_hist holds h = num / den so far (W, bias are None): project over all heads
+                o_hist[bi] = merge_full_width(o_hist[bi], self.W_full, self.bias_full)
         if parts:
             return o_loc + o_hist, o_loc, o_hist
         return o_loc + o_hist

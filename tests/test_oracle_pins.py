@@ -495,3 +495,37 @@ def test_relative_temporal_indices_eq8():
     assert oa.relative_temporal_indices(3, 21) == [1, 2, 3]
     assert oa.relative_temporal_indices(21, 21) == [19, 20, 21]
     assert oa.relative_temporal_indices(22, 21) == [19, 20, 21] and oa.relative_temporal_indices(600, 21) == [19, 20, 21]
+
+
+def test_full_width_merge_reduces_to_the_per_head_merge_and_to_scalar_loops():
+    """The one-matrix reading of Eq. 4's Linear: with a block-diagonal matrix it is the per-head projection (pinned
+    above); in general it is the plain double loop over output and input features of the concatenated heads."""
+    rng = np.random.default_rng(11)
+    H, T, d = 3, 5, 4
+    h = rng.standard_normal((H, T, d))
+    Wh = rng.standard_normal((H, d, d)); bh = rng.standard_normal((H, d))
+    W_full = np.zeros((H * d, H * d))
+    for i in range(H):
+        W_full[i * d:(i + 1) * d, i * d:(i + 1) * d] = Wh[i]
+    y = oa.merge_full_width(h, W_full, bh.reshape(-1))
+    for i in range(H):
+        assert np.allclose(y[i], h[i] @ Wh[i].T + bh[i][None, :], atol=1e-12)
+    W_full = rng.standard_normal((H * d, H * d)); b_full = rng.standard_normal(H * d)
+    y = oa.merge_full_width(h, W_full, b_full)
+    for t in range(T):
+        for ho in range(H):
+            for c in range(d):
+                acc = b_full[ho * d + c]
+                for hi in range(H):
+                    for a in range(d):
+                        acc += W_full[ho * d + c, hi * d + a] * h[hi, t, a]
+                assert abs(y[ho, t, c] - acc) < 1e-12
+    # and inside the stream: identity matrix = no projection at all
+    dd = 32                                     # (the canonical scorer wants a multiple of 32)
+    st_a = oa.HybridStream(1, H, dd, 2, 1, topk=1)
+    st_b = oa.HybridStream(1, H, dd, 2, 1, topk=1, W_full=np.eye(H * dd))
+    for c in range(3):
+        k = rng.standard_normal((1, H, 4, dd)); v = rng.standard_normal((1, H, 4, dd))
+        st_a.append(k, v); st_b.append(k, v)
+    q = rng.standard_normal((1, H, 4, dd)); k = rng.standard_normal((1, H, 4, dd)); v = rng.standard_normal((1, H, 4, dd))
+    assert np.allclose(st_a.forward(q, k, v), st_b.forward(q, k, v), atol=1e-12)
