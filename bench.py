@@ -286,6 +286,23 @@ def run_ours(args, w):
         contrast["note"] = ("one layer call, 4680 queries; dense = all key blocks kept (111 at window 9, 259 at window 21); the "
                             "paper reports 21.8 -> 29.5 whole-model FPS for dense window 9 -> hybrid and 15.4 for dense window 21")
 
+    # ---- the one-matrix reading of the history branch's Linear: read-out + projection over all heads + attention
+    if rank == 0:
+        wf = w.with_(layers=1)
+        cf = hf.Context(hf.make_config(wf, merge=hf.HF_MERGE_FULL_WIDTH), device=local)
+        Wfb, bfb = gen.merge_weights_full(wf, 0)
+        cf.hf_set_merge_weights(0, hf.bits_to_cuda(Wfb), hf.bits_to_cuda(bfb))
+        for c_ in range(wf.past_chunks + 1):
+            cf.hf_kv_append(0, kc[c_ % L], vc[c_ % L])
+        t_lin = timed(lambda r: cf.hf_linear_attn(0, q[r % L], o), 16)
+        t_fwd = timed(lambda r: cf.hf_hybrid_forward(0, q[r % L], k[r % L], v[r % L], o), 16)
+        hd = wf.heads * wf.head_dim
+        contrast["full_width_merge"] = {"linear_us": t_lin, "forward_us": t_fwd,
+                                        "projection_gflop": 2.0 * wf.batch * wf.chunk_tokens * hd * hd / 1e9,
+                                        "note": "history branch with one [H d, H d] projection over all heads: read-out kernel + projection kernel"
+                                                " (bf16 hi/lo operand, tcgen05), then the attention kernel adds the term"}
+        cf.close()
+
     # ---- end to end through the host-buffer entry points (H2D of q,k,v and D2H of o inside the timed region)
     e2e = None
     e2e_steps = max(1, min(args.steps, 2))

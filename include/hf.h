@@ -40,7 +40,7 @@ typedef enum {
 } hf_status;
 
 enum { HF_PHI_ELU1 = 0 };                                /* phi(x) = elu(x) + 1                 */
-enum { HF_MERGE_IDENTITY = 0, HF_MERGE_PER_HEAD = 1 };   /* "Linear" of Eq. 4: none | W[H,d,d]  */
+enum { HF_MERGE_IDENTITY = 0, HF_MERGE_PER_HEAD = 1, HF_MERGE_FULL_WIDTH = 2 };   /* "Linear" of Eq. 4: none | W[H,d,d] | W[H d, H d] */
 enum { HF_SWA_AUTO = 0, HF_SWA_MMA = 1, HF_SWA_TCGEN05 = 2, HF_SWA_TCGEN05_PINGPONG = 3 }; /* sparse-attention kernel choice */
 enum { HF_Z_SUM = 0, HF_Z_FRAME_MEAN = 1 };              /* z of Eq. 3: sum of phi(K) rows | per-frame means */
 
@@ -56,7 +56,7 @@ typedef struct {
     int layers;                      /* independent layer states held by the context                    */
     int phi;                         /* HF_PHI_ELU1                                                     */
     float eps;                       /* added to the denominator phi(q).z of Eq. 4                      */
-    int merge;                       /* HF_MERGE_IDENTITY | HF_MERGE_PER_HEAD                           */
+    int merge;                       /* HF_MERGE_IDENTITY | HF_MERGE_PER_HEAD | HF_MERGE_FULL_WIDTH     */
     int swa_kernel;                  /* HF_SWA_AUTO | HF_SWA_MMA | HF_SWA_TCGEN05 | HF_SWA_TCGEN05_PINGPONG */
     int z_mode;                      /* HF_Z_SUM: z += sum_t phi(K_ev[t]) (default).  HF_Z_FRAME_MEAN: Eq. 3 as printed,
                                         z += sum over evicted latent frames of the mean of phi(K) over the frame's
@@ -87,9 +87,14 @@ hf_status hf_destroy(hf_ctx* ctx);
 /* Empty the rolling cache and zero (S, z) of one layer (layer = -1: all layers). */
 hf_status hf_reset(hf_ctx* ctx, int layer, void* stream);
 
-/* Merge projection of the history branch ("Linear" in Eq. 4; the paper does not give its shape: here one
- * d x d matrix per head, y = W h + bias).  W: bf16 [H, d, d] row-major (row = output dim), bias: bf16 [H, d]
- * or NULL.  Copied into the context.  HF_ERR_STATE if the context was created with HF_MERGE_IDENTITY. */
+/* Merge projection of the history branch ("Linear" in Eq. 4; the paper does not give its shape).
+ *   HF_MERGE_PER_HEAD (default reading): one d x d matrix per head, y = W_h h + bias_h.  W: bf16 [H, d, d] row-major
+ *     (row = output dim), bias: bf16 [H, d] or NULL.  The matrix is folded into the state (S W_h^T), so it costs nothing
+ *     per call.
+ *   HF_MERGE_FULL_WIDTH: one matrix over the model width, y = W x + bias with x = the read-outs of all heads side by
+ *     side (head-major).  W: bf16 [H d, H d] row-major (row = output feature), bias: bf16 [H d] or NULL.  It couples the
+ *     heads: the read-out kernel is followed by a projection kernel, and the attention kernel adds the result.
+ * Copied into the context.  HF_ERR_STATE if the context was created with HF_MERGE_IDENTITY. */
 hf_status hf_set_merge_weights(hf_ctx* ctx, int layer, const void* W, const void* bias, void* stream);
 
 /* Rotation inside the linear branch (Eq. 3: RoPE(phi(K))^T V in the state; Eq. 4: RoPE(phi(Q)) in the numerator only, the

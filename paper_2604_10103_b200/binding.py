@@ -16,7 +16,7 @@ HF_OK = 0
 STATUS_NAMES = ["HF_OK", "HF_ERR_INVALID_ARG", "HF_ERR_SHAPE", "HF_ERR_STATE", "HF_ERR_UNSUPPORTED",
                 "HF_ERR_NOMEM", "HF_ERR_CUDA", "HF_ERR_DEVICE_TIMEOUT"]
 HF_PHI_ELU1 = 0
-HF_MERGE_IDENTITY, HF_MERGE_PER_HEAD = 0, 1
+HF_MERGE_IDENTITY, HF_MERGE_PER_HEAD, HF_MERGE_FULL_WIDTH = 0, 1, 2
 HF_SWA_AUTO, HF_SWA_MMA, HF_SWA_TCGEN05, HF_SWA_TCGEN05_PINGPONG = 0, 1, 2, 3
 HF_Z_SUM, HF_Z_FRAME_MEAN = 0, 1
 (HF_Q_CACHED_CHUNKS, HF_Q_KEY_BLOCKS, HF_Q_KEPT_BLOCKS, HF_Q_ABSORBED_TOKENS, HF_Q_QUERY_BLOCKS,

@@ -7,6 +7,7 @@
 #include "k_swa_tc5p.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
+#include "k_merge_full.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -44,6 +45,9 @@ struct LayerState {
     bf16* W = nullptr;           // [H, d, d]
     bf16* bias = nullptr;        // [H, d]
     bool has_w = false, has_bias = false;
+    bf16* W_full = nullptr;      // [H d, H d]: the one-matrix reading of Eq. 4's Linear (HF_MERGE_FULL_WIDTH); bias then [H d]
+    bool has_wfull = false;
+    CUtensorMap tm_wfull;        // [H d (in, contiguous), H d (out)], box = 64 columns x d rows
     uint32_t* mask = nullptr;    // last selection [B*H, T_m, mask_words]
     int32_t* idx = nullptr;      // [B*H, T_m, keep]
     int n_cached = 0, head = 0;  // head = slot of the oldest cached chunk
@@ -67,6 +71,8 @@ struct hf_ctx {
     float* pooled_q = nullptr;
     float* pooled_kcur = nullptr;
     float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
+    bf16* x_hi = nullptr;            // full-width merge: the read-out h of all heads as bf16 hi + lo, [B*H, T_c, d] each
+    bf16* x_lo = nullptr;
     float* partials = nullptr;       // absorb split partials
     int nsplit_max = 1;
     float z_scale = 1.f;             // 1 (z = sum of phi(K)) or 1 / tokens_per_frame (per-frame means)
@@ -116,7 +122,8 @@ hf_status validate(const hf_config& g) {
     if (g.topk < 0 || (g.topk == 0 && (g.keep_permille < 1 || g.keep_permille > 1000)))
         return fail(HF_ERR_SHAPE, "need topk > 0 or keep_permille in [1, 1000]");
     if (g.phi != HF_PHI_ELU1) return fail(HF_ERR_UNSUPPORTED, "phi %d unsupported", g.phi);
-    if (g.merge != HF_MERGE_IDENTITY && g.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_UNSUPPORTED, "merge %d unsupported", g.merge);
+    if (g.merge != HF_MERGE_IDENTITY && g.merge != HF_MERGE_PER_HEAD && g.merge != HF_MERGE_FULL_WIDTH)
+        return fail(HF_ERR_UNSUPPORTED, "merge %d unsupported", g.merge);
     if (!(g.eps >= 0.f)) return fail(HF_ERR_SHAPE, "eps must be >= 0");
     if (g.swa_kernel < HF_SWA_AUTO || g.swa_kernel > HF_SWA_TCGEN05_PINGPONG) return fail(HF_ERR_UNSUPPORTED, "swa_kernel %d unknown", g.swa_kernel);
     if (g.z_mode != HF_Z_SUM && g.z_mode != HF_Z_FRAME_MEAN) return fail(HF_ERR_UNSUPPORTED, "z_mode %d unknown", g.z_mode);
@@ -146,9 +153,9 @@ hf_status dmalloc(T** p, size_t count) {
 void free_all(hf_ctx* c) {
     for (auto& L : c->layers) {
         cudaFree(L.ring_k); cudaFree(L.ring_v); cudaFree(L.pooled_k); cudaFree(L.S); cudaFree(L.z);
-        cudaFree(L.sf_hi); cudaFree(L.sf_lo); cudaFree(L.W); cudaFree(L.bias); cudaFree(L.mask); cudaFree(L.idx);
+        cudaFree(L.sf_hi); cudaFree(L.sf_lo); cudaFree(L.W); cudaFree(L.W_full); cudaFree(L.bias); cudaFree(L.mask); cudaFree(L.idx);
     }
-    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials);
+    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -266,17 +273,33 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
 template <int D>
 hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16, float* out_f32, cudaStream_t st) {
     typedef ReadoutTc5<D> R;
+    // Full-width reading of Eq. 4's Linear: the read-out leaves h = phi(q) S / (phi(q).z + eps) of every head as bf16 hi + lo
+    // halves, and a second kernel applies the [H d, H d] matrix and the bias across the heads.
+    const bool full = c->cfg.merge == HF_MERGE_FULL_WIDTH && L.has_wfull;
     CUtensorMap tq;
     HF_TRY(make_map(c, &tq, q, 1));
     ReadoutTc5Params p;
     p.cos_q = c->rope_q[0]; p.sin_q = c->rope_q[1];
-    p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr; p.heads = c->cfg.heads; p.Tc = c->Tc;
+    p.z = L.z; p.bias = (L.has_bias && !full) ? L.bias : nullptr; p.heads = c->cfg.heads; p.Tc = c->Tc;
     p.Tm = (c->Tc + R::ROWS - 1) / R::ROWS; p.n_units = p.Tm * c->BH; p.eps = c->cfg.eps;
-    p.out_bf16 = out_bf16; p.out_f32 = out_f32; p.dev_status = c->dev_status;
+    p.out_bf16 = full ? c->x_hi : out_bf16; p.out_f32 = full ? nullptr : out_f32; p.out_lo = full ? c->x_lo : nullptr;
+    p.dev_status = c->dev_status;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     if (c->has_rope_q) k_readout_tc5<D, true><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
     else k_readout_tc5<D, false><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tq, L.tm_sfhi, L.tm_sflo, p);
-    return post_launch(c, "k_readout_tc5");
+    HF_TRY(post_launch(c, "k_readout_tc5"));
+    if (!full) return HF_OK;
+    typedef MergeFull<D> M;
+    CUtensorMap txh, txl;
+    HF_TRY(make_map(c, &txh, c->x_hi, 1));
+    HF_TRY(make_map(c, &txl, c->x_lo, 1));
+    MergeFullParams mp;
+    mp.heads = c->cfg.heads; mp.Tc = c->Tc; mp.Tm = (c->Tc + M::ROWS - 1) / M::ROWS;
+    mp.bias = L.has_bias ? L.bias : nullptr; mp.out_f32 = out_f32; mp.out_bf16 = out_f32 ? nullptr : out_bf16;
+    mp.dev_status = c->dev_status;
+    PdlLaunch pl(dim3(mp.Tm, c->cfg.heads, c->cfg.batch), dim3(M::THREADS), M::SMEM_BYTES, st, false);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_merge_full<D>, txh, txl, L.tm_wfull, mp));
+    return post_launch(c, "k_merge_full");
 }
 
 ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v_cur) {
@@ -501,7 +524,22 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK) s = dmalloc(&L.sf_hi, dd);
         if (s == HF_OK) s = dmalloc(&L.sf_lo, dd);
         if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.W, (size_t)cfg->heads * c->d * c->d);
-        if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
+        if (s == HF_OK && cfg->merge != HF_MERGE_IDENTITY) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
+        if (s == HF_OK && cfg->merge == HF_MERGE_FULL_WIDTH) {
+            const size_t hd = (size_t)cfg->heads * c->d;
+            s = dmalloc(&L.W_full, hd * hd);
+            if (s == HF_OK) {
+                const cuuint64_t dims[4] = {hd, hd, 1, 1};
+                const cuuint64_t strides[3] = {hd * 2, hd * hd * 2, hd * hd * 2};
+                const cuuint32_t box[4] = {64, (cuuint32_t)c->d, 1, 1};
+                const cuuint32_t es[4] = {1, 1, 1, 1};
+                CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_tiled)(&L.tm_wfull, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, L.W_full, dims,
+                                                                              strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                if (r != CUDA_SUCCESS) s = fail(HF_ERR_CUDA, "cuTensorMapEncodeTiled (merge matrix) failed with %d", (int)r);
+            }
+        }
         if (s == HF_OK) s = dmalloc(&L.mask, (size_t)c->BH * c->Tm * c->mask_words);
         if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
         if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_kring, L.ring_k, (int)slots);
@@ -515,6 +553,12 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     if (s == HF_OK) s = dmalloc(&c->pooled_q, c->pooled_elems);
     if (s == HF_OK) s = dmalloc(&c->pooled_kcur, c->pooled_elems);
     if (s == HF_OK) s = dmalloc(&c->hist, c->chunk_elems);
+    if (s == HF_OK && cfg->merge == HF_MERGE_FULL_WIDTH) s = dmalloc(&c->x_hi, c->chunk_elems);
+    if (s == HF_OK && cfg->merge == HF_MERGE_FULL_WIDTH) s = dmalloc(&c->x_lo, c->chunk_elems);
+    if (s == HF_OK && cfg->merge == HF_MERGE_FULL_WIDTH &&
+        (cudaFuncSetAttribute(k_merge_full<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, MergeFull<64>::SMEM_BYTES) != cudaSuccess ||
+         cudaFuncSetAttribute(k_merge_full<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, MergeFull<128>::SMEM_BYTES) != cudaSuccess))
+        s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_merge_full) failed");
     if (s == HF_OK) s = dmalloc(&c->partials, (size_t)c->BH * c->nsplit_max * ((size_t)c->d * c->d + c->d));
     if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)4);
     if (s == HF_OK && (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
@@ -572,11 +616,19 @@ hf_status hf_reset(hf_ctx* c, int layer, void* stream) {
 
 hf_status hf_set_merge_weights(hf_ctx* c, int layer, const void* W, const void* bias, void* stream) {
     HF_TRY(check_layer(c, layer));
-    if (c->cfg.merge != HF_MERGE_PER_HEAD) return fail(HF_ERR_STATE, "context was created with HF_MERGE_IDENTITY");
+    if (c->cfg.merge == HF_MERGE_IDENTITY) return fail(HF_ERR_STATE, "context was created with HF_MERGE_IDENTITY");
     HF_TRY(check_ptr(W, "W"));
     if (bias != nullptr) HF_TRY(check_ptr(bias, "bias"));
     cudaStream_t st = (cudaStream_t)stream;
     LayerState& L = c->layers[layer];
+    if (c->cfg.merge == HF_MERGE_FULL_WIDTH) {      // one [H d, H d] matrix: applied by its own kernel after the read-out
+        const size_t hd = (size_t)c->cfg.heads * c->d;
+        HF_CUDA(cudaMemcpyAsync(L.W_full, W, hd * hd * 2, cudaMemcpyDeviceToDevice, st));
+        if (bias) HF_CUDA(cudaMemcpyAsync(L.bias, bias, hd * 2, cudaMemcpyDeviceToDevice, st));
+        L.has_wfull = true;
+        L.has_bias = bias != nullptr;
+        return HF_OK;
+    }
     HF_CUDA(cudaMemcpyAsync(L.W, W, (size_t)c->cfg.heads * c->d * c->d * 2, cudaMemcpyDeviceToDevice, st));
     if (bias) HF_CUDA(cudaMemcpyAsync(L.bias, bias, (size_t)c->cfg.heads * c->d * 2, cudaMemcpyDeviceToDevice, st));
     L.has_w = true;
@@ -709,7 +761,8 @@ static hf_status attend_merge(hf_ctx* c, LayerState& L, const bf16* q, const bf1
     // At head_dim 128 the tcgen05 attention kernel forms the history term itself (three more tensor-core products per
     // query block against the folded state, which it keeps in shared memory): no read-out kernel, no scratch buffer.
     // The rotated variant of Eq. 4 (numerator and denominator see different phi(Q)) keeps the separate read-out.
-    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q)
+    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q &&
+        c->cfg.merge != HF_MERGE_FULL_WIDTH)
         return launch_swa_tc5_t<128>(c, L, q, k, v, idx, keep, nullptr, o, nullptr, st, true, after_select);
     // Otherwise the read-out kernel writes the history term to the context's scratch buffer and the attention kernel adds
     // it in its epilogue.
@@ -741,7 +794,8 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     HF_TRY(check_ptr(o, "o"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
-    const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q;
+    const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q &&
+                            c->cfg.merge != HF_MERGE_FULL_WIDTH;
     if (one_kernel) {
         HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
         return attend_merge(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, (bf16*)o, st, true);

@@ -275,8 +275,9 @@ struct ReadoutTc5Params {
     const bf16* bias;         // [H, D] or nullptr
     int heads, Tc, Tm, n_units;
     float eps;
-    bf16* out_bf16;           // exactly one of the two outputs is non-null: [B*H, T_c, D]
+    bf16* out_bf16;           // exactly one of out_bf16 / out_f32 is non-null: [B*H, T_c, D]
     float* out_f32;
+    bf16* out_lo;             // with out_bf16: the bf16 residual of the result (value = out_bf16 + out_lo to ~16 bits), or nullptr
     int* dev_status;
 };
 
@@ -496,10 +497,22 @@ k_readout_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         for (int v = 0; v < 8; ++v) dst[v] = make_float4(x[4 * v], x[4 * v + 1], x[4 * v + 2], x[4 * v + 3]);
                     } else {
                         uint4* dst = reinterpret_cast<uint4*>(p.out_bf16 + g + col);
+                        uint32_t hp[16];
 #pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            dst[v] = make_uint4(pack_bf16(x[8 * v], x[8 * v + 1]), pack_bf16(x[8 * v + 2], x[8 * v + 3]),
-                                                pack_bf16(x[8 * v + 4], x[8 * v + 5]), pack_bf16(x[8 * v + 6], x[8 * v + 7]));
+                        for (int e = 0; e < 16; ++e) hp[e] = pack_bf16(x[2 * e], x[2 * e + 1]);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) dst[v] = make_uint4(hp[4 * v], hp[4 * v + 1], hp[4 * v + 2], hp[4 * v + 3]);
+                        if (p.out_lo) {
+                            uint4* dlo = reinterpret_cast<uint4*>(p.out_lo + g + col);
+                            uint32_t lp[16];
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) {
+                                const float2 hf = unpack_bf16(hp[e]);
+                                lp[e] = pack_bf16(x[2 * e] - hf.x, x[2 * e + 1] - hf.y);
+                            }
+#pragma unroll
+                            for (int v = 0; v < 4; ++v) dlo[v] = make_uint4(lp[4 * v], lp[4 * v + 1], lp[4 * v + 2], lp[4 * v + 3]);
+                        }
                     }
                 }
             }

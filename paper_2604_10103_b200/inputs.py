@@ -149,6 +149,15 @@ def merge_weights(w: Workload, layer: int, with_bias: bool = True):
     return W, b
 
 
+def merge_weights_full(w: Workload, layer: int, with_bias: bool = True):
+    """Random-init projection over the model width (the one-matrix reading of the history branch's Linear):
+    W [H d, H d] ~ N(0, 1/(H d)), bias [H d] ~ N(0, 0.01)."""
+    hd = w.heads * w.head_dim
+    W = normal_bf16((hd, hd), w.seed, layer, 0, 1, T_W, scale=hd ** -0.5)
+    b = normal_bf16((hd,), w.seed, layer, 0, 1, T_BIAS, scale=0.1) if with_bias else None
+    return W, b
+
+
 def rotation_tables(w: Workload, which: int):
     """(cos, sin) float32 tables [T_c, d/2] of seeded angles ~ U(0, 2 pi): stand-ins for the position angles a model
     would supply to the linear branch's rotation.  `which`: T_ANGLE_Q or T_ANGLE_K."""

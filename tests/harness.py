@@ -22,9 +22,13 @@ def max_abs(a, b):
 
 
 def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, z_frame_mean: bool = False,
-                sink_chunks: int = 0, rope: bool = False):
-    W = b = None
-    if merge:
+                sink_chunks: int = 0, rope: bool = False, merge_full: bool = False):
+    W = b = Wf = bf = None
+    if merge_full:
+        Wb, bb = gen.merge_weights_full(w, layer, with_bias=bias)
+        Wf = gen.bf16_bits_to_f64(Wb)
+        bf = None if bb is None else gen.bf16_bits_to_f64(bb)
+    elif merge:
         Wb, bb = gen.merge_weights(w, layer, with_bias=bias)
         W = gen.bf16_bits_to_f64(Wb)
         b = None if bb is None else gen.bf16_bits_to_f64(bb)
@@ -32,7 +36,7 @@ def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool 
                            keep_permille=w.keep_permille, W=W, bias=b, eps=w.eps,
                            z_frame_tokens=w.tokens_per_frame if z_frame_mean else None, sink_chunks=sink_chunks,
                            rope_q=gen.rotation_tables(w, gen.T_ANGLE_Q) if rope else None,
-                           rope_k=gen.rotation_tables(w, gen.T_ANGLE_K) if rope else None)
+                           rope_k=gen.rotation_tables(w, gen.T_ANGLE_K) if rope else None, W_full=Wf, bias_full=bf)
 
 
 from paper_2604_10103_b200.binding import unpack_mask  # noqa: E402,F401
@@ -42,16 +46,21 @@ class GpuStream:
     """The library side of a one-layer stream (torch only for memory)."""
 
     def __init__(self, w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, swa_kernel: int = 0,
-                 layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0, rope: bool = False):
+                 layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0, rope: bool = False,
+                 merge_full: bool = False):
         import torch
         from paper_2604_10103_b200 import binding as hf
         self.torch, self.hf, self.w, self.layer = torch, hf, w, layer
         cfg = hf.make_config(w.with_(layers=layers or max(w.layers, layer + 1)),
-                             merge=hf.HF_MERGE_PER_HEAD if merge else hf.HF_MERGE_IDENTITY, swa_kernel=swa_kernel,
+                             merge=hf.HF_MERGE_FULL_WIDTH if merge_full else hf.HF_MERGE_PER_HEAD if merge else hf.HF_MERGE_IDENTITY,
+                             swa_kernel=swa_kernel,
                              z_mode=hf.HF_Z_FRAME_MEAN if z_frame_mean else hf.HF_Z_SUM,
                              sink_frames=sink_chunks * w.chunk_frames)
         self.ctx = hf.Context(cfg)
-        if merge:
+        if merge_full:
+            Wb, bb = gen.merge_weights_full(w, layer, with_bias=bias)
+            self.ctx.hf_set_merge_weights(layer, hf.bits_to_cuda(Wb), None if bb is None else hf.bits_to_cuda(bb))
+        elif merge:
             Wb, bb = gen.merge_weights(w, layer, with_bias=bias)
             self.ctx.hf_set_merge_weights(layer, hf.bits_to_cuda(Wb), None if bb is None else hf.bits_to_cuda(bb))
         if rope:

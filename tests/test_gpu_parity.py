@@ -516,3 +516,27 @@ def test_lse_output_of_the_tcgen05_kernel():
                 assert np.abs(lse[0, h, rows] - ref).max() < 2e-3
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,b,tpf,heads,batch,bias", [(128, 128, 300, 3, 2, True), (64, 16, 64, 2, 1, True), (64, 128, 200, 4, 1, False)])
+def test_full_width_merge_projection(d, b, tpf, heads, batch, bias):
+    """Eq. 4's Linear read as one [H d, H d] matrix over all heads: read-out (bf16 hi + lo) -> projection kernel ->
+    history term, against the oracle; hf_linear_attn alone and the whole forward, over a stream with evictions."""
+    w = gen.Workload("fullw", batch=batch, heads=heads, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=2,
+                     block=b, topk=0, keep_permille=500, seed=47)
+    gpu = hz.GpuStream(w, merge_full=True, bias=bias); ora = hz.make_oracle(w, merge_full=True, bias=bias)
+    try:
+        for c in range(4):
+            qb, kb, vb = gen.qkv(w, 0, c, 0)
+            q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+            m_gpu, _, _ = gpu.select(q, k)
+            m_ref, _ = ora.select(f64(qb), f64(kb))
+            assert np.array_equal(m_gpu, m_ref)
+            o_ref, _, oh_ref = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, parts=True)
+            hz.assert_close_out(gpu.forward(q, k, v), o_ref, f"chunk {c} hybrid O, full-width merge")
+            hz.assert_close_out(gpu.linear(q), oh_ref, f"chunk {c} O_history, full-width merge")
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
