@@ -113,3 +113,27 @@ def test_sweep_subset(permille, window, d, blk, batch):
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+def test_full_width_merge_at_the_832x480_layer_shape():
+    """The projection over the model width at full size (12 heads x 128 = 1536 features, 4680 tokens): history term of
+    hf_linear_attn against the oracle after two evictions (the attention branch at this size is covered above)."""
+    from oracle import hybrid_attention as oa
+    w = gen.layer_832x480().with_(seed=53)
+    gpu = hz.GpuStream(w, merge_full=True); ora = hz.make_oracle(w, merge_full=True)
+    f64 = gen.bf16_bits_to_f64
+    try:
+        for c in range(4):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert ora.absorbed_tokens == 2 * w.chunk_tokens
+        qb, _, _ = gen.qkv(w, 0, 4, 0)
+        qf = f64(qb)
+        h = np.stack([oa.linear_readout(qf[0, hh], ora.S[0, hh], ora.z[0, hh], None, None, ora.eps) for hh in range(w.heads)])
+        ref = oa.merge_full_width(h, ora.W_full, ora.bias_full)[None]
+        hz.assert_close_out(gpu.linear(gpu.up(qb)), ref, "O_history, full-width merge, 832x480 layer")
+        S, z = gpu.state()
+        assert hz.rel_l2(S, ora.S) <= hz.STATE_REL_L2 and hz.rel_l2(z, ora.z) <= hz.STATE_REL_L2
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
