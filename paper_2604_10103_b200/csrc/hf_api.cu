@@ -234,8 +234,10 @@ hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
 
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
-    // after the partials kernel (nsplit > 0) the launch may overlap that kernel's epilogue; a fold on its own is ordinary
-    PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, nsplit > 0);
+    // An ordinary launch, on purpose: launched programmatically under the partials kernel's epilogue, this grid (up to
+    // several hundred blocks that would sit on the SMs waiting) made thread blocks of the partials kernel run into their
+    // wait limits at batch 4 (measured; the mechanism was not established).
+    PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, false);
     HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D>, (const float*)c->partials, nsplit, L.S, L.z, c->z_scale,
                                (const bf16*)(L.has_w ? L.W : nullptr), c->cfg.heads, L.sf_hi, L.sf_lo));
     return post_launch(c, "k_reduce_fold");

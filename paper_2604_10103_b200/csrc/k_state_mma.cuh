@@ -143,12 +143,11 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
     const int cp = threadIdx.x;
     const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr;
     uint4 wq[D / 8];
-    if (with_w) {       // (W is a parameter set long before: read ahead of the wait below)
+    if (with_w) {
         const uint4* wrow = reinterpret_cast<const uint4*>(W + ((size_t)h * D + cp) * D);     // W_h[c'][.]
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
     }
-    pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
     const float* base = partials + (size_t)bh * nsplit * PART_FLOATS;
     float sum[ROWS];
 #pragma unroll

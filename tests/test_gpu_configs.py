@@ -137,3 +137,37 @@ def test_full_width_merge_at_the_832x480_layer_shape():
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+def test_many_cache_commits_at_batch_4_leave_a_clean_status():
+    """Back-to-back cache commits with evictions at batch 4 (48 batch*head pairs, 64-token blocks, head_dim 64): the
+    absorb, reduce/fold and copy kernels of consecutive commits overlap on two streams; no bounded wait may run out, and
+    the state must match a context that absorbed the same evicted chunks one call at a time."""
+    import torch
+    from paper_2604_10103_b200 import binding as hf
+    w = gen.layer_832x480().with_(name="commits", batch=4, head_dim=64, block=64, layers=2, seed=59)
+    ctx = hf.Context(hf.make_config(w)); ref = hf.Context(hf.make_config(w.with_(layers=1)))
+    try:
+        shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
+        g = torch.Generator(device="cuda"); g.manual_seed(59)
+        chunks = [(torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16),
+                   torch.randn(shape, generator=g, device="cuda").to(torch.bfloat16)) for _ in range(3)]
+        n = 24
+        for r in range(n):
+            kk, vv = chunks[r % 3]
+            ctx.hf_kv_append(r % 2, kk, vv)
+        assert ctx.hf_get_device_status() == (0, 0)
+        # layer 0 saw commits r = 0, 2, 4, ...: all but the last two of them were evicted, in order
+        evicted = [r for r in range(0, n, 2)][:-w.past_chunks]
+        for r in evicted:
+            kk, vv = chunks[r % 3]
+            ref.hf_state_absorb(0, kk, vv, w.chunk_tokens)
+        S = torch.empty((w.batch, w.heads, 64, 64), dtype=torch.float32, device="cuda"); z = torch.empty((w.batch, w.heads, 64), dtype=torch.float32, device="cuda")
+        S2 = torch.empty_like(S); z2 = torch.empty_like(z)
+        ctx.hf_get_state(0, S, z); ref.hf_get_state(0, S2, z2)
+        torch.cuda.synchronize()
+        assert torch.equal(S, S2) and torch.equal(z, z2)
+        assert ctx.hf_query(0, hf.HF_Q_ABSORBED_TOKENS) == len(evicted) * w.chunk_tokens
+        assert ref.hf_get_device_status() == (0, 0)
+    finally:
+        ctx.close(); ref.close()
