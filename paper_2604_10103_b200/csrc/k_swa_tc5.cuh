@@ -67,7 +67,7 @@ struct SwaTc5 {
 
 struct Tc5Params {
     const int32_t* idx;      // [B*H, T_m, keep]
-    int keep, Tc, n_b, n_cached, ring_head, P;   // P: physical ring slots (one more than the window holds); the sink slots follow them
+    int keep, Tc, n_b, n_cached, ring_head, P;   // P: ring slots (the cache's past chunks); the sink slots follow them
     int n_sink;              // sink chunks held (logical chunks 0 .. n_sink - 1)
     int Tm, n_units;         // units = (batch*head, query block) pairs, unit u = bh * Tm + i
     float scale_log2;
@@ -150,7 +150,10 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     // Everything above (barriers, tensor memory) may overlap the tail of the kernel before this one in the stream when the
     // launch allows it; the index list it wrote is read from here on.
     pdl_wait();
-    pdl_trigger();              // the next kernel in the stream may be made resident on SMs this grid has left; it waits itself
+    // The next kernel in the stream may be made resident on SMs this grid has left (it waits itself) -- only where a thread
+    // block of this kernel takes all of an SM's shared memory, so that no waiting block of the dependent grid ever sits
+    // beside a working block of this one.
+    if (C::SMEM_BYTES > 200 * 1024) pdl_trigger();
 
     if (warp == C::WARP_LOAD_K || warp == C::WARP_LOAD_V) {
         // ================================================================= TMA producers
