@@ -143,7 +143,11 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
         constexpr int HT = C::TT / C::NQ;                       // tokens per thread and tile
         bool ok = true;
         float zacc = 0.f;
-        for (int i = 0; ok && i < n_local; ++i) {
+        // Warps whose lanes lie past the head dimension (the upper two quadrants at head_dim 64) have no part in the tile
+        // loop and must stay out of it: they would wait on the stage barriers without ever arriving on the "free" ones, so
+        // nothing would keep the pipeline from running more than a ring ahead of them, and a warp that falls NST tiles
+        // behind waits on a phase parity that has come round again -- until its wait limit.  (`active` is warp-uniform.)
+        for (int i = 0; ok && active && i < n_local; ++i) {
             const int s = i % C::NST, ab = i & 1;
             ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, (i / C::NST) & 1, abort_flag, p.dev_status, 35));
             if (!ok) break;
