@@ -336,7 +336,7 @@ def run_ours(args, w):
                 "config": {"workload": w.name, "layers": w.layers, "denoise_steps": w.steps, "batch": w.batch, "heads": w.heads,
                            "head_dim": w.head_dim, "chunk_tokens": w.chunk_tokens, "window_frames": w.window_frames,
                            "block": w.block, "keep_permille": w.keep_permille,
-                           "l2": "inputs larger than L2 (distinct q/k/v per layer, 1.3 GB per pass; caches 3.5 GB)",
+                           "l2": "inputs larger than L2 (distinct q/k/v per layer, 1.3 GB per pass; caches 5.2 GB)",
                            "swa_kernel": {1: "mma.sync", 2: "tcgen05"}.get(ctx.hf_query(0, hf.HF_Q_SWA_KERNEL))},
                 "clocks": clocks, "gpu_launches": int(launches), "e2e": e2e, "roofline": roof, "stages": stage, "contrast": contrast,
                 "cpu_baseline": {"value": cpu_fps, "unit": UNIT, "cores": thr, "kind": "oracle", "sample": desc},

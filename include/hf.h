@@ -107,9 +107,11 @@ hf_status hf_set_merge_weights(hf_ctx* ctx, int layer, const void* W, const void
 hf_status hf_set_rope(hf_ctx* ctx, const float* cos_q, const float* sin_q, const float* cos_k, const float* sin_k, void* stream);
 
 /* Alg. 2, cache commit of a clean chunk: k, v bf16 [B,H,T_c,d].  If the cache already holds P chunks the oldest
- * is first folded into the state (Eq. 3: S += phi(K_ev)^T V_ev, z += sum phi(K_ev)) and its slot reused; the
- * chunk's K, V are copied in and its per-block K means stored.  With P = 0 the chunk goes straight into the
- * state and nothing is cached.  Device memory per layer: (P + sink chunks) x 2 x B*H*T_c*d bf16. */
+ * is folded into the state (Eq. 3: S += phi(K_ev)^T V_ev, z += sum phi(K_ev)) and leaves the window; the chunk's
+ * K, V are copied in and its per-block K means stored.  The ring has P + 1 slots per layer (a spare one), so the copy
+ * of the new chunk and the state update of the old one run side by side; when the call's work is done in stream order
+ * both have happened, and the evicted chunk's slot is not written before the next commit.  With P = 0 the chunk goes
+ * straight into the state and nothing is cached.  Device memory per layer: (P + 1 + sink chunks) x 2 x B*H*T_c*d bf16. */
 hf_status hf_kv_append(hf_ctx* ctx, int layer, const void* k, const void* v, void* stream);
 
 /* Eq. 3 on caller-supplied tokens: k_ev, v_ev bf16 [B,H,n_tokens,d], any n_tokens >= 1. */

@@ -65,7 +65,7 @@ struct hf_ctx {
     hf_config cfg;
     int device = 0, sm_count = 0;
     int BH = 0, Tc = 0, n_b = 0, P = 0, R = 0, Tm = 0, max_Tn = 0, mask_words = 0, d = 0;
-    int n_sink_max = 0;              // sink chunks of the configuration; ring (R = P slots) and sink share one allocation
+    int n_sink_max = 0;              // sink chunks of the configuration; ring (R = P + 1 slots: the window's P past chunks and a spare) and sink share one allocation
     size_t chunk_elems = 0, pooled_elems = 0;
     std::vector<LayerState> layers;
     float* pooled_q = nullptr;
@@ -234,20 +234,18 @@ hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
 
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
-    // An ordinary launch, on purpose: launched programmatically under the partials kernel's epilogue, this grid (up to
-    // several hundred blocks that would sit on the SMs waiting) made thread blocks of the partials kernel run into their
-    // wait limits at batch 4 (measured; the mechanism was not established).
-    PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, false);
+    // after the partials kernel (nsplit > 0) the launch may overlap that kernel's epilogue; a fold on its own is ordinary
+    PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, nsplit > 0);
     HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D>, (const float*)c->partials, nsplit, L.S, L.z, c->z_scale,
                                (const bf16*)(L.has_w ? L.W : nullptr), c->cfg.heads, L.sf_hi, L.sf_lo));
     return post_launch(c, "k_reduce_fold");
 }
 
-// fold_on_side: the reduce/fold kernel goes to the context's side stream (the caller has more work for `st` that only
-// needs the partials kernel to be done, and joins with ev_join afterwards).
+// on_side: both kernels go to the context's side stream, ordered after what `st` holds so far (the caller has
+// independent work for `st` and joins with ev_join afterwards).
 template <int D>
 hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, int n_tokens, cudaStream_t st,
-                        bool fold_on_side = false) {
+                        bool on_side = false) {
     typedef AbsorbTc5<D> A;
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     const int nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
@@ -257,15 +255,18 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     AbsorbTc5Params p;
     p.n_tokens = n_tokens; p.partials = c->partials; p.dev_status = c->dev_status;
     p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc;
-    PdlLaunch pl(dim3(nsplit, c->BH), dim3(A::THREADS), A::SMEM_BYTES, st, true);
+    cudaStream_t run = st;
+    if (on_side) {
+        HF_CUDA(cudaEventRecord(c->ev_fork, st));
+        HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        run = c->side;
+    }
+    PdlLaunch pl(dim3(nsplit, c->BH), dim3(A::THREADS), A::SMEM_BYTES, run, !on_side);   // (an event wait sits before it on the side stream)
     if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, true>, tk, tv, p));
     else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_tc5<D, false>, tk, tv, p));
     HF_TRY(post_launch(c, "k_absorb_tc5"));
-    if (!fold_on_side) return launch_fold<D>(c, L, nsplit, st);
-    HF_CUDA(cudaEventRecord(c->ev_fork, st));
-    HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
-    HF_TRY(launch_fold<D>(c, L, nsplit, c->side));
-    HF_CUDA(cudaEventRecord(c->ev_join, c->side));
+    HF_TRY(launch_fold<D>(c, L, nsplit, run));
+    if (on_side) HF_CUDA(cudaEventRecord(c->ev_join, c->side));
     return HF_OK;
 }
 
@@ -488,7 +489,7 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->n_b = (c->Tc + cfg->block - 1) / cfg->block;
     c->Tm = c->n_b;
     c->P = cfg->window_frames / cfg->chunk_frames - 1;
-    c->R = c->P;        // physical ring slots (kept apart from P: a spare slot was tried, see the cache commit)
+    c->R = c->P > 0 ? c->P + 1 : 0;     // physical ring slots: one more than the window holds (see the cache commit)
     c->n_sink_max = cfg->sink_frames / cfg->chunk_frames;
     c->max_Tn = (c->P + c->n_sink_max + 1) * c->n_b;
     c->mask_words = (c->max_Tn + 31) / 32;
@@ -693,22 +694,20 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
         L.cache_epoch++;
         return HF_OK;
     }
-    // Cache full: the state is updated before the evicted chunk's slot is reused.  The slot may be overwritten as soon as
-    // the partials kernel has read it (same stream); adding the partials to the state and folding it runs beside the
-    // copy, on the side stream.  (A spare ring slot, with the whole state update beside the copy, was 10 % faster but
-    // made thread blocks of the absorb kernel run into their wait limits now and then at batch 4 when the copy kernel's
-    // blocks shared the SMs with them: taken out.)
-    int slot;
+    // The ring has one slot more than the window holds, so the new chunk never lands on the chunk that leaves: the state
+    // update (Eq. 3) of the evicted chunk runs on the side stream beside the copy of the new one (the copy kernel's thread
+    // blocks fit on the SMs next to the absorb kernel's), and the call joins the two before it returns to the caller's
+    // stream.  The state is still updated before anything can overwrite the evicted chunk: the slot it sits in is the
+    // target of the NEXT commit, which is ordered after this call's join.
+    const int slot = (L.head + L.n_cached) % c->R;
     bool evicted = false;
     if (L.n_cached == c->P) {
-        slot = L.head;
-        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)slot * c->chunk_elems,
-                             L.ring_v + (size_t)slot * c->chunk_elems, c->Tc, st, true));
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, L.ring_k + (size_t)L.head * c->chunk_elems,
+                             L.ring_v + (size_t)L.head * c->chunk_elems, c->Tc, st, true));
         evicted = true;
         L.absorbed += c->Tc;
         L.head = (L.head + 1) % c->R;
     } else {
-        slot = (L.head + L.n_cached) % c->R;
         L.n_cached++;
     }
     PoolJobs jobs;

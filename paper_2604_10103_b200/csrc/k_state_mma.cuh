@@ -148,6 +148,7 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
     }
+    pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
     const float* base = partials + (size_t)bh * nsplit * PART_FLOATS;
     float sum[ROWS];
 #pragma unroll

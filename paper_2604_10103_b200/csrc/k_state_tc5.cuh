@@ -198,6 +198,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
         }
         // ---- epilogue: the accumulator goes through a padded staging tile in shared memory (the pipeline stages are
         // idle by now: every TMA copy has been consumed) so that the partial is written with coalesced stores
+        pdl_trigger();          // the reduce/fold kernel may be launched now: it waits for this grid before it reads a partial
         if (ok && active) {
             z_x[part * D + a] = zacc;
             mbar_arrive(bar_z);

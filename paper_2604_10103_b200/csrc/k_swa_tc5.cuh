@@ -67,7 +67,7 @@ struct SwaTc5 {
 
 struct Tc5Params {
     const int32_t* idx;      // [B*H, T_m, keep]
-    int keep, Tc, n_b, n_cached, ring_head, P;   // P: ring slots (the cache's past chunks); the sink slots follow them
+    int keep, Tc, n_b, n_cached, ring_head, P;   // P: physical ring slots (one more than the window holds); the sink slots follow them
     int n_sink;              // sink chunks held (logical chunks 0 .. n_sink - 1)
     int Tm, n_units;         // units = (batch*head, query block) pairs, unit u = bh * Tm + i
     float scale_log2;
