@@ -210,13 +210,25 @@ hf_status hf_query(hf_ctx* ctx, int layer, int what, int64_t* value);
 
 /* Synchronises the device and reports the device status word.  Flag 1: a bounded wait inside a kernel ran out
  * (detail = where), HF_ERR_DEVICE_TIMEOUT.  Flag 2: a caller's index list held a block index outside [0, T_n)
- * (detail = batch*head and query block of the row, as one number), HF_ERR_INVALID_ARG.  Flag 4: the tcgen05 attention
- * kernel (HF_SWA_TCGEN05) fixes a query row's softmax reference at the row maximum of its first kept key block times
- * 2^60 and keeps no running maximum; a row whose later blocks rise more than about 100 natural-log units above the first
- * one would overflow fp32 and is reported instead (detail = the query block), HF_ERR_UNSUPPORTED: HF_SWA_TCGEN05_PINGPONG
- * and HF_SWA_MMA keep a running maximum and take any input.  In every case the result of that launch is invalid, the
- * word is cleared and the context stays usable. */
+ * (detail = batch*head and query block of the row, as one number), HF_ERR_INVALID_ARG.  In both cases the result of
+ * that launch is invalid, the word is cleared and the context stays usable. */
 hf_status hf_get_device_status(hf_ctx* ctx, int* flags, int* detail);
+
+/* Alg. 3 keeps a running row maximum m (m_new = max(m, rowmax S)) and rescales l and O by e^{m - m_new}.  The tcgen05
+ * attention kernel (HF_SWA_TCGEN05, what HF_SWA_AUTO resolves to) instead fixes a row's reference after its first kept
+ * key block (softmax does not depend on the reference), which covers rows whose later blocks rise up to about 100
+ * natural-log units above the first; a (batch*head, query block) unit with a row beyond that is computed a second time
+ * inside the same launch with the running maximum, so o is the softmax of Eq. 6 for every finite input and no status has
+ * to be polled.  This call synchronises the device and reports how many units have taken that second pass since the
+ * context was created (a diagnostic: such units cost several times a normal one). */
+hf_status hf_slow_path_units(hf_ctx* ctx, int64_t* units);
+
+/* Self-test of the failure path all kernels share (no counterpart in the paper).  Every wait inside a kernel is bounded:
+ * when its limit runs out the thread block raises flag 1 of the status word and leaves in the ordinary way.  This call
+ * launches a one-warp kernel that waits, under a limit of about a millisecond, on a barrier nothing ever arrives on, so
+ * the wait runs out by construction; the next hf_get_device_status must then report HF_ERR_DEVICE_TIMEOUT with detail 77
+ * and clear the word, and the context must work as before.  Nothing in it can hang or fault the device. */
+hf_status hf_selftest_wait_limit(hf_ctx* ctx, void* stream);
 
 /* Number of kernels the library has launched since the context was created. */
 hf_status hf_launch_count(hf_ctx* ctx, int64_t* launches);

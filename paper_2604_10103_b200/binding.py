@@ -28,7 +28,7 @@ EXPORTS = [
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
     "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
-    "hf_sparse_swa_merged",
+    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit",
 ]
 
 
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
     L.hf_query.argtypes = [vp, ip, ip, C.POINTER(C.c_int64)]
     L.hf_get_device_status.argtypes = [vp, C.POINTER(ip), C.POINTER(ip)]
     L.hf_launch_count.argtypes = [vp, C.POINTER(C.c_int64)]
+    L.hf_slow_path_units.argtypes = [vp, C.POINTER(C.c_int64)]
+    L.hf_selftest_wait_limit.argtypes = [vp, vp]
     L.hf_state_absorb_noalloc.argtypes = [vp, vp, ip, ip, ip, vp, vp, vp]
     L.hf_status_string.argtypes = [ip]
     L.hf_status_string.restype = C.c_char_p
@@ -199,6 +201,14 @@ class Context:
         f, d = C.c_int(), C.c_int()
         _check(lib().hf_get_device_status(self._h, C.byref(f), C.byref(d)))
         return f.value, d.value
+
+    def hf_selftest_wait_limit(self):
+        _check(lib().hf_selftest_wait_limit(self._h, _stream()))
+
+    def hf_slow_path_units(self) -> int:
+        v = C.c_int64()
+        _check(lib().hf_slow_path_units(self._h, C.byref(v)))
+        return v.value
 
     def hf_launch_count(self) -> int:
         v = C.c_int64()

@@ -8,6 +8,7 @@
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
 #include "k_merge_full.cuh"
+#include "k_selftest.cuh"
 
 #include <cmath>
 #include <cstdarg>
@@ -374,6 +375,7 @@ hf_status launch_swa_tc5_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* 
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
     p.heads = c->cfg.heads; p.eps = c->cfg.eps;
     p.q = q; p.z = L.z; p.bias = L.has_bias ? L.bias : nullptr;
+    p.tab = make_table(c, L, k_cur, v_cur); p.sf_hi = L.sf_hi; p.sf_lo = L.sf_lo;
     const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
     const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
@@ -407,6 +409,7 @@ hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16*
     p.P = c->R;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
     p.hist = hist; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
+    memset(&p.tab, 0, sizeof(p.tab)); p.sf_hi = nullptr; p.sf_lo = nullptr;
     const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
     const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
     p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
@@ -560,13 +563,13 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
          cudaFuncSetAttribute(k_merge_full<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, MergeFull<128>::SMEM_BYTES) != cudaSuccess))
         s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_merge_full) failed");
     if (s == HF_OK) s = dmalloc(&c->partials, (size_t)c->BH * c->nsplit_max * ((size_t)c->d * c->d + c->d));
-    if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)4);
+    if (s == HF_OK) s = dmalloc(&c->dev_status, (size_t)8);     // status word [4] + self-test results [4]
     if (s == HF_OK && (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
                        cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
                        cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess))
         s = fail(HF_ERR_CUDA, "could not create the context's side stream / events");
     if (s == HF_OK) {
-        cudaMemset(c->dev_status, 0, 16);
+        cudaMemset(c->dev_status, 0, 32);
         s = set_swa_attr<16, 64>();
         if (s == HF_OK) s = set_swa_attr<16, 128>();
         if (s == HF_OK) s = set_swa_attr<64, 64>();
@@ -996,17 +999,29 @@ hf_status hf_get_device_status(hf_ctx* c, int* flags, int* detail) {
     if (flags) *flags = h[0];
     if (detail) *detail = h[1];
     if (h[0] != 0) {
-        HF_CUDA(cudaMemset(c->dev_status, 0, 16));
+        HF_CUDA(cudaMemset(c->dev_status, 0, 8));      // flags and detail; the counters behind them run on
         if (h[0] & HF_DEV_TIMEOUT_FLAG)
             return fail(HF_ERR_DEVICE_TIMEOUT, "a device-side wait ran out (flags %d, detail %d)", h[0], h[1]);
-        if (h[0] & HF_DEV_RANGE_FLAG)
-            return fail(HF_ERR_UNSUPPORTED, "attention logits of a query row rose by more than ~100 (natural log units) above those of "
-                        "its first kept block (unit %d): beyond the fixed-reference softmax of the tcgen05 kernel; "
-                        "HF_SWA_TCGEN05_PINGPONG and HF_SWA_MMA keep a running maximum", h[1]);
         return fail(HF_ERR_INVALID_ARG, "an index list held a block index outside [0, T_n) (unit %d); block 0 was read in its place",
                     h[1]);
     }
     return HF_OK;
+}
+
+hf_status hf_slow_path_units(hf_ctx* c, int64_t* units) {
+    if (c == nullptr || units == nullptr) return fail(HF_ERR_INVALID_ARG, "null argument");
+    int h[4] = {0, 0, 0, 0};
+    HF_CUDA(cudaDeviceSynchronize());
+    HF_CUDA(cudaMemcpy(h, c->dev_status, 16, cudaMemcpyDeviceToHost));
+    *units = h[2];
+    return HF_OK;
+}
+
+hf_status hf_selftest_wait_limit(hf_ctx* c, void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    // the kernel's two result words go to the reserved half of the status buffer's second line
+    k_selftest_wait<<<1, 32, 0, (cudaStream_t)stream>>>(c->dev_status, 77, c->dev_status + 4);
+    return post_launch(c, "k_selftest_wait");
 }
 
 hf_status hf_launch_count(hf_ctx* c, int64_t* launches) {

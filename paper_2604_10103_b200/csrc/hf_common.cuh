@@ -17,8 +17,9 @@ struct ChunkTable {
     int n_chunks;
 };
 
-// Device status word layout (int[4]): [0] flags, [1] detail, [2..3] reserved.
-enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2, HF_DEV_RANGE_FLAG = 4 };
+// Device status word layout (int[4]): [0] flags, [1] detail, [2] units the tcgen05 attention kernel computed a second
+// time with a running maximum (a counter, not an error), [3] reserved.
+enum { HF_DEV_TIMEOUT_FLAG = 1, HF_DEV_BAD_INDEX_FLAG = 2 };
 
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may start while its predecessor
 // in the stream still runs (once every block of the predecessor has called pdl_trigger or exited); pdl_wait returns when the

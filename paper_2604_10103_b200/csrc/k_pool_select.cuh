@@ -139,12 +139,18 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
         }
     }
     __syncthreads();
+    // Rank under a TOTAL order: a NaN score (a NaN anywhere in the query block or the key block) compares false both
+    // ways, which would give every NaN rank 0 and more than `keep` entries per row; here NaN ranks below every number
+    // (NaNs among themselves by block index), so that exactly `keep` blocks are kept whatever the inputs hold.
     for (int j = threadIdx.x; j < Tn; j += 256) {
         const float s = sc[j];
+        const bool s_nan = s != s;
         int rank = 0;
         for (int jj = 0; jj < Tn; ++jj) {
             const float s2 = sc[jj];
-            rank += (s2 > s) || (s2 == s && jj < j);
+            const bool s2_nan = s2 != s2;
+            const bool tie = (s2 == s) || (s_nan && s2_nan);
+            rank += (s2 > s) || (s_nan && !s2_nan) || (tie && jj < j);
         }
         keepf[j] = rank < keep;
     }
@@ -161,8 +167,10 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
             }
             if (f) {
                 const int pos = running + __popc(word & ((1u << lane) - 1u));
-                idx[row * keep + pos] = j;
-                if (idx_out) idx_out[row * keep + pos] = j;
+                if (pos < keep) {       // (always true under the total order above; the store never leaves the row)
+                    idx[row * keep + pos] = j;
+                    if (idx_out) idx_out[row * keep + pos] = j;
+                }
             }
             running += __popc(word);
         }

@@ -31,26 +31,30 @@ __device__ __forceinline__ void swa_load_tile(uint32_t smem_tile, const bf16* __
     }
 }
 
-// hist: optional fp32 [B*H, T_c, D] added to the normalised output before the single rounding to bf16.
+// One (batch*head, query block) unit with the first SwaMma::THREADS threads of the thread block (thread index tid), in the
+// shared-memory window starting at `smem` (SwaMma::SMEM_BYTES, 128-byte aligned).  The participating threads meet on
+// named barrier 1, so the function can run inside a larger thread block (the tcgen05 kernel calls it for the units it
+// hands back, see k_swa_tc5.cuh) as well as be the whole body of k_swa_mma.
+// hist_rows: optional fp32 rows [nq, D] of the unit (row stride D; global or shared memory), added to the normalised
+// output before the single rounding to bf16.
 template <int BLK, int D>
-__global__ void __launch_bounds__(SwaMma<BLK, D>::THREADS)
-k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict__ idx, int keep,
-          int Tc, int n_b, float scale_log2, const float* __restrict__ hist,
-          bf16* __restrict__ o, float* __restrict__ lse, int* dev_status) {
+__device__ __forceinline__ void swa_mma_unit(uint8_t* smem, const bf16* __restrict__ q, const ChunkTable& tab,
+                                             const int32_t* __restrict__ my_idx, int keep, int Tc, int n_b, float scale_log2,
+                                             const float* hist_rows, bf16* __restrict__ o, float* __restrict__ lse,
+                                             int* dev_status, int i, int bh, int unit) {
     typedef SwaMma<BLK, D> C;
-    extern __shared__ __align__(128) uint8_t smem[];
+    auto sync_unit = [] { asm volatile("bar.sync 1, %0;\n" ::"n"(C::THREADS) : "memory"); };
+    typedef SwaMma<BLK, D> C;
     const uint32_t sQ = smem_u32(smem);
     const uint32_t sKV = sQ + C::TILE_BYTES;   // stage s: K at sKV + s*2*TILE, V right after
 
-    const int i = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int q0 = i * BLK;
     const int nq = min(BLK, Tc - q0);
-    const int32_t* my_idx = idx + ((size_t)bh * gridDim.x + i) * keep;
 
     const int Tn = tab.n_chunks * n_b;
     auto issue = [&](int it, int stage) {
-        const int j = checked_block(my_idx[it], Tn, dev_status, bh * gridDim.x + i);
+        const int j = checked_block(my_idx[it], Tn, dev_status, unit);
         const int c = j / n_b, jb = j - c * n_b;
         const int nv = min(BLK, Tc - jb * BLK);
         const size_t off = ((size_t)bh * Tc + (size_t)jb * BLK) * D;
@@ -73,7 +77,7 @@ k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict_
         if (it + 1 < keep) issue(it + 1, stage ^ 1);
         cp_async_commit();
         cp_async_wait<1>();
-        __syncthreads();
+        sync_unit();
 
         const int j = checked_block(my_idx[it], Tn, nullptr, 0);
         const int jb = j % n_b;
@@ -155,7 +159,7 @@ k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict_
                 mma_bf16(o_acc[2 * dp + 1], a0, a1, a2, a3, b2, b3);
             }
         }
-        __syncthreads();   // every warp is done with this stage before the next prefetch overwrites it
+        sync_unit();       // every warp is done with this stage before the next prefetch overwrites it
     }
     cp_async_wait<0>();
 
@@ -176,11 +180,24 @@ k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict_
         for (int n = 0; n < D / 8; ++n) {
             const int col = n * 8 + 2 * (lane & 3);
             float x0 = o_acc[n][2 * r] * inv, x1 = o_acc[n][2 * r + 1] * inv;
-            if (hist) {
-                const float2 h = *reinterpret_cast<const float2*>(hist + g * D + col);
+            if (hist_rows) {
+                const float2 h = *reinterpret_cast<const float2*>(hist_rows + (size_t)row * D + col);
                 x0 += h.x; x1 += h.y;
             }
             *reinterpret_cast<uint32_t*>(o + g * D + col) = pack_bf16(x0, x1);
         }
     }
+}
+
+// hist: optional fp32 [B*H, T_c, D] added to the normalised output before the single rounding to bf16.
+template <int BLK, int D>
+__global__ void __launch_bounds__(SwaMma<BLK, D>::THREADS)
+k_swa_mma(const bf16* __restrict__ q, ChunkTable tab, const int32_t* __restrict__ idx, int keep,
+          int Tc, int n_b, float scale_log2, const float* __restrict__ hist,
+          bf16* __restrict__ o, float* __restrict__ lse, int* dev_status) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int i = blockIdx.x, bh = blockIdx.y;
+    const int unit = bh * gridDim.x + i;
+    swa_mma_unit<BLK, D>(smem, q, tab, idx + (size_t)unit * keep, keep, Tc, n_b, scale_log2,
+                         hist ? hist + ((size_t)bh * Tc + (size_t)i * BLK) * D : nullptr, o, lse, dev_status, i, bh, unit);
 }

@@ -26,8 +26,17 @@
 //                      Q copy once it has been read); then O / l (+ bias) -> bf16 -> shared memory -> bulk tensor store
 // Every wait is bounded (~1 s); on expiry the CTA raises the device status word and leaves through the
 // common exit (drains its copies, frees its TMEM).
+//
+// Range of the fixed reference, and what happens outside it.  Alg. 3 carries a running row maximum so that no input
+// overflows; here the reference is fixed after the first kept tile, which covers rows whose later tiles rise up to about
+// 100 natural-log units above the first one.  A unit with a row beyond that (row sum not finite or above 2^100 at the
+// unit's end -- a complete test: every P is a term of the row sum) is put on a list in shared memory, and when the
+// thread block has finished its tile stream it computes those units again with the running maximum, rescaling l and O as
+// Alg. 3 prints them (swa_redo_unit below: the warp-level code of k_swa_mma.cuh, plus the history term where this kernel
+// forms it), overwriting the rows the fast path left.  The result is therefore the softmax of Eq. 6 for every finite input.
 #pragma once
 #include "tc5_common.cuh"
+#include "k_swa_mma.cuh"
 
 
 template <int D, int NG>
@@ -82,6 +91,10 @@ struct Tc5Params {
     bf16* o;
     float* lse;
     int* dev_status;
+    // for the units that are computed again with a running maximum: the window as plain pointers, and the folded state
+    ChunkTable tab;
+    const bf16* sf_hi;       // [B*H, D, D] bf16 hi / lo halves of S W^T (HIST only)
+    const bf16* sf_lo;
 };
 
 // Ring position of item i in a ring of N stages: stage i % N, completed-phase parity (i / N) & 1, kept incrementally.
@@ -92,6 +105,74 @@ struct RingPos {
     __device__ __forceinline__ void advance() { if (++stage == N) { stage = 0; phase ^= 1u; } }
 };
 
+
+// One unit again, the way Alg. 3 prints it (running maximum m, rescaling of l and O), by threads 0 .. 255 of the thread
+// block, after the tile stream has drained (shared memory and the exchange buffers are free by then).  HIST: the history
+// term of Eq. 4 for the unit's rows is formed first, in fp32 on the CUDA cores, into a shared-memory tile that the
+// attention epilogue adds (Eq. 7).  Slow and rare by design.
+template <int D, bool HIST>
+__device__ __noinline__ void swa_redo_unit(uint8_t* s_gen, const Tc5Params& p, int u) {
+    typedef SwaMma<128, D> M;
+    constexpr int BLK = 128;
+    const int bh = u / p.Tm, i = u - bh * p.Tm;
+    const int q0 = i * BLK, nq = min(BLK, p.Tc - q0);
+    const int tid = threadIdx.x;
+    const float* hist_rows = p.hist ? p.hist + ((size_t)bh * p.Tc + q0) * D : nullptr;
+    asm volatile("bar.sync 1, 256;\n" ::: "memory");      // the previous unit's epilogue has read its history tile
+    if constexpr (HIST) {
+        constexpr int PS = D + 1;                                            // padded row of the phi(Q) tile
+        float* phi_t = reinterpret_cast<float*>(s_gen + M::TILE_BYTES);     // [128][D + 1], in the K / V stages (not yet in use)
+        float* den_t = phi_t + BLK * PS;                                    // [128]
+        float* hist_t = reinterpret_cast<float*>(s_gen + M::SMEM_BYTES);    // [128][D], behind the attention tiles
+        static_assert(M::TILE_BYTES + (BLK * PS + BLK) * 4 <= M::SMEM_BYTES, "phi(Q) tile must fit in the K / V stages");
+        {   // phi(q) of the unit's rows (zero past the chunk's end): thread = (row, half of the features)
+            const int row = tid >> 1, f0 = (tid & 1) * (D / 2);
+            const bf16* src = p.q + ((size_t)bh * p.Tc + q0 + row) * D + f0;
+            for (int c = 0; c < D / 2; c += 8) {
+                uint4 w = make_uint4(0, 0, 0, 0);
+                if (row < nq) w = __ldg(reinterpret_cast<const uint4*>(src + c));
+                const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 x = unpack_bf16(ws[e]);
+                    phi_t[row * PS + f0 + c + 2 * e] = row < nq ? phi_elu1(x.x) : 0.f;
+                    phi_t[row * PS + f0 + c + 2 * e + 1] = row < nq ? phi_elu1(x.y) : 0.f;
+                }
+            }
+        }
+        asm volatile("bar.sync 1, 256;\n" ::: "memory");
+        if (tid < BLK) {        // Eq. 4's denominator phi(q).z + eps, one row per thread
+            float dsum = 0.f;
+            const float* zr = p.z + (size_t)bh * D;
+            for (int a = 0; a < D; ++a) dsum = fmaf(phi_t[tid * PS + a], __ldg(zr + a), dsum);
+            den_t[tid] = dsum + p.eps;
+        }
+        {   // numerator phi(q) S' : thread = (output column, group of rows); S' = hi + lo halves of the folded state
+            constexpr int GROUPS = 256 / D, RPT = BLK / GROUPS;
+            const int c = tid % D, r0 = (tid / D) * RPT;
+            const bf16* sh = p.sf_hi + (size_t)bh * D * D + c;
+            const bf16* sl = p.sf_lo + (size_t)bh * D * D + c;
+            float acc[RPT];
+#pragma unroll
+            for (int r = 0; r < RPT; ++r) acc[r] = 0.f;
+            for (int a = 0; a < D; ++a) {
+                const float sv = __bfloat162float(sh[(size_t)a * D]) + __bfloat162float(sl[(size_t)a * D]);
+#pragma unroll
+                for (int r = 0; r < RPT; ++r) acc[r] = fmaf(phi_t[(r0 + r) * PS + a], sv, acc[r]);
+            }
+            asm volatile("bar.sync 1, 256;\n" ::: "memory");      // denominators written
+            const float b = p.bias ? __bfloat162float(p.bias[(size_t)(bh % p.heads) * D + c]) : 0.f;
+#pragma unroll
+            for (int r = 0; r < RPT; ++r) hist_t[(r0 + r) * D + c] = acc[r] / den_t[r0 + r] + b;
+        }
+        asm volatile("bar.sync 1, 256;\n" ::: "memory");          // tile complete; the K / V stages are free again
+        hist_rows = hist_t;
+    }
+    if (tid == 0) atomicAdd(p.dev_status + 2, 1);                 // count of units that took this path
+    swa_mma_unit<BLK, D>(s_gen, p.q, p.tab, p.idx + (size_t)u * p.keep, p.keep, p.Tc, p.n_b, p.scale_log2, hist_rows, p.o,
+                         p.lse, p.dev_status, i, bh, u);
+}
+
 // Persistent: CTA c processes units c, c + gridDim.x, ...
 // HIST: the history term is formed here (needs SwaTc5::FUSE and the tensor maps of S W^T); otherwise p.hist, if any, is added.
 template <int D, int NG, bool HIST>
@@ -99,7 +180,8 @@ __global__ void __launch_bounds__(SwaTc5<D, NG>::THREADS, 1)
 k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kring,
           const __grid_constant__ CUtensorMap tm_vring, const __grid_constant__ CUtensorMap tm_kcur,
           const __grid_constant__ CUtensorMap tm_vcur, const __grid_constant__ CUtensorMap tm_sh,
-          const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ CUtensorMap tm_o, const Tc5Params p) {
+          const __grid_constant__ CUtensorMap tm_sl, const __grid_constant__ CUtensorMap tm_o,
+          const __grid_constant__ Tc5Params p) {
     using namespace tc5;
     typedef SwaTc5<D, NG> C;
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -123,6 +205,14 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                    bar_h2 = bar0 + 256;                    // ... and its hi tile loaded (after the copy of Q has been read)
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 208);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 212);
+    // units whose rows left the range of the fixed reference: count, last unit listed, up to REDO_CAP local unit numbers
+    // (more than that: every unit of this thread block is computed again)
+    constexpr int REDO_CAP = 8;
+    int* redo_cnt = reinterpret_cast<int*>(s_gen + C::OFF_BAR + 264);
+    int* redo_last = redo_cnt + 1;
+    int* redo_list = redo_cnt + 2;
+    static_assert(264 + (2 + REDO_CAP) * 4 <= 320, "the list must fit in front of the exchange buffers");
+    static_assert(C::THREADS >= 256, "the second pass over a unit needs eight warps");
     float* x_max = reinterpret_cast<float*>(s_gen + C::OFF_XM);          // [2][NG][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -137,6 +227,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_ep, 128 * NG); mbar_init(bar_drain, 1);
         mbar_init(bar_rd, 128 * NG); mbar_init(bar_hf, 1); mbar_init(bar_he, 4 * NG); mbar_init(bar_af, 128 * NG); mbar_init(bar_ud, 1); mbar_init(bar_h2, 1);
         *abort_flag = 0;
+        *redo_cnt = 0; *redo_last = -1;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == C::WARP_MMA) {
@@ -324,6 +415,14 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
         // so every earlier completion of that barrier (tiles t - 5, t - 9, ...) has happened; and P.V of tile t + 3
         // cannot be issued before they have arrived on its P.  The barrier is therefore in completion (t - 1) >> 2 or
         // one past it, and the parity test is exact.
+        // All softmax threads test a unit's row sums between the same two block-wide exchanges, so listings of unit n all
+        // come before any listing of unit n + 1: the exchange on redo_last lets exactly one thread list a unit.
+        auto note_redo = [&](int n) {
+            if (atomicExch(redo_last, n) != n) {
+                const int slot = atomicAdd(redo_cnt, 1);
+                if (slot < REDO_CAP) redo_list[slot] = n;
+            }
+        };
         auto wait_pv_prev = [&](int where) -> bool {
             return __all_sync(0xffffffffu, mbar_wait(bar_pv + 8 * ((t - 1) & 3), ((t - 1) >> 2) & 1, abort_flag, p.dev_status, where));
         };
@@ -496,10 +595,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                 for (int g = 0; g < NG; ++g) { l_run += x_l[g * C::BLK + row]; den += x_d[g * C::BLK + row]; }
                 inv = 1.f / l_run;
-                if (!(l_run < 1e30f)) {     // overflow (or NaN): a later tile rose too far above the first one
-                    atomicOr(p.dev_status, HF_DEV_RANGE_FLAG);
-                    atomicExch(p.dev_status + 1, u);
-                }
+                if (!(l_run < 1e30f)) note_redo(n);     // overflow (or NaN): a later tile rose too far above the first one
                 const float fac = l_run / den;                      // O is divided by l at the end: pre-multiply the history term
                 // the S buffer two tiles on held P of the tile before the unit's last one: its P V must have read it
                 if (t >= 2) {
@@ -544,10 +640,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
                 if (!ok) break;
                 fence_after_sync();
                 inv = 1.f / l_run;
-                if (!(l_run < 1e30f)) {     // overflow (or NaN): a later tile rose too far above the first one
-                    atomicOr(p.dev_status, HF_DEV_RANGE_FLAG);
-                    atomicExch(p.dev_status + 1, u);
-                }
+                if (!(l_run < 1e30f)) note_redo(n);     // overflow (or NaN): a later tile rose too far above the first one
             }
             const bf16* bias_row = (fuse && p.bias) ? p.bias + (size_t)(bh % p.heads) * D : nullptr;
             const size_t g_row = (size_t)bh * p.Tc + q0 + row;
@@ -634,5 +727,16 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
     if (warp == C::WARP_MMA) {
         fence_after_sync();
         tmem_dealloc(tmem, C::TMEM_COLS);
+    }
+    // ---- second pass (rare): the listed units again, with the running maximum.  Every copy and tensor-core operation
+    // of the tile stream has completed (the roles above drain before the barrier), so shared memory is free.
+    const int n_redo = *redo_cnt;
+    if (n_redo > 0 && *abort_flag == 0 && threadIdx.x < 256) {
+        fence_proxy_async();                                  // the tile stream's bulk stores of these rows came first
+        const int total = n_redo > REDO_CAP ? my_units : n_redo;
+        for (int r = 0; r < total; ++r) {
+            const int n = n_redo > REDO_CAP ? r : redo_list[r];
+            swa_redo_unit<D, HIST>(s_gen, p, (int)blockIdx.x + n * (int)gridDim.x);
+        }
     }
 }

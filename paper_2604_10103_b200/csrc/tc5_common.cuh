@@ -33,8 +33,8 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
     return ok != 0;
 }
 // Bounded wait.  Returns false when the limit ran out or another role already gave up.  The polling loop is kept
-// out of line: the common case is a barrier that has already flipped.
-template <bool PARKED>
+// out of line: the common case is a barrier that has already flipped.  LIMIT: clock cycles before the wait gives up.
+template <bool PARKED, long long LIMIT>
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
     const long long t0 = clock64();
     for (;;) {
@@ -48,7 +48,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
                 if (mbar_try_wait(bar, parity)) return true;
         }
         if (*abort_flag) return false;
-        if (clock64() - t0 > WAIT_LIMIT_CYCLES) {
+        if (clock64() - t0 > LIMIT) {
             *abort_flag = 1;
             atomicOr(dev_status, HF_DEV_TIMEOUT_FLAG);
             atomicExch(dev_status + 1, where);
@@ -56,10 +56,10 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
         }
     }
 }
-template <bool PARKED = false>
+template <bool PARKED = false, long long LIMIT = WAIT_LIMIT_CYCLES>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* dev_status, int where) {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow<PARKED>(bar, parity, abort_flag, dev_status, where);
+    return mbar_wait_slow<PARKED, LIMIT>(bar, parity, abort_flag, dev_status, where);
 }
 
 // ----------------------------------------------------------------------------------------- TMA

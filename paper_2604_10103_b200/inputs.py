@@ -18,7 +18,7 @@ from dataclasses import dataclass, replace
 import numpy as np
 
 # tensor ids used in seeds
-T_Q, T_K, T_V, T_KCLEAN, T_VCLEAN, T_W, T_BIAS, T_ANGLE_Q, T_ANGLE_K = range(9)
+T_Q, T_K, T_V, T_KCLEAN, T_VCLEAN, T_W, T_BIAS, T_ANGLE_Q, T_ANGLE_K, T_DIR = range(10)
 
 
 @dataclass(frozen=True)
@@ -163,3 +163,20 @@ def rotation_tables(w: Workload, which: int):
     would supply to the linear branch's rotation.  `which`: T_ANGLE_Q or T_ANGLE_K."""
     th = _rng(w.seed, 0, 0, 0, which).uniform(0.0, 2.0 * np.pi, size=(w.chunk_tokens, w.head_dim // 2))
     return np.cos(th).astype(np.float32), np.sin(th).astype(np.float32)
+
+
+# ---------------------------------------------------------------------------
+# structured draws: peaked attention rows (trained attention maps are concentrated; i.i.d. N(0,1) gives flat ones)
+# ---------------------------------------------------------------------------
+
+def direction(w: Workload, layer: int) -> np.ndarray:
+    """One seeded N(0,1) vector per head, float32 [H, d]: queries and chosen key blocks are shifted along it, which
+    moves the logits of those blocks by (q shift) * (k shift) * |u|^2 / sqrt(d) ~ (q shift) * (k shift) * sqrt(d)."""
+    return _rng(w.seed, layer, 0, 0, T_DIR).standard_normal(size=(w.heads, w.head_dim), dtype=np.float32)
+
+
+def shifted(bits: np.ndarray, u: np.ndarray, amount: float, tokens: slice = slice(None), scale: float = 1.0) -> np.ndarray:
+    """bits [B, H, T, d] -> bf16 bits of (scale * x + amount * u[h]) on the token range `tokens`, x elsewhere."""
+    x = bf16_bits_to_f32(bits).copy()
+    x[:, :, tokens, :] = x[:, :, tokens, :] * np.float32(scale) + np.float32(amount) * u[None, :, None, :]
+    return f32_to_bf16_bits(x)

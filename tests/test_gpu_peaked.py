@@ -1,0 +1,227 @@
+"""GPU parity on PEAKED attention rows: the CUDA library against the CPU oracle on inputs whose logits spread over tens
+of natural-log units (scaled queries, one dominant key block per row, a first kept block far below or far above the
+rest), where the exponent range of P, the exp2 approximation and the softmax reference actually matter.  i.i.d. N(0,1)
+inputs give logits ~ N(0,1) and an almost flat softmax, which hides all of that.
+
+Alg. 3 keeps a running maximum; the tcgen05 kernel fixes the reference after the first kept block and hands the units
+that leave its range to a second pass with the running maximum.  Both must give the softmax of Eq. 6: masks bit-exact,
+outputs max-abs <= 2e-2 and rel-L2 <= 5e-3, on every attention kernel."""
+import numpy as np
+import pytest
+
+from paper_2604_10103_b200 import inputs as gen
+from tests import harness as hz
+
+pytestmark = pytest.mark.gpu
+
+f64 = gen.bf16_bits_to_f64
+KERNELS = [0, 3, 1]          # HF_SWA_AUTO (tcgen05 at 128-token blocks), tcgen05 ping-pong, warp-level
+
+
+def small(d=128, b=128, tpf=300, seed=51, permille=600, heads=2):
+    return gen.Workload("peaked", batch=1, heads=heads, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=3,
+                        block=b, topk=0, keep_permille=permille, seed=seed)
+
+
+def run_stream(w, kernel, make_qkv, make_clean, chunks, q_blocks=None, check_from=0, expect_slow=None):
+    """One forward (selection, O, O_local) + one cache commit per chunk on both sides.  make_qkv(c) / make_clean(c)
+    return bf16 bits.  expect_slow: None = don't care, False = the second pass must not have run, True = it must have."""
+    gpu = hz.GpuStream(w, swa_kernel=kernel); ora = hz.make_oracle(w)
+    worst = (0.0, 0.0)
+    try:
+        for c in range(chunks):
+            qb, kb, vb = make_qkv(c)
+            if c >= check_from:
+                q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+                m_gpu, _, sc_gpu = gpu.select(q, k)
+                m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+                assert np.array_equal(sc_gpu, sc_ref) and np.array_equal(m_gpu, m_ref), f"chunk {c}: selection differs"
+                o_ref, ol_ref, _ = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, q_blocks=q_blocks, parts=True)
+                assert np.isfinite(o_ref[~np.isnan(o_ref)]).all()
+                a = hz.assert_close_out(gpu.forward(q, k, v), o_ref, f"chunk {c} kernel {kernel} hybrid O")
+                b = hz.assert_close_out(gpu.swa(q, k, v), ol_ref, f"chunk {c} kernel {kernel} O_local")
+                worst = (max(worst[0], a[0], b[0]), max(worst[1], a[1], b[1]))
+            kc, vc = make_clean(c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+        slow = gpu.ctx.hf_slow_path_units()
+        if expect_slow is True:
+            assert slow > 0, "the running-maximum pass was expected to run"
+        if expect_slow is False:
+            assert slow == 0, f"{slow} units took the running-maximum pass"
+    finally:
+        gpu.close()
+    return worst
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("scale", [4.0, 8.0])
+def test_scaled_queries(kernel, scale):
+    """q ~ N(0, scale^2): logits with a standard deviation of 4 and 8, a handful of keys carry each row."""
+    w = small()
+    u = gen.direction(w, 0)
+    qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, 0.0, scale=scale), k, v))(*gen.qkv(w, 0, c, 0))
+    run_stream(w, kernel, qkv, lambda c: gen.clean_kv(w, 0, c), 5, expect_slow=False if kernel == 0 else None)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("d,b,amount", [(128, 128, 2.5), (64, 128, 3.0), (128, 64, 2.5), (64, 16, 3.0)])
+def test_newest_blocks_dominate_by_seventy_nats(kernel, d, b, amount):
+    """Queries and the current chunk's keys are shifted along one direction: the row's first kept blocks (older chunks)
+    lie ~70 natural-log units below the current chunk's.  Inside the range of the fixed softmax reference: the tcgen05
+    kernel must handle it in its tile stream."""
+    if kernel != 1 and b != 128:
+        pytest.skip("the tcgen05 kernels are selected by 128-token blocks")
+    w = small(d=d, b=b, tpf=300 if b == 128 else 150)
+    u = gen.direction(w, 0)
+    qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, amount), gen.shifted(k, u, amount), v))(*gen.qkv(w, 0, c, 0))
+    run_stream(w, kernel, qkv, lambda c: gen.clean_kv(w, 0, c), 5, check_from=2, expect_slow=False if kernel == 0 else None)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_oldest_block_dominates_by_sixty_nats(kernel):
+    """The first kept block of every row lies ~60 natural-log units ABOVE all the others: their terms underflow against
+    it and must vanish quietly (no NaN, no effect on the row)."""
+    w = small()
+    u = gen.direction(w, 0)
+    a = 2.3
+    qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, a), k, v))(*gen.qkv(w, 0, c, 0))
+    clean = lambda c: (lambda k, v: (gen.shifted(k, u, a, slice(0, 128)), v))(*gen.clean_kv(w, 0, c))
+    run_stream(w, kernel, qkv, clean, 5, check_from=2, expect_slow=False if kernel == 0 else None)
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("d,amount", [(128, 4.0), (64, 4.8)])
+def test_logits_beyond_the_fixed_reference_take_the_running_maximum_pass(kernel, d, amount):
+    """The current chunk's keys lie ~180 natural-log units above the cached ones: past what a reference fixed at the first
+    kept block covers in fp32.  The tcgen05 kernel must notice, compute those units again with the running maximum and
+    return the oracle's numbers (with and without the history term), with a clean status word."""
+    w = small(d=d, seed=52)
+    u = gen.direction(w, 0)
+    qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, amount), gen.shifted(k, u, amount), v))(*gen.qkv(w, 0, c, 0))
+    run_stream(w, kernel, qkv, lambda c: gen.clean_kv(w, 0, c), 5, check_from=2, expect_slow=True if kernel == 0 else None)
+
+
+def test_many_units_per_thread_block_beyond_the_reference():
+    """More out-of-range units in one thread block than its list holds (it then recomputes all of its units): nine units
+    per thread block, a short last block, bias and merge matrix in the history term.  Only the last two key blocks of the
+    current chunk are shifted, so that every row keeps a low first block beside them."""
+    w = gen.Workload("peaked_many", batch=2, heads=8, head_dim=128, tokens_per_frame=9620, chunk_frames=1, window_frames=2,
+                     block=128, topk=3, keep_permille=0, seed=53)
+    assert w.batch * w.heads * w.blocks_per_chunk > 8 * 148
+    u = gen.direction(w, 0)
+    qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, 4.0), gen.shifted(k, u, 4.0, slice(74 * 128, None)), v))(*gen.qkv(w, 0, c, 0))
+    run_stream(w, 0, qkv, lambda c: gen.clean_kv(w, 0, c), 3, check_from=2, q_blocks=[0, 37, 75], expect_slow=True)
+
+
+def test_a_single_row_beyond_the_reference():
+    """One query row per head is extreme, everything else is N(0,1): only that row's unit takes the second pass and its
+    neighbours keep the fast path's result."""
+    w = small(seed=54)
+    u = gen.direction(w, 0)
+
+    def qkv(c):
+        q, k, v = gen.qkv(w, 0, c, 0)
+        return gen.shifted(q, u, 16.0, slice(200, 201)), gen.shifted(k, u, 1.0), v
+
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        for c in range(3):
+            qb, kb, vb = qkv(c)
+            if c == 2:
+                q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+                m_gpu, _, _ = gpu.select(q, k)
+                m_ref, _ = ora.select(f64(qb), f64(kb))
+                assert np.array_equal(m_gpu, m_ref)
+                before = gpu.ctx.hf_slow_path_units()
+                hz.assert_close_out(gpu.forward(q, k, v), ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref), "one extreme row")
+                assert gpu.ctx.hf_slow_path_units() - before == w.heads      # query block 1 of each head
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
+
+
+def test_constant_tensors_three_hundred_nats_apart():
+    """q = 4, cached keys = -4, current keys = +4 in every component: logits of -181 and +181 in one row."""
+    w = gen.Workload("range", batch=1, heads=1, head_dim=128, tokens_per_frame=256, chunk_frames=1, window_frames=2,
+                     block=128, topk=0, keep_permille=1000, seed=37)
+    shape = (1, 1, 256, 128)
+    qb = gen.f32_to_bf16_bits(np.full(shape, 4.0, dtype=np.float32))
+    k_old = gen.f32_to_bf16_bits(np.full(shape, -4.0, dtype=np.float32))
+    k_new = gen.f32_to_bf16_bits(np.full(shape, 4.0, dtype=np.float32))
+    vb = gen.normal_bf16(shape, 37, 1)
+    for kernel in KERNELS:
+        gpu = hz.GpuStream(w, swa_kernel=kernel); ora = hz.make_oracle(w)
+        try:
+            gpu.append(gpu.up(k_old), gpu.up(vb)); ora.append(f64(k_old), f64(vb))
+            q, k, v = gpu.up(qb), gpu.up(k_new), gpu.up(vb)
+            gpu.select(q, k)
+            m_ref, _ = ora.select(f64(qb), f64(k_new))
+            o_ref, ol_ref, _ = ora.forward(f64(qb), f64(k_new), f64(vb), mask=m_ref, parts=True)
+            hz.assert_close_out(gpu.swa(q, k, v), ol_ref, f"kernel {kernel} O_local")
+            hz.assert_close_out(gpu.forward(q, k, v), o_ref, f"kernel {kernel} hybrid O")
+            assert gpu.ctx.hf_get_device_status() == (0, 0)
+            if kernel == 0:
+                assert gpu.ctx.hf_slow_path_units() == 4        # two query blocks, two calls
+        finally:
+            gpu.close()
+
+
+@pytest.mark.parametrize("mode", ["scaled4_dominant", "beyond"])
+def test_layer_832x480_peaked_rows_on_sampled_query_blocks(mode):
+    """The 832x480 layer shape (12 heads of 128, 4680 queries, 111 key blocks, 28 kept) with peaked rows: queries scaled
+    by 4 and shifted, the keys of the newest chunk's last 17 blocks shifted (dominant by ~45 nats, or by ~180 = beyond the
+    fixed reference; the other kept blocks of a row stay low);
+    all heads, query blocks 0, 17 and the ragged 36."""
+    w = gen.layer_832x480().with_(seed=55)
+    u = gen.direction(w, 0)
+    a = 2.0 if mode == "scaled4_dominant" else 4.0
+    qs = 4.0 if mode == "scaled4_dominant" else 1.0
+    gpu = hz.GpuStream(w); ora = hz.make_oracle(w)
+    try:
+        for c in range(4):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        qb, kb, vb = gen.qkv(w, 0, 4, 0)
+        qb = gen.shifted(qb, u, a, scale=qs); kb = gen.shifted(kb, u, a, slice(20 * 128, None))
+        q, k, v = gpu.up(qb), gpu.up(kb), gpu.up(vb)
+        m_gpu, _, sc_gpu = gpu.select(q, k)
+        m_ref, sc_ref = ora.select(f64(qb), f64(kb))
+        assert np.array_equal(sc_gpu, sc_ref) and np.array_equal(m_gpu, m_ref)
+        o_ref, ol_ref, _ = ora.forward(f64(qb), f64(kb), f64(vb), mask=m_ref, q_blocks=[0, 17, 36], parts=True)
+        hz.assert_close_out(gpu.forward(q, k, v), o_ref, "hybrid O")
+        hz.assert_close_out(gpu.swa(q, k, v), ol_ref, "O_local")
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+        slow = gpu.ctx.hf_slow_path_units()
+        assert (slow == 0) if mode == "scaled4_dominant" else (slow > 0)
+    finally:
+        gpu.close()
+
+
+def test_nan_in_a_query_block_keeps_exactly_k_blocks_and_raises_nothing():
+    """One NaN in q makes that query block's pooled mean, and with it every score of its row, NaN.  The selection must
+    still keep exactly k blocks per row (NaN ranks below every number, ties to the lower index), write nothing outside
+    the row, and the other rows must be what they are without the NaN."""
+    import torch
+    w = small(seed=56)
+    gpu = hz.GpuStream(w)
+    try:
+        for c in range(2):
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc))
+        qb, kb, vb = gen.qkv(w, 0, 2, 0)
+        q, k = gpu.up(qb), gpu.up(kb)
+        m0, idx0, _ = gpu.select(q, k)
+        keep = idx0.shape[-1]
+        q[0, 1, 130, 7] = float("nan")                 # head 1, query block 1
+        m1, idx1, sc1 = gpu.select(q, k)
+        assert np.isnan(sc1[0, 1, 1]).all()
+        assert (m1.sum(axis=-1) == keep).all()
+        assert np.array_equal(idx1[0, 1, 1], np.arange(keep))
+        other = np.ones(m0.shape[:3], dtype=bool); other[0, 1, 1] = False
+        assert np.array_equal(m1[other], m0[other]) and np.array_equal(idx1[other], idx0[other])
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
