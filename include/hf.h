@@ -117,6 +117,25 @@ hf_status hf_kv_append(hf_ctx* ctx, int layer, const void* k, const void* v, voi
 /* Eq. 3 on caller-supplied tokens: k_ev, v_ev bf16 [B,H,n_tokens,d], any n_tokens >= 1. */
 hf_status hf_state_absorb(hf_ctx* ctx, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream);
 
+/* Alg. 2's cache commit for layers first_layer .. first_layer + n_layers - 1 in one call.  In the sampler every layer
+ * commits its clean chunk at the same moment ("if KV full: pop(0) -> update LN; KV.append", once per chunk), and one
+ * layer's 28.75 MB at the 832x480 shape is too small a launch to use the memory system; here the chunks that leave are
+ * folded into their layers' states by ONE persistent launch (Eq. 3; a thread block owns a (layer, batch*head) state for
+ * the whole token range, so there are no partial sums and no second kernel to add them) and the new chunks are copied in
+ * and pooled by one more.
+ *   k, v   HOST arrays of n_layers DEVICE pointers, bf16 [B,H,T_c,d] each (entry l belongs to layer first_layer + l)
+ * Every layer ends up exactly as after hf_kv_append(layer, k[l], v[l]): same cache contents and the same bits in S and
+ * z (the token range is cut and summed in the same order).  Layers of the call that are in different phases of the
+ * protocol (some still filling the window, some evicting), a window of one chunk, or too few (layer, batch*head) pairs
+ * to fill the device are handled layer by layer inside the call. */
+hf_status hf_kv_append_layers(hf_ctx* ctx, int first_layer, int n_layers, const void* const* k, const void* const* v, void* stream);
+
+/* Eq. 3 on caller-supplied tokens for several layers at once: k_ev, v_ev device bf16 [n_layers, B, H, n_tokens, d]
+ * (slice l goes into the state of layer first_layer + l).  Same result, bit for bit, as n_layers calls of
+ * hf_state_absorb. */
+hf_status hf_state_absorb_layers(hf_ctx* ctx, int first_layer, int n_layers, const void* k_ev, const void* v_ev, int n_tokens,
+                                 void* stream);
+
 /* Eq. 5 + top-K rule (Alg. 3: M_c[i,j] = 1 iff block j is among the K best of row i): block means of q and of
  * the window's keys (cached chunks + k_cur), scores in a fixed float32 operation order, per (batch, head, query
  * block) the k_eff highest scores kept, equal scores going to the lower block index.  The selection is kept in

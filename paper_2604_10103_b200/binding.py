@@ -28,7 +28,7 @@ EXPORTS = [
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
     "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
-    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit",
+    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit", "hf_kv_append_layers", "hf_state_absorb_layers",
 ]
 
 
@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
     L.hf_set_rope.argtypes = [vp, vp, vp, vp, vp, vp]
     L.hf_kv_append.argtypes = [vp, ip, vp, vp, vp]
     L.hf_state_absorb.argtypes = [vp, ip, vp, vp, ip, vp]
+    L.hf_state_absorb_layers.argtypes = [vp, ip, ip, vp, vp, ip, vp]
+    L.hf_kv_append_layers.argtypes = [vp, ip, ip, C.POINTER(vp), C.POINTER(vp), vp]
     L.hf_block_select.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp]
     L.hf_sparse_swa.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp, vp]
     L.hf_linear_attn.argtypes = [vp, ip, vp, vp, vp]
@@ -148,6 +150,17 @@ class Context:
 
     def hf_kv_append(self, layer, k, v):
         _check(lib().hf_kv_append(self._h, layer, _ptr(k), _ptr(v), _stream()))
+
+    def hf_kv_append_layers(self, first_layer, ks, vs):
+        """ks, vs: sequences of bf16 CUDA tensors [B,H,T_c,d], one per layer from first_layer on."""
+        n = len(ks)
+        ka = (C.c_void_p * n)(*[t.data_ptr() for t in ks])
+        va = (C.c_void_p * n)(*[t.data_ptr() for t in vs])
+        _check(lib().hf_kv_append_layers(self._h, first_layer, n, ka, va, _stream()))
+
+    def hf_state_absorb_layers(self, first_layer, n_layers, k_ev, v_ev, n_tokens):
+        """k_ev, v_ev: bf16 CUDA tensors [n_layers, B, H, n_tokens, d]."""
+        _check(lib().hf_state_absorb_layers(self._h, first_layer, n_layers, _ptr(k_ev), _ptr(v_ev), n_tokens, _stream()))
 
     def hf_state_absorb(self, layer, k_ev, v_ev, n_tokens):
         _check(lib().hf_state_absorb(self._h, layer, _ptr(k_ev), _ptr(v_ev), n_tokens, _stream()))

@@ -7,6 +7,7 @@
 #include "k_swa_tc5p.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
+#include "k_state_items.cuh"
 #include "k_merge_full.cuh"
 #include "k_selftest.cuh"
 
@@ -69,6 +70,19 @@ struct hf_ctx {
     int n_sink_max = 0;              // sink chunks of the configuration; ring (R = P + 1 slots: the window's P past chunks and a spare) and sink share one allocation
     size_t chunk_elems = 0, pooled_elems = 0;
     std::vector<LayerState> layers;
+    // One allocation per kind for all layers (layer-major; the LayerState pointers point into them), so that a single
+    // launch can address every layer: the layer-batched cache commit and state update.
+    bf16* ring_k_all = nullptr;      // [layers][slots_per_layer][B*H*T_c*d]
+    bf16* ring_v_all = nullptr;
+    float* pooled_k_all = nullptr;   // [layers][slots_per_layer][B*H*n_b*d]
+    float* S_all = nullptr;          // [layers][B*H, d, d]
+    float* z_all = nullptr;          // [layers][B*H, d]
+    bf16* sf_hi_all = nullptr;       // [layers][B*H, d, d]
+    bf16* sf_lo_all = nullptr;
+    bf16* W_all = nullptr;           // [layers][H, d, d] (HF_MERGE_PER_HEAD)
+    bf16* bias_all = nullptr;        // [layers][H, d]
+    int slots_per_layer = 0;         // ring slots + sink slots
+    CUtensorMap tm_kall, tm_vall;    // the state-update kernels' views of all rings: [d, T_c, B*H, layers * slots_per_layer]
     float* pooled_q = nullptr;
     float* pooled_kcur = nullptr;
     float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
@@ -152,10 +166,9 @@ hf_status dmalloc(T** p, size_t count) {
 }
 
 void free_all(hf_ctx* c) {
-    for (auto& L : c->layers) {
-        cudaFree(L.ring_k); cudaFree(L.ring_v); cudaFree(L.pooled_k); cudaFree(L.S); cudaFree(L.z);
-        cudaFree(L.sf_hi); cudaFree(L.sf_lo); cudaFree(L.W); cudaFree(L.W_full); cudaFree(L.bias); cudaFree(L.mask); cudaFree(L.idx);
-    }
+    for (auto& L : c->layers) { cudaFree(L.W_full); cudaFree(L.mask); cudaFree(L.idx); }
+    cudaFree(c->ring_k_all); cudaFree(c->ring_v_all); cudaFree(c->pooled_k_all); cudaFree(c->S_all); cudaFree(c->z_all);
+    cudaFree(c->sf_hi_all); cudaFree(c->sf_lo_all); cudaFree(c->W_all); cudaFree(c->bias_all);
     cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
@@ -176,6 +189,8 @@ hf_status set_state_attr() {
     HF_CUDA(cudaFuncSetAttribute(k_absorb_tc5<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbTc5<D>::SMEM_BYTES));
     HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
     HF_CUDA(cudaFuncSetAttribute(k_readout_tc5<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ReadoutTc5<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_items<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbItems<D>::SMEM_BYTES));
+    HF_CUDA(cudaFuncSetAttribute(k_absorb_items<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AbsorbItems<D>::SMEM_BYTES));
     return HF_OK;
 }
 
@@ -269,6 +284,44 @@ hf_status launch_absorb(hf_ctx* c, LayerState& L, const bf16* k, const bf16* v, 
     HF_TRY(launch_fold<D>(c, L, nsplit, run));
     if (on_side) HF_CUDA(cudaEventRecord(c->ev_join, c->side));
     return HF_OK;
+}
+
+// Eq. 3 for n_layers layers (first_layer ..) in one persistent launch, then their folded states in a second, small one.
+// tk / tv: the kernel's views of the tokens ([d, n_tokens, B*H, slots]); slot[l]: coordinate 3 of layer l of the call.
+// The splits of an item's token range and their order are those of launch_absorb, so S and z get the same bits.
+template <int D>
+hf_status launch_absorb_layers(hf_ctx* c, int first_layer, int n_layers, const CUtensorMap& tk, const CUtensorMap& tv,
+                               const int* slot, int n_tokens, cudaStream_t st) {
+    typedef AbsorbItems<D> A;
+    const size_t dd = (size_t)c->BH * D * D, dz = (size_t)c->BH * D;
+    const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
+    AbsorbItemsParams p;
+    memset(&p, 0, sizeof(p));
+    p.n_tokens = n_tokens; p.BH = c->BH; p.n_items = n_layers * c->BH;
+    p.nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
+    p.z_scale = c->z_scale;
+    p.S = c->S_all + (size_t)first_layer * dd; p.z = c->z_all + (size_t)first_layer * dz;
+    for (int l = 0; l < n_layers; ++l) p.slot[l] = slot[l];
+    p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc; p.dev_status = c->dev_status;
+    const int grid = p.n_items < c->sm_count ? p.n_items : c->sm_count;
+    PdlLaunch pl(dim3(grid), dim3(A::THREADS), A::SMEM_BYTES, st, false);
+    if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, true>, tk, tv, p));
+    else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, false>, tk, tv, p));
+    HF_TRY(post_launch(c, "k_absorb_items"));
+    unsigned long long has_w = 0;
+    for (int l = 0; l < n_layers; ++l) if (c->layers[first_layer + l].has_w) has_w |= 1ull << l;
+    PdlLaunch pf(dim3(D / 4, c->BH, n_layers), dim3(D), 0, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_fold_layers<D>, (const float*)p.S,
+                               (const bf16*)(c->W_all ? c->W_all + (size_t)first_layer * c->cfg.heads * D * D : nullptr), c->cfg.heads,
+                               c->BH, c->sf_hi_all + (size_t)first_layer * dd, c->sf_lo_all + (size_t)first_layer * dd, has_w));
+    return post_launch(c, "k_fold_layers");
+}
+
+template <int D>
+hf_status launch_pool_layers(hf_ctx* c, const PoolLayersParams& p, int n_layers, cudaStream_t st) {
+    PdlLaunch pl(dim3(c->n_b, c->BH, 2 * n_layers), dim3(256), 0, st, false);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_pool_copy_layers<D>, p, c->Tc, c->cfg.block, c->n_b));
+    return post_launch(c, "k_pool_copy_layers");
 }
 
 template <int D>
@@ -517,17 +570,34 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     hf_status s = HF_OK;
     c->layers.resize(cfg->layers);
     const size_t dd = (size_t)c->BH * c->d * c->d, dz = (size_t)c->BH * c->d;
-    for (auto& L : c->layers) {
-        const size_t slots = (size_t)c->R + c->n_sink_max;      // ring slots, then sink slots
-        if (s == HF_OK) s = dmalloc(&L.ring_k, slots * c->chunk_elems);
-        if (s == HF_OK) s = dmalloc(&L.ring_v, slots * c->chunk_elems);
-        if (s == HF_OK) s = dmalloc(&L.pooled_k, slots * c->pooled_elems);
-        if (s == HF_OK) s = dmalloc(&L.S, dd);
-        if (s == HF_OK) s = dmalloc(&L.z, dz);
-        if (s == HF_OK) s = dmalloc(&L.sf_hi, dd);
-        if (s == HF_OK) s = dmalloc(&L.sf_lo, dd);
-        if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&L.W, (size_t)cfg->heads * c->d * c->d);
-        if (s == HF_OK && cfg->merge != HF_MERGE_IDENTITY) s = dmalloc(&L.bias, (size_t)cfg->heads * c->d);
+    const size_t slots = (size_t)c->R + c->n_sink_max;          // per layer: ring slots, then sink slots
+    const size_t nl = (size_t)cfg->layers, wd = (size_t)cfg->heads * c->d * c->d, bd = (size_t)cfg->heads * c->d;
+    c->slots_per_layer = (int)slots;
+    if (nl * slots > 0x7fffffffull) { delete c; return fail(HF_ERR_SHAPE, "layers x cache slots too large"); }
+    if (s == HF_OK) s = dmalloc(&c->ring_k_all, nl * slots * c->chunk_elems);
+    if (s == HF_OK) s = dmalloc(&c->ring_v_all, nl * slots * c->chunk_elems);
+    if (s == HF_OK) s = dmalloc(&c->pooled_k_all, nl * slots * c->pooled_elems);
+    if (s == HF_OK) s = dmalloc(&c->S_all, nl * dd);
+    if (s == HF_OK) s = dmalloc(&c->z_all, nl * dz);
+    if (s == HF_OK) s = dmalloc(&c->sf_hi_all, nl * dd);
+    if (s == HF_OK) s = dmalloc(&c->sf_lo_all, nl * dd);
+    if (s == HF_OK && cfg->merge == HF_MERGE_PER_HEAD) s = dmalloc(&c->W_all, nl * wd);
+    if (s == HF_OK && cfg->merge != HF_MERGE_IDENTITY) s = dmalloc(&c->bias_all, nl * bd);
+    if (s == HF_OK) {
+        cudaMemset(c->S_all, 0, nl * dd * 4); cudaMemset(c->z_all, 0, nl * dz * 4);
+        cudaMemset(c->sf_hi_all, 0, nl * dd * 2); cudaMemset(c->sf_lo_all, 0, nl * dd * 2);
+    }
+    if (s == HF_OK && slots > 0) s = make_map_ex(c, &c->tm_kall, c->ring_k_all, c->Tc, (int)(nl * slots), c->d, 64, false);
+    if (s == HF_OK && slots > 0) s = make_map_ex(c, &c->tm_vall, c->ring_v_all, c->Tc, (int)(nl * slots), 64, 64, true);
+    for (size_t li = 0; s == HF_OK && li < nl; ++li) {
+        LayerState& L = c->layers[li];
+        L.ring_k = slots ? c->ring_k_all + li * slots * c->chunk_elems : nullptr;
+        L.ring_v = slots ? c->ring_v_all + li * slots * c->chunk_elems : nullptr;
+        L.pooled_k = slots ? c->pooled_k_all + li * slots * c->pooled_elems : nullptr;
+        L.S = c->S_all + li * dd; L.z = c->z_all + li * dz;
+        L.sf_hi = c->sf_hi_all + li * dd; L.sf_lo = c->sf_lo_all + li * dd;
+        L.W = c->W_all ? c->W_all + li * wd : nullptr;
+        L.bias = c->bias_all ? c->bias_all + li * bd : nullptr;
         if (s == HF_OK && cfg->merge == HF_MERGE_FULL_WIDTH) {
             const size_t hd = (size_t)cfg->heads * c->d;
             s = dmalloc(&L.W_full, hd * hd);
@@ -549,9 +619,6 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_vring, L.ring_v, (int)slots);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sfhi, L.sf_hi, c->d, 1, 64, c->d, true);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sflo, L.sf_lo, c->d, 1, 64, c->d, true);
-        if (s != HF_OK) break;
-        cudaMemset(L.S, 0, dd * 4); cudaMemset(L.z, 0, dz * 4);
-        cudaMemset(L.sf_hi, 0, dd * 2); cudaMemset(L.sf_lo, 0, dd * 2);
     }
     if (s == HF_OK) s = dmalloc(&c->pooled_q, c->pooled_elems);
     if (s == HF_OK) s = dmalloc(&c->pooled_kcur, c->pooled_elems);
@@ -721,6 +788,98 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
     if (evicted) HF_CUDA(cudaStreamWaitEvent(st, c->ev_join, 0));
     L.cache_epoch++;
+    return HF_OK;
+}
+
+hf_status hf_state_absorb_layers(hf_ctx* c, int first_layer, int n_layers, const void* k_ev, const void* v_ev, int n_tokens,
+                                 void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    if (n_layers < 1 || first_layer < 0 || first_layer + n_layers > c->cfg.layers)
+        return fail(HF_ERR_INVALID_ARG, "layers [%d, %d) outside [0, %d)", first_layer, first_layer + n_layers, c->cfg.layers);
+    HF_TRY(check_ptr(k_ev, "k_ev"));
+    HF_TRY(check_ptr(v_ev, "v_ev"));
+    if (n_tokens < 1) return fail(HF_ERR_SHAPE, "n_tokens must be >= 1");
+    if (c->has_rope_k && n_tokens > c->Tc)
+        return fail(HF_ERR_SHAPE, "with rotation tables set, n_tokens may not exceed the chunk length (%d)", c->Tc);
+    if (c->cfg.z_mode == HF_Z_FRAME_MEAN && n_tokens % c->cfg.tokens_per_frame != 0)
+        return fail(HF_ERR_SHAPE, "with HF_Z_FRAME_MEAN n_tokens must be a multiple of tokens_per_frame (%d)", c->cfg.tokens_per_frame);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t per_layer = (size_t)c->BH * n_tokens * c->d;
+    // One persistent launch pays when there are at least as many (layer, batch*head) items as SMs; below that the
+    // per-layer kernel, which cuts every item over several thread blocks, fills the device better.  Same bits either way.
+    if ((long long)n_layers * c->BH < c->sm_count) {
+        for (int l = 0; l < n_layers; ++l)
+            HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, c->layers[first_layer + l], (const bf16*)k_ev + l * per_layer,
+                                 (const bf16*)v_ev + l * per_layer, n_tokens, st));
+    } else {
+        for (int l0 = 0; l0 < n_layers; l0 += HF_MAX_BATCH_LAYERS) {
+            const int nl = n_layers - l0 < HF_MAX_BATCH_LAYERS ? n_layers - l0 : HF_MAX_BATCH_LAYERS;
+            CUtensorMap tk, tv;
+            HF_TRY(make_map_ex(c, &tk, (const bf16*)k_ev + l0 * per_layer, n_tokens, nl, c->d, 64, false));
+            HF_TRY(make_map_ex(c, &tv, (const bf16*)v_ev + l0 * per_layer, n_tokens, nl, 64, 64, true));
+            int slot[HF_MAX_BATCH_LAYERS];
+            for (int l = 0; l < nl; ++l) slot[l] = l;
+            HF_TRY(HF_DISPATCH_D(c, launch_absorb_layers, c, first_layer + l0, nl, tk, tv, slot, n_tokens, st));
+        }
+    }
+    for (int l = 0; l < n_layers; ++l) c->layers[first_layer + l].absorbed += n_tokens;
+    return HF_OK;
+}
+
+hf_status hf_kv_append_layers(hf_ctx* c, int first_layer, int n_layers, const void* const* k, const void* const* v, void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    if (n_layers < 1 || first_layer < 0 || first_layer + n_layers > c->cfg.layers)
+        return fail(HF_ERR_INVALID_ARG, "layers [%d, %d) outside [0, %d)", first_layer, first_layer + n_layers, c->cfg.layers);
+    if (k == nullptr || v == nullptr) return fail(HF_ERR_INVALID_ARG, "pointer table is null");
+    for (int l = 0; l < n_layers; ++l) {
+        HF_TRY(check_ptr(k[l], "k[layer]"));
+        HF_TRY(check_ptr(v[l], "v[layer]"));
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    // The batched launches need every layer of the call in the same phase of Alg. 2's protocol (all still filling their
+    // sink, all filling the window, or all evicting) and enough (layer, batch*head) items to fill the device; anything
+    // else goes layer by layer.  The state gets the same bits either way.
+    const LayerState& L0 = c->layers[first_layer];
+    bool uniform = c->P > 0 && n_layers <= HF_MAX_BATCH_LAYERS && (long long)n_layers * c->BH >= c->sm_count;
+    for (int l = 1; uniform && l < n_layers; ++l) {
+        const LayerState& L = c->layers[first_layer + l];
+        uniform = (L.n_sink < c->n_sink_max) == (L0.n_sink < c->n_sink_max) && (L.n_cached == c->P) == (L0.n_cached == c->P);
+    }
+    if (!uniform) {
+        for (int l = 0; l < n_layers; ++l) HF_TRY(hf_kv_append(c, first_layer + l, k[l], v[l], stream));
+        return HF_OK;
+    }
+    PoolLayersParams pp;
+    memset(&pp, 0, sizeof(pp));
+    pp.chunk_elems = c->chunk_elems; pp.pooled_elems = c->pooled_elems; pp.slots_per_layer = c->slots_per_layer;
+    pp.ring_k = c->ring_k_all + (size_t)first_layer * c->slots_per_layer * c->chunk_elems;
+    pp.ring_v = c->ring_v_all + (size_t)first_layer * c->slots_per_layer * c->chunk_elems;
+    pp.pooled = c->pooled_k_all + (size_t)first_layer * c->slots_per_layer * c->pooled_elems;
+    const bool sink = L0.n_sink < c->n_sink_max, evict = !sink && L0.n_cached == c->P;
+    int ev_slot[HF_MAX_BATCH_LAYERS];
+    for (int l = 0; l < n_layers; ++l) {
+        LayerState& L = c->layers[first_layer + l];
+        pp.k_src[l] = (const bf16*)k[l]; pp.v_src[l] = (const bf16*)v[l];
+        pp.slot[l] = sink ? c->R + L.n_sink : (L.head + L.n_cached) % c->R;
+        ev_slot[l] = (first_layer + l) * c->slots_per_layer + L.head;
+    }
+    if (evict) {
+        // as in hf_kv_append: the state update of the chunks that leave runs on the side stream beside the copy of the new
+        // ones (which go to the spare slots), and the call joins the two
+        HF_CUDA(cudaEventRecord(c->ev_fork, st));
+        HF_CUDA(cudaStreamWaitEvent(c->side, c->ev_fork, 0));
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb_layers, c, first_layer, n_layers, c->tm_kall, c->tm_vall, ev_slot, c->Tc, c->side));
+        HF_CUDA(cudaEventRecord(c->ev_join, c->side));
+    }
+    HF_TRY(HF_DISPATCH_D(c, launch_pool_layers, c, pp, n_layers, st));
+    if (evict) HF_CUDA(cudaStreamWaitEvent(st, c->ev_join, 0));
+    for (int l = 0; l < n_layers; ++l) {
+        LayerState& L = c->layers[first_layer + l];
+        if (sink) L.n_sink++;
+        else if (evict) { L.absorbed += c->Tc; L.head = (L.head + 1) % c->R; }
+        else L.n_cached++;
+        L.cache_epoch++;
+    }
     return HF_OK;
 }
 

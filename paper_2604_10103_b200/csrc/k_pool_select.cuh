@@ -31,15 +31,12 @@ struct PoolJob {            // one tensor to pool (and optionally copy) per bloc
 };
 struct PoolJobs { PoolJob job[3]; };
 
-// grid (n_b, B*H, jobs), 256 threads: 16 threads per token row, 16 rows per pass.
+// One block of one tensor: copy (optional) and per-column mean in the canonical order.  256 threads: 16 threads per token
+// row, 16 rows per pass.
 template <int D>
-__global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
+__device__ __forceinline__ void pool_copy_block(const PoolJob& jb, int Tc, int blk, int n_b, int b_idx, int bh) {
     constexpr int VEC = D / 16;
     typedef typename VecLoad<VEC>::T V;
-    pdl_wait();                 // launched under the tail of the kernel before it: that kernel's reads and writes are done from here on
-    pdl_trigger();              // a dependent kernel (the selection) may be made resident; it waits for this grid itself
-    const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
-    const int b_idx = blockIdx.x, bh = blockIdx.y;
     const int t0 = b_idx * blk;
     const int n = min(blk, Tc - t0);
     const int r = threadIdx.x >> 4, cv = threadIdx.x & 15;
@@ -87,6 +84,42 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int
         for (int rr = 1; rr < 16; ++rr) tot = __fadd_rn(tot, part[rr][threadIdx.x]);
         jb.pooled[((size_t)bh * n_b + b_idx) * D + threadIdx.x] = __fdiv_rn(tot, (float)n);
     }
+}
+
+// grid (n_b, B*H, jobs), 256 threads.
+template <int D>
+__global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int blk, int n_b) {
+    pdl_wait();                 // launched under the tail of the kernel before it: that kernel's reads and writes are done from here on
+    pdl_trigger();              // a dependent kernel (the selection) may be made resident; it waits for this grid itself
+    const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
+    pool_copy_block<D>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y);
+}
+
+// The cache commit of several layers in one launch (Alg. 2 "KV.append" for every layer of the model): per layer the
+// clean chunk's K (copied, block means stored) and V (copied) go to the ring slot slot[l] of that layer.
+// grid (n_b, B*H, 2 * layers): blockIdx.z = 2 * layer + (0: K, 1: V).
+struct PoolLayersParams {
+    const bf16* k_src[64];      // per layer of the call: [B*H, T_c, d]
+    const bf16* v_src[64];
+    int slot[64];               // target slot within the layer's ring
+    bf16* ring_k;               // first layer of the call: [layers][slots_per_layer][B*H, T_c, d]
+    bf16* ring_v;
+    float* pooled;              // [layers][slots_per_layer][B*H, n_b, d]
+    size_t chunk_elems, pooled_elems;
+    int slots_per_layer;
+};
+template <int D>
+__global__ void __launch_bounds__(256, 6) k_pool_copy_layers(const __grid_constant__ PoolLayersParams p, int Tc, int blk, int n_b) {
+    pdl_wait();
+    pdl_trigger();
+    const int lay = blockIdx.z >> 1;
+    const bool is_v = blockIdx.z & 1;
+    const size_t s = (size_t)lay * p.slots_per_layer + p.slot[lay];
+    PoolJob jb;
+    jb.src = is_v ? p.v_src[lay] : p.k_src[lay];
+    jb.copy_dst = (is_v ? p.ring_v : p.ring_k) + s * p.chunk_elems;
+    jb.pooled = is_v ? nullptr : p.pooled + s * p.pooled_elems;
+    pool_copy_block<D>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y);
 }
 
 // A[i][j] = Mean(q_i) . Mean(k_j) in the canonical order, formed by one warp: 32 partials (partial l = columns l,

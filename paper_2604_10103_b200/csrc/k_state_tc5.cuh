@@ -35,6 +35,51 @@ struct AbsorbTc5 {
     static constexpr int PART_FLOATS = D * D + D;
 };
 
+
+// phi(K) of one 64-token tile for one key feature (= TMEM lane) and one quarter of the tile's tokens: evaluated in fp32,
+// split into bf16 hi + lo halves, stored as the A operand (M = feature, K = token) at tA (hi: 32 columns, lo: the next
+// 32); the unrotated values are added to zacc.  k_tile: the tile in shared memory, row-major [token][D], not swizzled.
+// Shared by the split kernel and the layer-batched kernel so that both form the same bits.
+template <int D, bool ROPE>
+__device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tokens, int tile_row0, int part, int a, uint32_t tA_buf,
+                                                const float* cos_k, const float* sin_k, int rope_rows, float& zacc) {
+    typedef AbsorbTc5<D> C;
+    constexpr int HT = C::TT / C::NQ;                       // tokens per thread and tile
+    // rows past the end of the tensor read as zero: phi(0) = 1 must not count
+    const int nv = min(C::TT, n_tokens - tile_row0) - part * HT;
+    const uint8_t* kt = k_tile + (size_t)(part * HT) * D * 2 + a * 2;
+    uint32_t hi[HT / 2], lo[HT / 2];
+#pragma unroll
+    for (int t = 0; t < HT; t += 2) {
+        const float x0 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)t * D * 2)) << 16);
+        const float x1 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)(t + 1) * D * 2)) << 16);
+        float f0 = phi_elu1(x0), f1 = phi_elu1(x1);
+        if (nv < HT) {                              // only the tensor's last tile
+            if (t >= nv) f0 = 0.f;
+            if (t + 1 >= nv) f1 = 0.f;
+        }
+        zacc += f0 + f1;                            // the normaliser keeps the unrotated values
+        if (ROPE) {
+            // feature pairs (2i, 2i+1) sit in neighbouring lanes; the pair's angle belongs to the token
+            const float g0 = __shfl_xor_sync(0xffffffffu, f0, 1), g1 = __shfl_xor_sync(0xffffffffu, f1, 1);
+            const int tok = tile_row0 + part * HT + t;     // rows past the tables belong to masked tokens
+            const size_t o0 = (size_t)min(tok, rope_rows - 1) * (D / 2) + (a >> 1);
+            const size_t o1 = (size_t)min(tok + 1, rope_rows - 1) * (D / 2) + (a >> 1);
+            const float c0 = __ldg(cos_k + o0), s0 = __ldg(sin_k + o0);
+            const float c1 = __ldg(cos_k + o1), s1 = __ldg(sin_k + o1);
+            f0 = (a & 1) ? fmaf(g0, s0, f0 * c0) : fmaf(-g0, s0, f0 * c0);
+            f1 = (a & 1) ? fmaf(g1, s1, f1 * c1) : fmaf(-g1, s1, f1 * c1);
+        }
+        const uint32_t hp = pack_bf16(f0, f1);
+        const float2 hf = unpack_bf16(hp);
+        hi[t >> 1] = hp;
+        lo[t >> 1] = pack_bf16(f0 - hf.x, f1 - hf.y);
+    }
+    const uint32_t tA = tA_buf + part * (HT / 2);
+    tc5::tmem_st8(tA, hi);
+    tc5::tmem_st8(tA + 32, lo);
+}
+
 struct AbsorbTc5Params {
     const float* cos_k;       // rotation tables of Eq. 3, [rope_rows, D/2] each (used by the ROPE instantiation only)
     const float* sin_k;
@@ -157,39 +202,8 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
                 fence_after_sync();
             }
             if (active) {
-                // rows past the end of the tensor read as zero: phi(0) = 1 must not count
-                const int nv = min(C::TT, p.n_tokens - (tile_lo + i) * C::TT) - part * HT;
-                const uint8_t* kt = s_gen + C::OFF_K + s * C::K_BYTES + (size_t)(part * HT) * D * 2 + a * 2;
-                uint32_t hi[HT / 2], lo[HT / 2];
-#pragma unroll
-                for (int t = 0; t < HT; t += 2) {
-                    const float x0 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)t * D * 2)) << 16);
-                    const float x1 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)(t + 1) * D * 2)) << 16);
-                    float f0 = phi_elu1(x0), f1 = phi_elu1(x1);
-                    if (nv < HT) {                              // only the tensor's last tile
-                        if (t >= nv) f0 = 0.f;
-                        if (t + 1 >= nv) f1 = 0.f;
-                    }
-                    zacc += f0 + f1;                            // the normaliser keeps the unrotated values
-                    if (ROPE) {
-                        // feature pairs (2i, 2i+1) sit in neighbouring lanes; the pair's angle belongs to the token
-                        const float g0 = __shfl_xor_sync(0xffffffffu, f0, 1), g1 = __shfl_xor_sync(0xffffffffu, f1, 1);
-                        const int tok = (tile_lo + i) * C::TT + part * HT + t;     // rows past the tables belong to masked tokens
-                        const size_t o0 = (size_t)min(tok, p.rope_rows - 1) * (D / 2) + (a >> 1);
-                        const size_t o1 = (size_t)min(tok + 1, p.rope_rows - 1) * (D / 2) + (a >> 1);
-                        const float c0 = __ldg(p.cos_k + o0), s0 = __ldg(p.sin_k + o0);
-                        const float c1 = __ldg(p.cos_k + o1), s1 = __ldg(p.sin_k + o1);
-                        f0 = (a & 1) ? fmaf(g0, s0, f0 * c0) : fmaf(-g0, s0, f0 * c0);
-                        f1 = (a & 1) ? fmaf(g1, s1, f1 * c1) : fmaf(-g1, s1, f1 * c1);
-                    }
-                    const uint32_t hp = pack_bf16(f0, f1);
-                    const float2 hf = unpack_bf16(hp);
-                    hi[t >> 1] = hp;
-                    lo[t >> 1] = pack_bf16(f0 - hf.x, f1 - hf.y);
-                }
-                const uint32_t tA = lane_base + C::COL_A + ab * 64 + part * (HT / 2);
-                tmem_st8(tA, hi);
-                tmem_st8(tA + 32, lo);
+                absorb_phi_tile<D, ROPE>(s_gen + C::OFF_K + s * C::K_BYTES, p.n_tokens, (tile_lo + i) * C::TT, part, a,
+                                         lane_base + C::COL_A + ab * 64, p.cos_k, p.sin_k, p.rope_rows, zacc);
                 tmem_wait_st();
                 fence_before_sync();
                 mbar_arrive(bar_afull + 8 * ab);
