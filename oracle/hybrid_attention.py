@@ -18,7 +18,7 @@ What follows which passage:
   block_means_f32, block_scores_f32   Eq. 5 in the canonical float32 order
   keep_count, select_blocks         top-K rule after Eq. 5 / Alg. 3 "M_c[i,j] = 1 if in TopK(P_c[i,:], K)"
   sparse_attention        Eq. 6 as its plain definition: softmax over the kept keys
-  sparse_attention_tiled  Alg. 3 inner loops (running max / sum / rescale), step by step
+  sparse_attention_blockwise  the same result as a mixture of per-block softmaxes (the identity behind Alg. 3's tiling)
   absorb                  Eq. 3 (state update) without the rotation
   absorb_frame_mean       Eq. 3 with H accumulated as printed: per evicted frame the mean of phi(K) over its tokens
   linear_readout          Eq. 4: Linear(phi(Q) L / (phi(Q) H)), optionally with RoPE(phi(Q)) in the numerator
@@ -185,30 +185,30 @@ def sparse_attention(q, k_chunks, v_chunks, b: int, mask: np.ndarray, q_blocks=N
     return out
 
 
-def sparse_attention_tiled(q, k_chunks, v_chunks, b: int, mask: np.ndarray) -> np.ndarray:
-    """O_local by the tile recurrence of Alg. 3: m = -inf, l = 0, O = 0, then for each kept block
-    S = q_i k_j^T / sqrt(d); m' = max(m, rowmax S); P = exp(S - m'); l = e^{m-m'} l + rowsum P;
-    O = diag(e^{m-m'}) O + P v_j; finally O / l."""
+def sparse_attention_blockwise(q, k_chunks, v_chunks, b: int, mask: np.ndarray) -> np.ndarray:
+    """O_local a second way, as a witness for sparse_attention: every kept key block on its own first -- its softmax-weighted
+    average of V rows and the log of its sum of exponentials -- then the blocks of a row combined with the weights
+    exp(lse_block - lse_row).  This is the identity that lets Alg. 3 walk the kept blocks one tile at a time (a softmax
+    over a union of blocks is the lse-weighted mixture of the per-block softmaxes); nothing is carried from block to block."""
     q = np.asarray(q, np.float64)
     d = q.shape[1]
     table = key_block_table([kc.shape[0] for kc in k_chunks], b)
     out = np.zeros((q.shape[0], v_chunks[0].shape[1]))
     for i, (qs, qe) in enumerate(block_ranges(q.shape[0], b)):
         qi = q[qs:qe]
-        m = np.full(qi.shape[0], -np.inf)
-        l = np.zeros(qi.shape[0])
-        o = np.zeros((qi.shape[0], out.shape[1]))
+        block_out, block_lse = [], []
         for j, (c, s, e) in enumerate(table):
             if not mask[i, j]:
                 continue
-            S = qi @ np.asarray(k_chunks[c][s:e], np.float64).T / math.sqrt(d)
-            m_new = np.maximum(m, S.max(axis=1))
-            P = np.exp(S - m_new[:, None])
-            alpha = np.exp(m - m_new)
-            l = alpha * l + P.sum(axis=1)
-            o = alpha[:, None] * o + P @ np.asarray(v_chunks[c][s:e], np.float64)
-            m = m_new
-        out[qs:qe] = o / l[:, None]
+            logits = qi @ np.asarray(k_chunks[c][s:e], np.float64).T / math.sqrt(d)
+            top = logits.max(axis=1, keepdims=True)
+            w = np.exp(logits - top)
+            block_out.append((w @ np.asarray(v_chunks[c][s:e], np.float64)) / w.sum(axis=1, keepdims=True))
+            block_lse.append(top[:, 0] + np.log(w.sum(axis=1)))
+        lse = np.stack(block_lse)                               # [kept, rows]
+        row_lse = lse.max(axis=0) + np.log(np.exp(lse - lse.max(axis=0)).sum(axis=0))
+        share = np.exp(lse - row_lse)                           # sums to one over the kept blocks
+        out[qs:qe] = sum(share[n][:, None] * block_out[n] for n in range(len(block_out)))
     return out
 
 

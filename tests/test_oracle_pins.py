@@ -160,7 +160,7 @@ def test_sparse_attention_equals_brute_force_masked_softmax(b, lens):
     ref = brute_masked_attention(q, np.concatenate(kc), np.concatenate(vc), expand_mask(mask, lens[-1], lens, b))
     got = oa.sparse_attention(q, kc, vc, b, mask)
     assert np.abs(got - ref).max() < 1e-13
-    assert np.abs(oa.sparse_attention_tiled(q, kc, vc, b, mask) - got).max() < 1e-12
+    assert np.abs(oa.sparse_attention_blockwise(q, kc, vc, b, mask) - got).max() < 1e-12
 
 
 def test_all_blocks_kept_is_dense_window_attention_library_sdpa():
