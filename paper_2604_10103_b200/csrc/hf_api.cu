@@ -89,6 +89,8 @@ struct hf_ctx {
     bf16* x_hi = nullptr;            // full-width merge: the read-out h of all heads as bf16 hi + lo, [B*H, T_c, d] each
     bf16* x_lo = nullptr;
     float* partials = nullptr;       // absorb split partials
+    float* partials_layers = nullptr;    // layer-batched state update: one partial per (layer, batch*head, group)
+    size_t partials_layers_count = 0;
     int nsplit_max = 1;
     float z_scale = 1.f;             // 1 (z = sum of phi(K)) or 1 / tokens_per_frame (per-frame means)
     bf16* stage[4] = {nullptr, nullptr, nullptr, nullptr};   // q, k, v, o staging of the *_host calls
@@ -169,7 +171,7 @@ void free_all(hf_ctx* c) {
     for (auto& L : c->layers) { cudaFree(L.W_full); cudaFree(L.mask); cudaFree(L.idx); }
     cudaFree(c->ring_k_all); cudaFree(c->ring_v_all); cudaFree(c->pooled_k_all); cudaFree(c->S_all); cudaFree(c->z_all);
     cudaFree(c->sf_hi_all); cudaFree(c->sf_lo_all); cudaFree(c->W_all); cudaFree(c->bias_all);
-    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->x_hi); cudaFree(c->x_lo);
+    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -248,12 +250,16 @@ hf_status make_map(hf_ctx* c, CUtensorMap* m, const void* base, int slots) {
     return make_map_ex(c, m, base, c->Tc, slots, 64, 128, true);
 }
 
+// Groups of consecutive splits in which the partial sums of an item are added up (part of the summation order, so a
+// function of the split count alone -- see k_reduce_fold).
+inline int absorb_groups(int nsplit) { return nsplit < 2 ? nsplit : 2; }
+
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
     // after the partials kernel (nsplit > 0) the launch may overlap that kernel's epilogue; a fold on its own is ordinary
     PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, nsplit > 0);
-    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D>, (const float*)c->partials, nsplit, L.S, L.z, c->z_scale,
-                               (const bf16*)(L.has_w ? L.W : nullptr), c->cfg.heads, L.sf_hi, L.sf_lo));
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D, 4>, (const float*)c->partials, nsplit, absorb_groups(nsplit), L.S, L.z, c->z_scale,
+                               (const bf16*)(L.has_w ? L.W : nullptr), c->cfg.heads, c->BH, L.sf_hi, L.sf_lo, 1ull));
     return post_launch(c, "k_reduce_fold");
 }
 
@@ -297,24 +303,35 @@ hf_status launch_absorb_layers(hf_ctx* c, int first_layer, int n_layers, const C
     const int n_tiles = (n_tokens + A::TT - 1) / A::TT;
     AbsorbItemsParams p;
     memset(&p, 0, sizeof(p));
-    p.n_tokens = n_tokens; p.BH = c->BH; p.n_items = n_layers * c->BH;
+    p.n_tokens = n_tokens; p.BH = c->BH;
     p.nsplit = n_tiles < c->nsplit_max ? n_tiles : c->nsplit_max;
-    p.z_scale = c->z_scale;
-    p.S = c->S_all + (size_t)first_layer * dd; p.z = c->z_all + (size_t)first_layer * dz;
+    p.ngroup = absorb_groups(p.nsplit);
+    p.n_units = n_layers * c->BH * p.ngroup;
+    // scratch for one partial per (item, group), grown on first use (never inside a later call of the same size)
+    const size_t need = (size_t)n_layers * c->BH * p.ngroup * ((size_t)D * D + D);
+    if (need > c->partials_layers_count) {
+        HF_CUDA(cudaStreamSynchronize(st));
+        cudaFree(c->partials_layers);
+        c->partials_layers = nullptr; c->partials_layers_count = 0;
+        HF_TRY(dmalloc(&c->partials_layers, need));
+        c->partials_layers_count = need;
+    }
+    p.partials = c->partials_layers;
     for (int l = 0; l < n_layers; ++l) p.slot[l] = slot[l];
     p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc; p.dev_status = c->dev_status;
-    const int grid = p.n_items < c->sm_count ? p.n_items : c->sm_count;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     PdlLaunch pl(dim3(grid), dim3(A::THREADS), A::SMEM_BYTES, st, false);
     if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, true>, tk, tv, p));
     else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, false>, tk, tv, p));
     HF_TRY(post_launch(c, "k_absorb_items"));
     unsigned long long has_w = 0;
     for (int l = 0; l < n_layers; ++l) if (c->layers[first_layer + l].has_w) has_w |= 1ull << l;
-    PdlLaunch pf(dim3(D / 4, c->BH, n_layers), dim3(D), 0, st, true);
-    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_fold_layers<D>, (const float*)p.S,
+    PdlLaunch pf(dim3(D / 16, c->BH, n_layers), dim3(D), 0, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_reduce_fold<D, 16>, (const float*)c->partials_layers, p.ngroup, p.ngroup,
+                               c->S_all + (size_t)first_layer * dd, c->z_all + (size_t)first_layer * dz, c->z_scale,
                                (const bf16*)(c->W_all ? c->W_all + (size_t)first_layer * c->cfg.heads * D * D : nullptr), c->cfg.heads,
                                c->BH, c->sf_hi_all + (size_t)first_layer * dd, c->sf_lo_all + (size_t)first_layer * dd, has_w));
-    return post_launch(c, "k_fold_layers");
+    return post_launch(c, "k_reduce_fold (layers)");
 }
 
 template <int D>

@@ -102,5 +102,7 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
 }
-// phi(x) = elu(x) + 1
-__device__ __forceinline__ float phi_elu1(float x) { return x > 0.f ? x + 1.f : __expf(x); }
+// phi(x) = elu(x) + 1.  The exponential is ex2.approx.ftz of x log2(e) (2 ulp; results below 2^-126 flush to zero, which
+// is below anything the state or the read-out can resolve): the non-flushing form costs several more instructions
+// per value, and the state update is bound by exactly these.
+__device__ __forceinline__ float phi_elu1(float x) { return x > 0.f ? x + 1.f : fast_exp2(x * 1.4426950408889634f); }

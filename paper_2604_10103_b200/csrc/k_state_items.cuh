@@ -4,18 +4,20 @@
 // not depend on anything else, so the evicted chunks of L layers go through ONE persistent launch: 30 x 28.75 MB at the
 // 832x480 shape instead of thirty 28.75 MB launches that are each over before the memory pipeline has filled.
 //
-// Work item = (layer, batch*head): the thread block that takes an item owns its state for the whole token range, so
-// nothing is written to scratch and no second kernel adds partial sums:
+// The token range of a (layer, batch*head) item is cut into `nsplit` splits, and the splits into `ngroup` groups of
+// consecutive splits (the same cuts, and the same order of additions, as k_absorb_tc5 + k_reduce_fold use for one layer:
+// same operations on the same operands in the same order, so both paths leave the same bits in S and z).
+// Work unit = (item, group); thread block c takes units c, c + gridDim.x, ... and sums a unit's splits on chip:
 //   TMA warp        K (row-major) and V (128-byte swizzle) tiles of 64 tokens, ring of four stages, running ahead over
-//                   split and item boundaries
+//                   split and unit boundaries
 //   16 phi warps    phi(K) of a tile in fp32 -> bf16 hi + lo halves -> tensor memory (A operand, M = key feature,
 //                   K = token), sum of phi(K) per feature in a register        [absorb_phi_tile, shared with k_absorb_tc5]
 //   MMA warp        P_s += A_hi V + A_lo V over the tiles of split s, two P accumulators in tensor memory alternating
-//   4 merge warps   R = S (loaded when the item starts); after each split R += P_s, z_sum += the split's phi(K) sums; when
-//                   the item ends S = R, z += z_sum * z_scale.  They run beside the next split's tiles.
-// The token range of an item is cut into the same `nsplit` splits, and the splits are added to the state in the same
-// ascending order, as k_absorb_tc5 + k_reduce_fold do for one layer: same operations on the same operands in the same
-// order, so both paths leave the same bits in S and z.
+//   4 merge warps   R = P of the unit's first split, R += P_s for the others, likewise the phi(K) sums; when the unit ends R
+//                   and the sums go to the unit's slot of the scratch buffer.  They run beside the next split's tiles.
+// k_reduce_fold then adds the ngroup slots of every item to its state in ascending order and refolds S W^T.  With two
+// groups per item the scratch traffic is 2 x 66 KB per item (against 2.4 MB of K, V read), and 720 units spread over the
+// SMs within 3 % of evenly where 360 whole items would leave a third of them idle for the last third of the launch.
 // Tensor memory (512 columns at head dim 128): R [0, D), P_0 [D, 2D), P_1 [2D, 3D), A_0 / A_1 (hi 32 + lo 32 columns each).
 // Every wait is bounded and reports through the device status word; nothing traps.
 #pragma once
@@ -41,11 +43,9 @@ struct AbsorbItems {
 
 struct AbsorbItemsParams {
     int n_tokens;             // tokens per item
-    int BH, n_items;          // items = layers of the call x B*H; item i: layer i / BH (of the call), batch*head i % BH
-    int nsplit;               // splits of an item's token range (the summation order)
-    float z_scale;
-    float* S;                 // [layers of the call][B*H][D][D], updated in place
-    float* z;                 // [layers of the call][B*H][D]
+    int BH, n_units;          // units = layers of the call x B*H x ngroup; unit u: item u / ngroup (layer item / BH, batch*head item % BH), group u % ngroup
+    int nsplit, ngroup;       // splits of an item's token range and groups of consecutive splits (the summation order)
+    float* partials;          // [items][ngroup][D*D + D]: per unit the sum of its splits' phi(K)^T V, then of their phi(K) sums
     int slot[HF_MAX_BATCH_LAYERS];   // coordinate 3 of the tensor maps for each layer of the call
     const float* cos_k;       // rotation tables (ROPE instantiation only)
     const float* sin_k;
@@ -53,7 +53,7 @@ struct AbsorbItemsParams {
     int* dev_status;
 };
 
-// grid: min(n_items, SMs); thread block c takes items c, c + gridDim.x, ...
+// grid: min(n_units, SMs); thread block c takes units c, c + gridDim.x, ...
 // tm_k: [D, n_tokens, B*H, slots] box {D, 64}, no swizzle.  tm_v: same tensor, box {64, 64}, 128-byte swizzle.
 template <int D, bool ROPE>
 __global__ void __launch_bounds__(AbsorbItems<D>::THREADS, 1)
@@ -74,8 +74,10 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = (p.n_tokens + C::TT - 1) / C::TT;
     const int nsplit = p.nsplit;
-    const int my_items = (p.n_items - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
-    auto split_lo = [&](int s) { return (int)(((long long)n_tiles * s) / nsplit); };
+    const int ngroup = p.ngroup;
+    const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    auto split_lo = [&](int s) { return (int)(((long long)n_tiles * s) / nsplit); };       // first tile of split s
+    auto group_lo = [&](int g) { return (int)(((long long)nsplit * g) / ngroup); };        // first split of group g
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_kfree + 8 * s, C::NQ * D); mbar_init(bar_vfree + 8 * s, 1); }
@@ -101,11 +103,13 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         if (lane == 0) {
             bool ok = true;
             int g = 0;                                        // tiles issued so far
-            for (int n = 0; ok && n < my_items; ++n) {
-                const int item = blockIdx.x + n * gridDim.x;
+            for (int n = 0; ok && n < my_units; ++n) {
+                const int unit = blockIdx.x + n * gridDim.x;
+                const int item = unit / ngroup, grp = unit - item * ngroup;
                 const int lay = item / p.BH, bh = item - lay * p.BH;
                 const int slot = p.slot[lay];
-                for (int tile = 0; ok && tile < n_tiles; ++tile, ++g) {
+                const int t_lo = split_lo(group_lo(grp)), t_hi = split_lo(group_lo(grp + 1));
+                for (int tile = t_lo; ok && tile < t_hi; ++tile, ++g) {
                     const int s = g % C::NST;
                     if (g >= C::NST) {
                         const uint32_t par_free = ((g / C::NST) & 1) ^ 1;
@@ -131,8 +135,9 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint64_t dv0 = smem_desc_sw128(sV, C::VSUB_BYTES, 1024);
         bool ok = true;
         int g = 0, q = 0;                                     // tiles / splits so far
-        for (int n = 0; ok && n < my_items; ++n) {
-            for (int sp = 0; ok && sp < nsplit; ++sp, ++q) {
+        for (int n = 0; ok && n < my_units; ++n) {
+            const int grp = (blockIdx.x + n * gridDim.x) % ngroup;
+            for (int sp = group_lo(grp); ok && sp < group_lo(grp + 1); ++sp, ++q) {
                 const int lo = split_lo(sp), hi = split_lo(sp + 1);
                 const int pb = q & 1;
                 // the accumulator of this split was read by the merge warps two splits ago
@@ -169,51 +174,45 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint32_t lane_base = tmem + ((uint32_t)(quad * 32) << 16);
         bool ok = true;
         int q = 0;
-        for (int n = 0; ok && active && n < my_items; ++n) {
-            const int item = blockIdx.x + n * gridDim.x;
-            float* S_row = p.S + ((size_t)item * D + a) * D;
-            // R = S: the thread's row, 32 columns at a time (R is this role's own: nothing else reads or writes it)
-#pragma unroll 1
-            for (int c = 0; c < D; c += 32) {
-                uint32_t r[32];
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    const float4 x = *reinterpret_cast<const float4*>(S_row + c + 4 * v);
-                    r[4 * v] = __float_as_uint(x.x); r[4 * v + 1] = __float_as_uint(x.y);
-                    r[4 * v + 2] = __float_as_uint(x.z); r[4 * v + 3] = __float_as_uint(x.w);
-                }
-                tmem_st32(lane_base + C::COL_R + c, r);
-            }
-            tmem_wait_st();
+        for (int n = 0; ok && active && n < my_units; ++n) {
+            const int unit = blockIdx.x + n * gridDim.x;
+            const int grp = unit % ngroup;
+            float* out = p.partials + (size_t)unit * (D * D + D);
             float zsum = 0.f;
-            for (int sp = 0; ok && sp < nsplit; ++sp, ++q) {
+            const int sp0 = group_lo(grp), sp1 = group_lo(grp + 1);
+            for (int sp = sp0; ok && sp < sp1; ++sp, ++q) {
                 const int pb = q & 1;
                 const uint32_t par = (q >> 1) & 1;
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_dfull + 8 * pb, par, abort_flag, p.dev_status, 66));
-                if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_zfull + 8 * pb, par, abort_flag, p.dev_status, 67));
+                ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_dfull + 8 * pb, par, abort_flag, p.dev_status, 66));
+                if (ok) ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_zfull + 8 * pb, par, abort_flag, p.dev_status, 67));
                 if (!ok) break;
                 fence_after_sync();
+                // R = P for the unit's first split, R += P for the others (R is this role's own: nothing else touches it)
 #pragma unroll 1
                 for (int c = 0; c < D; c += 32) {
                     uint32_t r[32], x[32];
-                    tmem_ld32(lane_base + C::COL_R + c, r);
                     tmem_ld32(lane_base + C::COL_P + pb * D + c, x);
-                    tmem_wait_ld();
+                    if (sp > sp0) {
+                        tmem_ld32(lane_base + C::COL_R + c, r);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__fadd_rn(__uint_as_float(r[e]), __uint_as_float(x[e])));
-                    tmem_st32(lane_base + C::COL_R + c, r);
+                        for (int e = 0; e < 32; ++e) x[e] = __float_as_uint(__fadd_rn(__uint_as_float(r[e]), __uint_as_float(x[e])));
+                    } else {
+                        tmem_wait_ld();
+                    }
+                    tmem_st32(lane_base + C::COL_R + c, x);
                 }
                 const float* zp = z_x + pb * C::NQ * D;
                 float zs = zp[a];
 #pragma unroll
                 for (int w = 1; w < C::NQ; ++w) zs += zp[w * D + a];
-                zsum += zs;
+                zsum = sp > sp0 ? zsum + zs : zs;
                 tmem_wait_st();
                 fence_before_sync();
                 mbar_arrive(bar_pfree + 8 * pb);
             }
             if (!ok) break;
-            // S = R, z += z_sum * z_scale
+            // the unit's sums to its slot of the scratch buffer (row a of the matrix: 4 D contiguous bytes per thread)
 #pragma unroll 1
             for (int c = 0; c < D; c += 32) {
                 uint32_t r[32];
@@ -221,10 +220,10 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 tmem_wait_ld();
 #pragma unroll
                 for (int v = 0; v < 8; ++v)
-                    *reinterpret_cast<float4*>(S_row + c + 4 * v) =
+                    *reinterpret_cast<float4*>(out + (size_t)a * D + c + 4 * v) =
                         make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
             }
-            p.z[(size_t)item * D + a] += zsum * p.z_scale;
+            out[D * D + a] = zsum;
         }
     } else {
         // ================================================================= phi(K) into tensor memory
@@ -236,8 +235,9 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         bool ok = true;
         int g = 0, q = 0;
-        for (int n = 0; ok && active && n < my_items; ++n) {
-            for (int sp = 0; ok && sp < nsplit; ++sp, ++q) {
+        for (int n = 0; ok && active && n < my_units; ++n) {
+            const int grp = (blockIdx.x + n * gridDim.x) % ngroup;
+            for (int sp = group_lo(grp); ok && sp < group_lo(grp + 1); ++sp, ++q) {
                 const int lo = split_lo(sp), hi = split_lo(sp + 1);
                 const int pb = q & 1;
                 float zacc = 0.f;
@@ -274,64 +274,5 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     if (warp == C::WARP_MMA) {
         fence_after_sync();
         tmem_dealloc(tmem, C::TMEM_COLS);
-    }
-}
-
-// Folded state of several layers in one launch: S'_l = S_l W_l^T as bf16 hi + lo halves (k_reduce_fold's second half).
-// grid (D / 4, B*H, layers); S, sf_hi, sf_lo: [layers][B*H][D][D]; W: [layers][H][D][D] or nullptr (identity).
-template <int D>
-__global__ void __launch_bounds__(D)
-k_fold_layers(const float* __restrict__ S, const bf16* __restrict__ W, int heads, int BH, bf16* __restrict__ sf_hi,
-              bf16* __restrict__ sf_lo, unsigned long long has_w_mask) {
-    constexpr int ROWS = 4;
-    __shared__ float rows[ROWS][D];
-    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, lay = blockIdx.z, h = bh % heads;
-    const int cp = threadIdx.x;
-    const bool with_w = W != nullptr && ((has_w_mask >> lay) & 1ull);
-    uint4 wq[D / 8];
-    if (with_w) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(W + (((size_t)lay * heads + h) * D + cp) * D);
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
-    }
-    pdl_wait();
-    const size_t base = ((size_t)lay * BH + bh) * D * D;
-    float sum[ROWS], out[ROWS];
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) sum[r] = S[base + (size_t)(a0 + r) * D + cp];
-    if (!with_w) {
-#pragma unroll
-        for (int r = 0; r < ROWS; ++r) out[r] = sum[r];
-    } else {
-#pragma unroll
-        for (int r = 0; r < ROWS; ++r) rows[r][cp] = sum[r];
-        __syncthreads();
-#pragma unroll
-        for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
-#pragma unroll
-        for (int i = 0; i < D / 8; ++i) {
-            float w[8];
-            float2 t;
-            t = unpack_bf16(wq[i].x); w[0] = t.x; w[1] = t.y;
-            t = unpack_bf16(wq[i].y); w[2] = t.x; w[3] = t.y;
-            t = unpack_bf16(wq[i].z); w[4] = t.x; w[5] = t.y;
-            t = unpack_bf16(wq[i].w); w[6] = t.x; w[7] = t.y;
-#pragma unroll
-            for (int r = 0; r < ROWS; ++r) {
-                const float4 s0 = *reinterpret_cast<const float4*>(&rows[r][i * 8]);
-                const float4 s1 = *reinterpret_cast<const float4*>(&rows[r][i * 8 + 4]);
-                out[r] = fmaf(s0.x, w[0], out[r]); out[r] = fmaf(s0.y, w[1], out[r]);
-                out[r] = fmaf(s0.z, w[2], out[r]); out[r] = fmaf(s0.w, w[3], out[r]);
-                out[r] = fmaf(s1.x, w[4], out[r]); out[r] = fmaf(s1.y, w[5], out[r]);
-                out[r] = fmaf(s1.z, w[6], out[r]); out[r] = fmaf(s1.w, w[7], out[r]);
-            }
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(out[r]);
-        const size_t o = base + (size_t)(a0 + r) * D + cp;
-        sf_hi[o] = hi;
-        sf_lo[o] = __float2bfloat16_rn(out[r] - __bfloat162float(hi));
     }
 }

@@ -2,7 +2,7 @@
 //   k_absorb_mma   Eq. 3, first half, on the warp-level tensor path (ldmatrix + mma.sync): per (batch, head) the token
 //                  range is split over thread blocks, each writing its partial phi(K_ev)^T V_ev and sum_t phi(K_ev[t])
 //                  to scratch.  Used by the entry point that may not allocate; the context's path is k_absorb_tc5.
-//   k_reduce_fold  Eq. 3, second half: S, z += the partials in ascending split order (deterministic), then
+//   k_reduce_fold  Eq. 3, second half: S, z += the partials in a fixed order (deterministic), then
 //                  S' = S W^T split into bf16 hi/lo halves (the per-row divisor of Eq. 4 commutes with W)
 // phi(K) is carried as a bf16 hi + lo pair so that the products keep ~16 mantissa bits; accumulation is fp32.
 #pragma once
@@ -127,44 +127,62 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
     }
 }
 
-// grid (D/4, B*H), D threads.  Adds the nsplit partials of a (batch, head) to S (rows a0 .. a0+3 per block) and z
-// (block 0) in ascending split order, then folds the updated rows: Sf = S W_h^T (or S when W == nullptr) as bf16
-// hi and lo halves.  nsplit == 0: fold only.  sf_hi == nullptr: state update only.  z_scale: 1 for z = sum of phi(K)
-// rows, 1 / tokens-per-frame for the per-frame-mean reading of Eq. 3.
+// grid (D / ROWS, B*H, layers), D threads.  Adds the nsplit partials of every (layer, batch*head) to S (rows a0 .. a0 + ROWS - 1
+// per block) and z (block 0), then folds the updated rows: Sf = S W_h^T (or S where the layer has no matrix) as bf16 hi and lo
+// halves.  Order of the additions (it fixes the bits of the state, whichever kernel produced the partials): the splits are
+// taken in `ngroup` groups of consecutive splits, group g = splits [nsplit g / ngroup, nsplit (g + 1) / ngroup); a group is
+// summed from its first split upwards, and the group sums are added to the state in ascending g.  (The layer-batched
+// kernel sums a group on chip and hands over one partial per group: nsplit == ngroup there.)
+// nsplit == 0: fold only.  sf_hi == nullptr: state update only.  z_scale: 1 for z = sum of phi(K) rows, 1 / tokens-per-frame
+// for the per-frame-mean reading of Eq. 3.  partials: [layers][B*H][nsplit][D*D + D]; S, sf_hi, sf_lo: [layers][B*H][D][D];
+// z: [layers][B*H][D]; W: [layers][H][D][D] or nullptr, used for the layers whose bit is set in has_w_mask.
 // Thread c' owns output column c': its row of W_h is fetched first (all loads in flight while the partials are summed).
-template <int D>
+// ROWS: 4 for one layer (many small blocks: latency), 16 for many layers (W_h is fetched D / ROWS times per head).
+template <int D, int ROWS>
 __global__ void __launch_bounds__(D)
-k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict__ S, float* __restrict__ z, float z_scale,
-              const bf16* __restrict__ W, int heads, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo) {
-    constexpr int ROWS = 4;
+k_reduce_fold(const float* __restrict__ partials, int nsplit, int ngroup, float* __restrict__ S, float* __restrict__ z, float z_scale,
+              const bf16* __restrict__ W, int heads, int BH, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo,
+              unsigned long long has_w_mask) {
     constexpr int PART_FLOATS = D * D + D;
     __shared__ float rows[ROWS][D];
-    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, h = bh % heads;
+    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, lay = blockIdx.z, h = bh % heads;
+    const size_t item = (size_t)lay * BH + bh;
     const int cp = threadIdx.x;
-    const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr;
+    const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr && ((has_w_mask >> lay) & 1ull);
     uint4 wq[D / 8];
     if (with_w) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(W + ((size_t)h * D + cp) * D);     // W_h[c'][.]
+        const uint4* wrow = reinterpret_cast<const uint4*>(W + (((size_t)lay * heads + h) * D + cp) * D);     // W_h[c'][.]
 #pragma unroll
         for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
     }
     pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
-    const float* base = partials + (size_t)bh * nsplit * PART_FLOATS;
+    const float* base = partials + item * nsplit * PART_FLOATS;
+    float* S_it = S + item * D * D;
     float sum[ROWS];
 #pragma unroll
-    for (int r = 0; r < ROWS; ++r) sum[r] = S[((size_t)bh * D + a0 + r) * D + cp];
-    float zsum = 0.f;           // this call's sum of phi(K) rows; enters z scaled (1, or 1 / tokens per frame)
+    for (int r = 0; r < ROWS; ++r) sum[r] = S_it[(size_t)(a0 + r) * D + cp];
+    float ztot = 0.f;           // this call's sum of phi(K) rows; enters z scaled (1, or 1 / tokens per frame)
     const bool do_z = blockIdx.x == 0 && nsplit > 0;
-#pragma unroll 8
-    for (int s = 0; s < nsplit; ++s) {      // ascending split order per element; several splits' loads in flight
+    for (int g = 0; g < ngroup && nsplit > 0; ++g) {
+        const int s0 = (int)(((long long)nsplit * g) / ngroup), s1 = (int)(((long long)nsplit * (g + 1)) / ngroup);
+        float sg[ROWS], zg = 0.f;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) sum[r] += __ldcg(base + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
-        if (do_z) zsum += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
+        for (int r = 0; r < ROWS; ++r) sg[r] = __ldcg(base + (size_t)s0 * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+        if (do_z) zg = __ldcg(base + (size_t)s0 * PART_FLOATS + D * D + cp);
+#pragma unroll 2
+        for (int s = s0 + 1; s < s1; ++s) {      // ascending split order per element; several splits' loads in flight
+#pragma unroll
+            for (int r = 0; r < ROWS; ++r) sg[r] += __ldcg(base + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+            if (do_z) zg += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
+        }
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) sum[r] += sg[r];
+        ztot += zg;
     }
     if (nsplit > 0) {
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) S[((size_t)bh * D + a0 + r) * D + cp] = sum[r];
-        if (do_z) z[(size_t)bh * D + cp] += zsum * z_scale;
+        for (int r = 0; r < ROWS; ++r) S_it[(size_t)(a0 + r) * D + cp] = sum[r];
+        if (do_z) z[item * D + cp] += ztot * z_scale;
     }
     if (!fold) return;
     float out[ROWS];
@@ -199,7 +217,7 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, float* __restrict_
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
         const __nv_bfloat16 hi = __float2bfloat16_rn(out[r]);
-        const size_t o = ((size_t)bh * D + a0 + r) * D + cp;
+        const size_t o = (item * D + a0 + r) * D + cp;
         sf_hi[o] = hi;
         sf_lo[o] = __float2bfloat16_rn(out[r] - __bfloat162float(hi));
     }

@@ -49,11 +49,16 @@ __device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tok
     const int nv = min(C::TT, n_tokens - tile_row0) - part * HT;
     const uint8_t* kt = k_tile + (size_t)(part * HT) * D * 2 + a * 2;
     uint32_t hi[HT / 2], lo[HT / 2];
+    constexpr float LOG2E = 1.4426950408889634f;
 #pragma unroll
     for (int t = 0; t < HT; t += 2) {
         const float x0 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)t * D * 2)) << 16);
         const float x1 = __uint_as_float((uint32_t)(*reinterpret_cast<const uint16_t*>(kt + (size_t)(t + 1) * D * 2)) << 16);
-        float f0 = phi_elu1(x0), f1 = phi_elu1(x1);
+        // phi(x) = x > 0 ? x + 1 : exp(x) for the two tokens at once (packed fp32 add / multiply: one instruction each)
+        const float2 xs = make_float2(x0, x1);
+        const float2 lin = fadd2(xs, make_float2(1.f, 1.f));
+        const float2 arg = ffma2(xs, make_float2(LOG2E, LOG2E), make_float2(0.f, 0.f));
+        float f0 = x0 > 0.f ? lin.x : fast_exp2(arg.x), f1 = x1 > 0.f ? lin.y : fast_exp2(arg.y);
         if (nv < HT) {                              // only the tensor's last tile
             if (t >= nv) f0 = 0.f;
             if (t + 1 >= nv) f1 = 0.f;
@@ -72,8 +77,9 @@ __device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tok
         }
         const uint32_t hp = pack_bf16(f0, f1);
         const float2 hf = unpack_bf16(hp);
+        const float2 res = fadd2(make_float2(f0, f1), make_float2(-hf.x, -hf.y));      // exact: the bf16 rounding error
         hi[t >> 1] = hp;
-        lo[t >> 1] = pack_bf16(f0 - hf.x, f1 - hf.y);
+        lo[t >> 1] = pack_bf16(res.x, res.y);
     }
     const uint32_t tA = tA_buf + part * (HT / 2);
     tc5::tmem_st8(tA, hi);
