@@ -257,8 +257,8 @@ inline int absorb_groups(int nsplit) { return nsplit < 2 ? nsplit : 2; }
 template <int D>
 hf_status launch_fold(hf_ctx* c, LayerState& L, int nsplit, cudaStream_t st) {
     // after the partials kernel (nsplit > 0) the launch may overlap that kernel's epilogue; a fold on its own is ordinary
-    PdlLaunch pl(dim3(D / 4, c->BH), dim3(D), 0, st, nsplit > 0);
-    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D, 4>, (const float*)c->partials, nsplit, absorb_groups(nsplit), L.S, L.z, c->z_scale,
+    PdlLaunch pl(dim3(D / 16, c->BH), dim3(D), 0, st, nsplit > 0);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_reduce_fold<D>, (const float*)c->partials, nsplit, absorb_groups(nsplit), L.S, L.z, c->z_scale,
                                (const bf16*)(L.has_w ? L.W : nullptr), c->cfg.heads, c->BH, L.sf_hi, L.sf_lo, 1ull));
     return post_launch(c, "k_reduce_fold");
 }
@@ -327,7 +327,7 @@ hf_status launch_absorb_layers(hf_ctx* c, int first_layer, int n_layers, const C
     unsigned long long has_w = 0;
     for (int l = 0; l < n_layers; ++l) if (c->layers[first_layer + l].has_w) has_w |= 1ull << l;
     PdlLaunch pf(dim3(D / 16, c->BH, n_layers), dim3(D), 0, st, true);
-    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_reduce_fold<D, 16>, (const float*)c->partials_layers, p.ngroup, p.ngroup,
+    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_reduce_fold<D>, (const float*)c->partials_layers, p.ngroup, p.ngroup,
                                c->S_all + (size_t)first_layer * dd, c->z_all + (size_t)first_layer * dz, c->z_scale,
                                (const bf16*)(c->W_all ? c->W_all + (size_t)first_layer * c->cfg.heads * D * D : nullptr), c->cfg.heads,
                                c->BH, c->sf_hi_all + (size_t)first_layer * dd, c->sf_lo_all + (size_t)first_layer * dd, has_w));

@@ -65,7 +65,7 @@ hf_status run(const bf16* k, const bf16* v, int bh, int n_tokens, float* S, floa
     k_absorb_mma<D><<<dim3(nsplit, bh), A::THREADS, A::SMEM_BYTES, st>>>(k, v, n_tokens, partials);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) {
-        k_reduce_fold<D, 4><<<dim3(D / 4, bh), D, 0, st>>>(partials, nsplit, nsplit < 2 ? nsplit : 2, S, z, 1.f, nullptr, 1, bh, nullptr, nullptr, 0ull);
+        k_reduce_fold<D><<<dim3(D / 16, bh), D, 0, st>>>(partials, nsplit, nsplit < 2 ? nsplit : 2, S, z, 1.f, nullptr, 1, bh, nullptr, nullptr, 0ull);
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) return nfail(HF_ERR_CUDA, "kernel launch failed with error %lld", (long long)e);

@@ -240,7 +240,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
             for (int sp = group_lo(grp); ok && sp < group_lo(grp + 1); ++sp, ++q) {
                 const int lo = split_lo(sp), hi = split_lo(sp + 1);
                 const int pb = q & 1;
-                float zacc = 0.f;
+                float2 zacc = make_float2(0.f, 0.f);
                 for (int tile = lo; ok && tile < hi; ++tile, ++g) {
                     const int s = g % C::NST, ab = g & 1;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, (g / C::NST) & 1, abort_flag, p.dev_status, 68));
@@ -263,7 +263,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * pb, ((q >> 1) & 1) ^ 1, abort_flag, p.dev_status, 70));
                     if (!ok) break;
                 }
-                z_x[(pb * C::NQ + part) * D + a] = zacc;
+                z_x[(pb * C::NQ + part) * D + a] = zacc.x + zacc.y;
                 mbar_arrive(bar_zfull + 8 * pb);
             }
         }

@@ -127,33 +127,41 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
     }
 }
 
-// grid (D / ROWS, B*H, layers), D threads.  Adds the nsplit partials of every (layer, batch*head) to S (rows a0 .. a0 + ROWS - 1
-// per block) and z (block 0), then folds the updated rows: Sf = S W_h^T (or S where the layer has no matrix) as bf16 hi and lo
+// grid (D / 16, B*H, layers), D threads.  Adds the nsplit partials of every (layer, batch*head) to S (rows a0 .. a0 + 15 per
+// block) and z (block 0), then folds the updated rows: Sf = S W_h^T (or S where the layer has no matrix) as bf16 hi and lo
 // halves.  Order of the additions (it fixes the bits of the state, whichever kernel produced the partials): the splits are
 // taken in `ngroup` groups of consecutive splits, group g = splits [nsplit g / ngroup, nsplit (g + 1) / ngroup); a group is
 // summed from its first split upwards, and the group sums are added to the state in ascending g.  (The layer-batched
 // kernel sums a group on chip and hands over one partial per group: nsplit == ngroup there.)
+// The fold is a 16 x D x D product per block on the warp-level tensor path: the fp32 rows are split exactly into three bf16
+// terms (hi + mid + lo = all 24 mantissa bits), W_h is bf16 already, so every product is exact and only the fp32
+// accumulation of mma.sync rounds; warp w owns output columns [32 w, 32 w + 32).
 // nsplit == 0: fold only.  sf_hi == nullptr: state update only.  z_scale: 1 for z = sum of phi(K) rows, 1 / tokens-per-frame
 // for the per-frame-mean reading of Eq. 3.  partials: [layers][B*H][nsplit][D*D + D]; S, sf_hi, sf_lo: [layers][B*H][D][D];
 // z: [layers][B*H][D]; W: [layers][H][D][D] or nullptr, used for the layers whose bit is set in has_w_mask.
-// Thread c' owns output column c': its row of W_h is fetched first (all loads in flight while the partials are summed).
-// ROWS: 4 for one layer (many small blocks: latency), 16 for many layers (W_h is fetched D / ROWS times per head).
-template <int D, int ROWS>
+template <int D>
 __global__ void __launch_bounds__(D)
 k_reduce_fold(const float* __restrict__ partials, int nsplit, int ngroup, float* __restrict__ S, float* __restrict__ z, float z_scale,
               const bf16* __restrict__ W, int heads, int BH, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo,
               unsigned long long has_w_mask) {
+    constexpr int ROWS = 16;
     constexpr int PART_FLOATS = D * D + D;
-    __shared__ float rows[ROWS][D];
+    constexpr int ROW_BYTES = D * 2;
+    __shared__ __align__(128) uint8_t sW[D * ROW_BYTES];            // W_h [c'][c], 16-byte chunks XOR-swizzled by the row
+    __shared__ __align__(128) uint8_t sA[3][ROWS * ROW_BYTES];      // the block's rows of S as bf16 hi / mid / lo, same swizzle
     const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, lay = blockIdx.z, h = bh % heads;
     const size_t item = (size_t)lay * BH + bh;
-    const int cp = threadIdx.x;
+    const int cp = threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr && ((has_w_mask >> lay) & 1ull);
-    uint4 wq[D / 8];
-    if (with_w) {
-        const uint4* wrow = reinterpret_cast<const uint4*>(W + (((size_t)lay * heads + h) * D + cp) * D);     // W_h[c'][.]
+    if (with_w) {       // the matrix does not depend on the kernel before this one: fetched while that kernel drains
+        const bf16* wsrc = W + ((size_t)lay * heads + h) * D * D;
+        constexpr int CPR = D / 8;                                  // 16-byte chunks per row
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) wq[i] = __ldg(wrow + i);
+        for (int i = 0; i < CPR; ++i) {
+            const int id = threadIdx.x + i * D, row = id / CPR, ch = id % CPR;
+            cp_async16(smem_u32(sW) + swz<ROW_BYTES>(row, ch), wsrc + (size_t)row * D + ch * 8, true);
+        }
+        cp_async_commit();
     }
     pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
     const float* base = partials + item * nsplit * PART_FLOATS;
@@ -185,40 +193,62 @@ k_reduce_fold(const float* __restrict__ partials, int nsplit, int ngroup, float*
         if (do_z) z[item * D + cp] += ztot * z_scale;
     }
     if (!fold) return;
-    float out[ROWS];
     if (!with_w) {
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) out[r] = sum[r];
-    } else {
+        for (int r = 0; r < ROWS; ++r) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(sum[r]);
+            const size_t o = (item * D + a0 + r) * D + cp;
+            sf_hi[o] = hi;
+            sf_lo[o] = __float2bfloat16_rn(sum[r] - __bfloat162float(hi));
+        }
+        return;
+    }
+    // ---- the rows as three bf16 terms (each difference is exact in fp32), column cp of every row
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) rows[r][cp] = sum[r];
-        __syncthreads();
+    for (int r = 0; r < ROWS; ++r) {
+        const __nv_bfloat16 t0 = __float2bfloat16_rn(sum[r]);
+        const float r1 = sum[r] - __bfloat162float(t0);
+        const __nv_bfloat16 t1 = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 t2 = __float2bfloat16_rn(r1 - __bfloat162float(t1));
+        const uint32_t off = swz<ROW_BYTES>(r, cp >> 3) + (cp & 7) * 2;
+        *reinterpret_cast<__nv_bfloat16*>(sA[0] + off) = t0;
+        *reinterpret_cast<__nv_bfloat16*>(sA[1] + off) = t1;
+        *reinterpret_cast<__nv_bfloat16*>(sA[2] + off) = t2;
+    }
+    cp_async_wait<0>();
+    __syncthreads();
+    // ---- out[a][c'] = sum_c S[a][c] W_h[c'][c]: A = the rows (16 x D), B = W_h as stored ([n][k], k contiguous)
+    float acc[4][4];
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) out[r] = 0.f;
+    for (int n = 0; n < 4; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
+    const int n0 = warp * 32;
 #pragma unroll
-        for (int i = 0; i < D / 8; ++i) {
-            float w[8];
-            float2 t;
-            t = unpack_bf16(wq[i].x); w[0] = t.x; w[1] = t.y;
-            t = unpack_bf16(wq[i].y); w[2] = t.x; w[3] = t.y;
-            t = unpack_bf16(wq[i].z); w[4] = t.x; w[5] = t.y;
-            t = unpack_bf16(wq[i].w); w[6] = t.x; w[7] = t.y;
+    for (int ks = 0; ks < D / 16; ++ks) {
+        uint32_t af[3][4];
 #pragma unroll
-            for (int r = 0; r < ROWS; ++r) {
-                const float4 s0 = *reinterpret_cast<const float4*>(&rows[r][i * 8]);
-                const float4 s1 = *reinterpret_cast<const float4*>(&rows[r][i * 8 + 4]);
-                out[r] = fmaf(s0.x, w[0], out[r]); out[r] = fmaf(s0.y, w[1], out[r]);
-                out[r] = fmaf(s0.z, w[2], out[r]); out[r] = fmaf(s0.w, w[3], out[r]);
-                out[r] = fmaf(s1.x, w[4], out[r]); out[r] = fmaf(s1.y, w[5], out[r]);
-                out[r] = fmaf(s1.z, w[6], out[r]); out[r] = fmaf(s1.w, w[7], out[r]);
+        for (int t = 0; t < 3; ++t)
+            ldsm_x4(smem_u32(sA[t]) + swz<ROW_BYTES>(lane & 15, ks * 2 + (lane >> 4)), af[t][0], af[t][1], af[t][2], af[t][3]);
+#pragma unroll
+        for (int np = 0; np < 2; ++np) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(smem_u32(sW) + swz<ROW_BYTES>(n0 + np * 16 + (lane & 7) + ((lane >> 4) << 3), ks * 2 + ((lane >> 3) & 1)), b0, b1, b2, b3);
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                mma_bf16(acc[2 * np], af[t][0], af[t][1], af[t][2], af[t][3], b0, b1);
+                mma_bf16(acc[2 * np + 1], af[t][0], af[t][1], af[t][2], af[t][3], b2, b3);
             }
         }
     }
 #pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-        const __nv_bfloat16 hi = __float2bfloat16_rn(out[r]);
-        const size_t o = (item * D + a0 + r) * D + cp;
-        sf_hi[o] = hi;
-        sf_lo[o] = __float2bfloat16_rn(out[r] - __bfloat162float(hi));
+    for (int n = 0; n < 4; ++n) {
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const float x0 = acc[n][2 * half], x1 = acc[n][2 * half + 1];
+            const uint32_t hp = pack_bf16(x0, x1);
+            const float2 hf = unpack_bf16(hp);
+            const size_t o = (item * D + a0 + (lane >> 2) + half * 8) * D + n0 + n * 8 + 2 * (lane & 3);
+            *reinterpret_cast<uint32_t*>(sf_hi + o) = hp;
+            *reinterpret_cast<uint32_t*>(sf_lo + o) = pack_bf16(x0 - hf.x, x1 - hf.y);
+        }
     }
 }

@@ -40,13 +40,11 @@ struct AbsorbTc5 {
 // split into bf16 hi + lo halves, stored as the A operand (M = feature, K = token) at tA (hi: 32 columns, lo: the next
 // 32); the unrotated values are added to zacc.  k_tile: the tile in shared memory, row-major [token][D], not swizzled.
 // Shared by the split kernel and the layer-batched kernel so that both form the same bits.
-template <int D, bool ROPE>
-__device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tokens, int tile_row0, int part, int a, uint32_t tA_buf,
-                                                const float* cos_k, const float* sin_k, int rope_rows, float& zacc) {
+template <int D, bool ROPE, bool TAIL>
+__device__ __forceinline__ void absorb_phi_tile_t(const uint8_t* k_tile, int nv, int tile_row0, int part, int a, uint32_t tA_buf,
+                                                  const float* cos_k, const float* sin_k, int rope_rows, float2& zacc2) {
     typedef AbsorbTc5<D> C;
     constexpr int HT = C::TT / C::NQ;                       // tokens per thread and tile
-    // rows past the end of the tensor read as zero: phi(0) = 1 must not count
-    const int nv = min(C::TT, n_tokens - tile_row0) - part * HT;
     const uint8_t* kt = k_tile + (size_t)(part * HT) * D * 2 + a * 2;
     uint32_t hi[HT / 2], lo[HT / 2];
     constexpr float LOG2E = 1.4426950408889634f;
@@ -59,11 +57,11 @@ __device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tok
         const float2 lin = fadd2(xs, make_float2(1.f, 1.f));
         const float2 arg = ffma2(xs, make_float2(LOG2E, LOG2E), make_float2(0.f, 0.f));
         float f0 = x0 > 0.f ? lin.x : fast_exp2(arg.x), f1 = x1 > 0.f ? lin.y : fast_exp2(arg.y);
-        if (nv < HT) {                              // only the tensor's last tile
+        if (TAIL) {                                 // only the tensor's last tile
             if (t >= nv) f0 = 0.f;
             if (t + 1 >= nv) f1 = 0.f;
         }
-        zacc += f0 + f1;                            // the normaliser keeps the unrotated values
+        zacc2 = fadd2(zacc2, make_float2(f0, f1));  // the normaliser keeps the unrotated values (even / odd tokens apart)
         if (ROPE) {
             // feature pairs (2i, 2i+1) sit in neighbouring lanes; the pair's angle belongs to the token
             const float g0 = __shfl_xor_sync(0xffffffffu, f0, 1), g1 = __shfl_xor_sync(0xffffffffu, f1, 1);
@@ -84,6 +82,17 @@ __device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tok
     const uint32_t tA = tA_buf + part * (HT / 2);
     tc5::tmem_st8(tA, hi);
     tc5::tmem_st8(tA + 32, lo);
+}
+// zacc2: running sums of phi(K) over the thread's even and odd tokens; a split's sum is zacc2.x + zacc2.y.
+template <int D, bool ROPE>
+__device__ __forceinline__ void absorb_phi_tile(const uint8_t* k_tile, int n_tokens, int tile_row0, int part, int a, uint32_t tA_buf,
+                                                const float* cos_k, const float* sin_k, int rope_rows, float2& zacc2) {
+    typedef AbsorbTc5<D> C;
+    constexpr int HT = C::TT / C::NQ;
+    // rows past the end of the tensor read as zero: phi(0) = 1 must not count (only the tensor's last tile has any)
+    const int nv = min(C::TT, n_tokens - tile_row0) - part * HT;
+    if (nv >= HT) absorb_phi_tile_t<D, ROPE, false>(k_tile, nv, tile_row0, part, a, tA_buf, cos_k, sin_k, rope_rows, zacc2);
+    else absorb_phi_tile_t<D, ROPE, true>(k_tile, nv, tile_row0, part, a, tA_buf, cos_k, sin_k, rope_rows, zacc2);
 }
 
 struct AbsorbTc5Params {
@@ -193,7 +202,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
         const uint32_t lane_base = tmem + ((uint32_t)((warp & 3) * 32) << 16);
         constexpr int HT = C::TT / C::NQ;                       // tokens per thread and tile
         bool ok = true;
-        float zacc = 0.f;
+        float2 zacc = make_float2(0.f, 0.f);
         // Warps whose lanes lie past the head dimension (the upper two quadrants at head_dim 64) have no part in the tile
         // loop and must stay out of it: they would wait on the stage barriers without ever arriving on the "free" ones, so
         // nothing would keep the pipeline from running more than a ring ahead of them, and a warp that falls NST tiles
@@ -220,7 +229,7 @@ k_absorb_tc5(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ C
         // idle by now: every TMA copy has been consumed) so that the partial is written with coalesced stores
         pdl_trigger();          // the reduce/fold kernel may be launched now: it waits for this grid before it reads a partial
         if (ok && active) {
-            z_x[part * D + a] = zacc;
+            z_x[part * D + a] = zacc.x + zacc.y;
             mbar_arrive(bar_z);
         }
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar_dfull, 0, abort_flag, p.dev_status, 37));
