@@ -65,7 +65,9 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const uint32_t s_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t sK = s_base + C::OFF_K, sV = s_base + C::OFF_V, bar0 = s_base + C::OFF_BAR;
-    const uint32_t bar_full = bar0, bar_kfree = bar0 + 32, bar_vfree = bar0 + 64, bar_afull = bar0 + 96, bar_afree = bar0 + 112,
+    // bar_full[s] completes for a tile when its K / V bytes have landed AND the A buffer the tile will use is free again
+    // (the tensor core has consumed the tile two before it): one wait per tile for the phi warps instead of two.
+    const uint32_t bar_full = bar0, bar_kfree = bar0 + 32, bar_vfree = bar0 + 64, bar_afull = bar0 + 96,
                    bar_dfull = bar0 + 128, bar_pfree = bar0 + 144, bar_zfull = bar0 + 160;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 176);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 180);
@@ -78,15 +80,21 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
     const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
     auto split_lo = [&](int s) { return (int)(((long long)n_tiles * s) / nsplit); };       // first tile of split s
     auto group_lo = [&](int g) { return (int)(((long long)nsplit * g) / ngroup); };        // first split of group g
+    int my_tiles = 0;                                                                       // tiles of all units of this thread block
+    for (int n = 0; n < my_units; ++n) {
+        const int grp = (blockIdx.x + n * gridDim.x) % ngroup;
+        my_tiles += split_lo(group_lo(grp + 1)) - split_lo(group_lo(grp));
+    }
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_kfree + 8 * s, C::NQ * D); mbar_init(bar_vfree + 8 * s, 1); }
+        for (int s = 0; s < C::NST; ++s) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_kfree + 8 * s, C::NQ * D); mbar_init(bar_vfree + 8 * s, 1); }
         for (int s = 0; s < 2; ++s) {
-            mbar_init(bar_afull + 8 * s, C::NQ * D); mbar_init(bar_afree + 8 * s, 1);
+            mbar_init(bar_afull + 8 * s, C::NQ * D);
             mbar_init(bar_dfull + 8 * s, 1); mbar_init(bar_pfree + 8 * s, D); mbar_init(bar_zfull + 8 * s, C::NQ * D);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        mbar_arrive(bar_full); mbar_arrive(bar_full + 8);     // the A buffers of the first two tiles are free from the start
     }
     if (warp == C::WARP_MMA) {
         tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
@@ -158,7 +166,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                             mma_ts(tP, tA + ks * 8, db, IDESC, tile > lo || ks > 0);        // hi half
                             mma_ts(tP, tA + 32 + ks * 8, db, IDESC, true);                  // lo half
                         }
-                        mma_commit(bar_afree + 8 * ab);
+                        if (g + 2 < my_tiles) mma_commit(bar_full + 8 * ((g + 2) % C::NST));    // this tile's A buffer is the next-but-one's
                         mma_commit(bar_vfree + 8 * s);
                         if (tile == hi - 1) mma_commit(bar_dfull + 8 * pb);
                     }
@@ -245,11 +253,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                     const int s = g % C::NST, ab = g & 1;
                     ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, (g / C::NST) & 1, abort_flag, p.dev_status, 68));
                     if (!ok) break;
-                    if (g >= 2) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(bar_afree + 8 * ab, ((g >> 1) & 1) ^ 1, abort_flag, p.dev_status, 69));
-                        if (!ok) break;
-                        fence_after_sync();
-                    }
+                    fence_after_sync();
                     absorb_phi_tile<D, ROPE>(s_gen + C::OFF_K + s * C::K_BYTES, p.n_tokens, tile * C::TT, part, a,
                                              lane_base + C::COL_A + ab * 64, p.cos_k, p.sin_k, p.rope_rows, zacc);
                     tmem_wait_st();

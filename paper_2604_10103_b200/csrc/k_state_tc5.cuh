@@ -75,9 +75,8 @@ __device__ __forceinline__ void absorb_phi_tile_t(const uint8_t* k_tile, int nv,
         }
         const uint32_t hp = pack_bf16(f0, f1);
         const float2 hf = unpack_bf16(hp);
-        const float2 res = fadd2(make_float2(f0, f1), make_float2(-hf.x, -hf.y));      // exact: the bf16 rounding error
         hi[t >> 1] = hp;
-        lo[t >> 1] = pack_bf16(res.x, res.y);
+        lo[t >> 1] = pack_bf16(f0 - hf.x, f1 - hf.y);       // (the differences are exact: the bf16 rounding errors)
     }
     const uint32_t tA = tA_buf + part * (HT / 2);
     tc5::tmem_st8(tA, hi);
