@@ -481,6 +481,35 @@ def run_sweep(args):
         out.close()
 
 
+def run_profile_stage(args):
+    """A small stand-alone run of one stage, for profilers: the layer-batched state update on 13 layers of the
+    832x480 layer shape (156 (layer, head) items, under 1 GB on the device; no cache ring is allocated)."""
+    import torch
+    from paper_2604_10103_b200 import binding as hf, build as hfbuild
+    hfbuild.build()
+    L = 13
+    w = gen.layer_832x480().with_(layers=L, window_frames=3)        # window == chunk: no ring
+    ctx = hf.Context(hf.make_config(w))
+    for l in range(L):
+        Wb, bb = gen.merge_weights(w, l)
+        ctx.hf_set_merge_weights(l, hf.bits_to_cuda(Wb), hf.bits_to_cuda(bb))
+    g = torch.Generator(device="cuda"); g.manual_seed(99)
+    shape = (L, w.batch, w.heads, w.chunk_tokens, w.head_dim)
+    k = torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    v = torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        if i == 2:
+            a.record()
+        ctx.hf_state_absorb_layers(0, L, k, v, w.chunk_tokens)
+    b.record(); torch.cuda.synchronize()
+    nbytes = 2 * k.numel() * 2
+    us = a.elapsed_time(b) * 1e3
+    print(json.dumps({"stage": "absorb_layers", "layers": L, "us": us, "gbs": nbytes / (us * 1e-6) / 1e9, "status": ctx.hf_get_device_status()}))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -498,9 +527,13 @@ def main():
                     help="instead of the benchmark line: per-stage times over the keep x window x head_dim x block x batch grid, "
                          "one JSON line per point (1 GPU)")
     ap.add_argument("--sweep-out", default=None, help="file for the sweep's JSON lines (default: stdout)")
+    ap.add_argument("--profile-stage", default=None, choices=["absorb_layers"],
+                    help="instead of the benchmark line: a small run of one stage alone (for ncu captures)")
     args = ap.parse_args()
     w = gen.full_depth_832x480(layers=args.layers, steps=args.denoise_steps)
-    if args.sweep:
+    if args.profile_stage:
+        run_profile_stage(args)
+    elif args.sweep:
         run_sweep(args)
     elif args.impl == "reference":
         run_reference(args, w)
