@@ -12,6 +12,12 @@
  * synchronise.  Every call returns an hf_status; an invalid argument never launches a kernel.
  * Nothing here throws, aborts or traps the device.
  *
+ * Concurrency: ONE stream per context at a time.  The scratch buffers (pooled means, split partial sums, the history
+ * term of the two-kernel forward path, the staging buffers of the *_host calls), the side stream and its two events
+ * belong to the context, not to a layer: two calls on the same context whose work may overlap on the device -- two
+ * streams, or two host threads -- race on them, even for different layers.  Calls on one stream, in any order of layers,
+ * are safe; so are different contexts on different streams.  To change streams, synchronise the old one first.
+ *
  * Logical key-block order seen by selection and attention: oldest cached chunk first, newest cached
  * chunk, then the current chunk.  Every chunk is cut into blocks of `block` tokens from its own first
  * token; a short last block is legal (its mean uses its own length).
@@ -193,7 +199,7 @@ hf_status hf_kv_append_host(hf_ctx* ctx, int layer, const void* k_host, const vo
  *   S           device float [batch_heads, head_dim, head_dim], updated in place (caller initialises it)
  *   z           device float [batch_heads, head_dim], updated in place
  * Limits: head_dim in {64, 128}; 1 <= batch_heads <= 1024 and batch_heads * (head_dim^2 + head_dim) * 4 bytes must
- * fit in 16 MiB - 4 KiB (253 batch*heads at head_dim 128, 1007 at head_dim 64); anything larger returns HF_ERR_SHAPE
+ * fit in 16 MiB - 4 KiB (253 batch*heads at head_dim 128, 1008 at head_dim 64); anything larger returns HF_ERR_SHAPE
  * and launches nothing.  All pointers 16-byte aligned (else HF_ERR_INVALID_ARG).
  * The first call on a device looks up the device address of the scratch array and sets a kernel attribute; make
  * that first call outside any stream capture.  No call here uses cudaMalloc, cudaFree or an allocating library routine.

@@ -251,7 +251,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 float2 zacc = make_float2(0.f, 0.f);
                 for (int tile = lo; ok && tile < hi; ++tile, ++g) {
                     const int s = g % C::NST, ab = g & 1;
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_full + 8 * s, (g / C::NST) & 1, abort_flag, p.dev_status, 68));
+                    ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_full + 8 * s, (g / C::NST) & 1, abort_flag, p.dev_status, 68));
                     if (!ok) break;
                     fence_after_sync();
                     absorb_phi_tile<D, ROPE>(s_gen + C::OFF_K + s * C::K_BYTES, p.n_tokens, tile * C::TT, part, a,
@@ -264,7 +264,7 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                 if (!ok) break;
                 // the split's sums: the buffer was read by the merge warps two splits ago
                 if (q >= 2) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(bar_pfree + 8 * pb, ((q >> 1) & 1) ^ 1, abort_flag, p.dev_status, 70));
+                    ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_pfree + 8 * pb, ((q >> 1) & 1) ^ 1, abort_flag, p.dev_status, 70));
                     if (!ok) break;
                 }
                 z_x[(pb * C::NQ + part) * D + a] = zacc.x + zacc.y;
