@@ -5,6 +5,7 @@
 #include "k_swa_mma.cuh"
 #include "k_swa_tc5.cuh"
 #include "k_swa_tc5p.cuh"
+#include "k_swa_tc5g.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
 #include "k_state_items.cuh"
@@ -88,6 +89,9 @@ struct hf_ctx {
     float* hist = nullptr;           // fp32 [B*H, T_c, d]: history term handed to the attention epilogue
     bf16* x_hi = nullptr;            // full-width merge: the read-out h of all heads as bf16 hi + lo, [B*H, T_c, d] each
     bf16* x_lo = nullptr;
+    uint32_t* union_entries = nullptr;   // small-block tcgen05 attention: merged kept lists [B*H * units, max tiles, G] ...
+    int* union_tiles = nullptr;          // ... and tiles per unit
+    int union_max_tiles = 0;
     float* partials = nullptr;       // absorb split partials
     float* partials_layers = nullptr;    // layer-batched state update: one partial per (layer, batch*head, group)
     size_t partials_layers_count = 0;
@@ -171,7 +175,7 @@ void free_all(hf_ctx* c) {
     for (auto& L : c->layers) { cudaFree(L.W_full); cudaFree(L.mask); cudaFree(L.idx); }
     cudaFree(c->ring_k_all); cudaFree(c->ring_v_all); cudaFree(c->pooled_k_all); cudaFree(c->S_all); cudaFree(c->z_all);
     cudaFree(c->sf_hi_all); cudaFree(c->sf_lo_all); cudaFree(c->W_all); cudaFree(c->bias_all);
-    cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
+    cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
@@ -488,8 +492,53 @@ hf_status launch_swa_tc5p_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16*
     return post_launch(c, "k_swa_tc5p");
 }
 
+// Blocks of 16 or 64 tokens on the tcgen05 path: merge the kept lists of the query blocks that share a 128-row unit
+// (k_union_tiles), then the attention kernel over 128-key tiles made of 128 / BLK key blocks each.
+template <int D, int BLK>
+hf_status launch_swa_tc5g_t(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
+                            int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    typedef SwaTc5<D, 2> C;
+    constexpr int G = 128 / BLK;
+    const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
+    const int Tmt = (c->Tc + 127) / 128;
+    const int uni = G * keep < Tn ? G * keep : Tn;
+    const int max_tiles = (uni + G - 1) / G;
+    if (max_tiles > c->union_max_tiles) return fail(HF_ERR_SHAPE, "tile list of %d tiles exceeds the %d the context was sized for", max_tiles, c->union_max_tiles);
+    PdlLaunch pu(dim3(Tmt, c->BH), dim3(256), 0, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pu.cfg, k_union_tiles<BLK>, idx, keep, c->Tm, Tn, c->n_b, c->Tc, max_tiles, c->union_entries, c->union_tiles,
+                               c->dev_status));
+    HF_TRY(post_launch(c, "k_union_tiles"));
+    CUtensorMap tq, tk, tv, to;
+    HF_TRY(make_map(c, &tq, q, 1));
+    HF_TRY(make_map_ex(c, &tk, k_cur, c->Tc, 1, 64, BLK, true));
+    HF_TRY(make_map_ex(c, &tv, v_cur, c->Tc, 1, 64, BLK, true));
+    HF_TRY(make_map_ex(c, &to, o, c->Tc, 1, 64, 32, true));
+    Tc5GParams p;
+    memset(&p, 0, sizeof(p));
+    p.entries = c->union_entries; p.tiles = c->union_tiles; p.max_tiles = max_tiles;
+    p.Tmt = Tmt; p.n_units = Tmt * c->BH;
+    p.idx = idx; p.keep = keep; p.Tm = c->Tm;
+    p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.P = c->R; p.n_sink = L.n_sink;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D));
+    p.hist = hist; p.q = q; p.o = o; p.lse = lse; p.dev_status = c->dev_status;
+    p.tab = make_table(c, L, k_cur, v_cur);
+    const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_tc5g<D, BLK>, tq, rk, rv, tk, tv, to, p));
+    return post_launch(c, "k_swa_tc5g");
+}
+
 hf_status launch_swa(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx,
                      int keep, const float* hist, bf16* o, float* lse, cudaStream_t st) {
+    if (c->swa_kernel == HF_SWA_TCGEN05 && c->cfg.block != 128) {
+        const int b = c->cfg.block, d = c->d;
+        if (b == 64 && d == 128) return launch_swa_tc5g_t<128, 64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+        if (b == 64 && d == 64) return launch_swa_tc5g_t<64, 64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+        if (b == 16 && d == 128) return launch_swa_tc5g_t<128, 16>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+        return launch_swa_tc5g_t<64, 16>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
+    }
     if (c->swa_kernel == HF_SWA_TCGEN05_PINGPONG) {
         if (c->d == 128) return launch_swa_tc5p_t<128>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
         return launch_swa_tc5p_t<64>(c, L, q, k_cur, v_cur, idx, keep, hist, o, lse, st);
@@ -572,8 +621,8 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
     c->nsplit_max = c->sm_count / c->BH;          // one wave: the absorb kernel runs one thread block per SM
     if (c->nsplit_max > 32) c->nsplit_max = 32;
     if (c->nsplit_max < 1) c->nsplit_max = 1;
-    if ((cfg->swa_kernel == HF_SWA_TCGEN05 || cfg->swa_kernel == HF_SWA_TCGEN05_PINGPONG) && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the tcgen05 attention kernels need block == 128"); }
-    c->swa_kernel = (cfg->swa_kernel == HF_SWA_MMA || cfg->block != 128) ? HF_SWA_MMA
+    if (cfg->swa_kernel == HF_SWA_TCGEN05_PINGPONG && cfg->block != 128) { delete c; return fail(HF_ERR_UNSUPPORTED, "the ping-pong attention kernel needs block == 128"); }
+    c->swa_kernel = cfg->swa_kernel == HF_SWA_MMA ? HF_SWA_MMA
                     : (cfg->swa_kernel == HF_SWA_TCGEN05_PINGPONG ? HF_SWA_TCGEN05_PINGPONG : HF_SWA_TCGEN05);
     {
         cudaDriverEntryPointQueryResult qres;
@@ -632,10 +681,17 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
         }
         if (s == HF_OK) s = dmalloc(&L.mask, (size_t)c->BH * c->Tm * c->mask_words);
         if (s == HF_OK) s = dmalloc(&L.idx, (size_t)c->BH * c->Tm * c->max_Tn);
-        if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_kring, L.ring_k, (int)slots);
-        if (s == HF_OK && slots > 0) s = make_map(c, &L.tm_vring, L.ring_v, (int)slots);
+        // the attention kernels fetch key blocks: boxes of `block` rows
+        if (s == HF_OK && slots > 0) s = make_map_ex(c, &L.tm_kring, L.ring_k, c->Tc, (int)slots, 64, cfg->block, true);
+        if (s == HF_OK && slots > 0) s = make_map_ex(c, &L.tm_vring, L.ring_v, c->Tc, (int)slots, 64, cfg->block, true);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sfhi, L.sf_hi, c->d, 1, 64, c->d, true);
         if (s == HF_OK) s = make_map_ex(c, &L.tm_sflo, L.sf_lo, c->d, 1, 64, c->d, true);
+    }
+    if (s == HF_OK && cfg->block != 128) {
+        const int G = 128 / cfg->block, Tmt = (c->Tc + 127) / 128;
+        c->union_max_tiles = (c->max_Tn + G - 1) / G;
+        s = dmalloc(&c->union_entries, (size_t)c->BH * Tmt * c->union_max_tiles * G);
+        if (s == HF_OK) s = dmalloc(&c->union_tiles, (size_t)c->BH * Tmt);
     }
     if (s == HF_OK) s = dmalloc(&c->pooled_q, c->pooled_elems);
     if (s == HF_OK) s = dmalloc(&c->pooled_kcur, c->pooled_elems);
@@ -666,6 +722,11 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
             if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5<128, Tc5Groups<128>::N, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, Tc5Groups<128>::N>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5<128, history>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<64, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<64, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<64>) failed");
         if (s == HF_OK && cudaFuncSetAttribute(k_swa_tc5p<128, HF_TC5P_COLGROUPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5P<128, HF_TC5P_COLGROUPS>::SMEM_BYTES) != cudaSuccess) s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5p<128>) failed");
+        if (s == HF_OK && (cudaFuncSetAttribute(k_swa_tc5g<64, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, 2>::SMEM_BYTES) != cudaSuccess ||
+                           cudaFuncSetAttribute(k_swa_tc5g<64, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<64, 2>::SMEM_BYTES) != cudaSuccess ||
+                           cudaFuncSetAttribute(k_swa_tc5g<128, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, 2>::SMEM_BYTES) != cudaSuccess ||
+                           cudaFuncSetAttribute(k_swa_tc5g<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, 2>::SMEM_BYTES) != cudaSuccess))
+            s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5g) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }
@@ -940,7 +1001,7 @@ static hf_status attend_merge(hf_ctx* c, LayerState& L, const bf16* q, const bf1
     // At head_dim 128 the tcgen05 attention kernel forms the history term itself (three more tensor-core products per
     // query block against the folded state, which it keeps in shared memory): no read-out kernel, no scratch buffer.
     // The rotated variant of Eq. 4 (numerator and denominator see different phi(Q)) keeps the separate read-out.
-    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q &&
+    if (c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && c->cfg.block == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q &&
         c->cfg.merge != HF_MERGE_FULL_WIDTH)
         return launch_swa_tc5_t<128>(c, L, q, k, v, idx, keep, nullptr, o, nullptr, st, true, after_select);
     // Otherwise the read-out kernel writes the history term to the context's scratch buffer and the attention kernel adds
@@ -973,8 +1034,8 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     HF_TRY(check_ptr(o, "o"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
-    const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE && !c->has_rope_q &&
-                            c->cfg.merge != HF_MERGE_FULL_WIDTH;
+    const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && c->cfg.block == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE &&
+                            !c->has_rope_q && c->cfg.merge != HF_MERGE_FULL_WIDTH;
     if (one_kernel) {
         HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
         return attend_merge(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, (bf16*)o, st, true);

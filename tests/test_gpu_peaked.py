@@ -15,7 +15,7 @@ from tests import harness as hz
 pytestmark = pytest.mark.gpu
 
 f64 = gen.bf16_bits_to_f64
-KERNELS = [0, 3, 1]          # HF_SWA_AUTO (tcgen05 at 128-token blocks), tcgen05 ping-pong, warp-level
+KERNELS = [0, 3, 1]          # HF_SWA_AUTO (tcgen05), tcgen05 ping-pong (128-token blocks only), warp-level
 
 
 def small(d=128, b=128, tpf=300, seed=51, permille=600, heads=2):
@@ -70,8 +70,8 @@ def test_newest_blocks_dominate_by_seventy_nats(kernel, d, b, amount):
     """Queries and the current chunk's keys are shifted along one direction: the row's first kept blocks (older chunks)
     lie ~70 natural-log units below the current chunk's.  Inside the range of the fixed softmax reference: the tcgen05
     kernel must handle it in its tile stream."""
-    if kernel != 1 and b != 128:
-        pytest.skip("the tcgen05 kernels are selected by 128-token blocks")
+    if kernel == 3 and b != 128:
+        pytest.skip("the ping-pong kernel takes 128-token blocks only")
     w = small(d=d, b=b, tpf=300 if b == 128 else 150)
     u = gen.direction(w, 0)
     qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, amount), gen.shifted(k, u, amount), v))(*gen.qkv(w, 0, c, 0))
@@ -91,12 +91,14 @@ def test_oldest_block_dominates_by_sixty_nats(kernel):
 
 
 @pytest.mark.parametrize("kernel", KERNELS)
-@pytest.mark.parametrize("d,amount", [(128, 4.0), (64, 4.8)])
-def test_logits_beyond_the_fixed_reference_take_the_running_maximum_pass(kernel, d, amount):
+@pytest.mark.parametrize("d,b,amount", [(128, 128, 4.0), (64, 128, 4.8), (128, 64, 4.0), (64, 16, 4.8), (128, 16, 4.0)])
+def test_logits_beyond_the_fixed_reference_take_the_running_maximum_pass(kernel, d, b, amount):
     """The current chunk's keys lie ~180 natural-log units above the cached ones: past what a reference fixed at the first
-    kept block covers in fp32.  The tcgen05 kernel must notice, compute those units again with the running maximum and
+    kept block covers in fp32.  The tcgen05 kernels must notice, compute those units again with the running maximum and
     return the oracle's numbers (with and without the history term), with a clean status word."""
-    w = small(d=d, seed=52)
+    if kernel == 3 and b != 128:
+        pytest.skip("the ping-pong kernel takes 128-token blocks only")
+    w = small(d=d, b=b, tpf=300 if b == 128 else 150, seed=52)
     u = gen.direction(w, 0)
     qkv = lambda c: (lambda q, k, v: (gen.shifted(q, u, amount), gen.shifted(k, u, amount), v))(*gen.qkv(w, 0, c, 0))
     run_stream(w, kernel, qkv, lambda c: gen.clean_kv(w, 0, c), 5, check_from=2, expect_slow=True if kernel == 0 else None)
