@@ -31,7 +31,7 @@ def test_small_blocks_resolve_to_the_tcgen05_kernel():
 @pytest.mark.parametrize("d,b,tpf,cf,wf,B,H,permille", [
     (64, 16, 64, 1, 3, 1, 2, 170),       # the tiny configuration's shape (top-2 of 12)
     (128, 64, 1560, 1, 3, 1, 3, 250),    # 25 query blocks of 64 (24 full + 24 tokens): units of two query blocks, ragged last unit
-    (64, 64, 1000, 1, 9, 2, 2, 100),     # eight cached chunks, sparse lists: tiles with a single useful block
+    (64, 64, 1000, 1, 8, 2, 2, 100),     # seven cached chunks, sparse lists: tiles with a single useful block
     (128, 16, 300, 1, 3, 1, 2, 500),     # 19 query blocks of 16: last unit holds 3 of 8 row groups, 12-token tail block
     (64, 16, 520, 1, 2, 1, 3, 1000),     # everything kept: every tile fully used
     (128, 64, 200, 1, 1, 1, 2, 1000),    # window == chunk
