@@ -126,8 +126,9 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy_layers(const __grid_consta
 // l + 32, ... ascending, product and sum rounded separately; lane l holds partial l, so the loads of a key row are
 // coalesced), then the butterfly p[l] + p[l ^ off], off = 16 .. 1: both partners get the same value (IEEE addition
 // commutes), so lane 0 ends with the fold of the upper half onto the lower half level by level, bit for bit.
-// grid (T_m, B*H), 256 threads.  One query-block row: T_n scores, rank-based top-K under the total order
-// (score descending, block index ascending), bit mask + ascending index list.
+// grid (T_m, B*H), 256 threads.  One query-block row: T_n scores, top-K under the total order (score descending, block
+// index ascending; by counting for short rows, by a bitonic sort of (score, index) keys for long ones), bit mask +
+// ascending index list.
 template <int D>
 __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __restrict__ pooled_q,
                                                 int n_b, int Tm, int Tn, int keep, int mask_words,
@@ -136,6 +137,7 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
                                                 float* __restrict__ scores_out) {
     __shared__ float sc[HF_MAX_TN];
     __shared__ uint8_t keepf[HF_MAX_TN];
+    __shared__ unsigned long long keys[HF_MAX_TN];
     const int i = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const size_t row = (size_t)bh * Tm + i;
@@ -172,20 +174,53 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
         }
     }
     __syncthreads();
-    // Rank under a TOTAL order: a NaN score (a NaN anywhere in the query block or the key block) compares false both
-    // ways, which would give every NaN rank 0 and more than `keep` entries per row; here NaN ranks below every number
-    // (NaNs among themselves by block index), so that exactly `keep` blocks are kept whatever the inputs hold.
-    for (int j = threadIdx.x; j < Tn; j += 256) {
-        const float s = sc[j];
-        const bool s_nan = s != s;
-        int rank = 0;
-        for (int jj = 0; jj < Tn; ++jj) {
-            const float s2 = sc[jj];
-            const bool s2_nan = s2 != s2;
-            const bool tie = (s2 == s) || (s_nan && s2_nan);
-            rank += (s2 > s) || (s_nan && !s2_nan) || (tie && jj < j);
+    // Keep the `keep` best under a TOTAL order: score descending, then block index ascending; +0 and -0 tie; a NaN score (a
+    // NaN anywhere in the query block or the key block) compares false both ways and would otherwise rank first everywhere:
+    // here it ranks below every number, NaNs among themselves by block index, so that exactly `keep` blocks are kept whatever
+    // the inputs hold.
+    if (Tn <= 128) {
+        // short rows: count, for every block, the blocks that come before it
+        for (int j = threadIdx.x; j < Tn; j += 256) {
+            const float s = sc[j];
+            const bool s_nan = s != s;
+            int rank = 0;
+            for (int jj = 0; jj < Tn; ++jj) {
+                const float s2 = sc[jj];
+                const bool s2_nan = s2 != s2;
+                const bool tie = (s2 == s) || (s_nan && s2_nan);
+                rank += (s2 > s) || (s_nan && !s2_nan) || (tie && jj < j);
+            }
+            keepf[j] = rank < keep;
         }
-        keepf[j] = rank < keep;
+    } else {
+        // long rows (counting is quadratic in T_n): sort 64-bit keys (order-preserving image of the score, then the
+        // complement of the index) in shared memory with a bitonic network and compare every block with the keep-th key
+        auto key_of = [](float s, int j) -> unsigned long long {
+            uint32_t u = __float_as_uint(s);
+            if (s != s) u = 0u;                                         // NaN: below -inf
+            else {
+                if (u == 0x80000000u) u = 0u;                           // -0 ties with +0
+                u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);         // ascending integers = ascending floats
+            }
+            return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)j);
+        };
+        int n2 = 256;
+        while (n2 < Tn) n2 <<= 1;
+        for (int j = threadIdx.x; j < n2; j += 256) keys[j] = j < Tn ? key_of(sc[j], j) : 0ull;      // padding sorts last
+        __syncthreads();
+        for (int size = 2; size <= n2; size <<= 1) {
+            for (int stride = size >> 1; stride > 0; stride >>= 1) {
+                for (int x = threadIdx.x; x < (n2 >> 1); x += 256) {
+                    const int lo = 2 * x - (x & (stride - 1)), hi = lo + stride;      // the pair (lo, lo + stride)
+                    const bool descending = (lo & size) == 0;
+                    const unsigned long long a = keys[lo], b = keys[hi];
+                    if ((a < b) == descending) { keys[lo] = b; keys[hi] = a; }
+                }
+                __syncthreads();
+            }
+        }
+        const unsigned long long kth = keys[keep - 1];
+        for (int j = threadIdx.x; j < Tn; j += 256) keepf[j] = key_of(sc[j], j) >= kth;
     }
     __syncthreads();
     if (warp == 0) {
