@@ -24,6 +24,9 @@ What follows which passage:
   linear_readout          Eq. 4: Linear(phi(Q) L / (phi(Q) H)), optionally with RoPE(phi(Q)) in the numerator
   rotate_pairs, absorb_rope        the rotation of Eq. 3 / Eq. 4 on feature pairs (2i, 2i+1); angles are inputs
   relative_temporal_indices        Eq. 8 (capped relative temporal index)
+  window_temporal_indices, rotate_temporal   Sec. 3.3: the indices of cached chunks follow their offset to the current chunk;
+                          the temporal rotation of the softmax branch's queries and keys
+  rotate_temporal_f32     the same rotation in the canonical float32 order with the bf16 rounding the cache applies
   HybridStream            Alg. 2 cache protocol (evict -> update state -> append) around Alg. 3, Eq. 7 sum
 
 Readings taken where the paper is silent or inconsistent (all listed again in the
@@ -259,6 +262,66 @@ def relative_temporal_indices(i: int, t0: int):
     return [i - 2, i - 1, i] if i <= t0 else [t0 - 2, t0 - 1, t0]
 
 
+def window_temporal_indices(cur_last_frame: int, chunk_last_frames, t0: int, chunk_frames: int):
+    """Sec. 3.3 ("the temporal RoPE indices in the KV cache are updated based on the offsets to the current chunk"):
+    the current chunk, whose last frame is the stream's (1-based) frame cur_last_frame, takes Eq. 8's indices; a cached
+    chunk whose last frame was frame f keeps its distance to it: its last frame has index top - (cur_last_frame - f),
+    top = min(cur_last_frame, T_0).  Returns (indices of the current chunk's frames, [indices per cached chunk])."""
+    cur = relative_temporal_indices(cur_last_frame, t0) if chunk_frames == 3 else \
+        [min(cur_last_frame, t0) - chunk_frames + 1 + i for i in range(chunk_frames)]
+    top = cur[-1]
+    cached = [[top - (cur_last_frame - f) - chunk_frames + 1 + i for i in range(chunk_frames)] for f in chunk_last_frames]
+    return cur, cached
+
+
+def temporal_tables(frame_indices, tokens_per_frame: int, d: int, first_pair: int, omegas):
+    """cos / sin tables [T, d/2] of a chunk for rotate_pairs: pair first_pair + n turns by index * omegas[n], where index
+    is the temporal index of the token's frame; every other pair is left alone (their rotation, by the spatial
+    coordinates, is the caller's and does not change while a key sits in the cache)."""
+    omegas = np.asarray(omegas, np.float64)
+    idx = np.repeat(np.asarray(frame_indices, np.float64), tokens_per_frame)
+    cos = np.ones((idx.shape[0], d // 2)); sin = np.zeros((idx.shape[0], d // 2))
+    ang = idx[:, None] * omegas[None, :]
+    cos[:, first_pair:first_pair + omegas.shape[0]] = np.cos(ang)
+    sin[:, first_pair:first_pair + omegas.shape[0]] = np.sin(ang)
+    return cos, sin
+
+
+def rotate_temporal(x, frame_indices, tokens_per_frame: int, first_pair: int, omegas) -> np.ndarray:
+    """Temporal RoPE of the softmax branch: x [T, d] (T = frames * tokens_per_frame), one index per frame."""
+    cos, sin = temporal_tables(frame_indices, tokens_per_frame, np.asarray(x).shape[1], first_pair, omegas)
+    return rotate_pairs(x, cos, sin)
+
+
+def bf16_round_f32(x: np.ndarray) -> np.ndarray:
+    """float32 -> nearest bf16 (ties to even) -> float32; finite input."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    r = (u + (np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1)))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32)
+
+
+def rotate_temporal_f32(x: np.ndarray, frame_steps, tokens_per_frame: int, first_pair: int, cos_tab: np.ndarray,
+                        sin_tab: np.ndarray) -> np.ndarray:
+    """The rotation as the cache stores it (part of the bit-exact selection contract, like the float32 scorer): x float32
+    [T, d] holding bf16 values; frame f turns by frame_steps[f] index steps (negative: backwards), the angle's cosine and
+    sine taken from the float32 tables cos_tab / sin_tab [steps, pairs] at |steps| (sine negated for a backward turn);
+    x0' = x0 c - x1 s and x1' = x0 s + x1 c with every product and the sum rounded separately in float32; the result
+    rounded to bf16.  Pairs outside [first_pair, first_pair + pairs) pass through."""
+    x = np.asarray(x)
+    assert x.dtype == np.float32
+    out = x.copy()
+    n = cos_tab.shape[1]
+    steps = np.repeat(np.asarray(frame_steps, np.int64), tokens_per_frame)
+    c = cos_tab[np.abs(steps)].astype(F32)
+    s_ = (sin_tab[np.abs(steps)] * np.where(steps < 0, F32(-1.0), F32(1.0))[:, None]).astype(F32)
+    x0 = x[:, 2 * first_pair:2 * (first_pair + n):2]; x1 = x[:, 2 * first_pair + 1:2 * (first_pair + n):2]
+    y0 = (x0 * c).astype(F32) - (x1 * s_).astype(F32)
+    y1 = (x0 * s_).astype(F32) + (x1 * c).astype(F32)
+    out[:, 2 * first_pair:2 * (first_pair + n):2] = bf16_round_f32(y0.astype(F32))
+    out[:, 2 * first_pair + 1:2 * (first_pair + n):2] = bf16_round_f32(y1.astype(F32))
+    return out
+
+
 def linear_readout(q, S, z, W=None, bias=None, eps: float = 1e-6, cos_q=None, sin_q=None) -> np.ndarray:
     """O_history (Eq. 4): h = phi(q) S / (phi(q) . z + eps) per query row, then Linear: y = W h + bias.
     With cos_q / sin_q [T, d/2] the numerator uses RoPE(phi(q)) (Eq. 4 as printed); the denominator never rotates."""
@@ -298,7 +361,7 @@ class HybridStream:
 
     def __init__(self, batch, heads, d, b, past_chunks, topk=0, keep_permille=0,
                  W=None, bias=None, eps=1e-6, z_frame_tokens=None, sink_chunks=0, rope_q=None, rope_k=None,
-                 W_full=None, bias_full=None):
+                 W_full=None, bias_full=None, temporal=None):
         self.B, self.H, self.d, self.b, self.P = batch, heads, d, b, past_chunks
         self.z_frame_tokens = z_frame_tokens     # None: z is the plain sum of phi(K); n: per-frame means of n tokens (Eq. 3 literal)
         self.topk, self.keep_permille, self.eps = topk, keep_permille, eps
@@ -315,13 +378,64 @@ class HybridStream:
         self.S = np.zeros((batch, heads, d, d))
         self.z = np.zeros((batch, heads, d))
         self.absorbed_tokens = 0
+        # Relative temporal RoPE of the softmax branch (Sec. 3.3, Eq. 8), or None.  dict(t0, first_pair, cos_tab, sin_tab
+        # [steps, pairs] float32, tokens_per_frame, chunk_frames).  q, k then arrive WITHOUT temporal rotation.  The cache is a
+        # bf16 store: a key enters it rotated to the index it will have while the NEXT chunk is generated, and is turned
+        # further (and rounded to bf16 again) whenever the cap of Eq. 8 makes the window's indices slide; the queries and the
+        # current chunk's keys are rotated to Eq. 8's indices and rounded to bf16 as well (they are the attention kernel's
+        # bf16 operands).  All of it in the canonical float32 order (rotate_temporal_f32), because these values decide the
+        # block selection.  Sink chunks keep the indices they had when they were generated.
+        self.temporal = temporal
+        self.frames_committed = 0
 
     # -- Alg. 2, cache commit
+    def _turn(self, x, frame_steps):
+        """x [B, H, T, d] -> rotated by frame_steps (one entry per frame) in the canonical order, as fp64 of bf16 values."""
+        t = self.temporal
+        out = np.empty(np.asarray(x).shape)
+        for bi in range(self.B):
+            for h in range(self.H):
+                out[bi, h] = rotate_temporal_f32(np.asarray(x[bi, h], np.float64).astype(F32), frame_steps, t["tokens_per_frame"],
+                                                 t["first_pair"], t["cos_tab"], t["sin_tab"])
+        return out
+
+    def current_indices(self):
+        """Eq. 8 for the chunk being generated now."""
+        t = self.temporal
+        c = t["chunk_frames"]
+        top = min(self.frames_committed + c, t["t0"])
+        return [top - c + 1 + i for i in range(c)]
+
+    def rotated_inputs(self, q, k_cur):
+        """(q, k_cur) as the attention sees them: unchanged without temporal rotation, else turned to Eq. 8's indices."""
+        if self.temporal is None:
+            return q, k_cur
+        idx = self.current_indices()
+        return self._turn(q, idx), self._turn(k_cur, idx)
+
     def append(self, k_clean, v_clean):
+        k_clean = np.asarray(k_clean, np.float64)
+        if self.temporal is not None:
+            t = self.temporal
+            c, t0 = t["chunk_frames"], t["t0"]
+            last = self.frames_committed + c                    # (1-based) number of this chunk's last frame
+            top_now, top_next = min(last, t0), min(last + c, t0)
+            self.frames_committed = last
+            if len(self.sink) < self.sink_chunks:               # a sink chunk keeps its own indices for good
+                k_clean = self._turn(k_clean, [top_now - c + 1 + i for i in range(c)])
+            else:
+                # indices during the next chunk: this chunk sits c frames behind it; older chunks slide by the same amount
+                k_clean = self._turn(k_clean, [top_next - 2 * c + 1 + i for i in range(c)])
+                slide = top_next - top_now - c                  # 0 until the cap is reached, then -c
+                if slide != 0:
+                    # all but the chunk that is about to leave (it is folded into the state as the window last saw it)
+                    keep_from = 1 if len(self.past) >= self.P else 0
+                    for n in range(keep_from, len(self.past)):
+                        self.past[n] = (self._turn(self.past[n][0], [slide] * c), self.past[n][1])
         if len(self.sink) < self.sink_chunks:
-            self.sink.append((np.asarray(k_clean, np.float64), np.asarray(v_clean, np.float64)))
+            self.sink.append((k_clean, np.asarray(v_clean, np.float64)))
             return
-        self.past.append((np.asarray(k_clean, np.float64), np.asarray(v_clean, np.float64)))
+        self.past.append((k_clean, np.asarray(v_clean, np.float64)))
         while len(self.past) > self.P:
             k_ev, v_ev = self.past.pop(0)
             for bi in range(self.B):
@@ -344,6 +458,7 @@ class HybridStream:
         """Masks [B, H, T_m, T_n].  exact=False: canonical float32 scores (the bit-exact contract);
         exact=True: fp64 scores (the ideal the canonical order approximates)."""
         B, H = self.B, self.H
+        q, k_cur = self.rotated_inputs(q, k_cur)
         n_kb = self.n_key_blocks(k_cur.shape[2])
         k = keep_count(self.topk, self.keep_permille, n_kb)
         masks, scores = [], []
@@ -372,6 +487,7 @@ class HybridStream:
         q = np.asarray(q, np.float64); k_cur = np.asarray(k_cur, np.float64); v_cur = np.asarray(v_cur, np.float64)
         if mask is None:
             mask, _ = self.select(q, k_cur)
+        q, k_cur = self.rotated_inputs(q, k_cur)        # (both branches see the queries with their temporal rotation)
         o_loc = np.empty_like(q); o_hist = np.empty_like(q)
         for bi in range(self.B):
             for h in range(self.H):

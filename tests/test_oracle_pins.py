@@ -529,3 +529,105 @@ def test_full_width_merge_reduces_to_the_per_head_merge_and_to_scalar_loops():
         st_a.append(k, v); st_b.append(k, v)
     q = rng.standard_normal((1, H, 4, dd)); k = rng.standard_normal((1, H, 4, dd)); v = rng.standard_normal((1, H, 4, dd))
     assert np.allclose(st_a.forward(q, k, v), st_b.forward(q, k, v), atol=1e-12)
+
+
+# --------------------------------------------------------------------------- Sec. 3.3 / Eq. 8: relative temporal RoPE
+def _temporal(t0=9, d=32, first_pair=2, pairs=5, tpf=4, c=3, steps=64):
+    om = 1.0 / (50.0 ** (np.arange(pairs) / pairs))
+    n = np.arange(steps)
+    return dict(t0=t0, first_pair=first_pair, cos_tab=np.cos(n[:, None] * om[None, :]).astype(np.float32),
+                sin_tab=np.sin(n[:, None] * om[None, :]).astype(np.float32), tokens_per_frame=tpf, chunk_frames=c), om
+
+
+def test_window_temporal_indices_hand_values():
+    """Eq. 8 with T_0 = 21 and the rule for cached chunks (offsets to the current chunk), by hand."""
+    assert oa.window_temporal_indices(9, [6, 3], 21, 3) == ([7, 8, 9], [[4, 5, 6], [1, 2, 3]])          # below the cap: absolute
+    assert oa.window_temporal_indices(21, [18, 15], 21, 3) == ([19, 20, 21], [[16, 17, 18], [13, 14, 15]])
+    assert oa.window_temporal_indices(24, [21, 18], 21, 3) == ([19, 20, 21], [[16, 17, 18], [13, 14, 15]])  # capped: window slides
+    assert oa.window_temporal_indices(600, [597, 594], 21, 3) == ([19, 20, 21], [[16, 17, 18], [13, 14, 15]])
+    # T_0 -> infinity: every frame keeps its absolute number
+    assert oa.window_temporal_indices(600, [597, 594], 10 ** 9, 3) == ([598, 599, 600], [[595, 596, 597], [592, 593, 594]])
+    assert oa.window_temporal_indices(5, [4], 21, 1) == ([5], [[4]])
+
+
+def test_temporal_rotation_depends_on_index_differences_only():
+    """<R_a q, R_b k> = <R_(a+s) q, R_(b+s) k>: what makes relative indices meaningful; other pairs are untouched."""
+    t, om = _temporal()
+    q = rnd((12, 32), 90); k = rnd((12, 32), 91)
+    a = oa.rotate_temporal(q, [7, 8, 9], 4, 2, om) @ oa.rotate_temporal(k, [1, 2, 3], 4, 2, om).T
+    b = oa.rotate_temporal(q, [19, 20, 21], 4, 2, om) @ oa.rotate_temporal(k, [13, 14, 15], 4, 2, om).T
+    c = oa.rotate_temporal(q, [7, 8, 9], 4, 2, om) @ oa.rotate_temporal(k, [2, 3, 4], 4, 2, om).T
+    blocks = lambda m: np.stack([m[4 * i:4 * i + 4, 4 * i:4 * i + 4] for i in range(3)])     # frame i of q against frame i of k
+    assert np.abs(blocks(a) - blocks(b)).max() < 1e-12
+    assert np.abs(blocks(a) - blocks(c)).max() > 1e-3
+    r = oa.rotate_temporal(q, [5, 6, 7], 4, 2, om)
+    assert np.array_equal(r[:, :4], q[:, :4]) and np.array_equal(r[:, 14:], q[:, 14:])
+    # one pair, by hand: angle = index * omega
+    th = 6 * om[1]
+    assert np.isclose(r[4, 6], q[4, 6] * np.cos(th) - q[4, 7] * np.sin(th)) and np.isclose(r[4, 7], q[4, 6] * np.sin(th) + q[4, 7] * np.cos(th))
+
+
+def test_canonical_temporal_rotation_is_the_ideal_one_up_to_bf16_rounding():
+    t, om = _temporal()
+    x = oa.bf16_round_f32(rnd((12, 32), 92).astype(np.float32))
+    got = oa.rotate_temporal_f32(x, [4, 5, 6], 4, 2, t["cos_tab"], t["sin_tab"]).astype(np.float64)
+    ideal = oa.rotate_temporal(x.astype(np.float64), [4, 5, 6], 4, 2, om)
+    assert np.abs(got - ideal).max() <= 2.0 ** -8 * np.abs(ideal).max() + 1e-6
+    assert np.array_equal(got[:, :4], x[:, :4].astype(np.float64))
+    assert np.array_equal(oa.bf16_round_f32(got.astype(np.float32)).astype(np.float64), got)       # values are bf16
+    # a backward turn undoes a forward turn up to two roundings
+    back = oa.rotate_temporal_f32(got.astype(np.float32), [-4, -5, -6], 4, 2, t["cos_tab"], t["sin_tab"])
+    assert np.abs(back - x).max() <= 2.0 ** -7 * np.abs(x).max()
+    # bf16 rounding: ties to even, by hand (1 + 2^-8 is a tie between 1 and 1 + 2^-7 -> 1; 1 + 3 * 2^-8 -> 1 + 2^-6)
+    assert oa.bf16_round_f32(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, 1 + 2.0 ** -9], np.float32)).tolist() == [1.0, 1 + 2.0 ** -6, 1.0]
+
+
+def test_stream_with_capped_relative_indices():
+    """Alg. 2 with the relative temporal RoPE: (a) the cache holds every key at the index Eq. 8 and the offset rule give it
+    for the chunk being generated, within the roundings of the bf16 store; (b) below the cap nothing is ever re-rotated;
+    (c) with identical chunks, the attention output no longer changes from chunk to chunk once the stream is past T_0
+    (the softmax branch sees only index differences); (d) sink chunks keep their own indices."""
+    t, om = _temporal(t0=9)
+    B, H, d, tpf, c = 1, 2, 32, 4, 3
+    bf = lambda x: oa.bf16_round_f32(x.astype(np.float32)).astype(np.float64)
+    q = bf(rnd((B, H, tpf * c, d), 93)); k = bf(rnd((B, H, tpf * c, d), 94)); v = bf(rnd((B, H, tpf * c, d), 95))
+    st = oa.HybridStream(B, H, d, 4, 2, topk=3, temporal=t, sink_chunks=1)
+    outs = []
+    for n in range(8):
+        o, o_loc, _ = st.forward(q, k, v, parts=True)
+        outs.append(o_loc)
+        st.append(k, v)
+        last = st.frames_committed
+        frames = [last - 3 * j for j in range(len(st.past))][::-1]
+        _, cached = oa.window_temporal_indices(last + c, frames, 9, c)
+        for (kp, _), idx in zip(st.past, cached):
+            ideal = oa.rotate_temporal(k[0, 0], idx, tpf, 2, om)
+            assert np.abs(kp[0, 0] - ideal).max() <= 3 * 2.0 ** -8 * np.abs(ideal).max()
+        sink_ideal = oa.rotate_temporal(k[0, 0], [1, 2, 3], tpf, 2, om)
+        assert np.abs(st.sink[0][0][0, 0] - sink_ideal).max() <= 2.0 ** -8 * np.abs(sink_ideal).max()
+        if last + c <= 9 and len(st.past) == 2:       # below the cap: a single rounding, exactly the canonical rotation of the raw keys
+            assert np.array_equal(st.past[0][0][0, 0], oa.rotate_temporal_f32(k[0, 0].astype(np.float32), cached[0], tpf, 2,
+                                                                             t["cos_tab"], t["sin_tab"]).astype(np.float64))
+    assert st.absorbed_tokens == 5 * tpf * c           # eight commits: one sink chunk, two still cached, five folded into the state
+    # past the cap with a full window (chunks 5, 6, 7 are generated at frames 18, 21, 24 > T_0 = 9): same softmax output up to the
+    # roundings of the re-rotated keys; the first chunks (growing window, absolute indices) differ
+    assert np.abs(outs[6] - outs[5]).max() < 2e-2 and np.abs(outs[7] - outs[6]).max() < 2e-2
+    assert np.abs(outs[2] - outs[1]).max() > 5e-2
+
+
+def test_stream_without_cap_is_absolute_indexing():
+    """T_0 -> infinity: the stored keys are the raw keys rotated once by their absolute frame numbers, never touched again."""
+    t, om = _temporal(t0=10 ** 6, steps=64)
+    B, H, d, tpf, c = 1, 1, 32, 4, 3
+    bf = lambda x: oa.bf16_round_f32(x.astype(np.float32)).astype(np.float64)
+    st = oa.HybridStream(B, H, d, 4, 2, topk=3, temporal=t)
+    ks = []
+    for n in range(5):
+        k = bf(rnd((B, H, tpf * c, d), 100 + n)); v = bf(rnd((B, H, tpf * c, d), 110 + n))
+        st.append(k, v); ks.append(k)
+        for j, (kp, _) in enumerate(st.past):
+            chunk_no = len(ks) - len(st.past) + j
+            idx = [3 * chunk_no + 1, 3 * chunk_no + 2, 3 * chunk_no + 3]
+            want = oa.rotate_temporal_f32(ks[chunk_no][0, 0].astype(np.float32), idx, tpf, 2, t["cos_tab"], t["sin_tab"])
+            assert np.array_equal(kp[0, 0], want.astype(np.float64))
+    assert st.current_indices() == [16, 17, 18]
