@@ -112,6 +112,25 @@ hf_status hf_set_merge_weights(hf_ctx* ctx, int layer, const void* W, const void
  * rotation off (the default).  With key tables set, hf_state_absorb accepts at most T_c tokens per call. */
 hf_status hf_set_rope(hf_ctx* ctx, const float* cos_q, const float* sin_q, const float* cos_k, const float* sin_k, void* stream);
 
+/* Relative temporal RoPE of the softmax branch (Sec. 3.3, Eq. 8): the temporal index of the chunk being generated counts
+ * up with the stream until it reaches t0 (21 in the paper) and stays there; the keys in the cache are re-indexed by their
+ * offset to the current chunk.  With this set, q and k are passed to every call WITHOUT temporal rotation (their spatial
+ * rotation is the caller's and never changes); the library turns feature pairs [first_pair, first_pair + n_pairs) -- pair p
+ * = features (2p, 2p+1) -- of every token by (index of its frame) x (frequency of the pair):
+ *   - the queries and the current chunk's keys of a forward call to Eq. 8's indices (the stream position is the number of
+ *     frames committed to that layer so far), in the pooling pass that the selection needs anyway; both branches see the
+ *     rotated queries;
+ *   - a committed chunk's keys to the indices they have while the NEXT chunk is generated; once the cap is reached every
+ *     commit turns the chunks that stay in the window back by chunk_frames index steps, in place (keys and block means);
+ *     the chunk that leaves is folded into the state as the window last saw it; sink chunks keep their own indices.
+ * The cache stores bf16, so each turn rounds once more (at most window/chunk roundings in a key's life).
+ *   cos_tab, sin_tab   device float [t0 + 1, n_pairs]: cosine and sine of (index steps) x (frequency of the pair); copied.
+ * Must be set while no chunk has been committed (HF_ERR_STATE otherwise); both tables NULL switches it off.
+ * The order of the float32 operations of a turn is fixed (the rotated values decide the block selection): x0' = x0 c - x1 s,
+ * x1' = x0 s + x1 c, products and sums rounded separately, result rounded to bf16. */
+hf_status hf_set_temporal_rope(hf_ctx* ctx, int t0, int first_pair, int n_pairs, const float* cos_tab, const float* sin_tab,
+                               void* stream);
+
 /* Alg. 2, cache commit of a clean chunk: k, v bf16 [B,H,T_c,d].  If the cache already holds P chunks the oldest
  * is folded into the state (Eq. 3: S += phi(K_ev)^T V_ev, z += sum phi(K_ev)) and leaves the window; the chunk's
  * K, V are copied in and its per-block K means stored.  The ring has P + 1 slots per layer (a spare one), so the copy

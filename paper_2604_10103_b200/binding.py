@@ -28,7 +28,7 @@ EXPORTS = [
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
     "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
-    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit", "hf_kv_append_layers", "hf_state_absorb_layers",
+    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit", "hf_kv_append_layers", "hf_state_absorb_layers", "hf_set_temporal_rope",
 ]
 
 
@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
     L.hf_reset.argtypes = [vp, ip, vp]
     L.hf_set_merge_weights.argtypes = [vp, ip, vp, vp, vp]
     L.hf_set_rope.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.hf_set_temporal_rope.argtypes = [vp, ip, ip, ip, vp, vp, vp]
     L.hf_kv_append.argtypes = [vp, ip, vp, vp, vp]
     L.hf_state_absorb.argtypes = [vp, ip, vp, vp, ip, vp]
     L.hf_state_absorb_layers.argtypes = [vp, ip, ip, vp, vp, ip, vp]
@@ -147,6 +148,10 @@ class Context:
     def hf_set_rope(self, cos_q=None, sin_q=None, cos_k=None, sin_k=None):
         """float32 CUDA tensors [T_c, d/2] (or None) -- see include/hf.h."""
         _check(lib().hf_set_rope(self._h, _ptr(cos_q), _ptr(sin_q), _ptr(cos_k), _ptr(sin_k), _stream()))
+
+    def hf_set_temporal_rope(self, t0, first_pair, n_pairs, cos_tab, sin_tab):
+        """float32 CUDA tensors [t0 + 1, n_pairs] -- see include/hf.h."""
+        _check(lib().hf_set_temporal_rope(self._h, t0, first_pair, n_pairs, _ptr(cos_tab), _ptr(sin_tab), _stream()))
 
     def hf_kv_append(self, layer, k, v):
         _check(lib().hf_kv_append(self._h, layer, _ptr(k), _ptr(v), _stream()))

@@ -56,6 +56,7 @@ struct LayerState {
     int n_cached = 0, head = 0;  // head = slot of the oldest cached chunk
     int n_sink = 0;              // sink chunks held (slots R, R + 1, ...)
     long long absorbed = 0;
+    long long frames = 0;        // latent frames committed so far (sink chunks included): the stream position of Eq. 8
     unsigned long long cache_epoch = 0, sel_epoch = ~0ull;
     int sel_keep = 0;
     CUtensorMap tm_kring, tm_vring;   // 4-D maps over the whole ring [slot, B*H, T_c, d]
@@ -102,6 +103,13 @@ struct hf_ctx {
     float* rope_q[2] = {nullptr, nullptr};   // cos / sin tables [T_c, d/2] of Eq. 4's numerator (nullptr: no rotation)
     float* rope_k[2] = {nullptr, nullptr};   // ... of Eq. 3, applied to a chunk when it is absorbed
     bool has_rope_q = false, has_rope_k = false;
+    // relative temporal RoPE of the softmax branch (Eq. 8): tables over index steps 0 .. t0, rotated copies of q / k_cur
+    bool has_trope = false;
+    int t0 = 0;
+    TemporalRope trope = {nullptr, nullptr, 0, 0, 1};
+    float* trope_tab[2] = {nullptr, nullptr};
+    bf16* q_rot = nullptr;
+    bf16* k_rot = nullptr;
     cudaStream_t side = nullptr;     // hf_hybrid_forward runs the history read-out here, beside pooling + selection
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     long long launches = 0;
@@ -178,6 +186,7 @@ void free_all(hf_ctx* c) {
     cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
+    cudaFree(c->trope_tab[0]); cudaFree(c->trope_tab[1]); cudaFree(c->q_rot); cudaFree(c->k_rot);
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
@@ -228,8 +237,31 @@ template <int D>
 hf_status launch_pool(hf_ctx* c, const PoolJobs& jobs, int njobs, cudaStream_t st) {
     dim3 grid(c->n_b, c->BH, njobs);
     PdlLaunch pl(grid, dim3(256), 0, st, true);
+    bool rot = false;
+    for (int i = 0; i < njobs; ++i) rot = rot || jobs.job[i].rot_on;
+    if (rot) {
+        HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_pool_copy_rot<D>, jobs, c->Tc, c->cfg.block, c->n_b, c->trope));
+        return post_launch(c, "k_pool_copy_rot");
+    }
     HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_pool_copy<D>, jobs, c->Tc, c->cfg.block, c->n_b));
     return post_launch(c, "k_pool_copy");
+}
+
+// Eq. 8: index of the last frame of the chunk that is generated when `frames` frames have been committed.
+inline int trope_top(const hf_ctx* c, long long frames) {
+    const long long last = frames + c->cfg.chunk_frames;
+    return (int)(last < c->t0 ? last : c->t0);
+}
+// q and k_cur turned to the current chunk's indices, into the context's rotated copies (no pooling); k_cur may be null.
+template <int D>
+hf_status launch_rotate_inputs(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, cudaStream_t st) {
+    PoolJobs jobs;
+    memset(&jobs, 0, sizeof(jobs));
+    const int base = trope_top(c, L.frames) - c->cfg.chunk_frames + 1;
+    int n = 0;
+    if (q) { jobs.job[n].src = q; jobs.job[n].copy_dst = c->q_rot; jobs.job[n].rot_on = 1; jobs.job[n].rot_base = base; jobs.job[n].rot_per_frame = 1; ++n; }
+    if (k_cur) { jobs.job[n].src = k_cur; jobs.job[n].copy_dst = c->k_rot; jobs.job[n].rot_on = 1; jobs.job[n].rot_base = base; jobs.job[n].rot_per_frame = 1; ++n; }
+    return launch_pool<D>(c, jobs, n, st);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -401,6 +433,11 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     memset(&jobs, 0, sizeof(jobs));
     jobs.job[0].src = q;     jobs.job[0].pooled = c->pooled_q;
     jobs.job[1].src = k_cur; jobs.job[1].pooled = c->pooled_kcur;
+    if (c->has_trope) {     // the block means are those of the rotated tensors, which the attention kernel reads afterwards
+        const int base = trope_top(c, L.frames) - c->cfg.chunk_frames + 1;
+        jobs.job[0].copy_dst = c->q_rot; jobs.job[1].copy_dst = c->k_rot;
+        for (int i = 0; i < 2; ++i) { jobs.job[i].rot_on = 1; jobs.job[i].rot_base = base; jobs.job[i].rot_per_frame = 1; }
+    }
     HF_TRY(launch_pool<D>(c, jobs, 2, st));
     const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     const int keep = keep_for(c, Tn);
@@ -757,7 +794,7 @@ hf_status hf_reset(hf_ctx* c, int layer, void* stream) {
         HF_CUDA(cudaMemsetAsync(L.z, 0, dz * 4, st));
         HF_CUDA(cudaMemsetAsync(L.sf_hi, 0, dd * 2, st));
         HF_CUDA(cudaMemsetAsync(L.sf_lo, 0, dd * 2, st));
-        L.n_cached = 0; L.head = 0; L.n_sink = 0; L.absorbed = 0; L.cache_epoch++; L.sel_epoch = ~0ull;
+        L.n_cached = 0; L.head = 0; L.n_sink = 0; L.absorbed = 0; L.frames = 0; L.cache_epoch++; L.sel_epoch = ~0ull;
     }
     return HF_OK;
 }
@@ -803,6 +840,34 @@ hf_status hf_set_rope(hf_ctx* c, const float* cos_q, const float* sin_q, const f
     return HF_OK;
 }
 
+hf_status hf_set_temporal_rope(hf_ctx* c, int t0, int first_pair, int n_pairs, const float* cos_tab, const float* sin_tab, void* stream) {
+    if (c == nullptr) return fail(HF_ERR_INVALID_ARG, "ctx is null");
+    for (const LayerState& L : c->layers)
+        if (L.frames != 0) return fail(HF_ERR_STATE, "the temporal rotation must be set before the first chunk is committed (or after hf_reset)");
+    if (cos_tab == nullptr && sin_tab == nullptr) { c->has_trope = false; return HF_OK; }
+    HF_TRY(check_ptr(cos_tab, "cos_tab"));
+    HF_TRY(check_ptr(sin_tab, "sin_tab"));
+    if (t0 < c->cfg.chunk_frames) return fail(HF_ERR_SHAPE, "t0 (%d) must be at least chunk_frames (%d)", t0, c->cfg.chunk_frames);
+    if (first_pair < 0 || n_pairs < 1 || first_pair + n_pairs > c->d / 2)
+        return fail(HF_ERR_SHAPE, "pairs [%d, %d) outside the head's %d feature pairs", first_pair, first_pair + n_pairs, c->d / 2);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t count = (size_t)(t0 + 1) * n_pairs;
+    HF_CUDA(cudaStreamSynchronize(st));
+    const float* src[2] = {cos_tab, sin_tab};
+    for (int i = 0; i < 2; ++i) {
+        cudaFree(c->trope_tab[i]); c->trope_tab[i] = nullptr;
+        HF_TRY(dmalloc(&c->trope_tab[i], count));
+        HF_CUDA(cudaMemcpyAsync(c->trope_tab[i], src[i], count * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    }
+    if (c->q_rot == nullptr) HF_TRY(dmalloc(&c->q_rot, c->chunk_elems));
+    if (c->k_rot == nullptr) HF_TRY(dmalloc(&c->k_rot, c->chunk_elems));
+    c->trope.cos_tab = c->trope_tab[0]; c->trope.sin_tab = c->trope_tab[1];
+    c->trope.first_pair = first_pair; c->trope.n_pairs = n_pairs; c->trope.tokens_per_frame = c->cfg.tokens_per_frame;
+    c->t0 = t0;
+    c->has_trope = true;
+    return HF_OK;
+}
+
 hf_status hf_state_absorb(hf_ctx* c, int layer, const void* k_ev, const void* v_ev, int n_tokens, void* stream) {
     HF_TRY(check_layer(c, layer));
     HF_TRY(check_ptr(k_ev, "k_ev"));
@@ -824,21 +889,36 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     HF_TRY(check_ptr(v, "v"));
     LayerState& L = c->layers[layer];
     cudaStream_t st = (cudaStream_t)stream;
+    // Relative temporal RoPE (Eq. 8): a key enters the cache turned to the index it has while the NEXT chunk is generated;
+    // when the cap makes the window's indices slide, the chunks that stay are turned by the same amount, in place.
+    const int cf = c->cfg.chunk_frames;
+    const int top_now = c->has_trope ? trope_top(c, L.frames) : 0, top_next = c->has_trope ? trope_top(c, L.frames + cf) : 0;
     if (L.n_sink < c->n_sink_max) {   // the stream's first chunks are the attention sink: kept in slots of their own for good
         const int slot = c->R + L.n_sink;
         PoolJobs jobs;
         memset(&jobs, 0, sizeof(jobs));
         jobs.job[0].src = (const bf16*)k; jobs.job[0].copy_dst = L.ring_k + (size_t)slot * c->chunk_elems;
         jobs.job[0].pooled = L.pooled_k + (size_t)slot * c->pooled_elems;
+        if (c->has_trope) { jobs.job[0].rot_on = 1; jobs.job[0].rot_base = top_now - cf + 1; jobs.job[0].rot_per_frame = 1; }   // its own indices, for good
         jobs.job[1].src = (const bf16*)v; jobs.job[1].copy_dst = L.ring_v + (size_t)slot * c->chunk_elems;
         HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
         L.n_sink++;
+        L.frames += cf;
         L.cache_epoch++;
         return HF_OK;
     }
-    if (c->P == 0) {   // window == chunk: a committed chunk leaves the window at once
-        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, (const bf16*)k, (const bf16*)v, c->Tc, st));
+    if (c->P == 0) {   // window == chunk: a committed chunk leaves the window at once (as the window saw it: at its own indices)
+        const bf16* ks = (const bf16*)k;
+        if (c->has_trope) {
+            PoolJobs jobs;
+            memset(&jobs, 0, sizeof(jobs));
+            jobs.job[0].src = ks; jobs.job[0].copy_dst = c->k_rot; jobs.job[0].rot_on = 1; jobs.job[0].rot_base = top_now - cf + 1; jobs.job[0].rot_per_frame = 1;
+            HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 1, st));
+            ks = c->k_rot;
+        }
+        HF_TRY(HF_DISPATCH_D(c, launch_absorb, c, L, ks, (const bf16*)v, c->Tc, st));
         L.absorbed += c->Tc;
+        L.frames += cf;
         L.cache_epoch++;
         return HF_OK;
     }
@@ -862,9 +942,29 @@ hf_status hf_kv_append(hf_ctx* c, int layer, const void* k, const void* v, void*
     memset(&jobs, 0, sizeof(jobs));
     jobs.job[0].src = (const bf16*)k; jobs.job[0].copy_dst = L.ring_k + (size_t)slot * c->chunk_elems;
     jobs.job[0].pooled = L.pooled_k + (size_t)slot * c->pooled_elems;
+    if (c->has_trope) { jobs.job[0].rot_on = 1; jobs.job[0].rot_base = top_next - 2 * cf + 1; jobs.job[0].rot_per_frame = 1; }
     jobs.job[1].src = (const bf16*)v; jobs.job[1].copy_dst = L.ring_v + (size_t)slot * c->chunk_elems;
     HF_TRY(HF_DISPATCH_D(c, launch_pool, c, jobs, 2, st));
+    const int slide = c->has_trope ? top_next - top_now - cf : 0;       // 0 below the cap, then -chunk_frames
+    if (slide != 0) {
+        // the chunks that stay in the window (L.head is already past the one that left; the new chunk is not counted yet when
+        // the window was still filling): their keys and block means, turned in place
+        const int stay = evicted ? L.n_cached - 1 : L.n_cached - 1;
+        for (int i = 0; i < stay; i += 3) {
+            PoolJobs rj;
+            memset(&rj, 0, sizeof(rj));
+            int n = 0;
+            for (; n < 3 && i + n < stay; ++n) {
+                const int sl = (L.head + i + n) % c->R;
+                bf16* kp = L.ring_k + (size_t)sl * c->chunk_elems;
+                rj.job[n].src = kp; rj.job[n].copy_dst = kp; rj.job[n].pooled = L.pooled_k + (size_t)sl * c->pooled_elems;
+                rj.job[n].rot_on = 1; rj.job[n].rot_base = slide; rj.job[n].rot_per_frame = 0;
+            }
+            HF_TRY(HF_DISPATCH_D(c, launch_pool, c, rj, n, st));
+        }
+    }
     if (evicted) HF_CUDA(cudaStreamWaitEvent(st, c->ev_join, 0));
+    L.frames += cf;
     L.cache_epoch++;
     return HF_OK;
 }
@@ -918,7 +1018,7 @@ hf_status hf_kv_append_layers(hf_ctx* c, int first_layer, int n_layers, const vo
     // sink, all filling the window, or all evicting) and enough (layer, batch*head) items to fill the device; anything
     // else goes layer by layer.  The state gets the same bits either way.
     const LayerState& L0 = c->layers[first_layer];
-    bool uniform = c->P > 0 && n_layers <= HF_MAX_BATCH_LAYERS && (long long)n_layers * c->BH >= c->sm_count;
+    bool uniform = c->P > 0 && !c->has_trope && n_layers <= HF_MAX_BATCH_LAYERS && (long long)n_layers * c->BH >= c->sm_count;
     for (int l = 1; uniform && l < n_layers; ++l) {
         const LayerState& L = c->layers[first_layer + l];
         uniform = (L.n_sink < c->n_sink_max) == (L0.n_sink < c->n_sink_max) && (L.n_cached == c->P) == (L0.n_cached == c->P);
@@ -956,6 +1056,7 @@ hf_status hf_kv_append_layers(hf_ctx* c, int first_layer, int n_layers, const vo
         if (sink) L.n_sink++;
         else if (evict) { L.absorbed += c->Tc; L.head = (L.head + 1) % c->R; }
         else L.n_cached++;
+        L.frames += c->cfg.chunk_frames;
         L.cache_epoch++;
     }
     return HF_OK;
@@ -983,6 +1084,10 @@ hf_status hf_sparse_swa(hf_ctx* c, int layer, const void* q, const void* k_cur, 
         if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
         idx = L.idx;
     }
+    if (c->has_trope) {     // the queries and the current chunk's keys at their Eq. 8 indices
+        HF_TRY(HF_DISPATCH_D(c, launch_rotate_inputs, c, L, (const bf16*)q, (const bf16*)k_cur, (cudaStream_t)stream));
+        q = c->q_rot; k_cur = c->k_rot;
+    }
     return launch_swa(c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, nullptr, (bf16*)o_local, lse,
                       (cudaStream_t)stream);
 }
@@ -991,6 +1096,10 @@ hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void
     HF_TRY(check_layer(c, layer));
     HF_TRY(check_ptr(q, "q"));
     HF_TRY(check_ptr(o_hist, "o_hist"));
+    if (c->has_trope) {     // both branches see the queries with their temporal rotation
+        HF_TRY(HF_DISPATCH_D(c, launch_rotate_inputs, c, c->layers[layer], (const bf16*)q, (const bf16*)nullptr, (cudaStream_t)stream));
+        q = c->q_rot;
+    }
     return HF_DISPATCH_D(c, launch_readout, c, c->layers[layer], (const bf16*)q, (bf16*)o_hist, (float*)nullptr, (cudaStream_t)stream);
 }
 
@@ -1023,6 +1132,10 @@ hf_status hf_sparse_swa_merged(hf_ctx* c, int layer, const void* q, const void* 
         if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
         idx = L.idx;
     }
+    if (c->has_trope) {
+        HF_TRY(HF_DISPATCH_D(c, launch_rotate_inputs, c, L, (const bf16*)q, (const bf16*)k_cur, (cudaStream_t)stream));
+        q = c->q_rot; k_cur = c->k_rot;
+    }
     return attend_merge(c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, (bf16*)o, (cudaStream_t)stream, false);
 }
 
@@ -1036,9 +1149,12 @@ hf_status hf_hybrid_forward(hf_ctx* c, int layer, const void* q, const void* k, 
     cudaStream_t st = (cudaStream_t)stream;
     const bool one_kernel = c->swa_kernel == HF_SWA_TCGEN05 && c->d == 128 && c->cfg.block == 128 && SwaTc5<128, Tc5Groups<128>::N>::FUSE &&
                             !c->has_rope_q && c->cfg.merge != HF_MERGE_FULL_WIDTH;
-    if (one_kernel) {
+    if (one_kernel || c->has_trope) {
+        // (with the temporal rotation the selection's pooling pass also writes the rotated q and k that everything after it
+        // reads, so the history read-out cannot run beside it: one stream)
         HF_TRY(HF_DISPATCH_D(c, launch_select, c, L, (const bf16*)q, (const bf16*)k, (uint32_t*)nullptr, (int32_t*)nullptr, (float*)nullptr, st));
-        return attend_merge(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, (bf16*)o, st, true);
+        if (c->has_trope) { q = c->q_rot; k = c->k_rot; }
+        return attend_merge(c, L, (const bf16*)q, (const bf16*)k, (const bf16*)v, L.idx, L.sel_keep, (bf16*)o, st, one_kernel);
     }
     // Otherwise the history term depends on q and the state only: it runs on the context's side stream while pooling and
     // selection run on the caller's stream; the attention kernel, which adds it in its epilogue, waits for both.
@@ -1094,7 +1210,7 @@ hf_status hf_get_state(hf_ctx* c, int layer, float* S, float* z, void* stream) {
 // ---- checkpoint image: header, then per layer {counts, S, z, held chunks in logical order (K, V, pooled sums)}
 namespace {
 constexpr uint64_t IMAGE_MAGIC = 0x3145544154534648ull;   // "HFSTATE1"
-constexpr uint32_t IMAGE_VERSION = 1;
+constexpr uint32_t IMAGE_VERSION = 2;
 struct ImageHeader {
     uint64_t magic;
     uint32_t version, header_bytes;
@@ -1104,6 +1220,7 @@ struct ImageHeader {
 struct ImageLayer {
     int32_t n_sink, n_cached;
     int64_t absorbed;
+    int64_t frames;
 };
 size_t image_chunk_bytes(const hf_ctx* c) { return 2 * c->chunk_elems * sizeof(bf16) + c->pooled_elems * sizeof(float); }
 size_t image_state_bytes(const hf_ctx* c) { return ((size_t)c->BH * c->d * c->d + (size_t)c->BH * c->d) * sizeof(float); }
@@ -1143,7 +1260,7 @@ hf_status hf_state_export(hf_ctx* c, void* host_buf, size_t* bytes) {
     const size_t kv = c->chunk_elems * sizeof(bf16), pl = c->pooled_elems * sizeof(float);
     for (const LayerState& L : c->layers) {
         ImageLayer il;
-        il.n_sink = L.n_sink; il.n_cached = L.n_cached; il.absorbed = L.absorbed;
+        il.n_sink = L.n_sink; il.n_cached = L.n_cached; il.absorbed = L.absorbed; il.frames = L.frames;
         memcpy(out, &il, sizeof(il)); out += sizeof(il);
         HF_CUDA(cudaMemcpy(out, L.S, dd, cudaMemcpyDeviceToHost)); out += dd;
         HF_CUDA(cudaMemcpy(out, L.z, dz, cudaMemcpyDeviceToHost)); out += dz;
@@ -1179,7 +1296,7 @@ hf_status hf_state_import(hf_ctx* c, const void* host_buf, size_t bytes) {
         if (off + sizeof(ImageLayer) > h.total_bytes) return fail(HF_ERR_INVALID_ARG, "image ends inside layer %d", l);
         ImageLayer il;
         memcpy(&il, in + off, sizeof(il));
-        if (il.n_sink < 0 || il.n_sink > c->n_sink_max || il.n_cached < 0 || il.n_cached > c->P || il.absorbed < 0 ||
+        if (il.n_sink < 0 || il.n_sink > c->n_sink_max || il.n_cached < 0 || il.n_cached > c->P || il.absorbed < 0 || il.frames < 0 ||
             (il.n_cached > 0 && il.n_sink < c->n_sink_max))
             return fail(HF_ERR_INVALID_ARG, "layer %d of the image holds counts this configuration cannot have", l);
         off += sizeof(ImageLayer) + image_state_bytes(c) + (size_t)(il.n_sink + il.n_cached) * image_chunk_bytes(c);
@@ -1195,7 +1312,7 @@ hf_status hf_state_import(hf_ctx* c, const void* host_buf, size_t bytes) {
         memcpy(&il, in, sizeof(il)); in += sizeof(il);
         HF_CUDA(cudaMemcpy(L.S, in, dd, cudaMemcpyHostToDevice)); in += dd;
         HF_CUDA(cudaMemcpy(L.z, in, dz, cudaMemcpyHostToDevice)); in += dz;
-        L.n_sink = il.n_sink; L.n_cached = il.n_cached; L.head = 0; L.absorbed = il.absorbed;
+        L.n_sink = il.n_sink; L.n_cached = il.n_cached; L.head = 0; L.absorbed = il.absorbed; L.frames = il.frames;
         L.cache_epoch++; L.sel_epoch = ~0ull;
         for (int i = 0; i < L.n_sink + L.n_cached; ++i) {
             const int slot = held_slot(c, L, i);

@@ -26,15 +26,53 @@ template <> struct VecLoad<4> {
 
 struct PoolJob {            // one tensor to pool (and optionally copy) per blockIdx.z
     const bf16* src;        // [B*H, T_c, d]
-    bf16* copy_dst;         // same shape, or nullptr
+    bf16* copy_dst;         // same shape, or nullptr (may be src itself: every thread rewrites exactly what it read)
     float* pooled;          // [B*H, n_b, d] block means, or nullptr (copy only)
+    // temporal rotation (ROT instantiation): frame f of the chunk is turned by rot_base + rot_per_frame * f index steps
+    int rot_on, rot_base, rot_per_frame;
 };
 struct PoolJobs { PoolJob job[3]; };
 
+// Relative temporal RoPE of the softmax branch (Eq. 8): pairs [first_pair, first_pair + n_pairs) of a token's features
+// turn by (index steps) x (the pair's frequency); cosine and sine come from tables over integer steps 0 .. t0 (a backward
+// turn uses the entry of |steps| with the sine negated).  The arithmetic order is fixed, because the rotated values feed
+// the block selection: x0' = x0 c - x1 s, x1' = x0 s + x1 c, each product and each sum rounded separately in float32, the
+// result rounded to bf16 (the cache and the attention operands are bf16).
+struct TemporalRope {
+    const float* cos_tab;   // [t0 + 1][n_pairs]
+    const float* sin_tab;
+    int first_pair, n_pairs, tokens_per_frame;
+};
+
 // One block of one tensor: copy (optional) and per-column mean in the canonical order.  256 threads: 16 threads per token
 // row, 16 rows per pass.
-template <int D>
-__device__ __forceinline__ void pool_copy_block(const PoolJob& jb, int Tc, int blk, int n_b, int b_idx, int bh) {
+template <int VEC, typename V>
+__device__ __forceinline__ V rotate_vec(const V& u, int first_feature, int steps, const TemporalRope& tr) {
+    float f[VEC];
+    VecLoad<VEC>::widen(u, f);
+    const int a = steps < 0 ? -steps : steps;
+    uint32_t w[VEC / 2];
+#pragma unroll
+    for (int e = 0; e < VEC; e += 2) {
+        const int pr = (first_feature + e) / 2 - tr.first_pair;
+        float y0 = f[e], y1 = f[e + 1];
+        if (pr >= 0 && pr < tr.n_pairs) {
+            const float c = __ldg(tr.cos_tab + (size_t)a * tr.n_pairs + pr);
+            float sn = __ldg(tr.sin_tab + (size_t)a * tr.n_pairs + pr);
+            if (steps < 0) sn = -sn;
+            y0 = __fsub_rn(__fmul_rn(f[e], c), __fmul_rn(f[e + 1], sn));
+            y1 = __fadd_rn(__fmul_rn(f[e], sn), __fmul_rn(f[e + 1], c));
+        }
+        w[e / 2] = pack_bf16(y0, y1);
+    }
+    V out;
+    if constexpr (VEC == 8) { out.x = w[0]; out.y = w[1]; out.z = w[2]; out.w = w[3]; }
+    else { out.x = w[0]; out.y = w[1]; }
+    return out;
+}
+
+template <int D, bool ROT>
+__device__ __forceinline__ void pool_copy_block(const PoolJob& jb, int Tc, int blk, int n_b, int b_idx, int bh, const TemporalRope& tr) {
     constexpr int VEC = D / 16;
     typedef typename VecLoad<VEC>::T V;
     const int t0 = b_idx * blk;
@@ -54,7 +92,14 @@ __device__ __forceinline__ void pool_copy_block(const PoolJob& jb, int Tc, int b
 #pragma unroll
         for (int i = 0; i < BATCH; ++i) {
             const int t = r + 16 * (i0 + i);
-            if (t < n) u[i] = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
+            if (t < n) {
+                // (the rotating instantiation may work in place: plain loads there, the read-only path elsewhere)
+                if (ROT) u[i] = *reinterpret_cast<const V*>(jb.src + base + (size_t)t * D);
+                else u[i] = __ldg(reinterpret_cast<const V*>(jb.src + base + (size_t)t * D));
+                if (ROT) {
+                    if (jb.rot_on) u[i] = rotate_vec<VEC, V>(u[i], cv * VEC, jb.rot_base + jb.rot_per_frame * ((t0 + t) / tr.tokens_per_frame), tr);
+                }
+            }
         }
         if (jb.copy_dst) {
 #pragma unroll
@@ -92,7 +137,16 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy(PoolJobs jobs, int Tc, int
     pdl_wait();                 // launched under the tail of the kernel before it: that kernel's reads and writes are done from here on
     pdl_trigger();              // a dependent kernel (the selection) may be made resident; it waits for this grid itself
     const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];   // (no indexed copy of the parameter block)
-    pool_copy_block<D>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y);
+    TemporalRope none = {nullptr, nullptr, 0, 0, 1};
+    pool_copy_block<D, false>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y, none);
+}
+// The same with the temporal rotation applied to the jobs that ask for it (before the copy and the means).
+template <int D>
+__global__ void __launch_bounds__(256, 4) k_pool_copy_rot(PoolJobs jobs, int Tc, int blk, int n_b, TemporalRope tr) {
+    pdl_wait();
+    pdl_trigger();
+    const PoolJob jb = blockIdx.z == 0 ? jobs.job[0] : blockIdx.z == 1 ? jobs.job[1] : jobs.job[2];
+    pool_copy_block<D, true>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y, tr);
 }
 
 // The cache commit of several layers in one launch (Alg. 2 "KV.append" for every layer of the model): per layer the
@@ -119,7 +173,9 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy_layers(const __grid_consta
     jb.src = is_v ? p.v_src[lay] : p.k_src[lay];
     jb.copy_dst = (is_v ? p.ring_v : p.ring_k) + s * p.chunk_elems;
     jb.pooled = is_v ? nullptr : p.pooled + s * p.pooled_elems;
-    pool_copy_block<D>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y);
+    jb.rot_on = 0; jb.rot_base = 0; jb.rot_per_frame = 0;
+    TemporalRope none = {nullptr, nullptr, 0, 0, 1};
+    pool_copy_block<D, false>(jb, Tc, blk, n_b, blockIdx.x, blockIdx.y, none);
 }
 
 // A[i][j] = Mean(q_i) . Mean(k_j) in the canonical order, formed by one warp: 32 partials (partial l = columns l,

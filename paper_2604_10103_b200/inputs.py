@@ -180,3 +180,14 @@ def shifted(bits: np.ndarray, u: np.ndarray, amount: float, tokens: slice = slic
     x = bf16_bits_to_f32(bits).copy()
     x[:, :, tokens, :] = x[:, :, tokens, :] * np.float32(scale) + np.float32(amount) * u[None, :, None, :]
     return f32_to_bf16_bits(x)
+
+
+def temporal_rope_tables(head_dim: int, t0: int, first_pair: int = 0, pairs: int | None = None, base: float = 10000.0):
+    """Angle tables of the temporal rotary axis for integer index steps 0 .. t0: float32 (cos, sin) [t0 + 1, pairs] with the
+    usual rotary frequencies base ** (-n / pairs), plus the frequencies themselves (float64).  `pairs` defaults to the
+    share of the head's d/2 pairs that a (t, y, x) split gives the temporal axis (d/2 - 2 * (d/6))."""
+    if pairs is None:
+        pairs = head_dim // 2 - 2 * (head_dim // 6)
+    om = base ** (-np.arange(pairs, dtype=np.float64) / pairs)
+    n = np.arange(t0 + 1, dtype=np.float64)
+    return np.cos(n[:, None] * om[None, :]).astype(np.float32), np.sin(n[:, None] * om[None, :]).astype(np.float32), om

@@ -21,8 +21,15 @@ def max_abs(a, b):
     return float(np.abs(np.asarray(a, np.float64) - np.asarray(b, np.float64)).max())
 
 
+def temporal_setup(w: gen.Workload, t0: int, first_pair: int = 0, pairs=None):
+    """The tables both sides get for the relative temporal RoPE (Eq. 8): (dict for the oracle, (cos, sin) float32)."""
+    cos, sin, _ = gen.temporal_rope_tables(w.head_dim, t0, first_pair, pairs)
+    return dict(t0=t0, first_pair=first_pair, cos_tab=cos, sin_tab=sin, tokens_per_frame=w.tokens_per_frame,
+                chunk_frames=w.chunk_frames), (cos, sin)
+
+
 def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, z_frame_mean: bool = False,
-                sink_chunks: int = 0, rope: bool = False, merge_full: bool = False):
+                sink_chunks: int = 0, rope: bool = False, merge_full: bool = False, temporal=None):
     W = b = Wf = bf = None
     if merge_full:
         Wb, bb = gen.merge_weights_full(w, layer, with_bias=bias)
@@ -36,7 +43,8 @@ def make_oracle(w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool 
                            keep_permille=w.keep_permille, W=W, bias=b, eps=w.eps,
                            z_frame_tokens=w.tokens_per_frame if z_frame_mean else None, sink_chunks=sink_chunks,
                            rope_q=gen.rotation_tables(w, gen.T_ANGLE_Q) if rope else None,
-                           rope_k=gen.rotation_tables(w, gen.T_ANGLE_K) if rope else None, W_full=Wf, bias_full=bf)
+                           rope_k=gen.rotation_tables(w, gen.T_ANGLE_K) if rope else None, W_full=Wf, bias_full=bf,
+                           temporal=None if temporal is None else temporal_setup(w, *temporal)[0])
 
 
 from paper_2604_10103_b200.binding import unpack_mask  # noqa: E402,F401
@@ -47,7 +55,7 @@ class GpuStream:
 
     def __init__(self, w: gen.Workload, layer: int = 0, merge: bool = True, bias: bool = True, swa_kernel: int = 0,
                  layers: int | None = None, z_frame_mean: bool = False, sink_chunks: int = 0, rope: bool = False,
-                 merge_full: bool = False):
+                 merge_full: bool = False, temporal=None):
         import torch
         from paper_2604_10103_b200 import binding as hf
         self.torch, self.hf, self.w, self.layer = torch, hf, w, layer
@@ -67,6 +75,11 @@ class GpuStream:
             to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
             cq, sq = gen.rotation_tables(w, gen.T_ANGLE_Q); ck, sk = gen.rotation_tables(w, gen.T_ANGLE_K)
             self.ctx.hf_set_rope(to_dev(cq), to_dev(sq), to_dev(ck), to_dev(sk))
+            torch.cuda.synchronize()
+        if temporal is not None:        # (t0, first_pair, pairs)
+            t, (cos, sin) = temporal_setup(w, *temporal)
+            to_dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+            self.ctx.hf_set_temporal_rope(t["t0"], t["first_pair"], cos.shape[1], to_dev(cos), to_dev(sin))
             torch.cuda.synchronize()
         self.shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
 
