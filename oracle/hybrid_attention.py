@@ -421,7 +421,9 @@ class HybridStream:
             last = self.frames_committed + c                    # (1-based) number of this chunk's last frame
             top_now, top_next = min(last, t0), min(last + c, t0)
             self.frames_committed = last
-            if len(self.sink) < self.sink_chunks:               # a sink chunk keeps its own indices for good
+            if len(self.sink) < self.sink_chunks or self.P == 0:
+                # a sink chunk keeps its own indices for good; without a cache (window = one chunk) the chunk goes straight
+                # into the state, as the window last saw it: at its own indices
                 k_clean = self._turn(k_clean, [top_now - c + 1 + i for i in range(c)])
             else:
                 # indices during the next chunk: this chunk sits c frames behind it; older chunks slide by the same amount
