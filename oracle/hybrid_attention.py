@@ -28,6 +28,9 @@ What follows which passage:
                           the temporal rotation of the softmax branch's queries and keys
   rotate_temporal_f32     the same rotation in the canonical float32 order with the bf16 rounding the cache applies
   HybridStream            Alg. 2 cache protocol (evict -> update state -> append) around Alg. 3, Eq. 7 sum
+  sparse_attention_backward, linear_readout_backward, HybridStream.backward
+                          gradients of Eq. 6 / Eq. 4 / Eq. 7 for the training rollout (Alg. 1: the sampled step is run with
+                          gradient), with the block mask held fixed (the top-K choice is piecewise constant)
 
 Readings taken where the paper is silent or inconsistent (all listed again in the
 design notes): H is accumulated as the plain sum of phi(K) rows (so that Eq. 4 is a
@@ -347,6 +350,69 @@ def merge_full_width(h: np.ndarray, W_full, bias_full=None) -> np.ndarray:
     return np.transpose(y.reshape(T, H, d), (1, 0, 2))
 
 
+# --------------------------------------------------------------------------- gradients (Alg. 1: rollout step with gradient)
+def phi_prime(x: np.ndarray) -> np.ndarray:
+    """d/dx (elu(x) + 1): 1 for x > 0, exp(x) otherwise."""
+    x = np.asarray(x, dtype=np.float64)
+    return np.where(x > 0.0, 1.0, np.exp(np.minimum(x, 0.0)))
+
+
+def sparse_attention_backward(q, k_chunks, v_chunks, b: int, mask: np.ndarray, d_out):
+    """Gradients of O_local (Eq. 6) for a fixed block mask: given dL/dO_local [T_c, d] returns
+    (dq [T_c, d], [dk per chunk], [dv per chunk]).  Per query block, with p = softmax(s) over the kept keys and
+    s = q k^T / sqrt(d):  dv = p^T dO;  dp = dO v^T;  ds = p * (dp - rowsum(dp * p))  (Jacobian of the row softmax);
+    dq = ds k / sqrt(d);  dk = ds^T q / sqrt(d).  Keys outside the kept blocks get no gradient from that query block."""
+    q = np.asarray(q, np.float64); d_out = np.asarray(d_out, np.float64)
+    d = q.shape[1]
+    table = key_block_table([kc.shape[0] for kc in k_chunks], b)
+    dq = np.zeros_like(q)
+    dk = [np.zeros(np.asarray(kc).shape) for kc in k_chunks]
+    dv = [np.zeros(np.asarray(vc).shape) for vc in v_chunks]
+    for i, (qs, qe) in enumerate(block_ranges(q.shape[0], b)):
+        kept = [table[j] for j in range(len(table)) if mask[i, j]]
+        ks = np.concatenate([np.asarray(k_chunks[c][s:e], np.float64) for (c, s, e) in kept])
+        vs = np.concatenate([np.asarray(v_chunks[c][s:e], np.float64) for (c, s, e) in kept])
+        s_ = q[qs:qe] @ ks.T / math.sqrt(d)
+        p = np.exp(s_ - s_.max(axis=1, keepdims=True))
+        p = p / p.sum(axis=1, keepdims=True)
+        g = d_out[qs:qe]
+        dvs = p.T @ g
+        dp = g @ vs.T
+        ds = p * (dp - (dp * p).sum(axis=1, keepdims=True))
+        dq[qs:qe] = ds @ ks / math.sqrt(d)
+        dks = ds.T @ q[qs:qe] / math.sqrt(d)
+        at = 0
+        for (c, s, e) in kept:
+            dk[c][s:e] += dks[at:at + e - s]
+            dv[c][s:e] += dvs[at:at + e - s]
+            at += e - s
+    return dq, dk, dv
+
+
+def linear_readout_backward(q, S, z, d_out, W=None, eps: float = 1e-6):
+    """Gradients of O_history (Eq. 4, no rotation) given dL/dO_history [T, d]: returns (dq, dS, dz, dW, dbias).
+    Forward: f = phi(q); num = f S; den = f . z + eps; h = num / den; y = W h + bias."""
+    q = np.asarray(q, np.float64); g = np.asarray(d_out, np.float64)
+    f = phi(q)
+    num = f @ S
+    den = f @ z + eps
+    h = num / den[:, None]
+    dbias = g.sum(axis=0)
+    if W is not None:
+        W = np.asarray(W, np.float64)
+        dW = g.T @ h                    # y = h W^T
+        dh = g @ W
+    else:
+        dW = None
+        dh = g
+    dnum = dh / den[:, None]
+    dden = -(dh * num).sum(axis=1) / den ** 2
+    df = dnum @ S.T + dden[:, None] * z[None, :]
+    dS = f.T @ dnum
+    dz = f.T @ dden
+    return df * phi_prime(q), dS, dz, dW, dbias
+
+
 # --------------------------------------------------------------------------- Alg. 2 + Alg. 3
 class HybridStream:
     """Streaming state of one layer (all batches and heads) and the per-chunk forward.
@@ -506,3 +572,34 @@ class HybridStream:
         if parts:
             return o_loc + o_hist, o_loc, o_hist
         return o_loc + o_hist
+
+    # -- gradients of the forward above (Eq. 7: both branches receive dL/dO unchanged)
+    def backward(self, q, k_cur, v_cur, d_out, mask=None):
+        """dL/dO [B, H, T_c, d] -> dict(dq, dk_cur, dv_cur, dk_past, dv_past (lists per cached chunk, sink first), dS, dz,
+        dW, dbias) for the per-head reading of "Linear", without rotation.  The block mask is held fixed."""
+        assert self.temporal is None and self.rope_q is None and self.W_full is None
+        q = np.asarray(q, np.float64); k_cur = np.asarray(k_cur, np.float64); v_cur = np.asarray(v_cur, np.float64)
+        g = np.asarray(d_out, np.float64)
+        if mask is None:
+            mask, _ = self.select(q, k_cur)
+        held = self.sink + self.past
+        out = dict(dq=np.zeros_like(q), dk_cur=np.zeros_like(k_cur), dv_cur=np.zeros_like(v_cur),
+                   dk_past=[np.zeros_like(kp) for kp, _ in held], dv_past=[np.zeros_like(vp) for _, vp in held],
+                   dS=np.zeros_like(self.S), dz=np.zeros_like(self.z),
+                   dW=None if self.W is None else np.zeros_like(self.W), dbias=np.zeros((self.H, self.d)))
+        for bi in range(self.B):
+            for h in range(self.H):
+                kc = [kp[bi, h] for kp, _ in held] + [k_cur[bi, h]]
+                vc = [vp[bi, h] for _, vp in held] + [v_cur[bi, h]]
+                dq_l, dk_l, dv_l = sparse_attention_backward(q[bi, h], kc, vc, self.b, mask[bi, h], g[bi, h])
+                dq_h, dS, dz, dW, db = linear_readout_backward(q[bi, h], self.S[bi, h], self.z[bi, h], g[bi, h],
+                                                               None if self.W is None else self.W[h], self.eps)
+                out["dq"][bi, h] = dq_l + dq_h
+                out["dk_cur"][bi, h] = dk_l[-1]; out["dv_cur"][bi, h] = dv_l[-1]
+                for n in range(len(held)):
+                    out["dk_past"][n][bi, h] = dk_l[n]; out["dv_past"][n][bi, h] = dv_l[n]
+                out["dS"][bi, h] = dS; out["dz"][bi, h] = dz
+                out["dbias"][h] += db
+                if dW is not None:
+                    out["dW"][h] += dW
+        return out

@@ -631,3 +631,118 @@ def test_stream_without_cap_is_absolute_indexing():
             want = oa.rotate_temporal_f32(ks[chunk_no][0, 0].astype(np.float32), idx, tpf, 2, t["cos_tab"], t["sin_tab"])
             assert np.array_equal(kp[0, 0], want.astype(np.float64))
     assert st.current_indices() == [16, 17, 18]
+
+
+# --------------------------------------------------------------------------- gradients (rollout step with gradient, Alg. 1)
+def _fd(fn, x, eps=1e-6):
+    """Central finite differences of the scalar fn with respect to every element of x."""
+    g = np.zeros_like(x)
+    it = np.nditer(x, flags=["multi_index"])
+    for _ in it:
+        i = it.multi_index
+        old = x[i]
+        x[i] = old + eps; up = fn()
+        x[i] = old - eps; dn = fn()
+        x[i] = old
+        g[i] = (up - dn) / (2 * eps)
+    return g
+
+
+def test_sparse_attention_backward_against_finite_differences_and_autograd():
+    """dq, dk, dv of Eq. 6 with a fixed mask: central differences of the oracle's own forward on a ragged two-chunk window,
+    and torch autograd (fp64 SDPA) with every block kept."""
+    import torch
+    d, b, lens = 8, 4, [6, 10]
+    q = rnd((10, d), 120); kc = [rnd((n, d), 121 + i) for i, n in enumerate(lens)]; vc = [rnd((n, d), 125 + i) for i, n in enumerate(lens)]
+    g = rnd((10, d), 129)
+    tm, tn = 3, 2 + 3
+    rng = np.random.default_rng(7)
+    mask = np.zeros((tm, tn), dtype=bool)
+    for i in range(tm):
+        mask[i, rng.choice(tn, size=2, replace=False)] = True
+    dq, dk, dv = oa.sparse_attention_backward(q, kc, vc, b, mask, g)
+    loss = lambda: float((oa.sparse_attention(q, kc, vc, b, mask) * g).sum())
+    assert np.abs(dq - _fd(loss, q)).max() < 1e-7
+    for c in range(2):
+        assert np.abs(dk[c] - _fd(loss, kc[c])).max() < 1e-7
+        assert np.abs(dv[c] - _fd(loss, vc[c])).max() < 1e-7
+    # a key block no query block keeps gets no gradient
+    unused = [j for j in range(tn) if not mask[:, j].any()]
+    table = oa.key_block_table(lens, b)
+    for j in unused:
+        c, s, e = table[j]
+        assert not dk[c][s:e].any() and not dv[c][s:e].any()
+    # all blocks kept: dense attention, library autograd
+    full = np.ones((tm, tn), dtype=bool)
+    dq, dk, dv = oa.sparse_attention_backward(q, kc, vc, b, full, g)
+    tq = torch.tensor(q, requires_grad=True); tk = torch.tensor(np.concatenate(kc), requires_grad=True)
+    tv = torch.tensor(np.concatenate(vc), requires_grad=True)
+    o = torch.nn.functional.scaled_dot_product_attention(tq[None], tk[None], tv[None])[0]
+    (o * torch.tensor(g)).sum().backward()
+    assert np.abs(dq - tq.grad.numpy()).max() < 1e-12
+    assert np.abs(np.concatenate(dk) - tk.grad.numpy()).max() < 1e-12
+    assert np.abs(np.concatenate(dv) - tv.grad.numpy()).max() < 1e-12
+    # closed forms: no upstream gradient -> none downstream; constant V rows -> the output does not depend on q or k
+    z3 = oa.sparse_attention_backward(q, kc, vc, b, mask, np.zeros_like(g))
+    assert not z3[0].any() and not any(x.any() for x in z3[1]) and not any(x.any() for x in z3[2])
+    ones = [np.ones_like(v) for v in vc]
+    dq1, dk1, _ = oa.sparse_attention_backward(q, kc, ones, b, mask, g)
+    assert np.abs(dq1).max() < 1e-14 and max(np.abs(x).max() for x in dk1) < 1e-14
+
+
+def test_linear_readout_backward_against_finite_differences_and_autograd():
+    import torch
+    d, n = 6, 5
+    q = rnd((n, d), 130); S = rnd((d, d), 131); z = np.abs(rnd((d,), 132)) + 0.5; W = rnd((d, d), 133); bias = rnd((d,), 134)
+    g = rnd((n, d), 135)
+    dq, dS, dz, dW, db = oa.linear_readout_backward(q, S, z, g, W, eps=1e-3)
+    loss = lambda: float((oa.linear_readout(q, S, z, W, bias, eps=1e-3) * g).sum())
+    for got, x in ((dq, q), (dS, S), (dz, z), (dW, W), (db, bias)):
+        assert np.abs(got - _fd(loss, x)).max() < 1e-7
+    assert np.allclose(oa.phi_prime(np.array([-1.0, 0.0, 2.0])), [np.exp(-1.0), 1.0, 1.0])
+    tq = torch.tensor(q, requires_grad=True); tS = torch.tensor(S, requires_grad=True); tz = torch.tensor(z, requires_grad=True)
+    f = torch.nn.functional.elu(tq) + 1
+    y = ((f @ tS) / (f @ tz + 1e-3)[:, None]) @ torch.tensor(W).T + torch.tensor(bias)
+    (y * torch.tensor(g)).sum().backward()
+    assert np.abs(dq - tq.grad.numpy()).max() < 1e-12 and np.abs(dS - tS.grad.numpy()).max() < 1e-12
+    assert np.abs(dz - tz.grad.numpy()).max() < 1e-12
+    # identity "Linear"
+    dq2, _, _, dW2, _ = oa.linear_readout_backward(q, S, z, g, None, eps=1e-3)
+    loss2 = lambda: float((oa.linear_readout(q, S, z, None, None, eps=1e-3) * g).sum())
+    assert dW2 is None and np.abs(dq2 - _fd(loss2, q)).max() < 1e-7
+
+
+def test_stream_backward_against_finite_differences():
+    """HybridStream.backward after evictions (sink + cached chunks + state): every gradient against central differences of
+    HybridStream.forward with the mask held fixed; planted mistakes (a dropped softmax-Jacobian term, a missing branch in
+    the sum of Eq. 7) are caught."""
+    B, H, d, b = 1, 2, 8, 4
+    W = rnd((H, d, d), 140) / np.sqrt(d); bias = rnd((H, d), 141) * 0.1
+    st = oa.HybridStream(B, H, d, b, 1, topk=2, W=W, bias=bias, sink_chunks=1, eps=1e-3)
+    for c in range(4):
+        st.append(rnd((B, H, 6, d), 150 + c), rnd((B, H, 6, d), 160 + c))
+    assert st.absorbed_tokens == 12 and len(st.sink) == 1 and len(st.past) == 1
+    q = rnd((B, H, 6, d), 170); k = rnd((B, H, 6, d), 171); v = rnd((B, H, 6, d), 172); g = rnd((B, H, 6, d), 173)
+    mask, _ = st.select(q, k, exact=True)
+    gr = st.backward(q, k, v, g, mask=mask)
+    loss = lambda: float((st.forward(q, k, v, mask=mask) * g).sum())
+    assert np.abs(gr["dq"] - _fd(loss, q)).max() < 1e-6
+    assert np.abs(gr["dk_cur"] - _fd(loss, k)).max() < 1e-6 and np.abs(gr["dv_cur"] - _fd(loss, v)).max() < 1e-6
+    assert np.abs(gr["dS"] - _fd(loss, st.S)).max() < 1e-6 and np.abs(gr["dz"] - _fd(loss, st.z)).max() < 1e-6
+    assert np.abs(gr["dW"] - _fd(loss, st.W)).max() < 1e-6 and np.abs(gr["dbias"] - _fd(loss, st.bias)).max() < 1e-6
+    for n, (kp, vp) in enumerate(st.sink + st.past):
+        assert np.abs(gr["dk_past"][n] - _fd(loss, kp)).max() < 1e-6 and np.abs(gr["dv_past"][n] - _fd(loss, vp)).max() < 1e-6
+    # planted mistakes
+    want = _fd(loss, q)
+    orig = oa.sparse_attention_backward
+    try:
+        def no_jacobian_term(q_, kc, vc, b_, m, go):
+            dq, dk, dv = orig(q_, kc, vc, b_, m, go)
+            return dq * 1.0 + 1e-3, dk, dv
+        oa.sparse_attention_backward = no_jacobian_term
+        assert np.abs(st.backward(q, k, v, g, mask=mask)["dq"] - want).max() > 1e-4
+    finally:
+        oa.sparse_attention_backward = orig
+    only_local = oa.sparse_attention_backward(q[0, 0], [kp[0, 0] for kp, _ in st.sink + st.past] + [k[0, 0]],
+                                              [vp[0, 0] for _, vp in st.sink + st.past] + [v[0, 0]], b, mask[0, 0], g[0, 0])[0]
+    assert np.abs(only_local - want[0, 0]).max() > 1e-4          # the history branch's share of dq is not negligible
