@@ -182,6 +182,17 @@ hf_status hf_block_select(hf_ctx* ctx, int layer, const void* q, const void* k_c
 hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur,
                         const int32_t* idx, void* o_local, float* lse, void* stream);
 
+/* Gradient of Eq. 6 with respect to the queries: the first piece of the backward pass that the training rollout needs
+ * for the denoising step it runs with gradient (Alg. 1).  With p = softmax over the kept keys and g = dL/dO_local,
+ *   dq_r = (1 / sqrt(d)) sum_c p_rc (g_r . v_c - g_r . o_local_r) k_c      (the block mask is the forward's, held fixed)
+ *   q, k_cur, v_cur, idx   as for hf_sparse_swa (same cache contents, same selection)
+ *   o_local bf16 [B,H,T_c,d], lse float [B,H,T_c]   what hf_sparse_swa returned for them
+ *   d_o bf16 [B,H,T_c,d] = dL/dO_local;  dq bf16 [B,H,T_c,d] out
+ * 128-token blocks only (HF_ERR_UNSUPPORTED otherwise, and with the temporal rotation set).  dK, dV and the gradients of
+ * the history branch are not built yet. */
+hf_status hf_sparse_swa_backward_dq(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
+                                    const void* o_local, const float* lse, const void* d_o, void* dq, void* stream);
+
 /* Eq. 4 without rotation: o_hist[r] = W (phi(q_r) S / (phi(q_r) . z + eps)) + bias, bf16 [B,H,T_c,d]. */
 hf_status hf_linear_attn(hf_ctx* ctx, int layer, const void* q, void* o_hist, void* stream);
 

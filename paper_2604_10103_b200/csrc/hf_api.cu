@@ -6,6 +6,7 @@
 #include "k_swa_tc5.cuh"
 #include "k_swa_tc5p.cuh"
 #include "k_swa_tc5g.cuh"
+#include "k_swa_bwd.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
 #include "k_state_items.cuh"
@@ -93,6 +94,7 @@ struct hf_ctx {
     uint32_t* union_entries = nullptr;   // small-block tcgen05 attention: merged kept lists [B*H * units, max tiles, G] ...
     int* union_tiles = nullptr;          // ... and tiles per unit
     int union_max_tiles = 0;
+    float* bwd_delta = nullptr;          // backward pass: g . o_local per query row [B*H, T_c]
     float* partials = nullptr;       // absorb split partials
     float* partials_layers = nullptr;    // layer-batched state update: one partial per (layer, batch*head, group)
     size_t partials_layers_count = 0;
@@ -183,7 +185,7 @@ void free_all(hf_ctx* c) {
     for (auto& L : c->layers) { cudaFree(L.W_full); cudaFree(L.mask); cudaFree(L.idx); }
     cudaFree(c->ring_k_all); cudaFree(c->ring_v_all); cudaFree(c->pooled_k_all); cudaFree(c->S_all); cudaFree(c->z_all);
     cudaFree(c->sf_hi_all); cudaFree(c->sf_lo_all); cudaFree(c->W_all); cudaFree(c->bias_all);
-    cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
+    cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->bwd_delta); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     cudaFree(c->trope_tab[0]); cudaFree(c->trope_tab[1]); cudaFree(c->q_rot); cudaFree(c->k_rot);
@@ -590,6 +592,36 @@ hf_status launch_swa(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur,
     HF_SWA_CASE(16, 64); HF_SWA_CASE(16, 128); HF_SWA_CASE(64, 64); HF_SWA_CASE(64, 128); HF_SWA_CASE(128, 64); HF_SWA_CASE(128, 128);
 #undef HF_SWA_CASE
     return fail(HF_ERR_UNSUPPORTED, "no attention kernel for block %d, head_dim %d", b, d);
+}
+
+template <int D>
+hf_status launch_bwd_dq(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx, int keep,
+                               const bf16* o_local, const float* lse, const bf16* d_o, bf16* dq, cudaStream_t st) {
+    typedef SwaBwd<D> C;
+    if (c->bwd_delta == nullptr) {
+        HF_TRY(dmalloc(&c->bwd_delta, (size_t)c->BH * c->Tc));
+        HF_CUDA(cudaFuncSetAttribute(k_swa_bwd_dq<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    }
+    const long long rows = (long long)c->BH * c->Tc;
+    k_rowdot<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(d_o, o_local, c->bwd_delta, rows);
+    HF_TRY(post_launch(c, "k_rowdot"));
+    CUtensorMap tq, tdo, tk, tv;
+    HF_TRY(make_map(c, &tq, q, 1));
+    HF_TRY(make_map(c, &tdo, d_o, 1));
+    HF_TRY(make_map(c, &tk, k_cur, 1));
+    HF_TRY(make_map(c, &tv, v_cur, 1));
+    SwaBwdParams p;
+    memset(&p, 0, sizeof(p));
+    p.idx = idx; p.keep = keep; p.Tc = c->Tc; p.n_b = c->n_b; p.n_cached = L.n_cached; p.ring_head = L.head; p.P = c->R; p.n_sink = L.n_sink;
+    p.Tm = c->Tm; p.n_units = c->Tm * c->BH;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D)); p.scale = (float)(1.0 / std::sqrt((double)D));
+    p.lse = lse; p.delta = c->bwd_delta; p.dq = dq; p.dev_status = c->dev_status;
+    const CUtensorMap& rk = c->R + c->n_sink_max > 0 ? L.tm_kring : tk;
+    const CUtensorMap& rv = c->R + c->n_sink_max > 0 ? L.tm_vring : tv;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, false);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_bwd_dq<D>, tq, tdo, rk, rv, tk, tv, p));
+    return post_launch(c, "k_swa_bwd_dq");
 }
 
 hf_status ensure_staging(hf_ctx* c) {
@@ -1090,6 +1122,23 @@ hf_status hf_sparse_swa(hf_ctx* c, int layer, const void* q, const void* k_cur, 
     }
     return launch_swa(c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, nullptr, (bf16*)o_local, lse,
                       (cudaStream_t)stream);
+}
+
+hf_status hf_sparse_swa_backward_dq(hf_ctx* c, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
+                                    const void* o_local, const float* lse, const void* d_o, void* dq, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q")); HF_TRY(check_ptr(k_cur, "k_cur")); HF_TRY(check_ptr(v_cur, "v_cur"));
+    HF_TRY(check_ptr(o_local, "o_local")); HF_TRY(check_ptr(lse, "lse")); HF_TRY(check_ptr(d_o, "d_o")); HF_TRY(check_ptr(dq, "dq"));
+    if (c->cfg.block != 128) return fail(HF_ERR_UNSUPPORTED, "the backward kernel takes 128-token blocks");
+    if (c->has_trope) return fail(HF_ERR_UNSUPPORTED, "the backward kernel does not rotate its inputs (temporal RoPE is set)");
+    LayerState& L = c->layers[layer];
+    const int keep = keep_for(c, (L.n_sink + L.n_cached + 1) * c->n_b);
+    if (idx == nullptr) {
+        if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
+        idx = L.idx;
+    }
+    return HF_DISPATCH_D(c, launch_bwd_dq, c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, (const bf16*)o_local, lse,
+                         (const bf16*)d_o, (bf16*)dq, (cudaStream_t)stream);
 }
 
 hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void* stream) {
