@@ -32,7 +32,7 @@ from paper_2604_10103_b200 import inputs as gen, replicas  # noqa: E402
 METRIC = "hybrid-attn latent frames/s at 832x480 shape"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention kernel (history term inside) at this
 # workload's layer shape, from an ncu capture of that kernel; None when the kernel has changed since the capture.
-SWA_DRAM_BYTES_PER_LAUNCH = None
+SWA_DRAM_BYTES_PER_LAUNCH = 106.6e6
 UNIT = "latent frames/s"
 
 
