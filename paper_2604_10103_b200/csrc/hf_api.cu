@@ -97,7 +97,6 @@ struct hf_ctx {
     float* bwd_delta = nullptr;          // backward pass: g . o_local per query row [B*H, T_c]
     float* partials = nullptr;       // absorb split partials
     float* partials_layers = nullptr;    // layer-batched state update: one partial per (layer, batch*head, group)
-    int* item_arrivals = nullptr;        // ... and the groups of an item that have delivered (zero between launches)
     size_t partials_layers_count = 0;
     int nsplit_max = 1;
     float z_scale = 1.f;             // 1 (z = sum of phi(K)) or 1 / tokens_per_frame (per-frame means)
@@ -186,7 +185,7 @@ void free_all(hf_ctx* c) {
     for (auto& L : c->layers) { cudaFree(L.W_full); cudaFree(L.mask); cudaFree(L.idx); }
     cudaFree(c->ring_k_all); cudaFree(c->ring_v_all); cudaFree(c->pooled_k_all); cudaFree(c->S_all); cudaFree(c->z_all);
     cudaFree(c->sf_hi_all); cudaFree(c->sf_lo_all); cudaFree(c->W_all); cudaFree(c->bias_all);
-    cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->bwd_delta); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->item_arrivals); cudaFree(c->x_hi); cudaFree(c->x_lo);
+    cudaFree(c->union_entries); cudaFree(c->union_tiles); cudaFree(c->bwd_delta); cudaFree(c->pooled_q); cudaFree(c->pooled_kcur); cudaFree(c->hist); cudaFree(c->partials); cudaFree(c->partials_layers); cudaFree(c->x_hi); cudaFree(c->x_lo);
     cudaFree(c->dev_status);
     cudaFree(c->rope_q[0]); cudaFree(c->rope_q[1]); cudaFree(c->rope_k[0]); cudaFree(c->rope_k[1]);
     cudaFree(c->trope_tab[0]); cudaFree(c->trope_tab[1]); cudaFree(c->q_rot); cudaFree(c->k_rot);
@@ -350,29 +349,27 @@ hf_status launch_absorb_layers(hf_ctx* c, int first_layer, int n_layers, const C
     const size_t need = (size_t)n_layers * c->BH * p.ngroup * ((size_t)D * D + D);
     if (need > c->partials_layers_count) {
         HF_CUDA(cudaStreamSynchronize(st));
-        cudaFree(c->partials_layers); cudaFree(c->item_arrivals);
-        c->partials_layers = nullptr; c->item_arrivals = nullptr; c->partials_layers_count = 0;
+        cudaFree(c->partials_layers);
+        c->partials_layers = nullptr; c->partials_layers_count = 0;
         HF_TRY(dmalloc(&c->partials_layers, need));
-        HF_TRY(dmalloc(&c->item_arrivals, (size_t)n_layers * c->BH));
-        HF_CUDA(cudaMemsetAsync(c->item_arrivals, 0, (size_t)n_layers * c->BH * sizeof(int), st));
         c->partials_layers_count = need;
     }
     p.partials = c->partials_layers;
-    p.arrivals = c->item_arrivals;
-    // (the kernel leaves the counters at zero itself; cleared again here so that a launch that gave up on a wait cannot
-    // leave a later one miscounting)
-    HF_CUDA(cudaMemsetAsync(c->item_arrivals, 0, (size_t)n_layers * c->BH * sizeof(int), st));
-    p.S = c->S_all + (size_t)first_layer * dd; p.z = c->z_all + (size_t)first_layer * dz; p.z_scale = c->z_scale;
-    p.W = c->W_all ? c->W_all + (size_t)first_layer * c->cfg.heads * D * D : nullptr; p.heads = c->cfg.heads;
-    p.sf_hi = c->sf_hi_all + (size_t)first_layer * dd; p.sf_lo = c->sf_lo_all + (size_t)first_layer * dd;
-    for (int l = 0; l < n_layers; ++l) if (c->layers[first_layer + l].has_w) p.has_w_mask |= 1ull << l;
     for (int l = 0; l < n_layers; ++l) p.slot[l] = slot[l];
     p.cos_k = c->rope_k[0]; p.sin_k = c->rope_k[1]; p.rope_rows = c->Tc; p.dev_status = c->dev_status;
     const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
     PdlLaunch pl(dim3(grid), dim3(A::THREADS), A::SMEM_BYTES, st, false);
     if (c->has_rope_k) HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, true>, tk, tv, p));
     else HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_absorb_items<D, false>, tk, tv, p));
-    return post_launch(c, "k_absorb_items");
+    HF_TRY(post_launch(c, "k_absorb_items"));
+    unsigned long long has_w = 0;
+    for (int l = 0; l < n_layers; ++l) if (c->layers[first_layer + l].has_w) has_w |= 1ull << l;
+    PdlLaunch pf(dim3(D / 16, c->BH, n_layers), dim3(D), 0, st, true);
+    HF_CUDA(cudaLaunchKernelEx(&pf.cfg, k_reduce_fold<D>, (const float*)c->partials_layers, p.ngroup, p.ngroup,
+                               c->S_all + (size_t)first_layer * dd, c->z_all + (size_t)first_layer * dz, c->z_scale,
+                               (const bf16*)(c->W_all ? c->W_all + (size_t)first_layer * c->cfg.heads * D * D : nullptr), c->cfg.heads,
+                               c->BH, c->sf_hi_all + (size_t)first_layer * dd, c->sf_lo_all + (size_t)first_layer * dd, has_w));
+    return post_launch(c, "k_reduce_fold (layers)");
 }
 
 template <int D>

@@ -15,15 +15,13 @@
 //   MMA warp        P_s += A_hi V + A_lo V over the tiles of split s, two P accumulators in tensor memory alternating
 //   4 merge warps   R = P of the unit's first split, R += P_s for the others, likewise the phi(K) sums; when the unit ends R
 //                   and the sums go to the unit's slot of the scratch buffer.  They run beside the next split's tiles.
-// The thread block that delivers an item's last group sum then adds the item's ngroup slots to its state in ascending order
-// and refolds S W^T (the routines of k_reduce_fold, run by its merge warps beside the next unit's tiles): no second launch.
-// With two groups per item the scratch traffic is 2 x 66 KB per item (against 2.4 MB of K, V read), and 720 units spread
-// over the SMs within 3 % of evenly where 360 whole items would leave a third of them idle for the last third of the launch.
+// k_reduce_fold then adds the ngroup slots of every item to its state in ascending order and refolds S W^T.  With two
+// groups per item the scratch traffic is 2 x 66 KB per item (against 2.4 MB of K, V read), and 720 units spread over the
+// SMs within 3 % of evenly where 360 whole items would leave a third of them idle for the last third of the launch.
 // Tensor memory (512 columns at head dim 128): R [0, D), P_0 [D, 2D), P_1 [2D, 3D), A_0 / A_1 (hi 32 + lo 32 columns each).
 // Every wait is bounded and reports through the device status word; nothing traps.
 #pragma once
 #include "k_state_tc5.cuh"
-#include "k_state_mma.cuh"
 
 #define HF_MAX_BATCH_LAYERS 64
 
@@ -34,9 +32,7 @@ struct AbsorbItems {
     static constexpr int K_BYTES = A::K_BYTES, VSUB_BYTES = A::VSUB_BYTES, V_BYTES = A::V_BYTES;
     static constexpr int OFF_K = 0, OFF_V = NST * K_BYTES, OFF_BAR = OFF_V + NST * V_BYTES;
     static constexpr int OFF_Z = OFF_BAR + 256;          // phi(K) sums of a split, [2 buffers][NQ][D] floats
-    static constexpr int OFF_W = OFF_Z + 2 * NQ * D * 4; // reduce + fold of a finished item: W_h (bf16 [D][D]) ...
-    static constexpr int OFF_A = OFF_W + D * D * 2;      // ... and 16 rows of S as three bf16 terms
-    static constexpr int SMEM_BYTES = OFF_A + 3 * 16 * D * 2 + 1024;
+    static constexpr int SMEM_BYTES = OFF_Z + 2 * NQ * D * 4 + 1024;
     static constexpr int WARP_MERGE = 4 * NQ;            // four merge warps: warp index % 4 = TMEM lane quadrant
     static constexpr int WARP_TMA = 4 * NQ + 4, WARP_MMA = 4 * NQ + 5;
     static constexpr int THREADS = 32 * (4 * NQ + 6);
@@ -50,17 +46,6 @@ struct AbsorbItemsParams {
     int BH, n_units;          // units = layers of the call x B*H x ngroup; unit u: item u / ngroup (layer item / BH, batch*head item % BH), group u % ngroup
     int nsplit, ngroup;       // splits of an item's token range and groups of consecutive splits (the summation order)
     float* partials;          // [items][ngroup][D*D + D]: per unit the sum of its splits' phi(K)^T V, then of their phi(K) sums
-    // The thread block that delivers the LAST group sum of an item adds the item's group sums to its state and refolds it
-    // (reduce_fold_rows of k_state_mma.cuh, run by its merge warps): no second kernel.
-    int* arrivals;            // [items], zero between launches (the last arrival resets its counter)
-    float* S;                 // [layers of the call][B*H][D][D]
-    float* z;                 // [layers of the call][B*H][D]
-    float z_scale;
-    const bf16* W;            // [layers of the call][H][D][D] or nullptr
-    int heads;
-    bf16* sf_hi;              // [layers of the call][B*H][D][D]
-    bf16* sf_lo;
-    unsigned long long has_w_mask;
     int slot[HF_MAX_BATCH_LAYERS];   // coordinate 3 of the tensor maps for each layer of the call
     const float* cos_k;       // rotation tables (ROPE instantiation only)
     const float* sin_k;
@@ -86,7 +71,6 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                    bar_dfull = bar0 + 128, bar_pfree = bar0 + 144, bar_zfull = bar0 + 160;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 176);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 180);
-    volatile int* last_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 184);
     float* z_x = reinterpret_cast<float*>(s_gen + C::OFF_Z);            // [2][NQ][D]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -248,31 +232,6 @@ k_absorb_items(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
                         make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
             }
             out[D * D + a] = zsum;
-            // ---- the item is complete when all of its groups have delivered: the last one to arrive folds it into the state
-            __threadfence();
-            asm volatile("bar.sync 2, %0;\n" ::"n"(D) : "memory");
-            if (a == 0) {
-                const int item = unit / ngroup;
-                const int seen = atomicAdd(p.arrivals + item, 1);
-                if (seen == ngroup - 1) p.arrivals[item] = 0;
-                *last_flag = seen == ngroup - 1;
-                __threadfence();
-            }
-            asm volatile("bar.sync 2, %0;\n" ::"n"(D) : "memory");
-            if (*last_flag) {
-                const int item = unit / ngroup;
-                const int lay = item / p.BH, bh = item - lay * p.BH;
-                const bool with_w = p.W != nullptr && ((p.has_w_mask >> lay) & 1ull);
-                uint8_t* sW = s_gen + C::OFF_W;
-                uint8_t* sA = s_gen + C::OFF_A;
-                if (with_w) fold_fetch_w<D>(sW, p.W + ((size_t)lay * p.heads + bh % p.heads) * D * D, a);
-#pragma unroll 1
-                for (int a0 = 0; a0 < D; a0 += 16)
-                    reduce_fold_rows<D>(sW, sA, p.partials + (size_t)item * ngroup * (D * D + D), ngroup, ngroup, p.S + (size_t)item * D * D,
-                                        p.z + (size_t)item * D, p.z_scale, with_w, true, p.sf_hi + (size_t)item * D * D,
-                                        p.sf_lo + (size_t)item * D * D, a0, a, 2);
-                asm volatile("bar.sync 2, %0;\n" ::"n"(D) : "memory");      // W_h and the row buffers are free for the next item
-            }
         }
     } else {
         // ================================================================= phi(K) into tensor memory

@@ -139,45 +139,49 @@ k_absorb_mma(const bf16* __restrict__ k_ev, const bf16* __restrict__ v_ev, int n
 // nsplit == 0: fold only.  sf_hi == nullptr: state update only.  z_scale: 1 for z = sum of phi(K) rows, 1 / tokens-per-frame
 // for the per-frame-mean reading of Eq. 3.  partials: [layers][B*H][nsplit][D*D + D]; S, sf_hi, sf_lo: [layers][B*H][D][D];
 // z: [layers][B*H][D]; W: [layers][H][D][D] or nullptr, used for the layers whose bit is set in has_w_mask.
-// The two halves of k_reduce_fold as device routines for D cooperating threads (thread index cp = 0 .. D-1) that meet on
-// named barrier `bar_id`: the kernel below is one call of each per thread block; the layer-batched state update calls them
-// from its merge warps for the item whose last group sum it has just delivered.
 template <int D>
-__device__ __forceinline__ void fold_fetch_w(uint8_t* sW, const bf16* __restrict__ w_h, int cp) {
-    constexpr int CPR = D / 8, ROW_BYTES = D * 2;                   // 16-byte chunks per row
-#pragma unroll
-    for (int i = 0; i < CPR; ++i) {
-        const int id = cp + i * D, row = id / CPR, ch = id % CPR;
-        cp_async16(smem_u32(sW) + swz<ROW_BYTES>(row, ch), w_h + (size_t)row * D + ch * 8, true);
-    }
-    cp_async_commit();
-}
-// Rows a0 .. a0 + 15 of one (layer, batch*head) item: S += its partials (grouped order), z (when a0 == 0), then the fold.
-// part: the item's partials [nsplit][D*D + D]; w_ready: the caller has not yet waited for fold_fetch_w's copies.
-template <int D>
-__device__ __forceinline__ void reduce_fold_rows(uint8_t* sW, uint8_t* sA, const float* part, int nsplit, int ngroup,
-                                                 float* __restrict__ S_it, float* __restrict__ z_it, float z_scale, bool with_w, bool fold,
-                                                 bf16* __restrict__ sf_hi_it, bf16* __restrict__ sf_lo_it, int a0, int cp, int bar_id) {
+__global__ void __launch_bounds__(D)
+k_reduce_fold(const float* __restrict__ partials, int nsplit, int ngroup, float* __restrict__ S, float* __restrict__ z, float z_scale,
+              const bf16* __restrict__ W, int heads, int BH, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo,
+              unsigned long long has_w_mask) {
     constexpr int ROWS = 16;
     constexpr int PART_FLOATS = D * D + D;
     constexpr int ROW_BYTES = D * 2;
-    const int lane = cp & 31, warp = cp >> 5;
+    __shared__ __align__(128) uint8_t sW[D * ROW_BYTES];            // W_h [c'][c], 16-byte chunks XOR-swizzled by the row
+    __shared__ __align__(128) uint8_t sA[3][ROWS * ROW_BYTES];      // the block's rows of S as bf16 hi / mid / lo, same swizzle
+    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, lay = blockIdx.z, h = bh % heads;
+    const size_t item = (size_t)lay * BH + bh;
+    const int cp = threadIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr && ((has_w_mask >> lay) & 1ull);
+    if (with_w) {       // the matrix does not depend on the kernel before this one: fetched while that kernel drains
+        const bf16* wsrc = W + ((size_t)lay * heads + h) * D * D;
+        constexpr int CPR = D / 8;                                  // 16-byte chunks per row
+#pragma unroll
+        for (int i = 0; i < CPR; ++i) {
+            const int id = threadIdx.x + i * D, row = id / CPR, ch = id % CPR;
+            cp_async16(smem_u32(sW) + swz<ROW_BYTES>(row, ch), wsrc + (size_t)row * D + ch * 8, true);
+        }
+        cp_async_commit();
+    }
+    pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
+    const float* base = partials + item * nsplit * PART_FLOATS;
+    float* S_it = S + item * D * D;
     float sum[ROWS];
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) sum[r] = S_it[(size_t)(a0 + r) * D + cp];
     float ztot = 0.f;           // this call's sum of phi(K) rows; enters z scaled (1, or 1 / tokens per frame)
-    const bool do_z = a0 == 0 && nsplit > 0;
+    const bool do_z = blockIdx.x == 0 && nsplit > 0;
     for (int g = 0; g < ngroup && nsplit > 0; ++g) {
         const int s0 = (int)(((long long)nsplit * g) / ngroup), s1 = (int)(((long long)nsplit * (g + 1)) / ngroup);
         float sg[ROWS], zg = 0.f;
 #pragma unroll
-        for (int r = 0; r < ROWS; ++r) sg[r] = __ldcg(part + (size_t)s0 * PART_FLOATS + (size_t)(a0 + r) * D + cp);
-        if (do_z) zg = __ldcg(part + (size_t)s0 * PART_FLOATS + D * D + cp);
+        for (int r = 0; r < ROWS; ++r) sg[r] = __ldcg(base + (size_t)s0 * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+        if (do_z) zg = __ldcg(base + (size_t)s0 * PART_FLOATS + D * D + cp);
 #pragma unroll 2
         for (int s = s0 + 1; s < s1; ++s) {      // ascending split order per element; several splits' loads in flight
 #pragma unroll
-            for (int r = 0; r < ROWS; ++r) sg[r] += __ldcg(part + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
-            if (do_z) zg += __ldcg(part + (size_t)s * PART_FLOATS + D * D + cp);
+            for (int r = 0; r < ROWS; ++r) sg[r] += __ldcg(base + (size_t)s * PART_FLOATS + (size_t)(a0 + r) * D + cp);
+            if (do_z) zg += __ldcg(base + (size_t)s * PART_FLOATS + D * D + cp);
         }
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) sum[r] += sg[r];
@@ -186,21 +190,20 @@ __device__ __forceinline__ void reduce_fold_rows(uint8_t* sW, uint8_t* sA, const
     if (nsplit > 0) {
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) S_it[(size_t)(a0 + r) * D + cp] = sum[r];
-        if (do_z) z_it[cp] += ztot * z_scale;
+        if (do_z) z[item * D + cp] += ztot * z_scale;
     }
     if (!fold) return;
     if (!with_w) {
 #pragma unroll
         for (int r = 0; r < ROWS; ++r) {
             const __nv_bfloat16 hi = __float2bfloat16_rn(sum[r]);
-            const size_t o = (size_t)(a0 + r) * D + cp;
-            sf_hi_it[o] = hi;
-            sf_lo_it[o] = __float2bfloat16_rn(sum[r] - __bfloat162float(hi));
+            const size_t o = (item * D + a0 + r) * D + cp;
+            sf_hi[o] = hi;
+            sf_lo[o] = __float2bfloat16_rn(sum[r] - __bfloat162float(hi));
         }
         return;
     }
     // ---- the rows as three bf16 terms (each difference is exact in fp32), column cp of every row
-    asm volatile("bar.sync %0, %1;\n" ::"r"(bar_id), "n"(D) : "memory");     // the previous row tile's products have read sA
 #pragma unroll
     for (int r = 0; r < ROWS; ++r) {
         const __nv_bfloat16 t0 = __float2bfloat16_rn(sum[r]);
@@ -208,12 +211,12 @@ __device__ __forceinline__ void reduce_fold_rows(uint8_t* sW, uint8_t* sA, const
         const __nv_bfloat16 t1 = __float2bfloat16_rn(r1);
         const __nv_bfloat16 t2 = __float2bfloat16_rn(r1 - __bfloat162float(t1));
         const uint32_t off = swz<ROW_BYTES>(r, cp >> 3) + (cp & 7) * 2;
-        *reinterpret_cast<__nv_bfloat16*>(sA + off) = t0;
-        *reinterpret_cast<__nv_bfloat16*>(sA + ROWS * ROW_BYTES + off) = t1;
-        *reinterpret_cast<__nv_bfloat16*>(sA + 2 * ROWS * ROW_BYTES + off) = t2;
+        *reinterpret_cast<__nv_bfloat16*>(sA[0] + off) = t0;
+        *reinterpret_cast<__nv_bfloat16*>(sA[1] + off) = t1;
+        *reinterpret_cast<__nv_bfloat16*>(sA[2] + off) = t2;
     }
     cp_async_wait<0>();
-    asm volatile("bar.sync %0, %1;\n" ::"r"(bar_id), "n"(D) : "memory");
+    __syncthreads();
     // ---- out[a][c'] = sum_c S[a][c] W_h[c'][c]: A = the rows (16 x D), B = W_h as stored ([n][k], k contiguous)
     float acc[4][4];
 #pragma unroll
@@ -224,7 +227,7 @@ __device__ __forceinline__ void reduce_fold_rows(uint8_t* sW, uint8_t* sA, const
         uint32_t af[3][4];
 #pragma unroll
         for (int t = 0; t < 3; ++t)
-            ldsm_x4(smem_u32(sA) + t * ROWS * ROW_BYTES + swz<ROW_BYTES>(lane & 15, ks * 2 + (lane >> 4)), af[t][0], af[t][1], af[t][2], af[t][3]);
+            ldsm_x4(smem_u32(sA[t]) + swz<ROW_BYTES>(lane & 15, ks * 2 + (lane >> 4)), af[t][0], af[t][1], af[t][2], af[t][3]);
 #pragma unroll
         for (int np = 0; np < 2; ++np) {
             uint32_t b0, b1, b2, b3;
@@ -243,29 +246,9 @@ __device__ __forceinline__ void reduce_fold_rows(uint8_t* sW, uint8_t* sA, const
             const float x0 = acc[n][2 * half], x1 = acc[n][2 * half + 1];
             const uint32_t hp = pack_bf16(x0, x1);
             const float2 hf = unpack_bf16(hp);
-            const size_t o = (size_t)(a0 + (lane >> 2) + half * 8) * D + n0 + n * 8 + 2 * (lane & 3);
-            *reinterpret_cast<uint32_t*>(sf_hi_it + o) = hp;
-            *reinterpret_cast<uint32_t*>(sf_lo_it + o) = pack_bf16(x0 - hf.x, x1 - hf.y);
+            const size_t o = (item * D + a0 + (lane >> 2) + half * 8) * D + n0 + n * 8 + 2 * (lane & 3);
+            *reinterpret_cast<uint32_t*>(sf_hi + o) = hp;
+            *reinterpret_cast<uint32_t*>(sf_lo + o) = pack_bf16(x0 - hf.x, x1 - hf.y);
         }
     }
-}
-
-template <int D>
-__global__ void __launch_bounds__(D)
-k_reduce_fold(const float* __restrict__ partials, int nsplit, int ngroup, float* __restrict__ S, float* __restrict__ z, float z_scale,
-              const bf16* __restrict__ W, int heads, int BH, bf16* __restrict__ sf_hi, bf16* __restrict__ sf_lo,
-              unsigned long long has_w_mask) {
-    constexpr int ROWS = 16;
-    constexpr int PART_FLOATS = D * D + D;
-    constexpr int ROW_BYTES = D * 2;
-    __shared__ __align__(128) uint8_t sW[D * ROW_BYTES];            // W_h [c'][c], 16-byte chunks XOR-swizzled by the row
-    __shared__ __align__(128) uint8_t sA[3 * ROWS * ROW_BYTES];     // the block's rows of S as bf16 hi / mid / lo, same swizzle
-    const int a0 = blockIdx.x * ROWS, bh = blockIdx.y, lay = blockIdx.z, h = bh % heads;
-    const size_t item = (size_t)lay * BH + bh;
-    const bool fold = sf_hi != nullptr, with_w = fold && W != nullptr && ((has_w_mask >> lay) & 1ull);
-    // the matrix does not depend on the kernel before this one: fetched while that kernel drains
-    if (with_w) fold_fetch_w<D>(sW, W + ((size_t)lay * heads + h) * D * D, threadIdx.x);
-    pdl_wait();         // launched under the tail of the partials kernel: its partials (and the state) are complete from here on
-    reduce_fold_rows<D>(sW, sA, partials + item * nsplit * PART_FLOATS, nsplit, ngroup, S + item * D * D, z + item * D, z_scale, with_w, fold,
-                        fold ? sf_hi + item * D * D : nullptr, fold ? sf_lo + item * D * D : nullptr, a0, threadIdx.x, 1);
 }
