@@ -444,9 +444,8 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     const int Tn = (L.n_sink + L.n_cached + 1) * c->n_b;
     const int keep = keep_for(c, Tn);
     ChunkTable tab = make_table(c, L, k_cur, nullptr);
-    constexpr int QR = 4;       // query blocks scored per thread block (each pooled key row is fetched once per group)
-    PdlLaunch pl(dim3((c->Tm + QR - 1) / QR, c->BH), dim3(256), SelectSmem<QR>::BYTES, st, true);      // follows the pooling kernel launched above
-    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D, QR>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+    PdlLaunch pl(dim3(c->Tm, c->BH), dim3(256), 0, st, true);      // follows the pooling kernel launched above
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
                                L.mask, L.idx, mask_out, idx_out, scores_out));
     HF_TRY(post_launch(c, "k_select"));
     L.sel_epoch = L.cache_epoch;
@@ -797,9 +796,6 @@ hf_status hf_create(const hf_config* cfg, int device, hf_ctx** out) {
                            cudaFuncSetAttribute(k_swa_tc5g<128, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, 2>::SMEM_BYTES) != cudaSuccess ||
                            cudaFuncSetAttribute(k_swa_tc5g<128, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SwaTc5<128, 2>::SMEM_BYTES) != cudaSuccess))
             s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_swa_tc5g) failed");
-        if (s == HF_OK && (cudaFuncSetAttribute(k_select<64, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, SelectSmem<4>::BYTES) != cudaSuccess ||
-                           cudaFuncSetAttribute(k_select<128, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, SelectSmem<4>::BYTES) != cudaSuccess))
-            s = fail(HF_ERR_CUDA, "cudaFuncSetAttribute(k_select) failed");
         if (s == HF_OK) s = set_state_attr<64>();
         if (s == HF_OK) s = set_state_attr<128>();
     }

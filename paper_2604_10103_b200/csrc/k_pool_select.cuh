@@ -182,42 +182,29 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy_layers(const __grid_consta
 // l + 32, ... ascending, product and sum rounded separately; lane l holds partial l, so the loads of a key row are
 // coalesced), then the butterfly p[l] + p[l ^ off], off = 16 .. 1: both partners get the same value (IEEE addition
 // commutes), so lane 0 ends with the fold of the upper half onto the lower half level by level, bit for bit.
-// grid (ceil(T_m / QR), B*H), 256 threads, dynamic shared memory SelectSmem<QR>::BYTES.  A thread block scores QR
-// consecutive query blocks of a head against all T_n key blocks -- every pooled key row is fetched once per group of QR
-// query blocks (the traffic out of L2 is what bounds this kernel) -- and keeps, per query block, the top K under the total
-// order (score descending, block index ascending): bit mask + ascending index list.
-template <int QR>
-struct SelectSmem {
-    static constexpr int OFF_SC = 0;                                   // scores [QR][HF_MAX_TN] float
-    static constexpr int OFF_KEYS = OFF_SC + QR * HF_MAX_TN * 4;       // sort keys [QR][HF_MAX_TN] 64-bit
-    static constexpr int OFF_KEEP = OFF_KEYS + QR * HF_MAX_TN * 8;     // kept flags [QR][HF_MAX_TN] bytes
-    static constexpr int BYTES = OFF_KEEP + QR * HF_MAX_TN;
-};
-
-template <int D, int QR>
+// grid (T_m, B*H), 256 threads.  One query-block row: T_n scores, top-K under the total order (score descending, block
+// index ascending; by counting for short rows, by a bitonic sort of (score, index) keys for long ones), bit mask +
+// ascending index list.
+template <int D>
 __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __restrict__ pooled_q,
                                                 int n_b, int Tm, int Tn, int keep, int mask_words,
                                                 uint32_t* __restrict__ mask, int32_t* __restrict__ idx,
                                                 uint32_t* __restrict__ mask_out, int32_t* __restrict__ idx_out,
                                                 float* __restrict__ scores_out) {
-    extern __shared__ __align__(16) uint8_t sel_smem[];
-    typedef SelectSmem<QR> SM;
-    float* sc = reinterpret_cast<float*>(sel_smem + SM::OFF_SC);
-    unsigned long long* keys = reinterpret_cast<unsigned long long*>(sel_smem + SM::OFF_KEYS);
-    uint8_t* keepf = sel_smem + SM::OFF_KEEP;
-    const int i0 = blockIdx.x * QR, bh = blockIdx.y;
-    const int nq = min(QR, Tm - i0);                    // query blocks of this thread block
+    __shared__ float sc[HF_MAX_TN];
+    __shared__ uint8_t keepf[HF_MAX_TN];
+    __shared__ unsigned long long keys[HF_MAX_TN];
+    const int i = blockIdx.x, bh = blockIdx.y;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t row = (size_t)bh * Tm + i;
     pdl_trigger();              // the attention kernel may be made resident as blocks of this grid leave
     pdl_wait();                 // the pooled rows of the query and of the current chunk come from the kernel before
-    // One warp per key row, lane l = partial l.  All loads of a pass (the lane's columns of eight key rows) are issued before
-    // the first use; every key row then serves the QR query rows, whose lane columns sit in registers.
-    constexpr int NW = 8, PER = 8, M = D / 32;
-    float qv[QR][M];
+    // One warp per score, lane l = partial l.  All loads of a pass (the lane's columns of the query row and of sixteen key
+    // rows) are issued before the first use: one trip to memory per pass, and one pass covers 128 key blocks.
+    constexpr int NW = 8, PER = 16, M = D / 32;
+    float qv[M];
 #pragma unroll
-    for (int r = 0; r < QR; ++r)
-#pragma unroll
-        for (int m = 0; m < M; ++m) qv[r][m] = r < nq ? __ldg(pooled_q + ((size_t)bh * Tm + i0 + r) * D + lane + 32 * m) : 0.f;
+    for (int m = 0; m < M; ++m) qv[m] = __ldg(pooled_q + row * D + lane + 32 * m);
     for (int base = 0; base < Tn; base += NW * PER) {
         float kv[PER][M];
 #pragma unroll
@@ -230,18 +217,15 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
         }
 #pragma unroll
         for (int u = 0; u < PER; ++u) {
+            float p = __fmul_rn(qv[0], kv[u][0]);
+#pragma unroll
+            for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[m], kv[u][m]));
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, off));
             const int j = base + warp + NW * u;
-#pragma unroll
-            for (int r = 0; r < QR; ++r) {
-                float p = __fmul_rn(qv[r][0], kv[u][0]);
-#pragma unroll
-                for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[r][m], kv[u][m]));
-#pragma unroll
-                for (int off = 16; off >= 1; off >>= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, off));
-                if (lane == 0 && j < Tn && r < nq) {
-                    sc[r * HF_MAX_TN + j] = p;
-                    if (scores_out) scores_out[((size_t)bh * Tm + i0 + r) * Tn + j] = p;
-                }
+            if (lane == 0 && j < Tn) {
+                sc[j] = p;
+                if (scores_out) scores_out[row * Tn + j] = p;
             }
         }
     }
@@ -251,25 +235,22 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
     // here it ranks below every number, NaNs among themselves by block index, so that exactly `keep` blocks are kept whatever
     // the inputs hold.
     if (Tn <= 128) {
-        // short rows: count, for every (query block, key block), the key blocks that come before it
-        for (int e = threadIdx.x; e < nq * Tn; e += 256) {
-            const int r = e / Tn, j = e - r * Tn;
-            const float* row = sc + r * HF_MAX_TN;
-            const float s = row[j];
+        // short rows: count, for every block, the blocks that come before it
+        for (int j = threadIdx.x; j < Tn; j += 256) {
+            const float s = sc[j];
             const bool s_nan = s != s;
             int rank = 0;
             for (int jj = 0; jj < Tn; ++jj) {
-                const float s2 = row[jj];
+                const float s2 = sc[jj];
                 const bool s2_nan = s2 != s2;
                 const bool tie = (s2 == s) || (s_nan && s2_nan);
                 rank += (s2 > s) || (s_nan && !s2_nan) || (tie && jj < j);
             }
-            keepf[r * HF_MAX_TN + j] = rank < keep;
+            keepf[j] = rank < keep;
         }
     } else {
         // long rows (counting is quadratic in T_n): sort 64-bit keys (order-preserving image of the score, then the
-        // complement of the index) with a bitonic network, all query blocks of the thread block side by side, and compare
-        // every key block with its row's keep-th key
+        // complement of the index) in shared memory with a bitonic network and compare every block with the keep-th key
         auto key_of = [](float s, int j) -> unsigned long long {
             uint32_t u = __float_as_uint(s);
             if (s != s) u = 0u;                                         // NaN: below -inf
@@ -279,39 +260,30 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
             }
             return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)j);
         };
-        int n2 = 256, lg = 8;
-        while (n2 < Tn) { n2 <<= 1; ++lg; }
-        for (int e = threadIdx.x; e < nq * n2; e += 256) {
-            const int r = e >> lg, j = e & (n2 - 1);
-            keys[r * HF_MAX_TN + j] = j < Tn ? key_of(sc[r * HF_MAX_TN + j], j) : 0ull;      // padding sorts last
-        }
+        int n2 = 256;
+        while (n2 < Tn) n2 <<= 1;
+        for (int j = threadIdx.x; j < n2; j += 256) keys[j] = j < Tn ? key_of(sc[j], j) : 0ull;      // padding sorts last
         __syncthreads();
-        const int half = n2 >> 1;
         for (int size = 2; size <= n2; size <<= 1) {
             for (int stride = size >> 1; stride > 0; stride >>= 1) {
-                for (int e = threadIdx.x; e < nq * half; e += 256) {
-                    const int r = e / half, x = e - r * half;
+                for (int x = threadIdx.x; x < (n2 >> 1); x += 256) {
                     const int lo = 2 * x - (x & (stride - 1)), hi = lo + stride;      // the pair (lo, lo + stride)
                     const bool descending = (lo & size) == 0;
-                    unsigned long long* kr = keys + r * HF_MAX_TN;
-                    const unsigned long long a = kr[lo], b = kr[hi];
-                    if ((a < b) == descending) { kr[lo] = b; kr[hi] = a; }
+                    const unsigned long long a = keys[lo], b = keys[hi];
+                    if ((a < b) == descending) { keys[lo] = b; keys[hi] = a; }
                 }
                 __syncthreads();
             }
         }
-        for (int e = threadIdx.x; e < nq * Tn; e += 256) {
-            const int r = e / Tn, j = e - r * Tn;
-            keepf[r * HF_MAX_TN + j] = key_of(sc[r * HF_MAX_TN + j], j) >= keys[r * HF_MAX_TN + keep - 1];
-        }
+        const unsigned long long kth = keys[keep - 1];
+        for (int j = threadIdx.x; j < Tn; j += 256) keepf[j] = key_of(sc[j], j) >= kth;
     }
     __syncthreads();
-    for (int r = warp; r < nq; r += NW) {       // one warp per query block: mask words and the ascending list
-        const size_t row = (size_t)bh * Tm + i0 + r;
+    if (warp == 0) {
         int running = 0;
         for (int w = 0; w < mask_words; ++w) {
             const int j = w * 32 + lane;
-            const bool f = (j < Tn) && keepf[r * HF_MAX_TN + j];
+            const bool f = (j < Tn) && keepf[j];
             const uint32_t word = __ballot_sync(0xffffffffu, f);
             if (lane == 0) {
                 mask[row * mask_words + w] = word;
