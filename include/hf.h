@@ -188,10 +188,19 @@ hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur
  *   q, k_cur, v_cur, idx   as for hf_sparse_swa (same cache contents, same selection)
  *   o_local bf16 [B,H,T_c,d], lse float [B,H,T_c]   what hf_sparse_swa returned for them
  *   d_o bf16 [B,H,T_c,d] = dL/dO_local;  dq bf16 [B,H,T_c,d] out
- * 128-token blocks only (HF_ERR_UNSUPPORTED otherwise, and with the temporal rotation set).  dK, dV and the gradients of
- * the history branch are not built yet. */
+ * 128-token blocks only (HF_ERR_UNSUPPORTED otherwise, and with the temporal rotation set).  The gradients of the history
+ * branch are not built yet. */
 hf_status hf_sparse_swa_backward_dq(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
                                     const void* o_local, const float* lse, const void* d_o, void* dq, void* stream);
+
+/* Gradients of Eq. 6 with respect to the CURRENT chunk's keys and values (the cached chunks come from earlier,
+ * gradient-free passes of the rollout and receive none): with the notation above, for key token c of the current chunk
+ *   dv_c = sum_r p_rc g_r,     dk_c = (1 / sqrt(d)) sum_r p_rc (g_r . v_c - g_r . o_local_r) q_r
+ * over the query rows r whose query block keeps c's key block -- the context's last selection for this layer
+ * (hf_block_select or hf_hybrid_forward; HF_ERR_STATE if the cache changed since).  Arguments as for
+ * hf_sparse_swa_backward_dq; dk, dv bf16 [B,H,T_c,d] out (zero for a key block that no query block keeps). */
+hf_status hf_sparse_swa_backward_dkv(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const void* o_local,
+                                     const float* lse, const void* d_o, void* dk, void* dv, void* stream);
 
 /* Eq. 4 without rotation: o_hist[r] = W (phi(q_r) S / (phi(q_r) . z + eps)) + bias, bf16 [B,H,T_c,d]. */
 hf_status hf_linear_attn(hf_ctx* ctx, int layer, const void* q, void* o_hist, void* stream);

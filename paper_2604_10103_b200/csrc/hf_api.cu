@@ -598,10 +598,8 @@ template <int D>
 hf_status launch_bwd_dq(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const int32_t* idx, int keep,
                                const bf16* o_local, const float* lse, const bf16* d_o, bf16* dq, cudaStream_t st) {
     typedef SwaBwd<D> C;
-    if (c->bwd_delta == nullptr) {
-        HF_TRY(dmalloc(&c->bwd_delta, (size_t)c->BH * c->Tc));
-        HF_CUDA(cudaFuncSetAttribute(k_swa_bwd_dq<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-    }
+    if (c->bwd_delta == nullptr) HF_TRY(dmalloc(&c->bwd_delta, (size_t)c->BH * c->Tc));
+    HF_CUDA(cudaFuncSetAttribute(k_swa_bwd_dq<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
     const long long rows = (long long)c->BH * c->Tc;
     k_rowdot<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(d_o, o_local, c->bwd_delta, rows);
     HF_TRY(post_launch(c, "k_rowdot"));
@@ -622,6 +620,32 @@ hf_status launch_bwd_dq(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, false);
     HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_bwd_dq<D>, tq, tdo, rk, rv, tk, tv, p));
     return post_launch(c, "k_swa_bwd_dq");
+}
+
+template <int D>
+hf_status launch_bwd_dkv(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_cur, const bf16* v_cur, const bf16* o_local,
+                         const float* lse, const bf16* d_o, bf16* dk, bf16* dv, cudaStream_t st) {
+    typedef SwaBwdKV<D> C;
+    if (c->bwd_delta == nullptr) HF_TRY(dmalloc(&c->bwd_delta, (size_t)c->BH * c->Tc));
+    HF_CUDA(cudaFuncSetAttribute(k_swa_bwd_dkv<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+    const long long rows = (long long)c->BH * c->Tc;
+    k_rowdot<D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(d_o, o_local, c->bwd_delta, rows);
+    HF_TRY(post_launch(c, "k_rowdot"));
+    CUtensorMap tq, tdo, tk, tv;
+    HF_TRY(make_map(c, &tq, q, 1));
+    HF_TRY(make_map(c, &tdo, d_o, 1));
+    HF_TRY(make_map(c, &tk, k_cur, 1));
+    HF_TRY(make_map(c, &tv, v_cur, 1));
+    SwaBwdKVParams p;
+    memset(&p, 0, sizeof(p));
+    p.mask = L.mask; p.mask_words = c->mask_words; p.first_block = (L.n_sink + L.n_cached) * c->n_b;
+    p.Tc = c->Tc; p.n_b = c->n_b; p.Tm = c->Tm; p.n_units = c->BH * c->n_b;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)D)); p.scale = (float)(1.0 / std::sqrt((double)D));
+    p.lse = lse; p.delta = c->bwd_delta; p.dk = dk; p.dv = dv; p.dev_status = c->dev_status;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    PdlLaunch pl(dim3(grid), dim3(C::THREADS), C::SMEM_BYTES, st, false);
+    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_swa_bwd_dkv<D>, tq, tdo, tk, tv, p));
+    return post_launch(c, "k_swa_bwd_dkv");
 }
 
 hf_status ensure_staging(hf_ctx* c) {
@@ -1139,6 +1163,20 @@ hf_status hf_sparse_swa_backward_dq(hf_ctx* c, int layer, const void* q, const v
     }
     return HF_DISPATCH_D(c, launch_bwd_dq, c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, idx, keep, (const bf16*)o_local, lse,
                          (const bf16*)d_o, (bf16*)dq, (cudaStream_t)stream);
+}
+
+hf_status hf_sparse_swa_backward_dkv(hf_ctx* c, int layer, const void* q, const void* k_cur, const void* v_cur, const void* o_local,
+                                     const float* lse, const void* d_o, void* dk, void* dv, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q")); HF_TRY(check_ptr(k_cur, "k_cur")); HF_TRY(check_ptr(v_cur, "v_cur"));
+    HF_TRY(check_ptr(o_local, "o_local")); HF_TRY(check_ptr(lse, "lse")); HF_TRY(check_ptr(d_o, "d_o"));
+    HF_TRY(check_ptr(dk, "dk")); HF_TRY(check_ptr(dv, "dv"));
+    if (c->cfg.block != 128) return fail(HF_ERR_UNSUPPORTED, "the backward kernels take 128-token blocks");
+    if (c->has_trope) return fail(HF_ERR_UNSUPPORTED, "the backward kernels do not rotate their inputs (temporal RoPE is set)");
+    LayerState& L = c->layers[layer];
+    if (L.sel_epoch != L.cache_epoch) return fail(HF_ERR_STATE, "no block selection for the current cache contents; call hf_block_select first");
+    return HF_DISPATCH_D(c, launch_bwd_dkv, c, L, (const bf16*)q, (const bf16*)k_cur, (const bf16*)v_cur, (const bf16*)o_local, lse,
+                         (const bf16*)d_o, (bf16*)dk, (bf16*)dv, (cudaStream_t)stream);
 }
 
 hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void* stream) {

@@ -1,5 +1,6 @@
-"""The backward pass (training rollout's step with gradient, Alg. 1): dq of the block-sparse attention from the tcgen05
-kernel against the oracle's gradient (itself pinned by finite differences and autograd)."""
+"""The backward pass (training rollout's step with gradient, Alg. 1): dq, and dk / dv of the current chunk, of the
+block-sparse attention from the tcgen05 kernels against the oracle's gradients (themselves pinned by finite differences and
+autograd)."""
 import numpy as np
 import pytest
 
@@ -17,7 +18,7 @@ f64 = gen.bf16_bits_to_f64
     (64, 200, 2, 1000, 3, 2),      # head_dim 64, every block kept
     (128, 1300, 2, 150, 8, 2),     # more units than SMs (several units per thread block), sparse lists
 ])
-def test_dq_of_the_sparse_branch(d, tpf, wf, permille, heads, batch):
+def test_gradients_of_the_sparse_branch(d, tpf, wf, permille, heads, batch):
     import torch
     w = gen.Workload("bwd", batch=batch, heads=heads, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=wf,
                      block=128, topk=0, keep_permille=permille, seed=101)
@@ -48,6 +49,24 @@ def test_dq_of_the_sparse_branch(d, tpf, wf, permille, heads, batch):
                 ref[bi, h] = oa.sparse_attention_backward(f64(qb)[bi, h], kc_, vc_, w.block, m_ref[bi, h], f64(gb)[bi, h])[0]
         rl = hz.rel_l2(got, ref); ma = hz.max_abs(got, ref)
         assert rl <= 1e-2 and ma <= 2e-2 * max(1.0, np.abs(ref).max()), f"dq: rel-L2 {rl:.3e}, max-abs {ma:.3e} (max |dq| {np.abs(ref).max():.3f})"
+        # dk, dv of the current chunk (the transposed walk over the selection's bit mask)
+        dk = torch.empty_like(o); dv = torch.empty_like(o)
+        gpu.ctx.hf_sparse_swa_backward_dkv(0, q, k, v, o, lse, g, dk, dv)
+        torch.cuda.synchronize()
+        got_k, got_v = gpu.f64(dk), gpu.f64(dv)
+        ref_k = np.empty_like(got_k); ref_v = np.empty_like(got_v)
+        for bi in range(batch):
+            for h in range(heads):
+                kc_ = [kp[bi, h] for kp, _ in held] + [f64(kb)[bi, h]]
+                vc_ = [vp[bi, h] for _, vp in held] + [f64(vb)[bi, h]]
+                _, dks, dvs = oa.sparse_attention_backward(f64(qb)[bi, h], kc_, vc_, w.block, m_ref[bi, h], f64(gb)[bi, h])
+                ref_k[bi, h] = dks[-1]; ref_v[bi, h] = dvs[-1]
+        for name, a_, b_ in (("dk", got_k, ref_k), ("dv", got_v, ref_v)):
+            rl = hz.rel_l2(a_, b_); ma = hz.max_abs(a_, b_)
+            assert rl <= 1e-2 and ma <= 2e-2 * max(1.0, np.abs(b_).max()), f"{name}: rel-L2 {rl:.3e}, max-abs {ma:.3e} (max {np.abs(b_).max():.3f})"
+        unkept = ~m_ref[..., -w.blocks_per_chunk:].any(axis=2)           # [B, H, n_b]: key blocks of the current chunk nobody keeps
+        for bi, h, jb in zip(*np.nonzero(unkept)):
+            assert not got_k[bi, h, jb * 128:(jb + 1) * 128].any() and not got_v[bi, h, jb * 128:(jb + 1) * 128].any()
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
