@@ -294,6 +294,14 @@ def run_ours(args, w):
         stage["sparse_swa_us"] = timed(lambda r: ctx.hf_sparse_swa(r % L, q[r % L], k[r % L], v[r % L], o), reps)
         # the kernel the step loop launches: sparse attention with the history term formed inside (one launch per call)
         stage["swa_merged_us"] = timed(lambda r: ctx.hf_sparse_swa_merged(r % L, q[r % L], k[r % L], v[r % L], o), reps)
+        # the backward kernels of the sparse branch (layer 0's selection; lse from its forward), timed alone
+        lse = torch.empty(shape[:3], dtype=torch.float32, device="cuda")
+        g_out = torch.randn(shape, device="cuda").to(torch.bfloat16); dq_ = torch.empty_like(o); dk_ = torch.empty_like(o); dv_ = torch.empty_like(o)
+        ctx.hf_sparse_swa(0, q[0], k[0], v[0], o, lse=lse)
+        o_fwd = o.clone()
+        stage["backward_dq_us"] = timed(lambda r: ctx.hf_sparse_swa_backward_dq(0, q[0], k[0], v[0], o_fwd, lse, g_out, dq_), 16)
+        stage["backward_dkv_us"] = timed(lambda r: ctx.hf_sparse_swa_backward_dkv(0, q[0], k[0], v[0], o_fwd, lse, g_out, dk_, dv_), 16)
+        del g_out, dq_, dk_, dv_, o_fwd
         stage["linear_us"] = timed(lambda r: ctx.hf_linear_attn(r % L, q[r % L], o), reps)
         stage["forward_us"] = timed(lambda r: ctx.hf_hybrid_forward(r % L, q[r % L], k[r % L], v[r % L], o), reps)
         stage["absorb_us"] = timed(lambda r: ctx.hf_state_absorb(r % L, kc[r % L], vc[r % L], w.chunk_tokens), reps)
@@ -325,6 +333,12 @@ def run_ours(args, w):
                 "flops_per_launch": flops, "flops_kept_tiles": flops_swa, "flops_history": flops_hist,
                 "attention_alone_tflops": flops_swa / (stage["sparse_swa_us"] * 1e-6) / 1e12,
                 "traffic": SWA_DRAM_BYTES_PER_LAUNCH}
+        # backward: 6 d FLOP per (query row, kept key) pair for dq (S, dP, dQ); 8 d per pair with the key in the CURRENT chunk
+        # for dk / dv (S^T, dP^T, dV, dK)
+        m_bool = hf.unpack_mask(mask.cpu().numpy().view(np.uint32), tn)
+        m_cur = np.zeros_like(m_bool); m_cur[..., tn - w.blocks_per_chunk:] = m_bool[..., tn - w.blocks_per_chunk:]
+        stage["backward_dq_tflops"] = 1.5 * flops_swa / (stage["backward_dq_us"] * 1e-6) / 1e12
+        stage["backward_dkv_tflops"] = 2.0 * kept_flops(m_cur, w) / (stage["backward_dkv_us"] * 1e-6) / 1e12
         bytes_absorb = 2 * w.batch * w.heads * w.chunk_tokens * w.head_dim * 2
         stage["absorb_gbs"] = bytes_absorb / (stage["absorb_us"] * 1e-6) / 1e9
         stage["absorb_frac_hbm"] = stage["absorb_gbs"] / peaks["hbm_gbs"]
