@@ -71,6 +71,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);   // .x = lo (low 16 bits), .y = hi
     return *reinterpret_cast<uint32_t*>(&t);
 }
+// The same packing on the integer pipe (two adds and a byte permute), for loops whose conversion unit is the busy one:
+// round to nearest with ties away from zero, which differs from pack_bf16 only on exact ties.  Finite or infinite
+// inputs (an infinity stays one; a NaN stays a NaN).
+__device__ __forceinline__ uint32_t pack_bf16_alu(float lo, float hi) {
+    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
 __device__ __forceinline__ float2 unpack_bf16(uint32_t u) {
     return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xFFFF0000u));
 }

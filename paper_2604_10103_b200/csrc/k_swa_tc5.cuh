@@ -529,7 +529,7 @@ k_swa_tc5(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUte
 #pragma unroll
                         for (int u = 0; u < 4; ++u) rsum[u] = fadd2(rsum[u], pe[u]);
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) pk[(e0 >> 1) + u] = pack_bf16(pe[u].x, pe[u].y);
+                        for (int u = 0; u < 4; ++u) pk[(e0 >> 1) + u] = pack_bf16_alu(pe[u].x, pe[u].y);
                     }
                     tmem_st16(tS + grp * C::GCOLS + c * 16, pk);
                 }

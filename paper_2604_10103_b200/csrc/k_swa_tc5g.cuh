@@ -374,7 +374,7 @@ k_swa_tc5g(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
 #pragma unroll
                         for (int v = 0; v < 4; ++v) rsum[v] = fadd2(rsum[v], pe[v]);
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) pk[(e0 >> 1) + v] = pack_bf16(pe[v].x, pe[v].y);
+                        for (int v = 0; v < 4; ++v) pk[(e0 >> 1) + v] = pack_bf16_alu(pe[v].x, pe[v].y);
                     }
                     tmem_st16(tS + grp * C::GCOLS + c * 16, pk);
                 }
