@@ -301,6 +301,7 @@ def run_ours(args, w):
         o_fwd = o.clone()
         stage["backward_dq_us"] = timed(lambda r: ctx.hf_sparse_swa_backward_dq(0, q[0], k[0], v[0], o_fwd, lse, g_out, dq_), 16)
         stage["backward_dkv_us"] = timed(lambda r: ctx.hf_sparse_swa_backward_dkv(0, q[0], k[0], v[0], o_fwd, lse, g_out, dk_, dv_), 16)
+        stage["backward_dq_history_us"] = timed(lambda r: ctx.hf_linear_attn_backward_dq(0, q[0], g_out, dq_), 16)
         del g_out, dq_, dk_, dv_, o_fwd
         stage["linear_us"] = timed(lambda r: ctx.hf_linear_attn(r % L, q[r % L], o), reps)
         stage["forward_us"] = timed(lambda r: ctx.hf_hybrid_forward(r % L, q[r % L], k[r % L], v[r % L], o), reps)

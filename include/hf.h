@@ -188,8 +188,8 @@ hf_status hf_sparse_swa(hf_ctx* ctx, int layer, const void* q, const void* k_cur
  *   q, k_cur, v_cur, idx   as for hf_sparse_swa (same cache contents, same selection)
  *   o_local bf16 [B,H,T_c,d], lse float [B,H,T_c]   what hf_sparse_swa returned for them
  *   d_o bf16 [B,H,T_c,d] = dL/dO_local;  dq bf16 [B,H,T_c,d] out
- * 128-token blocks only (HF_ERR_UNSUPPORTED otherwise, and with the temporal rotation set).  The gradients of the history
- * branch are not built yet. */
+ * 128-token blocks only (HF_ERR_UNSUPPORTED otherwise, and with the temporal rotation set).  The history branch's share of
+ * dq comes from hf_linear_attn_backward_dq. */
 hf_status hf_sparse_swa_backward_dq(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const int32_t* idx,
                                     const void* o_local, const float* lse, const void* d_o, void* dq, void* stream);
 
@@ -201,6 +201,15 @@ hf_status hf_sparse_swa_backward_dq(hf_ctx* ctx, int layer, const void* q, const
  * hf_sparse_swa_backward_dq; dk, dv bf16 [B,H,T_c,d] out (zero for a key block that no query block keeps). */
 hf_status hf_sparse_swa_backward_dkv(hf_ctx* ctx, int layer, const void* q, const void* k_cur, const void* v_cur, const void* o_local,
                                      const float* lse, const void* d_o, void* dk, void* dv, void* stream);
+
+/* Gradient of Eq. 4 (hf_linear_attn, per-head or identity merge, no rotation) with respect to the queries.  With
+ * f = phi(q_r), den = f . z + eps, S' = S W^T and g_r = d_o[r] (the gradient with respect to o_hist[r], which by Eq. 7 is
+ * the gradient with respect to the merged output):
+ *   u = S' g_r,   df = (u - (f . u / den) z) / den,   dq[r] = df * phi'(q_r)   (phi' = 1 above zero, e^x otherwise).
+ * S, z and the cached chunks come from earlier, gradient-free passes and receive nothing.  The total gradient of the
+ * hybrid output with respect to q is this plus hf_sparse_swa_backward_dq's (the caller adds them).  q, d_o bf16
+ * [B,H,T_c,d] device; dq bf16 [B,H,T_c,d] out.  HF_ERR_UNSUPPORTED with the full-width merge or a rotation set. */
+hf_status hf_linear_attn_backward_dq(hf_ctx* ctx, int layer, const void* q, const void* d_o, void* dq, void* stream);
 
 /* Eq. 4 without rotation: o_hist[r] = W (phi(q_r) S / (phi(q_r) . z + eps)) + bias, bf16 [B,H,T_c,d]. */
 hf_status hf_linear_attn(hf_ctx* ctx, int layer, const void* q, void* o_hist, void* stream);

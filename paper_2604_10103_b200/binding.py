@@ -28,7 +28,7 @@ EXPORTS = [
     "hf_block_select", "hf_sparse_swa", "hf_linear_attn", "hf_hybrid_forward", "hf_hybrid_forward_host",
     "hf_kv_append_host", "hf_get_state", "hf_query", "hf_get_device_status", "hf_launch_count",
     "hf_status_string", "hf_last_error", "hf_state_absorb_noalloc", "hf_set_rope", "hf_state_export", "hf_state_import",
-    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit", "hf_kv_append_layers", "hf_state_absorb_layers", "hf_set_temporal_rope", "hf_sparse_swa_backward_dq", "hf_sparse_swa_backward_dkv",
+    "hf_sparse_swa_merged", "hf_slow_path_units", "hf_selftest_wait_limit", "hf_kv_append_layers", "hf_state_absorb_layers", "hf_set_temporal_rope", "hf_sparse_swa_backward_dq", "hf_sparse_swa_backward_dkv", "hf_linear_attn_backward_dq",
 ]
 
 
@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
     L.hf_linear_attn.argtypes = [vp, ip, vp, vp, vp]
     L.hf_sparse_swa_backward_dq.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.hf_sparse_swa_backward_dkv.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.hf_linear_attn_backward_dq.argtypes = [vp, ip, vp, vp, vp, vp]
     L.hf_sparse_swa_merged.argtypes = [vp, ip, vp, vp, vp, vp, vp, vp]
     L.hf_hybrid_forward.argtypes = [vp, ip, vp, vp, vp, vp, vp]
     L.hf_hybrid_forward_host.argtypes = [vp, ip, vp, vp, vp, vp, vp]
@@ -190,6 +191,9 @@ class Context:
     def hf_sparse_swa_backward_dkv(self, layer, q, k_cur, v_cur, o_local, lse, d_o, dk, dv):
         _check(lib().hf_sparse_swa_backward_dkv(self._h, layer, _ptr(q), _ptr(k_cur), _ptr(v_cur), _ptr(o_local), _ptr(lse), _ptr(d_o),
                                                 _ptr(dk), _ptr(dv), _stream()))
+
+    def hf_linear_attn_backward_dq(self, layer, q, d_o, dq):
+        _check(lib().hf_linear_attn_backward_dq(self._h, layer, _ptr(q), _ptr(d_o), _ptr(dq), _stream()))
 
     def hf_linear_attn(self, layer, q, o_hist):
         _check(lib().hf_linear_attn(self._h, layer, _ptr(q), _ptr(o_hist), _stream()))

@@ -7,6 +7,7 @@
 #include "k_swa_tc5p.cuh"
 #include "k_swa_tc5g.cuh"
 #include "k_swa_bwd.cuh"
+#include "k_readout_bwd.cuh"
 #include "k_state_mma.cuh"
 #include "k_state_tc5.cuh"
 #include "k_state_items.cuh"
@@ -409,6 +410,20 @@ hf_status launch_readout(hf_ctx* c, LayerState& L, const bf16* q, bf16* out_bf16
     PdlLaunch pl(dim3(mp.Tm, c->cfg.heads, c->cfg.batch), dim3(M::THREADS), M::SMEM_BYTES, st, false);
     HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_merge_full<D>, txh, txl, L.tm_wfull, mp));
     return post_launch(c, "k_merge_full");
+}
+
+template <int D>
+hf_status launch_readout_bwd(hf_ctx* c, LayerState& L, const bf16* q, const bf16* d_o, bf16* dq, cudaStream_t st) {
+    typedef ReadoutBwd<D> R;
+    HF_CUDA(cudaFuncSetAttribute(k_readout_bwd_dq<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, R::SMEM_BYTES));
+    CUtensorMap tg;
+    HF_TRY(make_map(c, &tg, d_o, 1));
+    ReadoutBwdParams p;
+    p.q = q; p.z = L.z; p.dq = dq; p.Tc = c->Tc; p.Tm = (c->Tc + R::ROWS - 1) / R::ROWS; p.n_units = p.Tm * c->BH;
+    p.eps = c->cfg.eps; p.dev_status = c->dev_status;
+    const int grid = p.n_units < c->sm_count ? p.n_units : c->sm_count;
+    k_readout_bwd_dq<D><<<grid, R::THREADS, R::SMEM_BYTES, st>>>(tg, L.tm_sfhi, L.tm_sflo, p);
+    return post_launch(c, "k_readout_bwd_dq");
 }
 
 ChunkTable make_table(hf_ctx* c, LayerState& L, const bf16* k_cur, const bf16* v_cur) {
@@ -1188,6 +1203,14 @@ hf_status hf_linear_attn(hf_ctx* c, int layer, const void* q, void* o_hist, void
         q = c->q_rot;
     }
     return HF_DISPATCH_D(c, launch_readout, c, c->layers[layer], (const bf16*)q, (bf16*)o_hist, (float*)nullptr, (cudaStream_t)stream);
+}
+
+hf_status hf_linear_attn_backward_dq(hf_ctx* c, int layer, const void* q, const void* d_o, void* dq, void* stream) {
+    HF_TRY(check_layer(c, layer));
+    HF_TRY(check_ptr(q, "q")); HF_TRY(check_ptr(d_o, "d_o")); HF_TRY(check_ptr(dq, "dq"));
+    if (c->cfg.merge == HF_MERGE_FULL_WIDTH) return fail(HF_ERR_UNSUPPORTED, "the read-out's backward takes the per-head (or identity) merge");
+    if (c->has_rope_q || c->has_trope) return fail(HF_ERR_UNSUPPORTED, "the read-out's backward does not rotate its inputs (a rotation is set)");
+    return HF_DISPATCH_D(c, launch_readout_bwd, c, c->layers[layer], (const bf16*)q, (const bf16*)d_o, (bf16*)dq, (cudaStream_t)stream);
 }
 
 // Eq. 6 + Eq. 4 + Eq. 7 for a selection that is already made.  after_select: the call follows launch_select in the same

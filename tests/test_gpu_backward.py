@@ -70,3 +70,38 @@ def test_gradients_of_the_sparse_branch(d, tpf, wf, permille, heads, batch):
         assert gpu.ctx.hf_get_device_status() == (0, 0)
     finally:
         gpu.close()
+
+
+@pytest.mark.parametrize("d,tpf,heads,batch,merge", [
+    (128, 300, 2, 1, True),        # per-head Linear folded into the state; 44-token tail tile
+    (64, 200, 3, 2, True),         # head_dim 64
+    (128, 1300, 8, 2, False),      # identity merge; several tiles per thread block, a new head in the middle of a range
+])
+def test_gradient_of_the_history_readout(d, tpf, heads, batch, merge):
+    """dq of Eq. 4 (u = S' g on the tensor cores, then the quotient rule per row) against the oracle's read-out gradient."""
+    import torch
+    w = gen.Workload("bwdh", batch=batch, heads=heads, head_dim=d, tokens_per_frame=tpf, chunk_frames=1, window_frames=2,
+                     block=128, topk=0, keep_permille=500, seed=103)
+    gpu = hz.GpuStream(w, merge=merge); ora = hz.make_oracle(w, merge=merge)
+    try:
+        for c in range(4):                         # three chunks absorbed
+            kc, vc = gen.clean_kv(w, 0, c)
+            gpu.append(gpu.up(kc), gpu.up(vc)); ora.append(f64(kc), f64(vc))
+        assert ora.absorbed_tokens == 3 * tpf
+        qb, _, _ = gen.qkv(w, 0, 5, 0)
+        gb = gen.normal_bf16(qb.shape, 103, 7, 7)
+        q, g = gpu.up(qb), gpu.up(gb)
+        dq = torch.empty_like(q)
+        gpu.ctx.hf_linear_attn_backward_dq(0, q, g, dq)
+        torch.cuda.synchronize()
+        got = gpu.f64(dq)
+        ref = np.empty_like(got)
+        for bi in range(batch):
+            for h in range(heads):
+                ref[bi, h] = oa.linear_readout_backward(f64(qb)[bi, h], ora.S[bi, h], ora.z[bi, h], f64(gb)[bi, h],
+                                                        W=None if ora.W is None else ora.W[h], eps=ora.eps)[0]
+        rl = hz.rel_l2(got, ref); ma = hz.max_abs(got, ref)
+        assert rl <= 1e-2 and ma <= 2e-2 * max(1.0, np.abs(ref).max()), f"dq_hist: rel-L2 {rl:.3e}, max-abs {ma:.3e} (max {np.abs(ref).max():.3e})"
+        assert gpu.ctx.hf_get_device_status() == (0, 0)
+    finally:
+        gpu.close()
