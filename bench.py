@@ -32,7 +32,7 @@ from paper_2604_10103_b200 import inputs as gen, replicas  # noqa: E402
 METRIC = "hybrid-attn latent frames/s at 832x480 shape"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the attention kernel (history term inside) at this
 # workload's layer shape, from an ncu capture of that kernel; None when the kernel has changed since the capture.
-SWA_DRAM_BYTES_PER_LAUNCH = 106.6e6
+SWA_DRAM_BYTES_PER_LAUNCH = 107.3e6
 UNIT = "latent frames/s"
 
 
@@ -287,6 +287,9 @@ def run_ours(args, w):
             dist.destroy_process_group()
         return
     if rank == 0:
+        # The kernel-alone figures below are burst measurements (batches of a few milliseconds each): one second of idle
+        # first, so that the board's power controller, which the step loop above has driven towards its cap, starts from rest
+        time.sleep(1.0)
         reps = 2 * L
         stage["select_us"] = timed(lambda r: ctx.hf_block_select(r % L, q[r % L], k[r % L]), reps)
         for l in range(L):
@@ -326,7 +329,7 @@ def run_ours(args, w):
         ach_loop = flops / (breakdown["forward_us_mean"] * 1e-6) / 1e12 if breakdown else None
         roof = {"bound": "tensor", "kernel": "k_swa_tc5 with the history term inside (hf_sparse_swa_merged)", "achieved": ach, "peak": peak,
                 "unit": "TFLOP/s", "frac": ach / peak,
-                "peak_source": f"{peaks['source']} (burst cuBLAS bf16: the kernel is timed alone over {reps} launches; sustained {peaks['bf16_tflops_sustained']})",
+                "peak_source": f"{peaks['source']} (burst cuBLAS bf16: the kernel is timed alone over {reps} launches after 1 s of idle; sustained {peaks['bf16_tflops_sustained']})",
                 "frac_of_sustained": ach / peaks["bf16_tflops_sustained"], "frac_of_datasheet_2250": ach / 2250.0,
                 # the whole forward (pooling + selection + attention) inside the seconds-long step loop, same FLOPs, against the sustained figure
                 "forward_in_step_loop_tflops": ach_loop,
@@ -496,11 +499,49 @@ def run_sweep(args):
         out.close()
 
 
+def run_profile_backward():
+    """A small stand-alone run of the backward kernels, for profilers: one layer of the 832x480 shape (window 9, two cached
+    chunks and one absorbed), three calls of each of dq, dk / dv and the read-out's dq."""
+    import torch
+    from paper_2604_10103_b200 import binding as hf, build as hfbuild
+    hfbuild.build()
+    w = gen.layer_832x480().with_(layers=1)
+    ctx = hf.Context(hf.make_config(w))
+    Wb, bb = gen.merge_weights(w, 0)
+    ctx.hf_set_merge_weights(0, hf.bits_to_cuda(Wb), hf.bits_to_cuda(bb))
+    g = torch.Generator(device="cuda"); g.manual_seed(98)
+    shape = (w.batch, w.heads, w.chunk_tokens, w.head_dim)
+    mk = lambda: torch.randn(shape, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    for _ in range(w.past_chunks + 1):
+        ctx.hf_kv_append(0, mk(), mk())
+    q, k, v, go = mk(), mk(), mk(), mk()
+    o = torch.empty_like(q); dq = torch.empty_like(q); dk = torch.empty_like(q); dv = torch.empty_like(q)
+    lse = torch.empty(shape[:3], dtype=torch.float32, device="cuda")
+    ctx.hf_block_select(0, q, k)
+    ctx.hf_sparse_swa(0, q, k, v, o, lse=lse)
+    out = {"stage": "backward"}
+    for name, fn in (("dq_us", lambda: ctx.hf_sparse_swa_backward_dq(0, q, k, v, o, lse, go, dq)),
+                     ("dkv_us", lambda: ctx.hf_sparse_swa_backward_dkv(0, q, k, v, o, lse, go, dk, dv)),
+                     ("dq_history_us", lambda: ctx.hf_linear_attn_backward_dq(0, q, go, dq))):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for i in range(3):
+            if i == 2:
+                a.record()
+            fn()
+        b.record(); torch.cuda.synchronize()
+        out[name] = a.elapsed_time(b) * 1e3
+    out["status"] = ctx.hf_get_device_status()
+    print(json.dumps(out))
+    ctx.close()
+
+
 def run_profile_stage(args):
     """A small stand-alone run of one stage, for profilers: the layer-batched state update on 13 layers of the
     832x480 layer shape (156 (layer, head) items, under 1 GB on the device; no cache ring is allocated)."""
     import torch
     from paper_2604_10103_b200 import binding as hf, build as hfbuild
+    if args.profile_stage == "backward":
+        return run_profile_backward()
     hfbuild.build()
     L = 13
     w = gen.layer_832x480().with_(layers=L, window_frames=3)        # window == chunk: no ring
@@ -542,7 +583,7 @@ def main():
                     help="instead of the benchmark line: per-stage times over the keep x window x head_dim x block x batch grid, "
                          "one JSON line per point (1 GPU)")
     ap.add_argument("--sweep-out", default=None, help="file for the sweep's JSON lines (default: stdout)")
-    ap.add_argument("--profile-stage", default=None, choices=["absorb_layers"],
+    ap.add_argument("--profile-stage", default=None, choices=["absorb_layers", "backward"],
                     help="instead of the benchmark line: a small run of one stage alone (for ncu captures)")
     args = ap.parse_args()
     w = gen.full_depth_832x480(layers=args.layers, steps=args.denoise_steps)
