@@ -7,13 +7,15 @@
 // and k_rowdot forms delta; the block mask is the forward's (held fixed: the top-K choice is piecewise constant).
 //
 // Per (batch*head, query block) unit and kept key tile t, three tensor-core products:
-//   S  = Q K_t^T          A = Q  (smem, K-major),  B = K_t (smem, K-major)          -> TMEM [0, 128)
+//   S  = Q K_t^T          A = Q  (smem, K-major),  B = K_t (smem, K-major)          -> TMEM [0, 128) / [384, 512), t even / odd
 //   dP = dO V_t^T         A = dO (smem, K-major),  B = V_t (smem, K-major)          -> TMEM [128, 256)
 //   dQ += dS K_t          A = dS (TMEM, bf16, written over S),  B = K_t (MN-major)   -> TMEM [256, 256 + D)
 // and between them, on the softmax warps (thread = query row x half of the 128 key columns):
 //   dS = exp2(S c - lse log2 e) * (dP - delta) / sqrt(d)        (columns past a short block's end: 0)
-// A first version: S, dP single-buffered (tensor core and softmax warps alternate); K and V tiles double-buffered so that
-// the loads run ahead.  Every wait is bounded and reports through the device status word.
+// The two score products of tile t + 1 are issued while the softmax warps work on tile t: S has two buffers, and the
+// softmax threads free dP's one buffer as soon as their share of it is in registers.  A K tile is held from S to dS K
+// (three stages), a V tile only until dP (two); with less, the latency of the tile loads (~3 000 clk here) is what a
+// tile costs.  Every wait is bounded and reports through the device status word.
 #pragma once
 #include "k_swa_tc5.cuh"
 
@@ -38,14 +40,17 @@ template <int D>
 struct SwaBwd {
     static constexpr int BLK = 128;
     static constexpr int SUB = D / 64, SUB_BYTES = BLK * 128, TILE_BYTES = SUB * SUB_BYTES;
-    static constexpr int STAGES = 2;
-    static constexpr int OFF_Q = 0, OFF_DO = TILE_BYTES, OFF_K = 2 * TILE_BYTES, OFF_V = OFF_K + STAGES * TILE_BYTES;
-    static constexpr int OFF_BAR = OFF_V + STAGES * TILE_BYTES;
+    // a K tile is held until its dS K product has completed, a V tile only until dP has: three and two stages
+    static constexpr int KST = 3, VST = 2;
+    static constexpr int OFF_Q = 0, OFF_DO = TILE_BYTES, OFF_K = 2 * TILE_BYTES, OFF_V = OFF_K + KST * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_V + VST * TILE_BYTES;
     static constexpr int USED_BYTES = OFF_BAR + 256;
     static constexpr int SMEM_BYTES = USED_BYTES + 1024;
     static constexpr int THREADS = 320;                  // warps 0-7: softmax (two column groups), 8: TMA, 9: MMA
     static constexpr int WARP_TMA = 8, WARP_MMA = 9;
-    static constexpr int COL_S = 0, COL_DP = 128, COL_DQ = 256, TMEM_COLS = 512;
+    // S alternates between two buffers (tile t in buffer t % 2, the bf16 dS written over it); dP has one, which the softmax
+    // threads free as soon as they hold their share of it in registers
+    static constexpr int COL_S = 0, COL_S1 = 384, COL_DP = 128, COL_DQ = 256, TMEM_COLS = 512;
 };
 
 struct SwaBwdParams {
@@ -71,18 +76,20 @@ k_swa_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
     uint8_t* s_gen = smem_raw + (s_base - smem_u32(smem_raw));
     const uint32_t sQ = s_base + C::OFF_Q, sDO = s_base + C::OFF_DO, sK = s_base + C::OFF_K, sV = s_base + C::OFF_V;
     const uint32_t bar0 = s_base + C::OFF_BAR;
-    const uint32_t bar_kf = bar0, bar_ke = bar0 + 16, bar_vf = bar0 + 32, bar_ve = bar0 + 48, bar_qf = bar0 + 64, bar_qe = bar0 + 72,
-                   bar_sd = bar0 + 80, bar_ds = bar0 + 88, bar_dqf = bar0 + 96, bar_dqe = bar0 + 104;
+    const uint32_t bar_kf = bar0 + 128, bar_ke = bar0 + 152, bar_vf = bar0 + 32, bar_ve = bar0 + 48, bar_qf = bar0 + 64, bar_qe = bar0 + 72,
+                   bar_sd = bar0 + 80, bar_ds = bar0 + 88, bar_dqf = bar0 + 96, bar_dqe = bar0 + 104, bar_dpf = bar0 + 120;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(s_gen + C::OFF_BAR + 112);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(s_gen + C::OFF_BAR + 116);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int keep = p.keep;
     const int my_units = (p.n_units - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int n_tiles = my_units * keep;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < C::STAGES; ++s) { mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1); mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); }
-        mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_sd, 1); mbar_init(bar_ds, 256); mbar_init(bar_dqf, 1); mbar_init(bar_dqe, 256);
+        for (int s = 0; s < C::KST; ++s) { mbar_init(bar_kf + 8 * s, 1); mbar_init(bar_ke + 8 * s, 1); }
+        for (int s = 0; s < C::VST; ++s) { mbar_init(bar_vf + 8 * s, 1); mbar_init(bar_ve + 8 * s, 1); }
+        mbar_init(bar_qf, 1); mbar_init(bar_qe, 1); mbar_init(bar_sd, 1); mbar_init(bar_ds, 256); mbar_init(bar_dqf, 1); mbar_init(bar_dqe, 256); mbar_init(bar_dpf, 256);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
@@ -123,19 +130,17 @@ k_swa_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                         if (c < p.n_sink) slot = p.P + c;
                         else { slot = p.ring_head + c - p.n_sink; if (slot >= p.P) slot -= p.P; }
                     }
-                    const int st = t % C::STAGES;
-                    const uint32_t par_free = ((t / C::STAGES) & 1) ^ 1;
-                    if (t >= C::STAGES) {
-                        if (!(ok = mbar_wait<true>(bar_ke + 8 * st, par_free, abort_flag, p.dev_status, 82))) break;
-                        if (!(ok = mbar_wait<true>(bar_ve + 8 * st, par_free, abort_flag, p.dev_status, 83))) break;
-                    }
-                    mbar_expect_tx(bar_kf + 8 * st, C::TILE_BYTES);
-                    mbar_expect_tx(bar_vf + 8 * st, C::TILE_BYTES);
+                    const int kst = t % C::KST, vst = t % C::VST;
+                    if (t >= C::VST && !(ok = mbar_wait<true>(bar_ve + 8 * vst, ((t / C::VST) & 1) ^ 1, abort_flag, p.dev_status, 83))) break;
+                    mbar_expect_tx(bar_vf + 8 * vst, C::TILE_BYTES);
 #pragma unroll
-                    for (int s = 0; s < C::SUB; ++s) {
-                        tma_load_4d(sK + st * C::TILE_BYTES + s * C::SUB_BYTES, cur ? &tm_kcur : &tm_kring, s * 64, jb * C::BLK, bh, slot, bar_kf + 8 * st);
-                        tma_load_4d(sV + st * C::TILE_BYTES + s * C::SUB_BYTES, cur ? &tm_vcur : &tm_vring, s * 64, jb * C::BLK, bh, slot, bar_vf + 8 * st);
-                    }
+                    for (int s = 0; s < C::SUB; ++s)
+                        tma_load_4d(sV + vst * C::TILE_BYTES + s * C::SUB_BYTES, cur ? &tm_vcur : &tm_vring, s * 64, jb * C::BLK, bh, slot, bar_vf + 8 * vst);
+                    if (t >= C::KST && !(ok = mbar_wait<true>(bar_ke + 8 * kst, ((t / C::KST) & 1) ^ 1, abort_flag, p.dev_status, 82))) break;
+                    mbar_expect_tx(bar_kf + 8 * kst, C::TILE_BYTES);
+#pragma unroll
+                    for (int s = 0; s < C::SUB; ++s)
+                        tma_load_4d(sK + kst * C::TILE_BYTES + s * C::SUB_BYTES, cur ? &tm_kcur : &tm_kring, s * 64, jb * C::BLK, bh, slot, bar_kf + 8 * kst);
                 }
             }
             if (!ok) {
@@ -153,30 +158,45 @@ k_swa_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
         const uint64_t dkm = smem_desc_sw128(sK, C::SUB_BYTES, 1024);        // the K tile again, as the MN-major operand of dS K
         const uint32_t hi_k = (uint32_t)(dq0 >> 32), hi_m = (uint32_t)(dkm >> 32);
         bool ok = true;
+        // S_t = Q K_t^T and dP_t = dO V_t^T, one tile ahead of the softmax warps: tile t + 1 is issued while they turn
+        // tile t into dS (S into the other buffer; dP as soon as they have taken tile t's out of tensor memory)
+        int n_s = 0, j_s = 0, t_s = 0;
+        auto issue_scores = [&]() -> bool {
+            if (j_s == 0 && !__all_sync(0xffffffffu, mbar_wait<true>(bar_qf, n_s & 1, abort_flag, p.dev_status, 84))) return false;
+            const int kst = t_s % C::KST, vst = t_s % C::VST;
+            if (!__all_sync(0xffffffffu, mbar_wait<true>(bar_kf + 8 * kst, (t_s / C::KST) & 1, abort_flag, p.dev_status, 85))) return false;
+            if (!__all_sync(0xffffffffu, mbar_wait<true>(bar_vf + 8 * vst, (t_s / C::VST) & 1, abort_flag, p.dev_status, 86))) return false;
+            fence_after_sync();
+            if (elect_one()) {
+                mma_ss_tile<D>(tmem + ((t_s & 1) ? C::COL_S1 : C::COL_S), (uint32_t)dq0, (uint32_t)dk0 + kst * TILE_STEP, hi_k, IDESC_S);
+                mma_ss_tile<D>(tmem + C::COL_DP, (uint32_t)dd0, (uint32_t)dv0 + vst * TILE_STEP, hi_k, IDESC_S);
+                mma_commit(bar_sd);
+                mma_commit(bar_ve + 8 * vst);
+                if (j_s == keep - 1) mma_commit(bar_qe);          // Q and dO of this unit have been read for the last time
+            }
+            __syncwarp();
+            ++t_s;
+            if (++j_s == keep) { j_s = 0; ++n_s; }
+            return true;
+        };
+        if (n_tiles > 0) ok = issue_scores();
         int t = 0;
         for (int n = 0; ok && n < my_units; ++n) {
-            if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_qf, n & 1, abort_flag, p.dev_status, 84)))) break;
             for (int j = 0; ok && j < keep; ++j, ++t) {
-                const int st = t % C::STAGES;
-                const uint32_t par = (t / C::STAGES) & 1;
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_kf + 8 * st, par, abort_flag, p.dev_status, 85)))) break;
-                if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_vf + 8 * st, par, abort_flag, p.dev_status, 86)))) break;
-                fence_after_sync();
-                if (elect_one()) {
-                    mma_ss_tile<D>(tmem + C::COL_S, (uint32_t)dq0, (uint32_t)dk0 + st * TILE_STEP, hi_k, IDESC_S);
-                    mma_ss_tile<D>(tmem + C::COL_DP, (uint32_t)dd0, (uint32_t)dv0 + st * TILE_STEP, hi_k, IDESC_S);
-                    mma_commit(bar_sd);
-                    mma_commit(bar_ve + 8 * st);
-                    if (j == keep - 1) mma_commit(bar_qe);          // Q and dO of this unit have been read for the last time
+                const int kst = t % C::KST;
+                if (t + 1 < n_tiles) {
+                    // dP of tile t is in the softmax threads' registers: the buffer may take tile t + 1
+                    if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_dpf, t & 1, abort_flag, p.dev_status, 91)))) break;
+                    if (!(ok = issue_scores())) break;
                 }
-                __syncwarp();
                 if (!(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_ds, t & 1, abort_flag, p.dev_status, 87)))) break;
                 // the accumulator of the previous unit has been read out before this unit's first product overwrites it
                 if (j == 0 && n >= 1 && !(ok = __all_sync(0xffffffffu, mbar_wait<true>(bar_dqe, (n - 1) & 1, abort_flag, p.dev_status, 88)))) break;
                 fence_after_sync();
                 if (elect_one()) {
-                    mma_ts_tile_split(tmem + C::COL_DQ, tmem + C::COL_S, tmem + C::COL_S + 64, (uint32_t)dkm + st * TILE_STEP, hi_m, IDESC_DQ, j > 0);
-                    mma_commit(bar_ke + 8 * st);
+                    const uint32_t tS = tmem + ((t & 1) ? C::COL_S1 : C::COL_S);
+                    mma_ts_tile_split(tmem + C::COL_DQ, tS, tS + 64, (uint32_t)dkm + kst * TILE_STEP, hi_m, IDESC_DQ, j > 0);
+                    mma_commit(bar_ke + 8 * kst);
                     if (j == keep - 1) mma_commit(bar_dqf);
                 }
                 __syncwarp();
@@ -206,24 +226,34 @@ k_swa_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ C
                 ok = __all_sync(0xffffffffu, mbar_wait(bar_sd, t & 1, abort_flag, p.dev_status, 89));
                 if (!ok) break;
                 fence_after_sync();
+                const uint32_t tS = lane_base + ((t & 1) ? C::COL_S1 : C::COL_S) + grp * 64;
+                // this thread's share of dP first, all of it: the MMA warp refills the buffer as soon as every thread has it
+                uint32_t dp[2][32], s[32];
+                tmem_ld32(lane_base + C::COL_DP + grp * 64, dp[0]);
+                tmem_ld32(lane_base + C::COL_DP + grp * 64 + 32, dp[1]);
+                tmem_ld32(tS, s);
+                tmem_wait_ld();
+                fence_before_sync();
+                mbar_arrive(bar_dpf);
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
-                    uint32_t s[32], dp[32], pk[16];
-                    tmem_ld32(lane_base + C::COL_S + grp * 64 + c * 32, s);
-                    tmem_ld32(lane_base + C::COL_DP + grp * 64 + c * 32, dp);
-                    tmem_wait_ld();
+                    uint32_t pk[16];
+                    if (c == 1) {
+                        tmem_ld32(tS + 32, s);
+                        tmem_wait_ld();
+                    }
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
                         const float p0 = fast_exp2(fmaf(__uint_as_float(s[e]), p.scale_log2, neg_lse2));
                         const float p1 = fast_exp2(fmaf(__uint_as_float(s[e + 1]), p.scale_log2, neg_lse2));
-                        float d0 = p0 * (__uint_as_float(dp[e]) - delta) * p.scale;
-                        float d1 = p1 * (__uint_as_float(dp[e + 1]) - delta) * p.scale;
+                        float d0 = p0 * (__uint_as_float(dp[c][e]) - delta) * p.scale;
+                        float d1 = p1 * (__uint_as_float(dp[c][e + 1]) - delta) * p.scale;
                         if (grp * 64 + c * 32 + e >= nv) d0 = 0.f;
                         if (grp * 64 + c * 32 + e + 1 >= nv) d1 = 0.f;
-                        pk[e >> 1] = pack_bf16(d0, d1);
+                        pk[e >> 1] = pack_bf16_alu(d0, d1);
                     }
                     // (all of this thread's S columns of the chunk are in registers: the bf16 dS may go over them)
-                    tmem_st16(lane_base + C::COL_S + grp * 64 + c * 16, pk);
+                    tmem_st16(tS + c * 16, pk);
                 }
                 tmem_wait_st();
                 fence_before_sync();
