@@ -460,8 +460,14 @@ hf_status launch_select(hf_ctx* c, LayerState& L, const bf16* q, const bf16* k_c
     const int keep = keep_for(c, Tn);
     ChunkTable tab = make_table(c, L, k_cur, nullptr);
     PdlLaunch pl(dim3(c->Tm, c->BH), dim3(256), 0, st, true);      // follows the pooling kernel launched above
-    HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
-                               L.mask, L.idx, mask_out, idx_out, scores_out));
+    // Two forms of the scoring loop, same arithmetic: the wide one keeps a pass's loads in flight (80 registers, three
+    // thread blocks per SM) and is ahead while the grid fits that; the narrow one (40 registers) fits twice the thread blocks.
+    if (c->Tm * c->BH <= 3 * c->sm_count)
+        HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D, true>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+                                   L.mask, L.idx, mask_out, idx_out, scores_out));
+    else
+        HF_CUDA(cudaLaunchKernelEx(&pl.cfg, k_select<D, false>, tab, (const float*)c->pooled_q, c->n_b, c->Tm, Tn, keep, c->mask_words,
+                                   L.mask, L.idx, mask_out, idx_out, scores_out));
     HF_TRY(post_launch(c, "k_select"));
     L.sel_epoch = L.cache_epoch;
     L.sel_keep = keep;

@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(256, 6) k_pool_copy_layers(const __grid_consta
 // grid (T_m, B*H), 256 threads.  One query-block row: T_n scores, top-K under the total order (score descending, block
 // index ascending; by counting for short rows, by a bitonic sort of (score, index) keys for long ones), bit mask +
 // ascending index list.
-template <int D>
+template <int D, bool WIDE>
 __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __restrict__ pooled_q,
                                                 int n_b, int Tm, int Tn, int keep, int mask_words,
                                                 uint32_t* __restrict__ mask, int32_t* __restrict__ idx,
@@ -215,17 +215,52 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
 #pragma unroll
             for (int m = 0; m < M; ++m) kv[u][m] = __ldg(kp + 32 * m);
         }
+        if constexpr (WIDE) {
+            // one butterfly per key row (the compiler keeps all loads of the pass in flight in front of them: ~80 registers)
 #pragma unroll
-        for (int u = 0; u < PER; ++u) {
-            float p = __fmul_rn(qv[0], kv[u][0]);
+            for (int u = 0; u < PER; ++u) {
+                float p = __fmul_rn(qv[0], kv[u][0]);
 #pragma unroll
-            for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[m], kv[u][m]));
+                for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[m], kv[u][m]));
 #pragma unroll
-            for (int off = 16; off >= 1; off >>= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, off));
-            const int j = base + warp + NW * u;
-            if (lane == 0 && j < Tn) {
-                sc[j] = p;
-                if (scores_out) scores_out[row * Tn + j] = p;
+                for (int off = 16; off >= 1; off >>= 1) p = __fadd_rn(p, __shfl_xor_sync(0xffffffffu, p, off));
+                const int j = base + warp + NW * u;
+                if (lane == 0 && j < Tn) {
+                    sc[j] = p;
+                    if (scores_out) scores_out[row * Tn + j] = p;
+                }
+            }
+        } else {
+            // The sixteen butterflies side by side.  At the step with lane offset `off` a lane keeps the half of its rows
+            // that its own bit of `off` names and hands the other half to its partner, which does the opposite: every sum
+            // is still own partial + partner's partial (IEEE addition commutes, so both orders give the same bits), level
+            // by level as in the one-row butterfly, with 8 + 4 + 2 + 1 + 1 shuffles instead of 16 x 5.  After the last
+            // step lanes 2u and 2u + 1 both hold the score of row u.  (The compiler pairs this form's loads with their
+            // products: ~40 registers, twice the resident thread blocks, more trips to memory per pass.)
+            float pa[PER];
+#pragma unroll
+            for (int u = 0; u < PER; ++u) {
+                float p = __fmul_rn(qv[0], kv[u][0]);
+#pragma unroll
+                for (int m = 1; m < M; ++m) p = __fadd_rn(p, __fmul_rn(qv[m], kv[u][m]));
+                pa[u] = p;
+            }
+#pragma unroll
+            for (int half = PER / 2, off = 16; half >= 1; half >>= 1, off >>= 1) {
+                const bool upper = (lane & off) != 0;
+#pragma unroll
+                for (int x = 0; x < half; ++x) {
+                    const float mine = upper ? pa[x + half] : pa[x];
+                    const float theirs = upper ? pa[x] : pa[x + half];
+                    pa[x] = __fadd_rn(mine, __shfl_xor_sync(0xffffffffu, theirs, off));
+                }
+            }
+            static_assert(PER == 16, "one row per lane pair after four halvings");
+            const float score = __fadd_rn(pa[0], __shfl_xor_sync(0xffffffffu, pa[0], 1));
+            const int j = base + warp + NW * (lane >> 1);
+            if ((lane & 1) == 0 && j < Tn) {
+                sc[j] = score;
+                if (scores_out) scores_out[row * Tn + j] = score;
             }
         }
     }
@@ -234,32 +269,41 @@ __global__ void __launch_bounds__(256) k_select(ChunkTable tab, const float* __r
     // NaN anywhere in the query block or the key block) compares false both ways and would otherwise rank first everywhere:
     // here it ranks below every number, NaNs among themselves by block index, so that exactly `keep` blocks are kept whatever
     // the inputs hold.
+    // 64-bit keys: an order-preserving image of the score (NaN lowest, -0 = +0), then the complement of the block index;
+    // all keys of a row are distinct and "comes before" is "has the larger key"
+    auto key_of = [](float s, int j) -> unsigned long long {
+        uint32_t u = __float_as_uint(s);
+        if (s != s) u = 0u;                                         // NaN: below -inf
+        else {
+            if (u == 0x80000000u) u = 0u;                           // -0 ties with +0
+            u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);         // ascending integers = ascending floats
+        }
+        return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)j);
+    };
     if (Tn <= 128) {
-        // short rows: count, for every block, the blocks that come before it
-        for (int j = threadIdx.x; j < Tn; j += 256) {
-            const float s = sc[j];
-            const bool s_nan = s != s;
+        // short rows: count, for every block, the blocks that come before it.  Two threads per block, one for the even and
+        // one for the odd competitors, four comparisons in flight each.
+        for (int j = threadIdx.x; j < Tn; j += 256) keys[j] = key_of(sc[j], j);
+        __syncthreads();
+        {
+            const int j = threadIdx.x >> 1, par = threadIdx.x & 1;
             int rank = 0;
-            for (int jj = 0; jj < Tn; ++jj) {
-                const float s2 = sc[jj];
-                const bool s2_nan = s2 != s2;
-                const bool tie = (s2 == s) || (s_nan && s2_nan);
-                rank += (s2 > s) || (s_nan && !s2_nan) || (tie && jj < j);
+            if (j < Tn) {
+                const unsigned long long mine = keys[j];
+                int r0 = 0, r1 = 0, r2 = 0, r3 = 0;
+                int jj = par;
+                for (; jj + 6 < Tn; jj += 8) {
+                    r0 += keys[jj] > mine; r1 += keys[jj + 2] > mine; r2 += keys[jj + 4] > mine; r3 += keys[jj + 6] > mine;
+                }
+                for (; jj < Tn; jj += 2) r0 += keys[jj] > mine;
+                rank = (r0 + r1) + (r2 + r3);
             }
-            keepf[j] = rank < keep;
+            rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+            if (par == 0 && j < Tn) keepf[j] = rank < keep;
         }
     } else {
-        // long rows (counting is quadratic in T_n): sort 64-bit keys (order-preserving image of the score, then the
-        // complement of the index) in shared memory with a bitonic network and compare every block with the keep-th key
-        auto key_of = [](float s, int j) -> unsigned long long {
-            uint32_t u = __float_as_uint(s);
-            if (s != s) u = 0u;                                         // NaN: below -inf
-            else {
-                if (u == 0x80000000u) u = 0u;                           // -0 ties with +0
-                u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);         // ascending integers = ascending floats
-            }
-            return ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (uint32_t)j);
-        };
+        // long rows (counting is quadratic in T_n): sort the keys in shared memory with a bitonic network and compare every
+        // block with the keep-th key
         int n2 = 256;
         while (n2 < Tn) n2 <<= 1;
         for (int j = threadIdx.x; j < n2; j += 256) keys[j] = j < Tn ? key_of(sc[j], j) : 0ull;      // padding sorts last
